@@ -1,0 +1,347 @@
+"""Pins for the float64 CPU oracle (no GPU needed).
+
+The paper (arXiv 1801.04928) prints no worked numbers, so the oracle is tied to what the
+mathematics fixes: the gradient is the derivative of the cost (central finite differences
+of C, which only needs the forward pass), closed forms of special networks, the structure
+Eq. bp3/bp4 impose, and Theorem 1 (every layer saved exactly once) together with a hand
+trace of Algorithm 1.  Each test names the mistake it is there to catch.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import lf_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _net(L, N, B, seed, y_kind="uniform"):
+    r = np.random.default_rng(seed)
+    w = r.normal(0.0, 1.0 / np.sqrt(N), size=(L, N, N))
+    b = r.normal(0.0, 1.0, size=(L, N))
+    x = r.uniform(0.0, 1.0, size=(B, N))
+    if y_kind == "uniform":
+        y = r.uniform(0.0, 1.0, size=(B, N))
+    else:
+        y = np.zeros((B, N))
+        y[np.arange(B), r.integers(0, N, size=B)] = 1.0
+    return w, b, x, y
+
+
+def _cost(w, b, x, y):
+    _, a = orc.forward(w, b, x)
+    return orc.cost(a, y)
+
+
+# ---- sigma ---------------------------------------------------------------------------------
+
+def test_sigmoid_values_and_symmetry():
+    # sigma(0) = 1/2, sigma(ln 3) = 3/4, sigma(-t) = 1 - sigma(t); no overflow far out.
+    assert orc.sigma(0.0) == 0.5
+    assert abs(orc.sigma(np.log(3.0)) - 0.75) < 1e-15
+    for t in (0.3, 2.0, 17.0, 700.0, 800.0):
+        assert abs(orc.sigma(-t) - (1.0 - orc.sigma(t))) < 1e-15
+        assert np.isfinite(orc.sigma(t)) and np.isfinite(orc.sigma(-t))
+    assert orc.sigma(800.0) == 1.0 and orc.sigma(-800.0) == 0.0
+    # sigma' peaks at 1/4 in 0 and matches a central difference of sigma elsewhere.
+    assert orc.sigma_prime(0.0) == 0.25
+    for t in (-3.0, -0.7, 0.4, 2.5):
+        h = 1e-6
+        fd = (orc.sigma(t + h) - orc.sigma(t - h)) / (2 * h)
+        assert abs(fd - orc.sigma_prime(t)) < 1e-9
+
+
+# ---- forward: closed forms -----------------------------------------------------------------
+
+def test_forward_zero_weights_gives_half_activations():
+    L, N, B = 3, 4, 2
+    w = np.zeros((L, N, N)); b = np.zeros((L, N))
+    x = np.random.default_rng(0).uniform(size=(B, N))
+    z, a = orc.forward(w, b, x)
+    assert np.array_equal(a[0], x)                    # Eq. x
+    assert np.all(z == 0.0) and np.all(a[1:] == 0.5)
+
+
+def test_forward_row_column_orientation():
+    # One non-zero weight w[j=2][k=0]: only neuron 2 sees input 0.  A transposed index
+    # would light up neuron 0 from input 2 instead.
+    N = 4
+    w = np.zeros((1, N, N)); w[0, 2, 0] = 3.0
+    b = np.zeros((1, N))
+    x = np.array([[1.0, 0.0, 5.0, 0.0]])
+    z, a = orc.forward(w, b, x)
+    assert np.array_equal(z[0, 0], np.array([0.0, 0.0, 3.0, 0.0]))
+    # bias is ADDED to the weighted input (the reading of Eq. z)
+    b[0, 1] = -2.0
+    z, _ = orc.forward(w, b, x)
+    assert np.array_equal(z[0, 0], np.array([0.0, -2.0, 3.0, 0.0]))
+
+
+def test_cost_definition():
+    a = np.zeros((2, 2, 3)); a[1] = [[1.0, 2.0, 3.0], [0.0, 0.0, 1.0]]
+    y = np.array([[0.0, 2.0, 1.0], [1.0, 0.0, 1.0]])
+    # 1/2 (1 + 0 + 4) + 1/2 (1 + 0 + 0) = 3: summed over samples, no 1/B.
+    assert orc.cost(a, y) == 3.0
+
+
+# ---- the gradient is the derivative of the cost --------------------------------------------
+
+@pytest.mark.parametrize("L,N,B,y_kind", [(1, 3, 1, "uniform"), (2, 4, 1, "onehot"),
+                                          (3, 5, 3, "uniform"), (4, 8, 1, "uniform"),
+                                          (4, 6, 3, "onehot")])
+def test_gradients_match_central_differences(L, N, B, y_kind):
+    # Catches: dropped term, wrong sign, transposed w in bp2, a^{l} used for a^{l-1} in
+    # bp4, sigma' taken at the wrong layer, a 1/B factor, missing bias.
+    w, b, x, y = _net(L, N, B, seed=100 * L + 10 * N + B, y_kind=y_kind)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    h = 1e-5
+    fd_w = np.empty_like(w)
+    for idx in np.ndindex(*w.shape):
+        wp = w.copy(); wp[idx] += h
+        wm = w.copy(); wm[idx] -= h
+        fd_w[idx] = (_cost(wp, b, x, y) - _cost(wm, b, x, y)) / (2 * h)
+    fd_b = np.empty_like(b)
+    for idx in np.ndindex(*b.shape):
+        bp = b.copy(); bp[idx] += h
+        bm = b.copy(); bm[idx] -= h
+        fd_b[idx] = (_cost(w, bp, x, y) - _cost(w, bm, x, y)) / (2 * h)
+    for l in range(L):  # per layer: deep layers have much smaller gradients
+        sw = np.max(np.abs(fd_w[l])); sb = np.max(np.abs(fd_b[l]))
+        assert np.max(np.abs(gw[l] - fd_w[l])) <= 2e-7 * sw + 1e-12
+        assert np.max(np.abs(gb[l] - fd_b[l])) <= 2e-7 * sb + 1e-12
+
+
+def test_delta_is_dC_dz_per_sample():
+    # delta^l_b = dC/dz^l_b: perturbing b^l shifts z^l of every sample, so a single-sample
+    # run's gb is that sample's delta.  The batch run must reproduce each sample's chain.
+    L, N, B = 3, 5, 4
+    w, b, x, y = _net(L, N, B, seed=7)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    gw_sum = np.zeros_like(gw)
+    for s in range(B):
+        zs, as_ = orc.forward(w, b, x[s:s + 1])
+        ds, gws, gbs = orc.backward_sequential(w, zs, as_, y[s:s + 1])
+        assert np.array_equal(zs[:, 0], z[:, s]) and np.array_equal(as_[:, 0], a[:, s])
+        assert np.array_equal(ds[:, 0], delta[:, s])
+        assert np.array_equal(gbs, ds[:, 0])          # Eq. bp3, B = 1
+        gw_sum += gws
+    assert np.allclose(gw, gw_sum, rtol=1e-14, atol=0)
+    assert np.allclose(gb, delta.sum(axis=1), rtol=1e-14, atol=0)
+
+
+# ---- structure imposed by Eq. bp3 / bp4 for a single sample --------------------------------
+
+def test_single_sample_invariants_rank_one():
+    L, N = 4, 7
+    w, b, x, y = _net(L, N, 1, seed=3)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    assert np.array_equal(gb, delta[:, 0, :])                       # Eq. bp3
+    for l in range(L):
+        g = gw[l]
+        assert np.linalg.matrix_rank(g, tol=1e-13 * np.max(np.abs(g))) == 1
+        # all 2x2 minors vanish
+        j0, k0 = np.unravel_index(np.argmax(np.abs(g)), g.shape)
+        minors = g * g[j0, k0] - np.outer(g[:, k0], g[j0, :])
+        assert np.max(np.abs(minors)) <= 1e-15 * np.max(np.abs(g)) ** 2 + 1e-300
+        # row sums: sum_k gw_jk = delta_j * sum_k a^{l-1}_k ; column sums likewise.  The
+        # row factor must be delta^l and the column factor a^{l-1} (NOT a^l).
+        assert np.allclose(g.sum(axis=1), delta[l, 0] * a[l, 0].sum(), rtol=1e-12, atol=0)
+        assert np.allclose(g.sum(axis=0), a[l, 0] * delta[l, 0].sum(), rtol=1e-12, atol=0)
+
+
+# ---- closed forms of the backward pass -----------------------------------------------------
+
+def test_single_layer_textbook_gradient():
+    # L = 1: dC/dw = ((sigma(wx+b) - y) sigma'(wx+b)) x^T, written here with numpy.
+    N = 6
+    w, b, x, y = _net(1, N, 1, seed=11)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    zz = w[0] @ x[0] + b[0]
+    s = 1.0 / (1.0 + np.exp(-zz))
+    d = (s - y[0]) * s * (1.0 - s)
+    assert np.allclose(z[0, 0], zz, rtol=1e-14)
+    assert np.allclose(delta[0, 0], d, rtol=1e-13)
+    assert np.allclose(gw[0], np.outer(d, x[0]), rtol=1e-13)
+    assert np.allclose(gb[0], d, rtol=1e-13)
+
+
+def test_zero_weights_closed_form():
+    # w = 0, b = 0: a^l = 1/2, sigma' = 1/4, delta^L = (1/2 - y)/4, delta^l = 0 below,
+    # gw^L = delta^L (a^{L-1})^T with a^{L-1} = 1/2 (or x when L = 1), gw^l = 0 below.
+    L, N = 3, 4
+    w = np.zeros((L, N, N)); b = np.zeros((L, N))
+    x = np.array([[0.1, 0.2, 0.3, 0.4]]); y = np.array([[1.0, 0.0, 0.25, 0.5]])
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    dL = (0.5 - y[0]) / 4.0
+    assert np.array_equal(delta[L - 1, 0], dL)
+    assert np.all(delta[:L - 1] == 0.0) and np.all(gw[:L - 1] == 0.0)
+    assert np.array_equal(gw[L - 1], np.outer(dL, np.full(N, 0.5)))
+
+
+def test_identity_weights_decouple_into_scalar_chains():
+    # w = I: neuron i only talks to neuron i; delta^l_i = delta^L_i prod_{m=l}^{L-1} sigma'(z^m_i).
+    L, N = 4, 5
+    r = np.random.default_rng(5)
+    w = np.stack([np.eye(N)] * L); b = r.normal(size=(L, N))
+    x = r.uniform(size=(1, N)); y = r.uniform(size=(1, N))
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    sp = a[1:, 0] * (1.0 - a[1:, 0])                                 # sigma'(z^l) via a^l
+    expect = (a[L, 0] - y[0]) * sp[L - 1]
+    assert np.allclose(delta[L - 1, 0], expect, rtol=1e-13)
+    for l in range(L - 1, 0, -1):
+        expect = expect * sp[l - 1]
+        assert np.allclose(delta[l - 1, 0], expect, rtol=1e-12)
+
+
+def test_bp2_uses_the_transpose():
+    # A single off-diagonal weight w^{2}[j=1][k=3] routes delta^2_1 to neuron 3 of layer 1
+    # (and to nobody else).  Using w instead of w^T would route delta^2_3 to neuron 1.
+    N = 4
+    w_up = np.zeros((N, N)); w_up[1, 3] = 2.0
+    d_up = np.array([[10.0, 20.0, 30.0, 40.0]])
+    z_l = np.zeros((1, N))                                           # sigma'(0) = 1/4
+    d = orc.delta_step(w_up, d_up, z_l)
+    assert np.array_equal(d[0], np.array([0.0, 0.0, 0.0, 2.0 * 20.0 * 0.25]))
+
+
+def test_scalar_network_product_chain():
+    # N = 1: everything is a scalar recurrence.
+    L = 5
+    r = np.random.default_rng(9)
+    w = r.normal(size=(L, 1, 1)); b = r.normal(size=(L, 1))
+    x = np.array([[0.7]]); y = np.array([[0.2]])
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    act = [0.7]
+    for l in range(L):
+        act.append(1.0 / (1.0 + np.exp(-(w[l, 0, 0] * act[-1] + b[l, 0]))))
+    d = (act[L] - 0.2) * act[L] * (1 - act[L])
+    for l in range(L, 0, -1):
+        assert np.isclose(delta[l - 1, 0, 0], d, rtol=1e-12)
+        assert np.isclose(gw[l - 1, 0, 0], d * act[l - 1], rtol=1e-12)
+        if l > 1:
+            d = d * w[l - 1, 0, 0] * act[l - 1] * (1 - act[l - 1])
+
+
+def test_step_functions_agree_with_full_backward():
+    L, N, B = 3, 6, 2
+    w, b, x, y = _net(L, N, B, seed=21)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    assert np.array_equal(orc.output_error(a[L], y, z[L - 1]), delta[L - 1])
+    assert np.array_equal(orc.delta_step(w[2], delta[2], z[1]), delta[1])
+    assert np.array_equal(orc.grad_b(delta[1]), gb[1])
+    assert np.array_equal(orc.grad_w(delta[1], a[1]), gw[1])
+    assert orc.grad_w_entry(delta[1], a[1], 4, 2) == gw[1, 4, 2]
+
+
+def test_float_weight_flavour_promotes_exactly():
+    L, N, B = 3, 8, 2
+    w, b, x, y = _net(L, N, B, seed=2)
+    w32 = w.astype(np.float32)
+    z64, a64 = orc.forward(w32.astype(np.float64), b, x)
+    z32, a32 = orc.forward(w32, b, x)
+    assert np.array_equal(z64, z32) and np.array_equal(a64, a32)
+    r64 = orc.backward_sequential(w32.astype(np.float64), z64, a64, y)
+    r32 = orc.backward_sequential(w32, z32, a32, y)
+    for u, v in zip(r64, r32):
+        assert np.array_equal(u, v)
+
+
+# ---- Algorithm 1: coverage, ownership, schedule invariance ---------------------------------
+
+def _simulate_algorithm1_paper_numbering(Lp, k):
+    """Integer-only walk of the printed pseudocode in the paper's own layer numbering
+    (layers 1..Lp, layer 1 = input).  Returns {paper layer: saver}, parent = -1."""
+    saver = {}
+    for i in range(Lp - 1, Lp - k, -1):          # i = L-1 ... L-k+1
+        if i >= 2:
+            saver[i] = -1
+    for t in range(k):
+        j = t
+        while j < Lp - k - 1:
+            i = 0
+            while i < k:
+                l = Lp - 1 - j - i
+                if i == k - 1:
+                    assert l not in saver
+                    saver[l] = t
+                i += 1
+            j += k
+    return saver
+
+
+def test_hand_trace_fixture_matches_pseudocode_walk():
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "algorithm1_trace_L8_k3.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    golden = {int(p): int(s) for p, s in rows}
+    sim = _simulate_algorithm1_paper_numbering(8, 3)
+    assert {p: s for p, s in golden.items() if s != -9} == sim
+    # and the oracle's literal run (library L = 7 weight layers) names the same savers
+    L, N, k = 7, 3, 3
+    w, b, x, y = _net(L, N, 1, seed=1)
+    z, a = orc.forward(w, b, x)
+    _, _, _, writer, writes, _ = orc.backward_leapfrog(w, z, a, y, k)
+    for p, s in golden.items():
+        l = p - 1
+        assert writer[l - 1] == (-1 if s == -9 else s)   # the top layer: parent (reading)
+    assert np.all(writes == 1)
+
+
+@pytest.mark.parametrize("threads", [True, False])
+def test_leapfrog_is_bitwise_the_sequential_result_for_every_k(threads):
+    L, N, B = 9, 5, 2
+    w, b, x, y = _net(L, N, B, seed=77)
+    z, a = orc.forward(w, b, x)
+    ref = orc.backward_sequential(w, z, a, y)
+    for k in range(1, L + 3):
+        delta, gw, gb, writer, writes, bp2 = orc.backward_leapfrog(w, z, a, y, k,
+                                                                   threads=threads)
+        assert np.array_equal(delta, ref[0]) and np.array_equal(gw, ref[1])
+        assert np.array_equal(gb, ref[2])
+        assert np.all(writes == 1)                                   # Theorem 1
+        ke = min(k, L)
+        for l in range(1, L + 1):
+            if l >= L - ke + 1:
+                assert writer[l - 1] == -1                           # parent's layers
+            else:
+                assert writer[l - 1] == (L - l) % ke                 # owner residue class
+
+
+def test_leapfrog_ownership_matches_pseudocode_for_many_sizes():
+    N = 2
+    for Lp in range(2, 22):
+        L = Lp - 1
+        w, b, x, y = _net(L, N, 1, seed=Lp)
+        z, a = orc.forward(w, b, x)
+        for k in range(1, Lp + 1):
+            sim = _simulate_algorithm1_paper_numbering(Lp, min(k, L))
+            _, _, _, writer, writes, _ = orc.backward_leapfrog(w, z, a, y, k, want_gw=False,
+                                                               threads=False)
+            assert np.all(writes == 1)
+            for p in range(2, Lp):                                   # below the top layer
+                assert sim[p] == writer[p - 2], (Lp, k, p)
+            assert writer[L - 1] == -1
+
+
+def test_leapfrog_recomputes_the_chain_in_every_thread():
+    # Every thread applies bp2 at every layer from its start down to its last save: the
+    # redundant work the cost model f' = f1 + f2 + f3/k leaves out.  Count it.
+    L, N, k = 12, 2, 4
+    w, b, x, y = _net(L, N, 1, seed=4)
+    z, a = orc.forward(w, b, x)
+    *_, bp2 = orc.backward_leapfrog(w, z, a, y, k, want_gw=False)
+    expect = k - 1                                                   # parent
+    for j in range(k):
+        jj = j
+        while jj < L - k:
+            expect += k
+            jj += k
+    assert bp2 == expect and bp2 > L - 1
