@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the leapfrog backward pass (arXiv 1801.04928) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--config 1..4] [--variant auto|streams|persistent|fused] [--k K]
+
+A step is one whole backward pass (Eq. bp1, the Eq. bp2 chain, Eq. bp3/bp4 of every layer
+under the leapfrog schedule) over one batch of synthetic inputs that are already resident in
+device memory.  The metric is backward layers per second (L / step time), reported with the
+achieved algorithmic HBM bandwidth of the dominant kernel against the measured copy peak.
+With N > 1 GPUs every rank runs an independent replica of the workload (the path does not
+shard: the delta chain is sequential in depth), so the aggregate is N times the per-GPU rate.
+
+One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "backward_layers_per_sec"
+UNIT = "layers/s"
+HBM_FALLBACK_GBS = 6650.0  # used only if MEASURED_PEAKS.json is absent
+VARIANT_NAMES = {"auto": 0, "streams": 1, "persistent": 2, "fused": 3}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=4000)
+    p.add_argument("--warmup", type=int, default=10)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--config", type=int, default=2)
+    p.add_argument("--variant", default="auto", choices=sorted(VARIANT_NAMES))
+    p.add_argument("--k", type=int, default=0, help="leapfrog workers (0 = the config's k)")
+    p.add_argument("--e2e-steps", type=int, default=5)
+    p.add_argument("--cpu-seconds", type=float, default=10.0)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-e2e", action="store_true")
+    return p.parse_args()
+
+
+def algorithmic_bytes(L, N, B):
+    """Bytes one backward pass must move: w^2..w^L read once, gw^1..gw^L written once, plus
+    the z/a/delta operand vectors (3 * 4NB per layer)."""
+    return 4 * N * N * (2 * L - 1) + 3 * 4 * N * B * L
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                d = json.load(f)
+            return float(d["hbm_gbs"]), "measured", d
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback", {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [c.strip() for c in r.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def time_oracle(cfg, tensors_cpu, seconds):
+    """Times the oracle's backward pass (Algorithm 1 taken literally with k threads, every
+    thread recomputing the delta chain) on the host, as it stands."""
+    import numpy as np
+    from oracle import lf_oracle as orc
+    w = tensors_cpu["w"].numpy(); b = tensors_cpu["b"].numpy()
+    x = tensors_cpu["x"].numpy(); y = tensors_cpu["y"].numpy()
+    L, N, B, k = cfg["L"], cfg["N"], cfg["B"], cfg["k"]
+    # bound the sample for the big workloads: fewer layers of the same width, same batch
+    L_s = L
+    per_layer_macs = 3.0 * N * N * B
+    while L_s > 2 and per_layer_macs * L_s * max(1, k) > 4e9 * seconds:
+        L_s //= 2
+    w_s = np.ascontiguousarray(w[:L_s]); b_s = np.ascontiguousarray(b[:L_s])
+    z, a = orc.forward(w_s, b_s, x)
+    reps, t_seq, t_lf = 0, 0.0, 0.0
+    t_end = time.perf_counter() + seconds
+    while True:
+        t0 = time.perf_counter()
+        orc.backward_sequential(w_s, z, a, y, want_gw=True)
+        t1 = time.perf_counter()
+        orc.backward_leapfrog(w_s, z, a, y, k, want_gw=True, threads=True)
+        t2 = time.perf_counter()
+        t_seq += t1 - t0; t_lf += t2 - t1; reps += 1
+        if time.perf_counter() > t_end or reps >= 50:
+            break
+    cores = os.cpu_count() or 1
+    return {
+        "value": L_s * reps / t_lf, "unit": UNIT, "cores": min(k, L_s, cores), "kind": "oracle",
+        "sample": (f"Algorithm 1 literal with k={k} pthreads, float64, L={L_s} of {L} layers, "
+                   f"N={N}, B={B}, {reps} repetitions"),
+        "sequential_value": L_s * reps / t_seq, "host_cores": cores,
+    }
+
+
+def run_reference(args):
+    """The reference arm: the float64 CPU oracle, timed as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import lf_inputs
+    cfg, cpu = lf_inputs.make_config(args.config)
+    if args.k:
+        cfg["k"] = args.k
+    per_step = max(1.0, min(15.0, 90.0 / max(1, args.steps + args.warmup)))
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(cfg, cpu, 0.01)
+    vals, t0 = [], time.perf_counter()
+    base = None
+    for _ in range(max(1, min(args.steps, 5))):
+        base = time_oracle(cfg, cpu, per_step)
+        vals.append(base["value"])
+    wall = time.perf_counter() - t0
+    v = statistics.median(vals)
+    base["value"] = v
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1000.0 * cfg["L"] / v, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(args.config, cfg), **cfg},
+            "cpu_baseline": base,
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "wall_s": wall}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_name(index, cfg):
+    return (f"configs[{index - 1}]: L={cfg['L']} N={cfg['N']} B={cfg['B']} k={cfg['k']} fp32, "
+            f"y={cfg['y']}")
+
+
+def run_ours(args):
+    import torch
+    import lf_inputs
+    import paper_1801_04928_b200 as lf
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg, cpu = lf_inputs.make_config(args.config)
+    if args.k:
+        cfg["k"] = args.k
+    L, N, B, k = cfg["L"], cfg["N"], cfg["B"], cfg["k"]
+    variant = VARIANT_NAMES[args.variant]
+
+    # Rotating buffer sets: consecutive steps touch different w / gw, so a step never finds
+    # its inputs in the 126 MB L2 left there by the step before.
+    set_bytes = 2 * 4 * L * N * N
+    n_sets = max(2, min(8, int((1 << 30) // max(set_bytes, 1))))
+    if set_bytes * n_sets > 64 << 30:
+        n_sets = 2
+    stream = torch.cuda.Stream(device=dev)
+    base = {kk: v.to(dev) for kk, v in cpu.items()}
+    sets = []
+    for i in range(n_sets):
+        t = {kk: (v if i == 0 else v.clone()) for kk, v in base.items()}
+        t["z"] = torch.empty((L, B, N), dtype=torch.float32, device=dev)
+        t["a"] = torch.empty((L + 1, B, N), dtype=torch.float32, device=dev)
+        t["delta"] = torch.empty((L, B, N), dtype=torch.float32, device=dev)
+        t["gw"] = torch.empty((L, N, N), dtype=torch.float32, device=dev)
+        t["gb"] = torch.empty((L, N), dtype=torch.float32, device=dev)
+        ctx = lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream)
+        ctx.set_option(lf.LF_OPT_VARIANT, variant)
+        t["ctx"] = ctx
+        sets.append(t)
+    torch.cuda.synchronize(dev)
+    for t in sets:
+        t["ctx"].forward(t["w"], t["b"], t["x"], t["z"], t["a"])
+        t["ctx"].sync()
+
+    def step(i):
+        t = sets[i % n_sets]
+        t["ctx"].backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        for i in range(max(3, args.warmup)):
+            step(i)
+        stream.synchronize()
+        barrier()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.25)
+        ev0 = torch.cuda.Event(enable_timing=True)
+        ev1 = torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        ev1.record(stream)
+        stream.synchronize()
+        barrier()
+        # keep the load on while the sampler collects a few more rows (short regions would
+        # otherwise be missed entirely); these extra steps are not timed
+        if rank == 0:
+            t_end = time.perf_counter() + 0.6
+            i = 0
+            while time.perf_counter() < t_end:
+                step(i); i += 1
+                if i % 64 == 0:
+                    stream.synchronize()
+            stream.synchronize()
+        clocks = sampler.stop() if rank == 0 else None
+    total_ms = ev0.elapsed_time(ev1)
+    for t in sets:
+        t["ctx"].sync()
+    stats = sets[0]["ctx"].stats()
+
+    tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    total_ms_max = float(tmax.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * L * args.steps / (total_ms_max * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    e2e = None
+    if not args.no_e2e:
+        t = sets[0]
+        host = {n: torch.empty_like(t[n], device="cpu").pin_memory() for n in
+                ("w", "z", "a", "y", "delta", "gw", "gb")}
+        for n in ("w", "z", "a", "y"):
+            host[n].copy_(t[n])
+        h2d = sum(host[n].numel() * 4 for n in ("w", "z", "a", "y"))
+        d2h = sum(host[n].numel() * 4 for n in ("delta", "gw", "gb"))
+        ctx = t["ctx"]
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                ctx.backward_host(*(host[n] for n in ("w", "z", "a", "y", "delta", "gw", "gb")))
+            ctx.sync()
+            barrier()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.e2e_steps):
+                ctx.backward_host(*(host[n] for n in ("w", "z", "a", "y", "delta", "gw", "gb")))
+            e1.record(stream)
+            ctx.sync()
+            barrier()
+        e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * L * args.e2e_steps / (float(e2e_ms.item()) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": float(e2e_ms.item()) / args.e2e_steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peak, peak_kind, peaks = measured_peaks()
+    alg = algorithmic_bytes(L, N, B)
+    launches_per_step = stats["launches_backward"]
+    if launches_per_step == 1:
+        kernel_name = "persistent backward kernel (one launch per step)"
+    else:
+        kernel_name = f"whole step ({launches_per_step} launches replayed from one CUDA graph)"
+    achieved = alg / (ms_per_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "kernel": kernel_name, "algorithmic_bytes_per_launch": alg,
+                "avg_launch_ms": ms_per_step,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        cpu_baseline = time_oracle(cfg, cpu, args.cpu_seconds)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(args.config, cfg), "L": L, "N": N, "B": B, "k": k,
+                   "variant": stats["variant"], "gw_math": stats["gw_math"],
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2_policy": f"{n_sets} rotating buffer sets of {set_bytes >> 20} MiB (w + gw); "
+                                "inputs larger than the 126 MB L2"},
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,164 @@
+/*
+ * leapfrog.h -- C ABI of the sm_100a library for one pass of an L-layer, N-wide sigmoid
+ * multi-layer perceptron with the weight-gradient work interleaved over k workers
+ * ("leapfrogging", arXiv 1801.04928).
+ *
+ * Indexing.  The library counts L WEIGHT layers l = 1..L with a^0 = x.  The paper numbers
+ * the input as its layer 1, so paper layer p is l = p - 1 here.  C arrays are zero-based:
+ * slab l-1 of an array holds the quantity of layer l.
+ *
+ * Layouts.  All tensors are float32, contiguous, 16-byte aligned and live in DEVICE memory
+ * owned by the caller (except for the *_host entry point, which says so).  With B samples:
+ *     w     [L][N][N]   w[l-1][j][k] = weight from neuron k of layer l-1 to neuron j of layer l
+ *     b     [L][N]
+ *     x, y  [B][N]      sample-major; B = 1 is the paper's vector form
+ *     z     [L][B][N]
+ *     a     [L+1][B][N] a[0] = x
+ *     delta [L][B][N]
+ *     gw    [L][N][N]   same indexing as w
+ *     gb    [L][N]
+ * N must be a multiple of 4 (128-bit accesses); other sizes are rejected with LF_EINVAL.
+ *
+ * Execution.  Calls enqueue work on the context's stream and return; lf_sync() waits for it
+ * and reports device-side status.  The library never allocates or frees tensors; a context
+ * owns only its workspace (flags, reduction scratch, helper streams and events).  Nothing
+ * here throws or aborts; every entry point returns LF_OK (0) or a negative code.  There is
+ * no CPU fallback: without a CUDA device every compute entry point fails with LF_ECUDA.
+ * A context is not thread-safe; use one per host thread.
+ */
+#ifndef LEAPFROG_H
+#define LEAPFROG_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lf_ctx lf_ctx;
+
+enum lf_status {
+    LF_OK = 0,
+    LF_EINVAL = -1,    /* L, N, B or k < 1, N not a multiple of 4, unknown option or value  */
+    LF_ENULL = -2,     /* a required pointer is NULL                                         */
+    LF_EALIGN = -3,    /* a tensor pointer is not 16-byte aligned                            */
+    LF_ERESOURCE = -4, /* the device cannot hold the requested configuration co-resident     */
+    LF_ECUDA = -5,     /* a CUDA call failed; lf_last_cuda_error() gives the cudaError_t     */
+    LF_ETIMEOUT = -6,  /* a bounded device-side wait ran out; outputs are undefined          */
+    LF_ENOMEM = -7     /* workspace allocation failed                                        */
+};
+
+/* How lf_backward schedules Eq. bp4 (the weight gradients) against the delta chain. */
+enum lf_variant {
+    LF_VARIANT_AUTO = 0,       /* pick from the built-in per-(N,B) table of measurements      */
+    LF_VARIANT_STREAMS = 1,    /* one launch per layer; the k leapfrog workers are k streams  */
+    LF_VARIANT_PERSISTENT = 2, /* one persistent launch; the k workers are k CTA groups       */
+    LF_VARIANT_FUSED = 3       /* one persistent launch; the pass that reads a tile of
+                                  w^{l+1} for Eq. bp2 also stores the same tile of gw^{l+1}   */
+};
+
+/* Arithmetic of the B > 1 weight-gradient contraction. */
+enum lf_gw_math {
+    LF_GW_MATH_AUTO = 0, /* TF32 tensor cores when B > 1 and the shape is supported          */
+    LF_GW_MATH_FP32 = 1, /* fp32 FMA on the CUDA cores                                        */
+    LF_GW_MATH_TF32 = 2  /* inputs rounded to TF32, fp32 accumulation in tensor memory        */
+};
+
+enum lf_option {
+    LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
+    LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
+    LF_OPT_WAIT_BUDGET_US = 3,/* upper bound of any device-side wait, microseconds (>= 1)     */
+    LF_OPT_USE_GRAPH = 4      /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
+};
+
+typedef struct lf_stats {
+    int L, N, B, k;           /* sizes the context was created with                           */
+    int k_effective;          /* min(k, L)                                                    */
+    int variant;              /* variant the last lf_backward used (enum lf_variant)          */
+    int gw_math;              /* arithmetic the last lf_backward used for Eq. bp4             */
+    int sm_count;             /* multiprocessors of the device                                */
+    int chain_ctas;           /* persistent variants: CTAs on the delta chain                 */
+    int worker_ctas;          /* persistent variants: CTAs per leapfrog worker group          */
+    int launches_forward;     /* kernels launched by the last lf_forward                      */
+    int launches_backward;    /* kernels launched by the last lf_backward                     */
+    unsigned int device_status; /* status word read by the last lf_sync (0 = clean)           */
+    long long workspace_bytes;  /* device memory owned by the context                         */
+} lf_stats;
+
+/*
+ * Create a context for networks of L weight layers, width N, B samples and k leapfrog
+ * workers (Section 3: "k threads"; here CTA groups or streams).  k > L is legal and acts as
+ * k = L.  Binds to the current CUDA device and allocates the workspace there.
+ * *out receives the context; on failure *out is NULL.
+ * Errors: LF_ENULL (out), LF_EINVAL (sizes), LF_ECUDA (no device / CUDA failure), LF_ENOMEM.
+ */
+int lf_create(lf_ctx** out, int L, int N, int B, int k);
+
+/*
+ * Use `cuda_stream` (a cudaStream_t, borrowed, must outlive the work enqueued on it) for
+ * all subsequent calls.  NULL selects the legacy default stream (the initial setting).
+ */
+int lf_set_stream(lf_ctx* ctx, void* cuda_stream);
+
+/* Set an option (enum lf_option).  LF_EINVAL for unknown keys or out-of-range values. */
+int lf_set_option(lf_ctx* ctx, int key, long long value);
+
+/*
+ * Forward pass, Section 2 Eq. x, z, a:  a^0 = x;  z^l = w^l a^{l-1} + b^l;  a^l = sigma(z^l),
+ * sigma(t) = 1 / (1 + e^{-t}).  (The printed Eq. z shows no bias; b^l is added, as Eq. bp3
+ * presupposes.)  Reads w, b, x; writes all L slabs of z and all L+1 slabs of a (a[0] := x).
+ */
+int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, float* z,
+               float* a);
+
+/*
+ * Backward pass under the quadratic cost C = 1/2 sum_b ||a^L_b - y_b||^2:
+ *   Eq. bp1  delta^L = (a^L - y) (.) sigma'(z^L)
+ *   Eq. bp2  delta^l = ((w^{l+1})^T delta^{l+1}) (.) sigma'(z^l),  l = L-1 .. 1
+ *   Eq. bp3  gb^l = sum_b delta^l_b
+ *   Eq. bp4  gw^l = sum_b delta^l_b (a^{l-1}_b)^T
+ * with Eq. bp3/bp4 of layer l done by leapfrog worker (L - l) mod k (Section 3, Algorithm 1;
+ * the delta chain itself is computed once, not once per worker).  The top layer L, which
+ * Algorithm 1 leaves out, is included.  z and a must be what lf_forward produced for the
+ * same w (sigma' may be taken from a as a (1 - a)).  Reads w (layers 2..L), z, a, y; writes
+ * every element of delta, gw and gb.  For B > 1 with TF32 math the inputs of Eq. bp4 are
+ * rounded to TF32 and accumulated in fp32; everything else is fp32.
+ */
+int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                float* delta, float* gw, float* gb);
+
+/*
+ * The same backward pass on HOST buffers (pageable or pinned; same layouts): copies w, z, a,
+ * y to device staging owned by the context (allocated on first use, counted in
+ * workspace_bytes), runs lf_backward, copies delta, gw, gb back, all on the context's
+ * stream.  The host buffers must stay valid until lf_sync() returns.
+ */
+int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a,
+                     const float* y, float* delta, float* gw, float* gb);
+
+/*
+ * Wait for everything enqueued on the context's stream and read the device status word.
+ * Returns LF_ETIMEOUT if a bounded device-side wait expired, LF_ECUDA on a CUDA error.
+ */
+int lf_sync(lf_ctx* ctx);
+
+/* Worker that performs Eq. bp3/bp4 of layer l (1-based): (L - l) mod min(k, L); -1 if out of range. */
+int lf_owner(const lf_ctx* ctx, int l);
+
+/* Copy the context's counters into *out. */
+int lf_get_stats(lf_ctx* ctx, lf_stats* out);
+
+/* cudaError_t of the last failed CUDA call of this context (0 if none). */
+int lf_last_cuda_error(const lf_ctx* ctx);
+
+/* Static English text for a status code. */
+const char* lf_strerror(int status);
+
+/* Library version, major * 100 + minor. */
+int lf_version(void);
+
+/* Synchronise the stream, free the workspace and the context.  NULL is LF_ENULL. */
+int lf_destroy(lf_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LEAPFROG_H */

@@ -1,0 +1,205 @@
+"""ctypes binding of ``libleapfrog.so``: argument marshalling only.
+
+Every function has the name and meaning of the C entry point declared in
+``include/leapfrog.h``; tensors are passed as raw device (or, for ``lf_backward_host``, host)
+addresses.  There is no fallback of any kind: if the shared library has not been built the
+import fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libleapfrog.so")
+
+LF_OK, LF_EINVAL, LF_ENULL, LF_EALIGN, LF_ERESOURCE, LF_ECUDA, LF_ETIMEOUT, LF_ENOMEM = (
+    0, -1, -2, -3, -4, -5, -6, -7)
+LF_VARIANT_AUTO, LF_VARIANT_STREAMS, LF_VARIANT_PERSISTENT, LF_VARIANT_FUSED = 0, 1, 2, 3
+LF_GW_MATH_AUTO, LF_GW_MATH_FP32, LF_GW_MATH_TF32 = 0, 1, 2
+LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH = 1, 2, 3, 4
+
+EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
+           "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
+           "lf_strerror", "lf_version", "lf_destroy")
+
+
+class lf_stats(ctypes.Structure):
+    _fields_ = [("L", ctypes.c_int), ("N", ctypes.c_int), ("B", ctypes.c_int),
+                ("k", ctypes.c_int), ("k_effective", ctypes.c_int), ("variant", ctypes.c_int),
+                ("gw_math", ctypes.c_int), ("sm_count", ctypes.c_int),
+                ("chain_ctas", ctypes.c_int), ("worker_ctas", ctypes.c_int),
+                ("launches_forward", ctypes.c_int), ("launches_backward", ctypes.c_int),
+                ("device_status", ctypes.c_uint), ("workspace_bytes", ctypes.c_longlong)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_1801_04928_b200.build` "
+            "(needs nvcc). There is no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, ll = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong
+    lib.lf_create.argtypes = [ctypes.POINTER(vp), i, i, i, i]
+    lib.lf_set_stream.argtypes = [vp, vp]
+    lib.lf_set_option.argtypes = [vp, i, ll]
+    lib.lf_forward.argtypes = [vp] * 6
+    lib.lf_backward.argtypes = [vp] * 8
+    lib.lf_backward_host.argtypes = [vp] * 8
+    lib.lf_sync.argtypes = [vp]
+    lib.lf_owner.argtypes = [vp, i]
+    lib.lf_get_stats.argtypes = [vp, ctypes.POINTER(lf_stats)]
+    lib.lf_last_cuda_error.argtypes = [vp]
+    lib.lf_strerror.argtypes = [i]
+    lib.lf_strerror.restype = ctypes.c_char_p
+    lib.lf_version.argtypes = []
+    lib.lf_destroy.argtypes = [vp]
+    for name in EXPORTS:
+        if name != "lf_strerror":
+            getattr(lib, name).restype = i
+    return lib
+
+
+_lib = _load()
+
+
+class LeapfrogError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        msg = f"{where}: {lf_strerror(status)} (status {status}"
+        msg += f", cudaError {cuda_error})" if cuda_error else ")"
+        super().__init__(msg)
+
+
+def _ptr(t) -> ctypes.c_void_p:
+    """Address of a tensor-like object (``data_ptr()``), an int, or None."""
+    if t is None:
+        return ctypes.c_void_p(None)
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+# ---- the C entry points, one to one -----------------------------------------------------------
+
+def lf_version() -> int:
+    return _lib.lf_version()
+
+
+def lf_strerror(status: int) -> str:
+    return _lib.lf_strerror(int(status)).decode()
+
+
+def lf_create(L: int, N: int, B: int, k: int):
+    """Returns (status, handle)."""
+    h = ctypes.c_void_p(None)
+    rc = _lib.lf_create(ctypes.byref(h), int(L), int(N), int(B), int(k))
+    return rc, h
+
+
+def lf_set_stream(ctx, cuda_stream: int | None) -> int:
+    return _lib.lf_set_stream(ctx, ctypes.c_void_p(cuda_stream or None))
+
+
+def lf_set_option(ctx, key: int, value: int) -> int:
+    return _lib.lf_set_option(ctx, int(key), int(value))
+
+
+def lf_forward(ctx, w, b, x, z, a) -> int:
+    return _lib.lf_forward(ctx, _ptr(w), _ptr(b), _ptr(x), _ptr(z), _ptr(a))
+
+
+def lf_backward(ctx, w, z, a, y, delta, gw, gb) -> int:
+    return _lib.lf_backward(ctx, _ptr(w), _ptr(z), _ptr(a), _ptr(y), _ptr(delta), _ptr(gw),
+                            _ptr(gb))
+
+
+def lf_backward_host(ctx, w, z, a, y, delta, gw, gb) -> int:
+    return _lib.lf_backward_host(ctx, _ptr(w), _ptr(z), _ptr(a), _ptr(y), _ptr(delta),
+                                 _ptr(gw), _ptr(gb))
+
+
+def lf_sync(ctx) -> int:
+    return _lib.lf_sync(ctx)
+
+
+def lf_owner(ctx, l: int) -> int:
+    return _lib.lf_owner(ctx, int(l))
+
+
+def lf_get_stats(ctx):
+    """Returns (status, dict)."""
+    st = lf_stats()
+    rc = _lib.lf_get_stats(ctx, ctypes.byref(st))
+    return rc, {f: getattr(st, f) for f, _ in lf_stats._fields_}
+
+
+def lf_last_cuda_error(ctx) -> int:
+    return _lib.lf_last_cuda_error(ctx)
+
+
+def lf_destroy(ctx) -> int:
+    return _lib.lf_destroy(ctx)
+
+
+# ---- a small convenience wrapper (still marshalling only) -------------------------------------
+
+class Leapfrog:
+    """Owns one ``lf_ctx``; raises :class:`LeapfrogError` on any non-zero status."""
+
+    def __init__(self, L: int, N: int, B: int = 1, k: int = 1, stream: int | None = None):
+        rc, self._h = lf_create(L, N, B, k)
+        if rc != LF_OK:
+            self._h = None
+            raise LeapfrogError(rc, "lf_create")
+        self.L, self.N, self.B, self.k = L, N, B, k
+        if stream is not None:
+            self.set_stream(stream)
+
+    def _check(self, rc: int, where: str):
+        if rc != LF_OK:
+            raise LeapfrogError(rc, where, lf_last_cuda_error(self._h))
+
+    def set_stream(self, cuda_stream: int | None):
+        self._check(lf_set_stream(self._h, cuda_stream), "lf_set_stream")
+
+    def set_option(self, key: int, value: int):
+        self._check(lf_set_option(self._h, key, value), "lf_set_option")
+
+    def forward(self, w, b, x, z, a):
+        self._check(lf_forward(self._h, w, b, x, z, a), "lf_forward")
+
+    def backward(self, w, z, a, y, delta, gw, gb):
+        self._check(lf_backward(self._h, w, z, a, y, delta, gw, gb), "lf_backward")
+
+    def backward_host(self, w, z, a, y, delta, gw, gb):
+        self._check(lf_backward_host(self._h, w, z, a, y, delta, gw, gb), "lf_backward_host")
+
+    def sync(self):
+        self._check(lf_sync(self._h), "lf_sync")
+
+    def owner(self, l: int) -> int:
+        return lf_owner(self._h, l)
+
+    def stats(self) -> dict:
+        rc, d = lf_get_stats(self._h)
+        self._check(rc, "lf_get_stats")
+        return d
+
+    def close(self):
+        if self._h is not None:
+            lf_destroy(self._h)
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,430 @@
+// C ABI of libleapfrog: context, validation, scheduling of the per-layer kernels.
+#include <new>
+#include <string.h>
+
+#include "lf_internal.h"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_ptrs(const void* const* ps, int n)
+{
+    for (int i = 0; i < n; ++i)
+        if (!ps[i]) return LF_ENULL;
+    for (int i = 0; i < n; ++i)
+        if (!aligned16(ps[i])) return LF_EALIGN;
+    return LF_OK;
+}
+
+inline size_t slab(const lf_ctx* c) { return (size_t)c->B * (size_t)c->N; }
+inline size_t mat(const lf_ctx* c) { return (size_t)c->N * (size_t)c->N; }
+
+int resolve_variant(const lf_ctx* c)
+{
+    if (c->opt_variant != LF_VARIANT_AUTO) return c->opt_variant;
+    return lf_auto_variant(c);
+}
+
+int resolve_gw_math(const lf_ctx* c)
+{
+    if (c->B == 1) return LF_GW_MATH_FP32;  // rank-1: one multiply per element, nothing to contract
+    if (c->opt_gw_math == LF_GW_MATH_FP32) return LF_GW_MATH_FP32;
+    return lf_tf32_supported(c) ? LF_GW_MATH_TF32 : LF_GW_MATH_FP32;
+}
+
+// Eq. bp4 (and, for a mini-batch, Eq. bp3) of layer l on stream s.
+int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, float* gw, float* gb,
+                      int gw_math, cudaStream_t s, int* launches)
+{
+    const float* d_l = delta + (size_t)(l - 1) * slab(c);
+    const float* a_prev = a + (size_t)(l - 1) * slab(c);
+    float* gw_l = gw + (size_t)(l - 1) * mat(c);
+    if (c->B == 1) {
+        LF_CUDA_TRY(c, lfk_gw_rank1(d_l, a_prev, gw_l, c->N, s));
+        *launches += 1;
+    } else {
+        if (gw_math == LF_GW_MATH_TF32) {
+            int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, s, launches);
+            if (rc != LF_OK) return rc;
+        } else {
+            LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, c->N, c->B, s));
+            *launches += 1;
+        }
+        LF_CUDA_TRY(c, lfk_grad_b_colsum(d_l, gb + (size_t)(l - 1) * c->N, c->N, c->B, s));
+        *launches += 1;
+    }
+    return LF_OK;
+}
+
+// One delta-chain step on stream s: Eq. bp1 for l = L, Eq. bp2 below.
+int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const float* y,
+                       float* delta, float* gb, cudaStream_t s, int* launches)
+{
+    const int L = c->L, N = c->N, B = c->B;
+    float* d_l = delta + (size_t)(l - 1) * slab(c);
+    const float* a_l = a + (size_t)l * slab(c);
+    float* gb_l = gb + (size_t)(l - 1) * N;
+    if (l == L) {
+        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, s));
+    } else {
+        const float* w_up = w + (size_t)l * mat(c);  // w^{l+1}
+        const float* d_up = delta + (size_t)l * slab(c);
+        if (B == 1)
+            LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, N, s));
+        else
+            LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, N, B, s));
+    }
+    *launches += 1;
+    return LF_OK;
+}
+
+// The leapfrog schedule with streams: the chain runs on the context's stream and signals
+// ready[l]; worker (L - l) mod k waits for it on its own stream and does Eq. bp3/bp4 there.
+int enqueue_backward_streams(lf_ctx* c, const float* w, const float* a, const float* y,
+                             float* delta, float* gw, float* gb, int gw_math, int* launches)
+{
+    cudaStream_t s = c->stream;
+    LF_CUDA_TRY(c, cudaEventRecord(c->fork_ev, s));
+    for (int j = 0; j < c->keff; ++j)
+        LF_CUDA_TRY(c, cudaStreamWaitEvent(c->wstreams[j], c->fork_ev, 0));
+    for (int l = c->L; l >= 1; --l) {
+        int rc = enqueue_chain_step(c, l, w, a, y, delta, gb, s, launches);
+        if (rc != LF_OK) return rc;
+        LF_CUDA_TRY(c, cudaEventRecord(c->ready_ev[l - 1], s));
+        int j = (c->L - l) % c->keff;
+        LF_CUDA_TRY(c, cudaStreamWaitEvent(c->wstreams[j], c->ready_ev[l - 1], 0));
+        rc = enqueue_gradients(c, l, a, delta, gw, gb, gw_math, c->wstreams[j], launches);
+        if (rc != LF_OK) return rc;
+    }
+    for (int j = 0; j < c->keff; ++j) {
+        LF_CUDA_TRY(c, cudaEventRecord(c->done_ev[j], c->wstreams[j]));
+        LF_CUDA_TRY(c, cudaStreamWaitEvent(s, c->done_ev[j], 0));
+    }
+    return LF_OK;
+}
+
+void drop_graph(lf_ctx* c)
+{
+    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    c->graph_exec = nullptr;
+    c->graph_valid = false;
+}
+
+int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, const float* y,
+                     float* delta, float* gw, float* gb, int gw_math)
+{
+    int launches = 0;
+    const bool graph_ok = c->use_graph && c->stream != nullptr &&
+                          c->stream != cudaStreamLegacy && c->stream != cudaStreamPerThread;
+    if (!graph_ok) {
+        int rc = enqueue_backward_streams(c, w, a, y, delta, gw, gb, gw_math, &launches);
+        c->stats.launches_backward = launches;
+        return rc;
+    }
+    lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math};
+    if (!(c->graph_valid && c->graph_key == key)) {
+        drop_graph(c);
+        LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+        int rc = enqueue_backward_streams(c, w, a, y, delta, gw, gb, gw_math, &launches);
+        cudaGraph_t g = nullptr;
+        cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+        if (rc != LF_OK) {
+            if (g) cudaGraphDestroy(g);
+            return rc;
+        }
+        if (e != cudaSuccess) {
+            c->last_cuda_error = (int)e;
+            return LF_ECUDA;
+        }
+        e = cudaGraphInstantiate(&c->graph_exec, g, 0);
+        cudaGraphDestroy(g);
+        if (e != cudaSuccess) {
+            c->last_cuda_error = (int)e;
+            c->graph_exec = nullptr;
+            return LF_ECUDA;
+        }
+        c->graph_key = key;
+        c->graph_valid = true;
+        c->graph_launches = launches;
+    }
+    LF_CUDA_TRY(c, cudaGraphLaunch(c->graph_exec, c->stream));
+    c->stats.launches_backward = c->graph_launches;
+    return LF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lf_version(void) { return 100; }
+
+const char* lf_strerror(int status)
+{
+    switch (status) {
+        case LF_OK: return "ok";
+        case LF_EINVAL: return "invalid argument (sizes must be >= 1, N a multiple of 4, option in range)";
+        case LF_ENULL: return "required pointer is NULL";
+        case LF_EALIGN: return "tensor pointer is not 16-byte aligned";
+        case LF_ERESOURCE: return "configuration cannot be made co-resident on this device";
+        case LF_ECUDA: return "CUDA call failed (see lf_last_cuda_error)";
+        case LF_ETIMEOUT: return "a bounded device-side wait expired; outputs are undefined";
+        case LF_ENOMEM: return "workspace allocation failed";
+        default: return "unknown status";
+    }
+}
+
+int lf_create(lf_ctx** out, int L, int N, int B, int k)
+{
+    if (!out) return LF_ENULL;
+    *out = nullptr;
+    if (L < 1 || N < 1 || B < 1 || k < 1 || (N & 3) != 0) return LF_EINVAL;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LF_ECUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return LF_ECUDA;
+
+    lf_ctx* c = new (std::nothrow) lf_ctx;
+    if (!c) return LF_ENOMEM;
+    memset(c, 0, sizeof(*c));
+    c->L = L; c->N = N; c->B = B; c->k = k; c->keff = k < L ? k : L;
+    c->device = dev;
+    c->sm_count = prop.multiProcessorCount;
+    c->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    c->stream = nullptr;
+    c->opt_variant = LF_VARIANT_AUTO;
+    c->opt_gw_math = LF_GW_MATH_AUTO;
+    c->wait_budget_us = 2000000;
+    c->use_graph = 1;
+
+    bool ok = true;
+    size_t ws = 0;
+    const int chunks = lfk_delta_row_chunks(N);
+    size_t partial_bytes = (size_t)chunks * N * sizeof(float);
+    size_t counter_bytes = (size_t)(N / 128 + 1) * sizeof(unsigned);
+    c->sync_words_count = lf_sync_words_needed(c);
+    ok = ok && cudaMalloc(&c->partial, partial_bytes) == cudaSuccess; ws += partial_bytes;
+    ok = ok && cudaMalloc(&c->counters, counter_bytes) == cudaSuccess; ws += counter_bytes;
+    ok = ok && cudaMalloc(&c->sync_words, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
+    ws += c->sync_words_count * sizeof(unsigned);
+    ok = ok && cudaMalloc(&c->status_dev, sizeof(unsigned)) == cudaSuccess; ws += sizeof(unsigned);
+    ok = ok && cudaMallocHost(&c->status_host, sizeof(unsigned)) == cudaSuccess;
+    if (ok) {
+        ok = ok && cudaMemset(c->counters, 0, counter_bytes) == cudaSuccess;
+        ok = ok && cudaMemset(c->sync_words, 0, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
+        ok = ok && cudaMemset(c->status_dev, 0, sizeof(unsigned)) == cudaSuccess;
+        *c->status_host = 0;
+    }
+    c->wstreams = new (std::nothrow) cudaStream_t[c->keff]();
+    c->ready_ev = new (std::nothrow) cudaEvent_t[L]();
+    c->done_ev = new (std::nothrow) cudaEvent_t[c->keff]();
+    ok = ok && c->wstreams && c->ready_ev && c->done_ev;
+    if (ok) {
+        for (int j = 0; j < c->keff && ok; ++j) {
+            ok = cudaStreamCreateWithFlags(&c->wstreams[j], cudaStreamNonBlocking) == cudaSuccess;
+            ok = ok && cudaEventCreateWithFlags(&c->done_ev[j], cudaEventDisableTiming) == cudaSuccess;
+        }
+        for (int l = 0; l < L && ok; ++l)
+            ok = cudaEventCreateWithFlags(&c->ready_ev[l], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaError_t e = cudaGetLastError();
+        bool oom = (e == cudaErrorMemoryAllocation);
+        lf_destroy(c);
+        return oom ? LF_ENOMEM : LF_ECUDA;
+    }
+    c->stats.L = L; c->stats.N = N; c->stats.B = B; c->stats.k = k;
+    c->stats.k_effective = c->keff;
+    c->stats.sm_count = c->sm_count;
+    c->stats.workspace_bytes = (long long)ws;
+    *out = c;
+    return LF_OK;
+}
+
+int lf_set_stream(lf_ctx* ctx, void* cuda_stream)
+{
+    if (!ctx) return LF_ENULL;
+    if (ctx->stream != (cudaStream_t)cuda_stream) drop_graph(ctx);
+    ctx->stream = (cudaStream_t)cuda_stream;
+    return LF_OK;
+}
+
+int lf_set_option(lf_ctx* ctx, int key, long long value)
+{
+    if (!ctx) return LF_ENULL;
+    switch (key) {
+        case LF_OPT_VARIANT:
+            if (value < LF_VARIANT_AUTO || value > LF_VARIANT_FUSED) return LF_EINVAL;
+            ctx->opt_variant = (int)value;
+            return LF_OK;
+        case LF_OPT_GW_MATH:
+            if (value < LF_GW_MATH_AUTO || value > LF_GW_MATH_TF32) return LF_EINVAL;
+            ctx->opt_gw_math = (int)value;
+            return LF_OK;
+        case LF_OPT_WAIT_BUDGET_US:
+            if (value < 1 || value > 60000000LL) return LF_EINVAL;
+            ctx->wait_budget_us = value;
+            return LF_OK;
+        case LF_OPT_USE_GRAPH:
+            if (value != 0 && value != 1) return LF_EINVAL;
+            ctx->use_graph = (int)value;
+            if (!value) drop_graph(ctx);
+            return LF_OK;
+        default:
+            return LF_EINVAL;
+    }
+}
+
+int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, float* z, float* a)
+{
+    if (!ctx) return LF_ENULL;
+    const void* ps[] = {w, b, x, z, a};
+    int rc = check_ptrs(ps, 5);
+    if (rc != LF_OK) return rc;
+    const int L = ctx->L, N = ctx->N, B = ctx->B;
+    cudaStream_t s = ctx->stream;
+    int launches = 0;
+    if (a != x) LF_CUDA_TRY(ctx, lfk_copy_input(x, a, slab(ctx), s));  // Eq. x
+    for (int l = 1; l <= L; ++l) {
+        const float* w_l = w + (size_t)(l - 1) * mat(ctx);
+        const float* b_l = b + (size_t)(l - 1) * N;
+        const float* a_prev = a + (size_t)(l - 1) * slab(ctx);
+        float* z_l = z + (size_t)(l - 1) * slab(ctx);
+        float* a_l = a + (size_t)l * slab(ctx);
+        if (B == 1)
+            LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, N, s));
+        else
+            LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, N, B, s));
+        ++launches;
+    }
+    ctx->stats.launches_forward = launches;
+    return LF_OK;
+}
+
+int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                float* delta, float* gw, float* gb)
+{
+    if (!ctx) return LF_ENULL;
+    const void* ps[] = {w, z, a, y, delta, gw, gb};
+    int rc = check_ptrs(ps, 7);
+    if (rc != LF_OK) return rc;
+    int variant = resolve_variant(ctx);
+    const int gw_math = resolve_gw_math(ctx);
+    if (variant != LF_VARIANT_STREAMS && !lf_persistent_supported(ctx, variant))
+        variant = LF_VARIANT_STREAMS;
+    ctx->stats.variant = variant;
+    ctx->stats.gw_math = gw_math;
+    if (variant == LF_VARIANT_STREAMS)
+        return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
+    return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
+}
+
+int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                     float* delta, float* gw, float* gb)
+{
+    if (!ctx) return LF_ENULL;
+    const void* ps[] = {w, z, a, y, delta, gw, gb};
+    for (int i = 0; i < 7; ++i)
+        if (!ps[i]) return LF_ENULL;
+    const size_t L = (size_t)ctx->L, S = slab(ctx), M = mat(ctx), N = (size_t)ctx->N;
+    // staging layout, every block a multiple of 4 floats: w | z | a | y | delta | gw | gb
+    const size_t n_w = L * M, n_z = L * S, n_a = (L + 1) * S, n_y = S, n_d = L * S, n_gw = L * M,
+                 n_gb = L * N;
+    const size_t total = n_w + n_z + n_a + n_y + n_d + n_gw + n_gb;
+    if (!ctx->stage) {
+        cudaError_t e = cudaMalloc(&ctx->stage, total * sizeof(float));
+        if (e != cudaSuccess) {
+            ctx->stage = nullptr;
+            ctx->last_cuda_error = (int)e;
+            cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? LF_ENOMEM : LF_ECUDA;
+        }
+        ctx->stage_bytes = total * sizeof(float);
+        ctx->stats.workspace_bytes += (long long)ctx->stage_bytes;
+    }
+    float* d_w = ctx->stage;
+    float* d_z = d_w + n_w;
+    float* d_a = d_z + n_z;
+    float* d_y = d_a + n_a;
+    float* d_d = d_y + n_y;
+    float* d_gw = d_d + n_d;
+    float* d_gb = d_gw + n_gw;
+    cudaStream_t s = ctx->stream;
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w, w, n_w * sizeof(float), cudaMemcpyHostToDevice, s));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_z, z, n_z * sizeof(float), cudaMemcpyHostToDevice, s));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, s));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, s));
+    int rc = lf_backward(ctx, d_w, d_z, d_a, d_y, d_d, d_gw, d_gb);
+    if (rc != LF_OK) return rc;
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(delta, d_d, n_d * sizeof(float), cudaMemcpyDeviceToHost, s));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw, d_gw, n_gw * sizeof(float), cudaMemcpyDeviceToHost, s));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, s));
+    return LF_OK;
+}
+
+int lf_sync(lf_ctx* ctx)
+{
+    if (!ctx) return LF_ENULL;
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(unsigned),
+                                     cudaMemcpyDeviceToHost, ctx->stream));
+    LF_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    unsigned st = *ctx->status_host;
+    ctx->stats.device_status = st;
+    if (st != 0) {
+        cudaMemsetAsync(ctx->status_dev, 0, sizeof(unsigned), ctx->stream);  // next call starts clean
+        if (st & (LF_DEV_TIMEOUT_FLAG | LF_DEV_TIMEOUT_BARRIER)) return LF_ETIMEOUT;
+        return LF_EINVAL;
+    }
+    return LF_OK;
+}
+
+int lf_owner(const lf_ctx* ctx, int l)
+{
+    if (!ctx || l < 1 || l > ctx->L) return -1;
+    return (ctx->L - l) % ctx->keff;
+}
+
+int lf_get_stats(lf_ctx* ctx, lf_stats* out)
+{
+    if (!ctx || !out) return LF_ENULL;
+    *out = ctx->stats;
+    return LF_OK;
+}
+
+int lf_last_cuda_error(const lf_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int lf_destroy(lf_ctx* ctx)
+{
+    if (!ctx) return LF_ENULL;
+    cudaStreamSynchronize(ctx->stream);
+    drop_graph(ctx);
+    if (ctx->wstreams) {
+        for (int j = 0; j < ctx->keff; ++j)
+            if (ctx->wstreams[j]) { cudaStreamSynchronize(ctx->wstreams[j]); cudaStreamDestroy(ctx->wstreams[j]); }
+        delete[] ctx->wstreams;
+    }
+    if (ctx->done_ev) {
+        for (int j = 0; j < ctx->keff; ++j)
+            if (ctx->done_ev[j]) cudaEventDestroy(ctx->done_ev[j]);
+        delete[] ctx->done_ev;
+    }
+    if (ctx->ready_ev) {
+        for (int l = 0; l < ctx->L; ++l)
+            if (ctx->ready_ev[l]) cudaEventDestroy(ctx->ready_ev[l]);
+        delete[] ctx->ready_ev;
+    }
+    if (ctx->fork_ev) cudaEventDestroy(ctx->fork_ev);
+    if (ctx->partial) cudaFree(ctx->partial);
+    if (ctx->counters) cudaFree(ctx->counters);
+    if (ctx->sync_words) cudaFree(ctx->sync_words);
+    if (ctx->status_dev) cudaFree(ctx->status_dev);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    if (ctx->stage) cudaFree(ctx->stage);
+    lf_persistent_release(ctx);
+    lf_tf32_release(ctx);
+    delete ctx;
+    return LF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+// Internal declarations shared by the translation units of libleapfrog (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "leapfrog.h"
+
+// Bits of the device status word (0 = clean).
+enum : unsigned {
+    LF_DEV_TIMEOUT_FLAG = 1u,     // a wait on a ready flag ran out
+    LF_DEV_TIMEOUT_BARRIER = 2u,  // a wait on a group barrier ran out
+    LF_DEV_BAD_CONFIG = 4u        // a kernel was launched with a shape it does not support
+};
+
+struct lf_graph_key {
+    const void *w, *z, *a, *y;
+    void *delta, *gw, *gb;
+    int variant, gw_math;
+    bool operator==(const lf_graph_key& o) const {
+        return w == o.w && z == o.z && a == o.a && y == o.y && delta == o.delta &&
+               gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math;
+    }
+};
+
+struct lf_ctx {
+    int L, N, B, k, keff;
+    int device;
+    int sm_count;
+    int smem_optin;  // max dynamic shared memory per block
+    cudaStream_t stream;
+
+    // options
+    int opt_variant;
+    int opt_gw_math;
+    long long wait_budget_us;
+    int use_graph;
+
+    // workspace (device)
+    float* partial;          // partial column sums of the delta matvec: [row_chunks][N]
+    unsigned* counters;      // arrival counters, one per column strip (self-resetting)
+    unsigned* sync_words;    // persistent kernels: ready flags + barrier words (zeroed per call)
+    size_t sync_words_count;
+    unsigned* status_dev;    // device status word
+    unsigned* status_host;   // pinned mirror
+    float* tf32_scratch;     // reserved for operand repacking of the tensor-core path
+
+    // leapfrog workers as streams
+    cudaStream_t* wstreams;  // keff streams
+    cudaEvent_t* ready_ev;   // L events: delta^l is complete
+    cudaEvent_t* done_ev;    // keff events: worker finished its layers
+    cudaEvent_t fork_ev;
+
+    // captured graph of the STREAMS variant
+    cudaGraphExec_t graph_exec;
+    lf_graph_key graph_key;
+    bool graph_valid;
+    int graph_launches;      // kernels inside the captured graph
+
+    // host-buffer entry point staging
+    float* stage;            // one allocation holding w, z, a, y, delta, gw, gb
+    size_t stage_bytes;
+
+    int last_cuda_error;
+    lf_stats stats;
+};
+
+#define LF_CUDA_TRY(ctx, expr)                                  \
+    do {                                                        \
+        cudaError_t e__ = (expr);                               \
+        if (e__ != cudaSuccess) {                               \
+            (ctx)->last_cuda_error = (int)e__;                  \
+            return LF_ECUDA;                                    \
+        }                                                       \
+    } while (0)
+
+// ---- launchers (each enqueues on `s` and returns the cudaError_t of the launch) -------------
+
+// B = 1 kernels
+cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* a_prev,
+                               float* z_l, float* a_l, int N, cudaStream_t s);
+cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s);
+cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
+                             int B, cudaStream_t s);
+int lfk_delta_row_chunks(int N);  // number of row chunks the delta matvec splits N rows into
+cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
+                             float* delta_l, float* gb_l, float* partial, unsigned* counters,
+                             int N, cudaStream_t s);
+cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
+                         cudaStream_t s);
+
+// B > 1 kernels (fp32 on the CUDA cores)
+cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
+                             float* z_l, float* a_l, int N, int B, cudaStream_t s);
+cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
+                           float* delta_l, int N, int B, cudaStream_t s);
+cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
+                             int B, cudaStream_t s);
+cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s);
+
+// ---- persistent single-launch backward (B = 1) ---------------------------------------------
+size_t lf_sync_words_needed(const lf_ctx* c);           // unsigned words of flag/barrier workspace
+bool lf_persistent_supported(const lf_ctx* c, int variant);
+int lf_auto_variant(const lf_ctx* c);                   // table lookup for LF_VARIANT_AUTO
+int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* z, const float* a,
+                           const float* y, float* delta, float* gw, float* gb);
+void lf_persistent_release(lf_ctx* c);
+
+// ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------
+bool lf_tf32_supported(const lf_ctx* c);
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l,
+                    cudaStream_t s, int* launches);
+void lf_tf32_release(lf_ctx* c);

@@ -1,0 +1,155 @@
+// Mini-batch (B > 1) kernels in fp32 on the CUDA cores.  With B samples as columns, Eq. z,
+// Eq. bp2 and Eq. bp4 each become one dense N x N x B contraction per layer:
+//     forward : Z[b][j]  = sum_k A[b][k]  W[j][k] + bias[j],  A' = sigma(Z)
+//     delta   : D'[b][k] = (sum_j D[b][j] W[j][k]) * a[b][k] (1 - a[b][k])
+//     grad_w  : G[j][k]  = sum_b D[b][j]  A[b][k]
+// One shared-memory tiled kernel serves all three; the operand orientation (which index is
+// contiguous in memory) and the epilogue are template parameters.
+#include "lf_internal.h"
+
+namespace {
+
+__device__ __forceinline__ float lf_sigmoid(float t) { return 1.0f / (1.0f + expf(-t)); }
+
+constexpr int BM = 64, BN = 64, BK = 16, PAD = 4;
+
+enum { EPI_PLAIN = 0, EPI_FORWARD = 1, EPI_DELTA = 2 };
+
+// C[m][n] = sum_k A(m,k) Bm(k,n).
+//   A_KMAJOR: A(m,k) = A[m*lda + k]   else A(m,k) = A[k*lda + m]
+//   B_KMAJOR: Bm(k,n) = Bm[n*ldb + k] else Bm(k,n) = Bm[k*ldb + n]
+// The contiguous extent of every operand (and Nn, ldc) must be a multiple of 4.
+template <bool A_KMAJOR, bool B_KMAJOR, int EPI>
+__global__ void __launch_bounds__(256)
+k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __restrict__ C,
+            float* __restrict__ C2, const float* __restrict__ aux, int M, int Nn, int K, int lda,
+            int ldb, int ldc)
+{
+    __shared__ __align__(16) float As[BK][BM + PAD];
+    __shared__ __align__(16) float Bs[BK][BN + PAD];
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        // ---- stage the A tile as As[k][m]
+        if (A_KMAJOR) {
+            int m = tid >> 2, kq = (tid & 3) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (m0 + m < M && k0 + kq < K)
+                v = *reinterpret_cast<const float4*>(A + (size_t)(m0 + m) * lda + k0 + kq);
+            As[kq + 0][m] = v.x; As[kq + 1][m] = v.y; As[kq + 2][m] = v.z; As[kq + 3][m] = v.w;
+        } else {
+            int kk = tid >> 4, mq = (tid & 15) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (k0 + kk < K && m0 + mq < M)
+                v = *reinterpret_cast<const float4*>(A + (size_t)(k0 + kk) * lda + m0 + mq);
+            *reinterpret_cast<float4*>(&As[kk][mq]) = v;
+        }
+        // ---- stage the B tile as Bs[k][n]
+        if (B_KMAJOR) {
+            int n = tid >> 2, kq = (tid & 3) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (n0 + n < Nn && k0 + kq < K)
+                v = *reinterpret_cast<const float4*>(Bm + (size_t)(n0 + n) * ldb + k0 + kq);
+            Bs[kq + 0][n] = v.x; Bs[kq + 1][n] = v.y; Bs[kq + 2][n] = v.z; Bs[kq + 3][n] = v.w;
+        } else {
+            int kk = tid >> 4, nq = (tid & 15) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (k0 + kk < K && n0 + nq < Nn)
+                v = *reinterpret_cast<const float4*>(Bm + (size_t)(k0 + kk) * ldb + n0 + nq);
+            *reinterpret_cast<float4*>(&Bs[kk][nq]) = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            float ar[4] = {av.x, av.y, av.z, av.w};
+            float br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    const int n = n0 + tx * 4;
+    if (n >= Nn) return;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+        float4 r = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        size_t off = (size_t)m * ldc + n;
+        if (EPI == EPI_FORWARD) {
+            float4 bb = *reinterpret_cast<const float4*>(aux + n);
+            r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
+            *reinterpret_cast<float4*>(C + off) = r;                       // z
+            *reinterpret_cast<float4*>(C2 + off) = make_float4(lf_sigmoid(r.x), lf_sigmoid(r.y),
+                                                               lf_sigmoid(r.z), lf_sigmoid(r.w));
+        } else if (EPI == EPI_DELTA) {
+            float4 av = *reinterpret_cast<const float4*>(aux + off);
+            r.x *= av.x * (1.0f - av.x); r.y *= av.y * (1.0f - av.y);
+            r.z *= av.z * (1.0f - av.z); r.w *= av.w * (1.0f - av.w);
+            *reinterpret_cast<float4*>(C + off) = r;
+        } else {
+            *reinterpret_cast<float4*>(C + off) = r;
+        }
+    }
+}
+
+// Eq. bp3 for a mini-batch: gb_j = sum_b delta_bj, samples added in index order.
+__global__ void k_grad_b_colsum(const float* __restrict__ delta_l, float* __restrict__ gb_l, int N,
+                                int B)
+{
+    int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= N) return;
+    float s = 0.f;
+    for (int b = 0; b < B; ++b) s += delta_l[(size_t)b * N + j];
+    gb_l[j] = s;
+}
+
+inline dim3 gemm_grid(int M, int Nn) { return dim3((Nn + BN - 1) / BN, (M + BM - 1) / BM); }
+
+}  // namespace
+
+cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
+                             float* z_l, float* a_l, int N, int B, cudaStream_t s)
+{
+    // M = B (samples), Nn = N (neuron j), K = N (neuron k of the layer below)
+    k_gemm_simt<true, true, EPI_FORWARD><<<gemm_grid(B, N), 256, 0, s>>>(
+        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N);
+    return cudaGetLastError();
+}
+
+cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
+                           float* delta_l, int N, int B, cudaStream_t s)
+{
+    // M = B, Nn = N (neuron k of layer l), K = N (neuron j of layer l+1); w_up[j][k] is n-contiguous
+    k_gemm_simt<true, false, EPI_DELTA><<<gemm_grid(B, N), 256, 0, s>>>(
+        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N);
+    return cudaGetLastError();
+}
+
+cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
+                             int B, cudaStream_t s)
+{
+    // M = N (j), Nn = N (k), K = B; both operands are contiguous along their M / N index
+    k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(N, N), 256, 0, s>>>(
+        delta_l, a_prev, gw_l, nullptr, nullptr, N, N, B, N, N, N);
+    return cudaGetLastError();
+}
+
+cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s)
+{
+    k_grad_b_colsum<<<(N + 127) / 128, 128, 0, s>>>(delta_l, gb_l, N, B);
+    return cudaGetLastError();
+}

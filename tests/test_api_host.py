@@ -1,0 +1,61 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every symbol the
+header declares, and its argument validation answers before any device work."""
+import ctypes
+import os
+import re
+
+import paper_1801_04928_b200 as lf
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "leapfrog.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lf_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(lf.LIB_PATH)
+    names = _declared_symbols()
+    assert "lf_backward" in names and "lf_create" in names and len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(lf.EXPORTS)
+
+
+def test_binding_has_the_same_names():
+    for n in _declared_symbols():
+        assert callable(getattr(lf, n)), n
+
+
+def test_strerror_and_version():
+    assert lf.lf_version() >= 100
+    assert lf.lf_strerror(lf.LF_OK) == "ok"
+    for code in range(-7, 0):
+        assert lf.lf_strerror(code) != "unknown status"
+    assert lf.lf_strerror(-99) == "unknown status"
+
+
+def test_create_rejects_bad_sizes_before_touching_the_device():
+    for args in [(0, 64, 1, 1), (4, 0, 1, 1), (4, 64, 0, 1), (4, 64, 1, 0), (4, 66, 1, 1),
+                 (-1, 64, 1, 1)]:
+        rc, h = lf.lf_create(*args)
+        assert rc == lf.LF_EINVAL and not h.value
+
+
+def test_null_context_is_an_error_not_a_crash():
+    assert lf.lf_sync(None) == lf.LF_ENULL
+    assert lf.lf_destroy(None) == lf.LF_ENULL
+    assert lf.lf_set_option(None, lf.LF_OPT_VARIANT, 1) == lf.LF_ENULL
+    assert lf.lf_forward(None, 16, 16, 16, 16, 16) == lf.LF_ENULL
+    assert lf.lf_backward(None, 16, 16, 16, 16, 16, 16, 16) == lf.LF_ENULL
+    assert lf.lf_owner(None, 1) == -1
+
+
+def test_no_device_means_an_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        return
+    rc, h = lf.lf_create(4, 64, 1, 2)
+    assert rc == lf.LF_ECUDA and not h.value
