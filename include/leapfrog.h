@@ -43,7 +43,8 @@ enum lf_status {
     LF_ERESOURCE = -4, /* the device cannot hold the requested configuration co-resident     */
     LF_ECUDA = -5,     /* a CUDA call failed; lf_last_cuda_error() gives the cudaError_t     */
     LF_ETIMEOUT = -6,  /* a bounded device-side wait ran out; outputs are undefined          */
-    LF_ENOMEM = -7     /* workspace allocation failed                                        */
+    LF_ENOMEM = -7,    /* workspace allocation failed                                        */
+    LF_ECAPACITY = -8  /* size is beyond the fixed capacity of an allocation-free entry point */
 };
 
 /* How lf_backward schedules Eq. bp4 (the weight gradients) against the delta chain. */
@@ -148,6 +149,40 @@ int lf_get_stats(lf_ctx* ctx, lf_stats* out);
 
 /* cudaError_t of the last failed CUDA call of this context (0 if none). */
 int lf_last_cuda_error(const lf_ctx* ctx);
+
+/*
+ * One delta-chain step (Eq. bp2, single sample) for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for the library's users.)
+ *
+ *     delta_l[k] = (sum_j w_up[j][k] * delta_up[j]) * a_l[k] * (1 - a_l[k]),   k = 0..N-1
+ *
+ * w_up is w^{l+1} [N][N] row-major, delta_up is delta^{l+1} [N], a_l is a^l = sigma(z^l) [N],
+ * delta_l receives delta^l [N]; all are device pointers, float32, 16-byte aligned, owned by
+ * the caller.  The result is the same as the delta slab lf_backward writes for that layer.
+ *
+ * Who needs it: a process that has handed all of the GPU's memory to its own pool (an
+ * inference server or a framework allocator that reserves HBM up front), where a cudaMalloc
+ * made behind its back fails or fragments the pool; and a latency-critical loop that cannot
+ * afford the device-wide synchronisation an allocation or a free implies.  Every other entry
+ * point needs an lf_ctx, and lf_create allocates.  This one takes no context and calls no
+ * allocating routine: the scratch its kernel needs (partial column sums and arrival counters)
+ * is a fixed array inside the library image, about 1 MiB, resident on every GPU that loads the
+ * library until the process exits.
+ *
+ * Limits and rules:
+ *  - N must be a multiple of 4 and at most 4096; a larger N is LF_ECAPACITY (nothing is run).
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current) and remembers it; make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  Calls whose kernels may overlap on the GPU
+ *    (different streams without an ordering between them, or several host threads) race on it
+ *    and give wrong results; keep calls on one stream or order them with events.
+ *  - `cuda_stream` is a cudaStream_t of the current device (NULL = legacy default stream).  The
+ *    call enqueues a small memset of the counters and one kernel, and returns without waiting.
+ * Errors: LF_ENULL, LF_EALIGN, LF_EINVAL (N), LF_ECAPACITY, LF_ERESOURCE (device ordinal
+ * >= 64), LF_ECUDA.
+ */
+int lf_delta_step_static(const float* w_up, const float* delta_up, const float* a_l,
+                         float* delta_l, int N, void* cuda_stream);
 
 /* Static English text for a status code. */
 const char* lf_strerror(int status);

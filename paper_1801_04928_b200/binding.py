@@ -15,13 +15,14 @@ LIB_PATH = os.path.join(_PKG, "libleapfrog.so")
 
 LF_OK, LF_EINVAL, LF_ENULL, LF_EALIGN, LF_ERESOURCE, LF_ECUDA, LF_ETIMEOUT, LF_ENOMEM = (
     0, -1, -2, -3, -4, -5, -6, -7)
+LF_ECAPACITY = -8
 LF_VARIANT_AUTO, LF_VARIANT_STREAMS, LF_VARIANT_PERSISTENT, LF_VARIANT_FUSED = 0, 1, 2, 3
 LF_GW_MATH_AUTO, LF_GW_MATH_FP32, LF_GW_MATH_TF32 = 0, 1, 2
 LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH = 1, 2, 3, 4
 
 EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
            "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
-           "lf_strerror", "lf_version", "lf_destroy")
+           "lf_strerror", "lf_version", "lf_destroy", "lf_delta_step_static")
 
 
 class lf_stats(ctypes.Structure):
@@ -54,6 +55,7 @@ def _load() -> ctypes.CDLL:
     lib.lf_strerror.restype = ctypes.c_char_p
     lib.lf_version.argtypes = []
     lib.lf_destroy.argtypes = [vp]
+    lib.lf_delta_step_static.argtypes = [vp, vp, vp, vp, i, vp]
     for name in EXPORTS:
         if name != "lf_strerror":
             getattr(lib, name).restype = i
@@ -141,6 +143,18 @@ def lf_last_cuda_error(ctx) -> int:
 
 def lf_destroy(ctx) -> int:
     return _lib.lf_destroy(ctx)
+
+
+def lf_delta_step_static(w_up, delta_up, a_l, delta_l, N: int, cuda_stream: int | None = None) -> int:
+    """One Eq. bp2 step without a context and without any allocation (see the header).
+
+    For processes that own all device memory through their own pool, or that cannot take the
+    device-wide stall of a cudaMalloc: the kernel's scratch is a fixed array inside the
+    library (N <= 4096, else LF_ECAPACITY).  Calls share that array, so do not let two of
+    them overlap on the GPU.  Returns the status code; the work is only enqueued.
+    """
+    return _lib.lf_delta_step_static(_ptr(w_up), _ptr(delta_up), _ptr(a_l), _ptr(delta_l), int(N),
+                                     ctypes.c_void_p(cuda_stream or None))
 
 
 # ---- a small convenience wrapper (still marshalling only) -------------------------------------

@@ -170,6 +170,7 @@ const char* lf_strerror(int status)
         case LF_ECUDA: return "CUDA call failed (see lf_last_cuda_error)";
         case LF_ETIMEOUT: return "a bounded device-side wait expired; outputs are undefined";
         case LF_ENOMEM: return "workspace allocation failed";
+        case LF_ECAPACITY: return "size exceeds the fixed capacity of this allocation-free entry point";
         default: return "unknown status";
     }
 }

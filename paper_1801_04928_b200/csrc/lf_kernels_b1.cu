@@ -2,6 +2,8 @@
 // the output error (Eq. bp1), the transposed matvec of the delta recurrence (Eq. bp2) and the
 // rank-1 weight-gradient writer (Eq. bp4).  All are HBM-bound streams over one N x N matrix:
 // 128-bit accesses, rows walked in the order they sit in memory.
+#include <mutex>
+
 #include "lf_internal.h"
 
 namespace {
@@ -230,4 +232,75 @@ cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l,
     if (grid < 1) grid = 1;
     k_gw_rank1<<<grid, GW1_THREADS, 0, s>>>(delta_l, a_prev, gw_l, N);
     return cudaGetLastError();
+}
+
+// ---- Eq. bp2 for callers that must not allocate -------------------------------------------------
+// The scratch of k_delta_matvec (partial column sums, then the per-strip arrival counters) lives
+// in a file-scope device array instead of a context's workspace.  Every GPU that loads this
+// library carries these LF_STATIC_SCRATCH_WORDS * 4 bytes (a little over 1 MiB) until exit.
+namespace {
+
+constexpr int LF_STATIC_MAX_N = 4096;                 // largest width the array is sized for
+constexpr int LF_STATIC_MAX_CHUNKS = 64;              // row chunks never exceed this for N <= 4096
+constexpr int LF_STATIC_COUNTER_WORDS = 64;           // >= column strips (N / 128) for N <= 4096
+constexpr int LF_STATIC_PARTIAL_WORDS = LF_STATIC_MAX_CHUNKS * LF_STATIC_MAX_N;
+constexpr int LF_STATIC_SCRATCH_WORDS = LF_STATIC_PARTIAL_WORDS + LF_STATIC_COUNTER_WORDS;
+
+static __device__ __align__(256) float lf_static_scratch[LF_STATIC_SCRATCH_WORDS];
+
+constexpr int LF_STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+float* g_static_scratch_addr[LF_STATIC_MAX_DEVICES];  // device address of the array, per device
+
+// In host code `lf_static_scratch` is only a handle for the runtime, not an address a kernel
+// could use; the device address has to be asked for, once per device, with that device current.
+int static_scratch_for_current_device(float** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LF_ECUDA;
+    if (dev < 0 || dev >= LF_STATIC_MAX_DEVICES) return LF_ERESOURCE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        float* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), lf_static_scratch);
+        if (e != cudaSuccess || !p) {
+            cudaGetLastError();
+            return LF_ECUDA;
+        }
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return LF_OK;
+}
+
+}  // namespace
+
+extern "C" int lf_delta_step_static(const float* w_up, const float* delta_up, const float* a_l,
+                                    float* delta_l, int N, void* cuda_stream)
+{
+    if (!w_up || !delta_up || !a_l || !delta_l) return LF_ENULL;
+    const void* ps[] = {w_up, delta_up, a_l, delta_l};
+    for (const void* p : ps)
+        if (reinterpret_cast<uintptr_t>(p) & 15u) return LF_EALIGN;
+    if (N < 1 || (N & 3) != 0) return LF_EINVAL;
+    if (N > LF_STATIC_MAX_N) return LF_ECAPACITY;
+    const int rows = dmv_rows_per_chunk(N);
+    const int chunks = (N + rows - 1) / rows;
+    const int strips = ((N >> 2) + DMV_STRIP4 - 1) / DMV_STRIP4;
+    if (chunks > LF_STATIC_MAX_CHUNKS || strips > LF_STATIC_COUNTER_WORDS) return LF_ECAPACITY;
+
+    float* scratch = nullptr;
+    int rc = static_scratch_for_current_device(&scratch);
+    if (rc != LF_OK) return rc;
+    float* partial = scratch;
+    unsigned* counters = reinterpret_cast<unsigned*>(scratch + LF_STATIC_PARTIAL_WORDS);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // The array keeps whatever the previous call left.  The partial sums are fully rewritten
+    // before they are read; the arrival counters must start at zero.
+    if (cudaMemsetAsync(counters, 0, LF_STATIC_COUNTER_WORDS * sizeof(unsigned), s) != cudaSuccess)
+        return LF_ECUDA;
+    dim3 grid(strips, chunks);
+    k_delta_matvec<<<grid, DMV_WARPS * 32, 0, s>>>(w_up, delta_up, a_l, delta_l, nullptr, partial,
+                                                  counters, N, rows, chunks);
+    return cudaGetLastError() == cudaSuccess ? LF_OK : LF_ECUDA;
 }
