@@ -57,6 +57,13 @@ struct lf_ctx {
     bool graph_valid;
     int graph_launches;      // kernels inside the captured graph
 
+    // persistent kernels: TMA descriptor of w (opaque 128-byte CUtensorMap) and the call epoch
+    alignas(64) unsigned char w_map_storage[128];
+    bool w_map_valid;
+    const void* w_map_ptr;
+    int w_map_wc;
+    unsigned epoch;
+
     // host-buffer entry point staging
     float* stage;            // one allocation holding w, z, a, y, delta, gw, gb
     size_t stage_bytes;

@@ -30,6 +30,7 @@ def test_single_sample_parity(L, N, k, variant):
     cfg = dict(L=L, N=N, B=1, k=k)
     t = _inputs(L, N, 1, seed=L * 1000 + N)
     out, stats = gpu_pass(cfg, t, variant=variant)
+    assert stats["variant"] == variant and stats["device_status"] == 0
     ref = oracle_pass(t)
     compare_all(cfg, out, ref)
     assert torch.equal(out["a"][0], t["x"])            # Eq. x
