@@ -63,6 +63,9 @@ struct lf_ctx {
     const void* w_map_ptr;
     int w_map_wc;
     unsigned epoch;
+#ifdef LF_PK_TRACE
+    unsigned long long* trace_dev;  // debug builds: per-step SM-clock stamps of two CTAs
+#endif
 
     // host-buffer entry point staging
     float* stage;            // one allocation holding w, z, a, y, delta, gw, gb

@@ -1,25 +1,29 @@
 // Persistent single-launch backward pass for one sample (B = 1): Eq. bp1, the Eq. bp2 chain and
 // Eq. bp3/bp4 of every layer in ONE kernel.
 //
-// Roles.  The grid is a row of thread-block clusters of 8 CTAs.
+// Grid.  A row of thread-block clusters of C CTAs (C = 2, 4 or 8: whichever puts the most SMs
+// to work), one CTA per SM, 256 threads per CTA.
 //   * Chain clusters.  Cluster q owns the column strip [q*Ws, (q+1)*Ws) of every weight matrix;
 //     inside it CTA c owns the rows [c*Hr, (c+1)*Hr).  For layer step s (reading w^s, producing
-//     delta^{s-1}) a CTA multiplies its tile by delta^s of its rows, the 8 CTAs of the cluster
-//     add their partial column sums through distributed shared memory (each CTA finishes 1/8 of
-//     the strip), apply sigma' and publish delta^{s-1}.  Weight tiles do not depend on delta, so
-//     they are fetched by TMA several sub-tiles (and layers) ahead of the chain.
-//   * Fused variant: the pass over a tile of w^s also stores the same tile of gw^s =
-//     delta^s (x) a^{s-1} (both already known); gw^1 is stored by a tail pass.
+//     delta^{s-1}) the CHAIN WARPS (0-3) of a CTA multiply its tile by delta^s of its rows, send
+//     their partial column sums through distributed shared memory to the CTA of the cluster that
+//     finishes those columns (each CTA finishes 1/C of the strip), which adds them, applies
+//     sigma' and publishes delta^{s-1}.  Weight tiles do not depend on delta, so they are
+//     fetched by TMA several sub-tiles (and layers) ahead of the chain.
+//   * Fused variant: the STORE WARPS (4-7) of the same CTA stream the tile of gw^s =
+//     delta^s (x) a^{s-1} out while the chain warps go on; gw^1 follows after the last step.
 //   * Leapfrog variant: extra worker clusters are split into k groups; group (L-l) mod k waits
 //     for delta^l and streams gw^l out (Section 3: each worker handles every k-th layer).  The
 //     chain CTAs then only read.
 //
-// delta crosses CTAs through an exchange buffer of 8-byte slots {value, epoch}: one 64-bit store
-// publishes a value together with its "ready" tag, one 64-bit load polls both, so no fence and no
-// separate flag is needed.  The epoch changes with every call, so the buffer is never cleared.
-// Every wait (slot poll, TMA barrier) is bounded by a time budget; on expiry the CTA raises the
-// status word, stops waiting for the rest of the launch and runs to completion with whatever it
-// has, so cluster barriers still see every thread and the kernel always ends.
+// Hand-offs.  delta crosses clusters through an exchange buffer of 8-byte slots {value, epoch}:
+// one 64-bit store publishes a value together with its "ready" tag and one 64-bit load polls
+// both, so no fence and no separate flag is needed; the epoch changes with every call, so the
+// buffer is never cleared.  Partial sums cross CTAs of a cluster by st.async, which writes the
+// data and credits its bytes to an mbarrier of the receiving CTA; chain and store warps of a CTA hand the delta buffers back and
+// forth through two pairs of mbarriers.  Every wait is bounded by a time budget; on expiry the
+// CTA raises the status word, stops waiting for the rest of the launch and runs to the end with
+// whatever it has, so the kernel always terminates.
 #include <cuda.h>
 
 #include "lf_internal.h"
@@ -27,14 +31,18 @@
 namespace {
 
 constexpr int PK_THREADS = 256;
-constexpr int PK_CLUSTER = 8;
-constexpr int PK_STAGE_FLOATS = 8192;  // 32 KiB per pipeline stage
+constexpr int PK_CHAIN_THREADS = 128;   // warps 0-3
+constexpr int PK_CHAIN_WARPS = 4;
+constexpr int PK_MAX_CLUSTER = 8;       // cluster sizes 2, 4 and 8 are used
+constexpr int PK_STAGE_FLOATS = 8192;   // 32 KiB per pipeline stage
 constexpr int PK_STAGES = 6;
-constexpr int PK_MAX_NCB = 4;          // column blocks per strip (strip width <= 4 * 256)
-constexpr int PK_MAX_SLICE = 128;      // strip columns finished per CTA (strip / 8)
+constexpr int PK_MAX_NCB = 4;           // column blocks per strip (strip width <= 4 * 256)
+constexpr int PK_MAX_SLICE = 128;       // strip columns finished per CTA (strip / C)
+constexpr int PK_DROWS = 2176;          // floats of delta held per CTA and buffer (tile rows, padded)
 
 struct PkParams {
     int L, N;
+    int C;         // CTAs per cluster
     int Qc;        // chain clusters
     int Qw;        // worker clusters (0 in the fused variant)
     int fused;     // 1: chain CTAs store gw tiles
@@ -44,7 +52,7 @@ struct PkParams {
     int Hr;        // rows per chain CTA
     int R;         // rows per sub-tile = PK_STAGE_FLOATS / Wc
     int nRB;       // row blocks per layer
-    int slice;     // Ws / 8
+    int slice;     // Ws / C
     int keff;      // effective leapfrog workers
     unsigned epoch;
     unsigned long long budget_ns;
@@ -55,6 +63,9 @@ struct PkParams {
     float* gb;
     unsigned long long* xch;  // [L][N] slots
     unsigned* status;
+#ifdef LF_PK_TRACE
+    unsigned long long* trace;  // [2 CTAs][L][16] SM-clock stamps (debug builds only)
+#endif
 };
 
 // ---- small PTX wrappers ----------------------------------------------------------------------
@@ -77,12 +88,28 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(unsigned bar)
+{
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
 {
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -103,6 +130,10 @@ __device__ __forceinline__ void cluster_sync_all()
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;"
                  ::: "memory");
 }
+__device__ __forceinline__ void chain_sync()   // the four chain warps only
+{
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+}
 __device__ __forceinline__ unsigned cluster_ctarank()
 {
     unsigned r;
@@ -115,9 +146,14 @@ __device__ __forceinline__ unsigned map_to_cta(unsigned local_addr, unsigned ran
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f32(unsigned addr, float v)
+// Store four floats into the shared memory of a CTA of the cluster and credit 16 bytes to an
+// mbarrier there (both addresses from mapa): data and "it has arrived" travel together, no fence.
+__device__ __forceinline__ void st_async_f32x4(unsigned cluster_addr, float4 v, unsigned cluster_bar)
 {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+    asm volatile(
+        "st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+        ::"r"(cluster_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(cluster_bar)
+        : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_slot(const unsigned long long* p)
 {
@@ -135,10 +171,31 @@ __device__ __forceinline__ void st_stream4(float* p, float4 v)
     __stcs(reinterpret_cast<float4*>(p), v);
 }
 
+// Debug builds (-DLF_PK_TRACE) record SM-clock stamps of each chain step of two CTAs.
+#ifdef LF_PK_TRACE
+#define PK_STAMP(slot)                                                                       \
+    do {                                                                                     \
+        if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == 77))                               \
+            P.trace[((blockIdx.x == 0 ? 0 : 1) * (size_t)P.L + (size_t)(P.L - s)) * 16 + (slot)] = \
+                (unsigned long long)clock64();                                               \
+    } while (0)
+#else
+#define PK_STAMP(slot) do { } while (0)
+#endif
+
 struct PkShared {
-    unsigned long long full[PK_STAGES];  // TMA arrival barriers
+    unsigned long long full[PK_STAGES];  // TMA arrival, one per stage
+    unsigned long long part_ready[2];    // partial sums of a step have landed here (by step parity)
+    unsigned long long d_ready[2];       // chain warps filled delta buffer p
+    unsigned long long d_free[2];        // store warps are done with delta buffer p
     volatile unsigned abort_flag;        // set once a wait of this CTA has run out
 };
+
+__device__ __forceinline__ void raise_timeout(const PkParams& P, PkShared* sh, unsigned bit)
+{
+    atomicOr(P.status, bit);
+    sh->abort_flag = 1u;
+}
 
 // Wait until slot *p carries this call's epoch; returns the value (0 after a timeout).
 __device__ __forceinline__ float wait_slot(const unsigned long long* p, const PkParams& P,
@@ -154,28 +211,29 @@ __device__ __forceinline__ float wait_slot(const unsigned long long* p, const Pk
         if ((unsigned)(v >> 32) == P.epoch) return __uint_as_float((unsigned)v);
         if ((++spins & 31u) == 0u) {
             if (sh->abort_flag) return 0.f;
-            if (globaltimer_ns() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
-                atomicOr(P.status, LF_DEV_TIMEOUT_FLAG);
-                sh->abort_flag = 1u;
+            if (globaltimer_ns() - t0 > P.budget_ns ||
+                (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
+                raise_timeout(P, sh, LF_DEV_TIMEOUT_FLAG);
                 return 0.f;
             }
         }
     }
 }
 
-__device__ __forceinline__ void wait_full(unsigned bar, unsigned parity, const PkParams& P,
-                                          PkShared* sh)
+// Bounded wait on an mbarrier of this CTA (CLUSTER = arrivals come from other CTAs).
+template <bool CLUSTER>
+__device__ __forceinline__ void wait_bar(unsigned bar, unsigned parity, const PkParams& P,
+                                         PkShared* sh)
 {
-    if (mbar_try_wait(bar, parity)) return;
+    if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return;
     if (sh->abort_flag) return;
     const unsigned long long t0 = globaltimer_ns();
     unsigned spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
+    while (!(CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity))) {
         if ((++spins & 15u) == 0u) {
             if (sh->abort_flag) return;
             if (globaltimer_ns() - t0 > P.budget_ns) {
-                atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
-                sh->abort_flag = 1u;
+                raise_timeout(P, sh, LF_DEV_TIMEOUT_BARRIER);
                 return;
             }
         }
@@ -211,39 +269,46 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     float* stages = reinterpret_cast<float*>(smem_raw);                       // PK_STAGES x 32 KiB
-    float* d_rows = stages + PK_STAGES * PK_STAGE_FLOATS;                     // nRB*R (<= 2304)
-    float* red = d_rows + 2304;                                               // 256 float4
-    float* recv = red + PK_THREADS * 4;                                       // [2][8][PK_MAX_SLICE]
-    PkShared* sh = reinterpret_cast<PkShared*>(recv + 2 * PK_CLUSTER * PK_MAX_SLICE);
+    float* d_rows = stages + PK_STAGES * PK_STAGE_FLOATS;                     // [2][PK_DROWS]
+    float4* red = reinterpret_cast<float4*>(d_rows + 2 * PK_DROWS);           // [2][4 warps][32 lanes]
+    float* recv = reinterpret_cast<float*>(red + 2 * PK_CHAIN_THREADS);       // [2][C][PK_MAX_SLICE]
+    PkShared* sh = reinterpret_cast<PkShared*>(recv + 2 * PK_MAX_CLUSTER * PK_MAX_SLICE);
 
-    const int tid = threadIdx.x;
-    const int N = P.N, L = P.L;
-    const int cluster_id = blockIdx.x / PK_CLUSTER;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int N = P.N, L = P.L, C = P.C;
+    const int cluster_id = blockIdx.x / C;
     const int c = (int)cluster_ctarank();
+    const bool is_chain_cluster = cluster_id < P.Qc;
 
     if (tid == 0) {
         for (int i = 0; i < PK_STAGES; ++i) mbar_init(smem_u32(&sh->full[i]), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&sh->part_ready[i]), 1);
+            mbar_init(smem_u32(&sh->d_ready[i]), PK_CHAIN_THREADS);
+            mbar_init(smem_u32(&sh->d_free[i]), PK_THREADS - PK_CHAIN_THREADS);
+        }
         sh->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    cluster_sync_all();   // every CTA's barriers exist before a peer can arrive on them
 
     // ===================== leapfrog worker clusters ==========================================
-    if (cluster_id >= P.Qc) {
-        const int Wn = P.Qw * PK_CLUSTER;
-        const int wi = (cluster_id - P.Qc) * PK_CLUSTER + c;
+    if (!is_chain_cluster) {
+        const int Wn = P.Qw * C;
+        const int wi = (cluster_id - P.Qc) * C + c;
         const int G = P.keff < Wn ? P.keff : Wn;     // groups that really exist
         const int g = wi % G, m = wi / G;
         const int Mg = (Wn - g + G - 1) / G;          // members of my group
         const int rpm = (N + Mg - 1) / Mg;            // rows per member
         const int row0 = m * rpm, row1 = min(N, row0 + rpm);
-        float* a_sm = stages;                         // N floats (N <= 16384 fits one... two stages)
+        float* a_sm = stages;                         // N floats (N <= 16384: two stages)
         float* dr = stages + 16384;                   // up to N floats
         for (int l = L; l >= 1; --l) {
             if ((((L - l) % P.keff) % G) != g) continue;   // not a layer of my group
             if (row0 < row1) worker_store_rows(P, l, row0, row1, dr, a_sm, sh);
         }
-        cluster_sync_all();   // matched by nothing else: keeps the cluster's CTAs exiting together
+        cluster_sync_all();   // the cluster's CTAs leave together
         return;
     }
 
@@ -251,163 +316,216 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
     const int q = cluster_id;
     const int Wc = P.Wc, nCB = P.nCB, R = P.R, nRB = P.nRB, Hr = P.Hr, Ws = P.Ws;
     const int WC4 = Wc >> 2;
-    const int RG = PK_THREADS / WC4;       // row groups
-    const int tcol = tid % WC4, trow = tid / WC4;
+    const int RG = PK_CHAIN_THREADS / WC4;    // row groups of the 128 threads of either half
+    const int ht = tid & (PK_CHAIN_THREADS - 1);   // thread index inside its half (chain / store)
+    const int tcol = ht % WC4, trow = ht / WC4;
     const int row_base = c * Hr;
     const int row_end = min(N, row_base + Hr);
     const int col_base = q * Ws;
-    const int nSub = nCB * nRB;
-    const int total = (L - 1) * nSub;
-    const unsigned stage_bytes = (unsigned)(R * Wc * sizeof(float));
     const int Hr_pad = nRB * R;
 
-    // producer: issue the TMA load of sub-tile `it` of this CTA's sequence
-    auto issue = [&](int it) {
-        const int step = it / nSub, sub = it - step * nSub;
-        const int s = L - step;                 // w^s
-        const int cb = sub / nRB, rb = sub - cb * nRB;
-        const int st = it % PK_STAGES;
-        const unsigned bar = smem_u32(&sh->full[st]);
-        mbar_expect_tx(bar, stage_bytes);
-        tma_load_3d(smem_u32(stages + (size_t)st * PK_STAGE_FLOATS), &w_map, bar,
-                    col_base + cb * Wc, row_base + rb * R, s - 1);
-    };
-    if (tid == 0) {
-        const int pre = total < PK_STAGES ? total : PK_STAGES;
-        for (int it = 0; it < pre; ++it) issue(it);
-    }
+    if (warp >= PK_CHAIN_WARPS) {
+        // ------------------------- store warps: gw^s = delta^s (x) a^{s-1} ---------------------
+        if (P.fused) {
+            float4 a4[PK_MAX_NCB], a4_next[PK_MAX_NCB];
+            auto load_a4 = [&](int l, float4* dst) {
+                const float* av = P.a + (size_t)l * N;
+#pragma unroll
+                for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
+                    dst[cb] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const int col = col_base + cb * Wc + tcol * 4;
+                    if (cb < nCB && col < N) dst[cb] = *reinterpret_cast<const float4*>(av + col);
+                }
+            };
+            load_a4(L - 1, a4);
+            for (int s = L; s >= 1; --s) {
+                const int p = s & 1;
+                const unsigned use = (unsigned)((L - s) >> 1);      // how often buffer p was used before
+                if (s >= 2) load_a4(s - 2, a4_next);
+                wait_bar<false>(smem_u32(&sh->d_ready[p]), use & 1u, P, sh);
+                const float* dr = d_rows + p * PK_DROWS;
+                float* gw_s = P.gw + (size_t)(s - 1) * N * N;
+#pragma unroll
+                for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
+                    if (cb >= nCB) break;
+                    const int col = col_base + cb * Wc + tcol * 4;
+                    if (col >= N) continue;
+                    const float4 av = a4[cb];
+                    float* out = gw_s + (size_t)row_base * N + col;
+                    const int rows = row_end - row_base;
+#pragma unroll 4
+                    for (int rr = trow; rr < rows; rr += RG) {
+                        const float d = dr[rr];
+                        st_stream4(out + (size_t)rr * N, make_float4(d * av.x, d * av.y, d * av.z, d * av.w));
+                    }
+                }
+                mbar_arrive(smem_u32(&sh->d_free[p]));
+#pragma unroll
+                for (int cb = 0; cb < PK_MAX_NCB; ++cb) a4[cb] = a4_next[cb];
+            }
+        }
+    } else {
+        // ------------------------- chain warps --------------------------------------------------
+        const int nSub = nCB * nRB;
+        const int total = (L - 1) * nSub;
+        const unsigned stage_bytes = (unsigned)(R * Wc * sizeof(float));
+        const int wpr = WC4 > 32 ? WC4 / 32 : 1;   // warps that share one tile row
 
-    // ---- Eq. bp1: delta^L for my rows (every cluster computes it for itself)
-    {
-        const float* aL = P.a + (size_t)L * N;
-        for (int r = tid; r < Hr_pad; r += PK_THREADS) {
-            const int row = row_base + r;
-            float d = 0.f;
-            if (r < Hr && row < N) {
-                const float av = aL[row];
-                d = (av - P.y[row]) * (av * (1.0f - av));
-                if (q == 0) {
-                    P.delta[(size_t)(L - 1) * N + row] = d;
-                    P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
-                    if (P.Qw > 0) st_slot(P.xch + (size_t)(L - 1) * N + row, d, P.epoch);
+        // producer state (thread 0): the next sub-tile to fetch, as (layer, column block, row block)
+        int is_s = L, is_cb = 0, is_rb = 0, is_it = 0;
+        auto issue_next = [&]() {
+            const int st = is_it % PK_STAGES;
+            const unsigned bar = smem_u32(&sh->full[st]);
+            mbar_expect_tx(bar, stage_bytes);
+            tma_load_3d(smem_u32(stages + (size_t)st * PK_STAGE_FLOATS), &w_map, bar,
+                        col_base + is_cb * Wc, row_base + is_rb * R, is_s - 1);
+            ++is_it;
+            if (++is_rb == nRB) { is_rb = 0; if (++is_cb == nCB) { is_cb = 0; --is_s; } }
+        };
+        if (tid == 0) {
+            const int pre = total < PK_STAGES ? total : PK_STAGES;
+            for (int i = 0; i < pre; ++i) issue_next();
+        }
+
+        const int my_col = col_base + c * P.slice + tid;   // the column this thread finishes (tid < slice)
+        const bool finisher = tid < P.slice && my_col < N;
+        float a_mine = finisher ? P.a[(size_t)(L - 1) * N + my_col] : 0.f;
+
+        // ---- Eq. bp1: delta^L for my rows (every cluster computes it for itself)
+        {
+            const float* aL = P.a + (size_t)L * N;
+            float* dr = d_rows + (L & 1) * PK_DROWS;
+            for (int r = tid; r < Hr_pad; r += PK_CHAIN_THREADS) {
+                const int row = row_base + r;
+                float d = 0.f;
+                if (r < Hr && row < N) {
+                    const float av = aL[row];
+                    d = (av - P.y[row]) * (av * (1.0f - av));
+                    if (q == 0) {
+                        P.delta[(size_t)(L - 1) * N + row] = d;
+                        P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
+                        if (P.Qw > 0) st_slot(P.xch + (size_t)(L - 1) * N + row, d, P.epoch);
+                    }
+                }
+                dr[r] = d;
+            }
+            mbar_arrive(smem_u32(&sh->d_ready[L & 1]));
+        }
+        chain_sync();
+
+        int it = 0;
+        for (int s = L; s >= 2; --s) {
+            PK_STAMP(0);
+            const int p = s & 1;
+            const float* dr = d_rows + p * PK_DROWS;
+            float* recv_p = recv + p * PK_MAX_CLUSTER * PK_MAX_SLICE;
+            const float a_mine_next = (finisher && s >= 3) ? P.a[(size_t)(s - 2) * N + my_col] : 0.f;
+            // this step's partial sums for my slice: C CTAs x slice floats will be credited
+            if (tid == 0) mbar_expect_tx(smem_u32(&sh->part_ready[p]), (unsigned)(C * P.slice * sizeof(float)));
+
+#pragma unroll
+            for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
+                if (cb >= nCB) break;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float4* red_p = red + (cb & 1) * PK_CHAIN_THREADS;
+                for (int rb = 0; rb < nRB; ++rb, ++it) {
+                    const int st = it % PK_STAGES;
+                    wait_bar<false>(smem_u32(&sh->full[st]), (unsigned)((it / PK_STAGES) & 1), P, sh);
+                    if (rb == 0 && cb == 0) PK_STAMP(1);
+                    const float4* tile = reinterpret_cast<const float4*>(stages + (size_t)st * PK_STAGE_FLOATS);
+                    const float* drb = dr + rb * R + trow;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        // row trow + i*RG of the sub-tile; RG * WC4 == 128, so the float4 index is
+                        const float4 wv = tile[tid + i * PK_CHAIN_THREADS];
+                        const float d = drb[i * RG];
+                        acc.x = fmaf(wv.x, d, acc.x);
+                        acc.y = fmaf(wv.y, d, acc.y);
+                        acc.z = fmaf(wv.z, d, acc.z);
+                        acc.w = fmaf(wv.w, d, acc.w);
+                    }
+                    if (rb == nRB - 1) {
+                        // partial column sums of this column block: first the row groups that
+                        // share a warp (shuffles, fixed order), then one entry per warp
+                        for (int off = WC4; off < 32; off <<= 1) {
+                            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off);
+                            acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+                            acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
+                            acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+                        }
+                        if (lane < WC4) red_p[warp * 32 + lane] = acc;
+                    }
+                    chain_sync();   // the stage is free again (and red_p is complete)
+                    if (tid == 0 && is_it < total && !sh->abort_flag) issue_next();
+                }
+                if (cb == 0) PK_STAMP(2);
+                if (tid < WC4) {
+                    // add the warps' entries in order; warps (tid>>5), +wpr, ... hold my columns
+                    const int l5 = tid & 31;
+                    int wq = tid >> 5;
+                    float4 sum = red_p[wq * 32 + l5];
+                    for (wq += wpr; wq < PK_CHAIN_WARPS; wq += wpr) {
+                        const float4 t = red_p[wq * 32 + l5];
+                        sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+                    }
+                    // hand the four columns to the CTA that finishes them and tell it
+                    const int cs = cb * Wc + tid * 4;            // column inside the strip
+                    const int owner = cs / P.slice, off = cs - owner * P.slice;
+                    st_async_f32x4(map_to_cta(smem_u32(recv_p + c * PK_MAX_SLICE + off), (unsigned)owner), sum,
+                                   map_to_cta(smem_u32(&sh->part_ready[p]), (unsigned)owner));
                 }
             }
-            d_rows[r] = d;
+            PK_STAMP(3);
+            // the partial sums for my slice of the strip, from every CTA of the cluster
+            wait_bar<true>(smem_u32(&sh->part_ready[p]), (unsigned)(((L - s) >> 1) & 1), P, sh);
+            PK_STAMP(4);
+            if (tid < P.slice) {
+                float v = recv_p[tid];
+                for (int cc = 1; cc < C; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
+                if (my_col < N) {
+                    const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
+                    st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
+                    P.delta[(size_t)(s - 2) * N + my_col] = d;
+                    P.gb[(size_t)(s - 2) * N + my_col] = d;           // Eq. bp3
+                }
+            }
+            a_mine = a_mine_next;
+            PK_STAMP(5);
+            // delta^{s-1} of my rows, from whichever clusters finished those columns, into the
+            // other delta buffer once the store warps have let go of it
+            {
+                const int pn = (s - 1) & 1;
+                const unsigned used = (unsigned)((L - (s - 1)) >> 1);   // earlier uses of buffer pn
+                if (P.fused && used > 0) wait_bar<false>(smem_u32(&sh->d_free[pn]), (used - 1) & 1u, P, sh);
+                float* dn = d_rows + pn * PK_DROWS;
+                const unsigned long long* slots = P.xch + (size_t)(s - 2) * N;
+                for (int r0 = 0; r0 < Hr_pad; r0 += 4 * PK_CHAIN_THREADS) {
+                    unsigned long long v[4];
+                    bool want[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {      // four polls in flight per thread
+                        const int r = r0 + u * PK_CHAIN_THREADS + tid;
+                        want[u] = r < Hr && row_base + r < N;
+                        v[u] = want[u] ? ld_slot(slots + row_base + r) : 0ull;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int r = r0 + u * PK_CHAIN_THREADS + tid;
+                        if (r >= Hr_pad) continue;
+                        float d = 0.f;
+                        if (want[u])
+                            d = ((unsigned)(v[u] >> 32) == P.epoch) ? __uint_as_float((unsigned)v[u])
+                                                                   : wait_slot(slots + row_base + r, P, sh);
+                        dn[r] = d;
+                    }
+                }
+                mbar_arrive(smem_u32(&sh->d_ready[pn]));
+            }
+            chain_sync();
+            PK_STAMP(6);
         }
     }
     __syncthreads();
-
-    int it = 0;
-    for (int s = L; s >= 2; --s) {
-        // a^{s-1}: columns of my strip (for the gw^s tile) and of my slice (for sigma')
-        const float* a_prev = P.a + (size_t)(s - 1) * N;
-        float4 a4[PK_MAX_NCB];
-#pragma unroll
-        for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
-            a4[cb] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const int col = col_base + cb * Wc + tcol * 4;
-            if (cb < nCB && P.fused && col < N) a4[cb] = *reinterpret_cast<const float4*>(a_prev + col);
-        }
-        const int my_col = col_base + c * P.slice + tid;   // the column this thread finishes (tid < slice)
-        float a_mine = 0.f;
-        if (tid < P.slice && my_col < N) a_mine = a_prev[my_col];
-
-        float* gw_s = P.gw + (size_t)(s - 1) * N * N;
-        const int par = s & 1;
-        float* recv_p = recv + par * PK_CLUSTER * PK_MAX_SLICE;
-
-#pragma unroll
-        for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
-            if (cb >= nCB) break;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            const int col = col_base + cb * Wc + tcol * 4;
-            const bool col_ok = col < N;
-            for (int rb = 0; rb < nRB; ++rb, ++it) {
-                const int st = it % PK_STAGES;
-                wait_full(smem_u32(&sh->full[st]), (unsigned)((it / PK_STAGES) & 1), P, sh);
-                const float4* tile = reinterpret_cast<const float4*>(stages + (size_t)st * PK_STAGE_FLOATS);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = trow + i * RG;            // row inside the sub-tile
-                    const float4 wv = tile[r * WC4 + tcol];
-                    const int rr = rb * R + r;              // row inside my chunk
-                    const float d = d_rows[rr];
-                    acc.x = fmaf(wv.x, d, acc.x);
-                    acc.y = fmaf(wv.y, d, acc.y);
-                    acc.z = fmaf(wv.z, d, acc.z);
-                    acc.w = fmaf(wv.w, d, acc.w);
-                    if (P.fused) {
-                        const int row = row_base + rr;
-                        if (col_ok && rr < Hr && row < row_end)
-                            st_stream4(gw_s + (size_t)row * N + col,
-                                       make_float4(d * a4[cb].x, d * a4[cb].y, d * a4[cb].z, d * a4[cb].w));
-                    }
-                }
-                __syncthreads();   // every thread is done with this stage
-                if (tid == 0 && it + PK_STAGES < total && !sh->abort_flag) issue(it + PK_STAGES);
-            }
-            // partial column sums of this column block: add the RG row groups in order
-            reinterpret_cast<float4*>(red)[tid] = acc;
-            __syncthreads();
-            if (tid < WC4) {
-                float4 sum = reinterpret_cast<const float4*>(red)[tid];
-                for (int gidx = 1; gidx < RG; ++gidx) {
-                    const float4 t = reinterpret_cast<const float4*>(red)[gidx * WC4 + tid];
-                    sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
-                }
-                // hand the four columns to the CTA that finishes them
-                const int cs = cb * Wc + tid * 4;            // column inside the strip
-                const int owner = cs / P.slice, off = cs - owner * P.slice;
-                const unsigned base = map_to_cta(smem_u32(recv_p + c * PK_MAX_SLICE + off), (unsigned)owner);
-                st_cluster_f32(base + 0, sum.x);
-                st_cluster_f32(base + 4, sum.y);
-                st_cluster_f32(base + 8, sum.z);
-                st_cluster_f32(base + 12, sum.w);
-            }
-            __syncthreads();
-        }
-        cluster_sync_all();   // all partial sums of the strip have landed
-        if (tid < P.slice) {
-            float v = recv_p[tid];
-#pragma unroll
-            for (int cc = 1; cc < PK_CLUSTER; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
-            if (my_col < N) {
-                const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
-                st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
-                P.delta[(size_t)(s - 2) * N + my_col] = d;
-                P.gb[(size_t)(s - 2) * N + my_col] = d;           // Eq. bp3
-            }
-        }
-        // delta^{s-1} of my rows, from whichever clusters finished those columns
-        {
-            const unsigned long long* slots = P.xch + (size_t)(s - 2) * N;
-            for (int r = tid; r < Hr_pad; r += PK_THREADS) {
-                const int row = row_base + r;
-                float d = 0.f;
-                if (r < Hr && row < N) d = wait_slot(slots + row, P, sh);
-                d_rows[r] = d;
-            }
-        }
-        __syncthreads();
-    }
-
-    // ---- tail: gw^1 = delta^1 (x) a^0 for my tile (fused variant)
-    if (P.fused) {
-        const float* a0 = P.a;
-#pragma unroll
-        for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
-            if (cb >= nCB) break;
-            const int col = col_base + cb * Wc + tcol * 4;
-            if (col >= N) continue;
-            const float4 av = *reinterpret_cast<const float4*>(a0 + col);
-            for (int rr = trow; rr < Hr; rr += RG) {
-                const int row = row_base + rr;
-                if (row >= row_end) break;
-                const float d = d_rows[rr];
-                st_stream4(P.gw + (size_t)row * N + col, make_float4(d * av.x, d * av.y, d * av.z, d * av.w));
-            }
-        }
-    }
     cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory
 }
 
@@ -433,49 +551,51 @@ encode_tiled_fn get_encode_fn()
     return fn;
 }
 
-constexpr size_t PK_SMEM_BYTES = (size_t)PK_STAGES * PK_STAGE_FLOATS * 4 + 2304 * 4 + PK_THREADS * 16 +
-                                 2 * PK_CLUSTER * PK_MAX_SLICE * 4 + 128;
+constexpr size_t PK_SMEM_BYTES = (size_t)PK_STAGES * PK_STAGE_FLOATS * 4 + (size_t)2 * PK_DROWS * 4 +
+                                 2 * PK_CHAIN_THREADS * 16 + 2 * PK_MAX_CLUSTER * PK_MAX_SLICE * 4 + 128;
 
 struct PkPlan {
     bool ok;
-    int Qmax, Qc, Qw, Wc, nCB, Ws, Hr, R, nRB, slice;
+    int C, Qmax, Qc, Qw, Wc, nCB, Ws, Hr, R, nRB, slice;
 };
 
-int max_active_clusters(const lf_ctx* c)
+void cluster_launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int C, int clusters)
 {
-    static int cached_dev = -1, cached = 0;
-    if (cached_dev == c->device) return cached;
-    if (cudaFuncSetAttribute(k_backward_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)PK_SMEM_BYTES) != cudaSuccess) {
-        cudaGetLastError();
-        return 0;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(PK_CLUSTER * 16);
-    cfg.blockDim = dim3(PK_THREADS);
-    cfg.dynamicSmemBytes = PK_SMEM_BYTES;
-    cudaLaunchAttribute at[1];
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3(C * clusters);
+    cfg->blockDim = dim3(PK_THREADS);
+    cfg->dynamicSmemBytes = PK_SMEM_BYTES;
     at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = PK_CLUSTER; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, k_backward_persistent, &cfg) != cudaSuccess) {
-        cudaGetLastError();
-        n = 0;
+    at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg->attrs = at; cfg->numAttrs = 1;
+}
+
+// How many clusters of C CTAs (one CTA per SM at this shared-memory size) fit on the device.
+int max_active_clusters(const lf_ctx* c, int C)
+{
+    static int cached_dev = -1, cached[PK_MAX_CLUSTER + 1];
+    if (cached_dev != c->device) {
+        for (int i = 0; i <= PK_MAX_CLUSTER; ++i) cached[i] = -1;
+        cached_dev = c->device;
     }
-    cached_dev = c->device;
-    cached = n;
+    if (cached[C] >= 0) return cached[C];
+    int n = 0;
+    if (cudaFuncSetAttribute(k_backward_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)PK_SMEM_BYTES) == cudaSuccess) {
+        cudaLaunchConfig_t cfg; cudaLaunchAttribute at[1];
+        cluster_launch_config(&cfg, at, C, 16);
+        if (cudaOccupancyMaxActiveClusters(&n, k_backward_persistent, &cfg) != cudaSuccess) n = 0;
+    }
+    cudaGetLastError();
+    cached[C] = n;
     return n;
 }
 
-PkPlan make_plan(const lf_ctx* c, int variant)
+PkPlan plan_for_cluster(const lf_ctx* c, int variant, int C)
 {
     PkPlan p = {};
-    if (c->B != 1) return p;
-    if ((size_t)c->smem_optin < PK_SMEM_BYTES) return p;
-    if (!get_encode_fn()) return p;
-    p.Qmax = max_active_clusters(c);
-    if (p.Qmax > 18) p.Qmax = 18;
+    p.C = C;
+    p.Qmax = max_active_clusters(c, C);
     int Qc_budget = p.Qmax;
     if (variant == LF_VARIANT_PERSISTENT) {
         if (p.Qmax < 2) return p;
@@ -493,13 +613,31 @@ PkPlan make_plan(const lf_ctx* c, int variant)
     p.Qc = (N + p.Ws - 1) / p.Ws;
     p.Qw = variant == LF_VARIANT_PERSISTENT ? p.Qmax - p.Qc : 0;
     p.R = PK_STAGE_FLOATS / Wc;
-    p.Hr = (N + PK_CLUSTER - 1) / PK_CLUSTER;
+    p.Hr = (N + C - 1) / C;
     p.nRB = (p.Hr + p.R - 1) / p.R;
-    p.slice = p.Ws / PK_CLUSTER;
-    if (p.slice > PK_MAX_SLICE || p.nRB * p.R > 2304) return p;
+    p.slice = p.Ws / C;
+    if (p.slice > PK_MAX_SLICE || p.slice < 4 || p.nRB * p.R > PK_DROWS) return p;
     if (variant == LF_VARIANT_PERSISTENT && N > 16384) return p;
     p.ok = true;
     return p;
+}
+
+// Pick the cluster size that puts the most CTAs (SMs) to work; ties go to the larger cluster,
+// whose strips are wider.
+PkPlan make_plan(const lf_ctx* c, int variant)
+{
+    PkPlan best = {};
+    if (c->B != 1) return best;
+    if ((size_t)c->smem_optin < PK_SMEM_BYTES) return best;
+    if (!get_encode_fn()) return best;
+    int best_ctas = 0;
+    for (int C = PK_MAX_CLUSTER; C >= 2; C >>= 1) {
+        PkPlan p = plan_for_cluster(c, variant, C);
+        if (!p.ok) continue;
+        const int ctas = (p.Qc + p.Qw) * C;
+        if (ctas > best_ctas) { best = p; best_ctas = ctas; }
+    }
+    return best;
 }
 
 }  // namespace
@@ -550,7 +688,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     if (c->epoch == 0) c->epoch = 1;
 
     PkParams P = {};
-    P.L = c->L; P.N = c->N; P.Qc = pl.Qc; P.Qw = pl.Qw;
+    P.L = c->L; P.N = c->N; P.C = pl.C; P.Qc = pl.Qc; P.Qw = pl.Qw;
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch;
@@ -558,24 +696,41 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
     P.xch = reinterpret_cast<unsigned long long*>(c->sync_words);
     P.status = c->status_dev;
+#ifdef LF_PK_TRACE
+    if (!c->trace_dev) cudaMalloc(&c->trace_dev, (size_t)2 * c->L * 16 * sizeof(unsigned long long));
+    cudaMemsetAsync(c->trace_dev, 0, (size_t)2 * c->L * 16 * sizeof(unsigned long long), c->stream);
+    P.trace = c->trace_dev;
+#endif
 
     LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)PK_SMEM_BYTES));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((pl.Qc + pl.Qw) * PK_CLUSTER);
-    cfg.blockDim = dim3(PK_THREADS);
-    cfg.dynamicSmemBytes = PK_SMEM_BYTES;
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[1];
+    cluster_launch_config(&cfg, at, pl.C, pl.Qc + pl.Qw);
     cfg.stream = c->stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = PK_CLUSTER; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
     const CUtensorMap* mp = reinterpret_cast<const CUtensorMap*>(c->w_map_storage);
     LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_persistent, *mp, P));
     c->stats.launches_backward = 1;
-    c->stats.chain_ctas = pl.Qc * PK_CLUSTER;
-    c->stats.worker_ctas = pl.Qw * PK_CLUSTER;
+    c->stats.chain_ctas = pl.Qc * pl.C;
+    c->stats.worker_ctas = pl.Qw * pl.C;
     return LF_OK;
 }
 
-void lf_persistent_release(lf_ctx*) {}
+void lf_persistent_release(lf_ctx* c)
+{
+#ifdef LF_PK_TRACE
+    if (c->trace_dev) cudaFree(c->trace_dev);
+#else
+    (void)c;
+#endif
+}
+
+#ifdef LF_PK_TRACE
+// Debug builds: copy the SM-clock stamps of the last persistent launch to `out` (2 * L * 16 words).
+extern "C" int lf_debug_read_trace(lf_ctx* c, unsigned long long* out)
+{
+    if (!c || !out || !c->trace_dev) return LF_ENULL;
+    cudaStreamSynchronize(c->stream);
+    return cudaMemcpy(out, c->trace_dev, (size_t)2 * c->L * 16 * sizeof(unsigned long long),
+                      cudaMemcpyDeviceToHost) == cudaSuccess ? LF_OK : LF_ECUDA;
+}
+#endif
