@@ -67,7 +67,10 @@ enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
     LF_OPT_WAIT_BUDGET_US = 3,/* upper bound of any device-side wait, microseconds (>= 1)     */
-    LF_OPT_USE_GRAPH = 4      /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
+    LF_OPT_USE_GRAPH = 4,     /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
+    LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
+                                 publish its share of delta, so the bounded waits of the others
+                                 expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
 };
 
 typedef struct lf_stats {

@@ -18,7 +18,7 @@ LF_OK, LF_EINVAL, LF_ENULL, LF_EALIGN, LF_ERESOURCE, LF_ECUDA, LF_ETIMEOUT, LF_E
 LF_ECAPACITY = -8
 LF_VARIANT_AUTO, LF_VARIANT_STREAMS, LF_VARIANT_PERSISTENT, LF_VARIANT_FUSED = 0, 1, 2, 3
 LF_GW_MATH_AUTO, LF_GW_MATH_FP32, LF_GW_MATH_TF32 = 0, 1, 2
-LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH = 1, 2, 3, 4
+LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH, LF_OPT_WITHHOLD = 1, 2, 3, 4, 5
 
 EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
            "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",

@@ -267,6 +267,10 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value < 1 || value > 60000000LL) return LF_EINVAL;
             ctx->wait_budget_us = value;
             return LF_OK;
+        case LF_OPT_WITHHOLD:
+            if (value != 0 && value != 1) return LF_EINVAL;
+            ctx->withhold = (int)value;
+            return LF_OK;
         case LF_OPT_USE_GRAPH:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->use_graph = (int)value;

@@ -35,6 +35,7 @@ struct lf_ctx {
     int opt_gw_math;
     long long wait_budget_us;
     int use_graph;
+    int withhold;            // test hook: one chain CTA withholds its published delta values
 
     // workspace (device)
     float* partial;          // partial column sums of the delta matvec: [row_chunks][N]

@@ -54,6 +54,7 @@ struct PkParams {
     int nRB;       // row blocks per layer
     int slice;     // Ws / C
     int keff;      // effective leapfrog workers
+    int withhold;  // test hook: chain CTA 0 publishes nothing (the others' waits must expire)
     unsigned epoch;
     unsigned long long budget_ns;
     const float* a;
@@ -83,9 +84,11 @@ __device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+// The barriers armed this way guard data written by TMA or st.async, never by the arriving
+// thread itself, so the arrive carries no release fence.
 __device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
 {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cta.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(unsigned bar)
@@ -484,7 +487,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 for (int cc = 1; cc < C; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
                 if (my_col < N) {
                     const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
-                    st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
+                    if (!(P.withhold && blockIdx.x == 0)) st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
                     P.delta[(size_t)(s - 2) * N + my_col] = d;
                     P.gb[(size_t)(s - 2) * N + my_col] = d;           // Eq. bp3
                 }
@@ -691,7 +694,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.L = c->L; P.N = c->N; P.C = pl.C; P.Qc = pl.Qc; P.Qw = pl.Qw;
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
-    P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch;
+    P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
     P.xch = reinterpret_cast<unsigned long long*>(c->sync_words);
