@@ -1,9 +1,366 @@
-// TF32 tensor-core contraction for the mini-batch weight gradient (Eq. bp4 summed over samples).
+// Mini-batch weight gradient (Eq. bp4 summed over the B samples) on the 5th-generation tensor
+// cores:  G[j][k] = sum_b D[b][j] * A[b][k],  D = delta^l [B][N], A = a^{l-1} [B][N], G = gw^l.
+//
+// An N x N x B contraction whose contraction index b is the SLOW index of both operands, i.e.
+// both are "MN-major".  One persistent CTA per SM works through 128 x 256 output tiles:
+//   warp 0     TMA producer: 32 samples of D (128 columns) and of A (256 columns) per stage, as
+//              boxes of 32 floats x 32 rows in the 128-byte swizzle with 32-byte atoms -- the one
+//              shared-memory layout the tensor core accepts for MN-major 32-bit operands -- so
+//              the [B][N] arrays are used as they are, with no repacking;
+//   warp 1     issues tcgen05.mma kind::tf32 (M = 128, N = 256, K = 8 per instruction), fp32
+//              accumulators in tensor memory, two accumulator buffers of 256 columns;
+//   warps 2-5  epilogue: tcgen05.ld the finished accumulator (one 32-lane quadrant per warp)
+//              and store it to gw while the next tile is being multiplied.
+// The tensor core takes the upper 19 bits of each fp32 operand (TF32); accumulation is fp32.
+// Ragged edges: TMA fills out-of-range columns / samples with zeros, stores are bounds-checked.
+// Every mbarrier wait is bounded; on expiry the status word is raised and the CTA drains out.
+#include <cuda.h>
+
 #include "lf_internal.h"
 
-bool lf_tf32_supported(const lf_ctx*) { return false; }
-int lf_gw_gemm_tf32(lf_ctx*, const float*, const float*, float*, cudaStream_t, int*)
+namespace {
+
+constexpr int TG_BM = 128, TG_BN = 256, TG_BK = 32;      // tile and samples per stage
+constexpr int TG_STAGES = 4;
+constexpr int TG_BOX_BYTES = 32 * TG_BK * 4;             // one 32-float x 32-row box: 4 KiB
+constexpr int TG_A_BYTES = (TG_BM / 32) * TG_BOX_BYTES;  // 16 KiB
+constexpr int TG_B_BYTES = (TG_BN / 32) * TG_BOX_BYTES;  // 32 KiB
+constexpr int TG_STAGE_BYTES = TG_A_BYTES + TG_B_BYTES;  // 48 KiB
+constexpr int TG_THREADS = 192;
+constexpr int TG_TMEM_COLS = 512;                        // two accumulators of 256 fp32 columns
+constexpr size_t TG_SMEM_BYTES = (size_t)TG_STAGES * TG_STAGE_BYTES + 1024 /*alignment slack*/ + 256;
+
+struct TgParams {
+    int N, B;
+    int tiles_m, tiles_n;
+    float* gw;
+    unsigned* status;
+    unsigned long long budget_ns;
+};
+
+struct TgShared {
+    unsigned long long full[TG_STAGES];
+    unsigned long long empty[TG_STAGES];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned tmem_base;
+    volatile unsigned abort_flag;
+};
+
+__device__ __forceinline__ unsigned tg_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long tg_timer()
 {
-    return LF_EINVAL;
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
+__device__ __forceinline__ void tg_mbar_init(unsigned bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void tg_mbar_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tg_mbar_arrive(unsigned bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool tg_mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; returns false once this CTA has given up.
+__device__ __forceinline__ bool tg_wait(unsigned bar, unsigned parity, const TgParams& P, TgShared* sh)
+{
+    if (tg_mbar_try_wait(bar, parity)) return true;
+    if (sh->abort_flag) return false;
+    const unsigned long long t0 = tg_timer();
+    unsigned spins = 0;
+    while (!tg_mbar_try_wait(bar, parity)) {
+        if ((++spins & 15u) == 0u) {
+            if (sh->abort_flag) return false;
+            if (tg_timer() - t0 > P.budget_ns) {
+                atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
+                sh->abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tg_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// Shared-memory matrix descriptor of an MN-major 32-bit operand (128-byte swizzle, 32-byte
+// atoms): 32 floats (128 B) run along M/N, four consecutive samples form one 512-byte swizzle
+// atom; the next 32 columns start `lbo` bytes further, the next four samples 512 bytes further.
+__device__ __forceinline__ unsigned long long tg_make_desc(unsigned smem_addr, unsigned lbo_bytes)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);          // start address, bits [0,14)
+    d |= (unsigned long long)((lbo_bytes >> 4) & 0x3FFFu) << 16;     // leading byte offset, bits [16,30)
+    d |= (unsigned long long)((512u >> 4) & 0x3FFFu) << 32;          // stride byte offset, bits [32,46)
+    d |= 1ull << 46;                                                 // descriptor version of this architecture
+    d |= 1ull << 61;                                                 // layout type: 128-byte swizzle, 32-byte atoms
+    return d;
+}
+// Instruction descriptor of kind::tf32: fp32 accumulator, TF32 x TF32, both operands MN-major.
+__device__ __forceinline__ unsigned tg_make_idesc(int M, int Nn)
+{
+    unsigned d = 0;
+    d |= 1u << 4;                       // accumulator format: F32
+    d |= 2u << 7;                       // A format: TF32
+    d |= 2u << 10;                      // B format: TF32
+    d |= 1u << 15;                      // A is MN-major
+    d |= 1u << 16;                      // B is MN-major
+    d |= (unsigned)(Nn >> 3) << 17;     // N / 8
+    d |= (unsigned)(M >> 4) << 24;      // M / 16
+    return d;
+}
+__device__ __forceinline__ void tg_mma_tf32(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                            unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrive once all tensor-core operations issued so far by this thread have completed
+__device__ __forceinline__ void tg_commit(unsigned bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tg_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tg_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 lanes x 32 consecutive fp32 columns of tensor memory -> 32 registers per thread
+__device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(TG_THREADS, 1)
+k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_a,
+               const TgParams P)
+{
+    extern __shared__ unsigned char tg_smem_raw[];
+    // operand stages must sit on 1024-byte boundaries (the swizzle atom)
+    unsigned char* stages = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(tg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    TgShared* sh = reinterpret_cast<TgShared*>(stages + (size_t)TG_STAGES * TG_STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = P.tiles_m * P.tiles_n;
+    const int n_k = (P.B + TG_BK - 1) / TG_BK;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < TG_STAGES; ++i) {
+            tg_mbar_init(tg_smem_u32(&sh->full[i]), 1);
+            tg_mbar_init(tg_smem_u32(&sh->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            tg_mbar_init(tg_smem_u32(&sh->tmem_full[i]), 1);
+            tg_mbar_init(tg_smem_u32(&sh->tmem_empty[i]), 128);
+        }
+        sh->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // tensor memory for both accumulators
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tg_smem_u32(&sh->tmem_base)), "r"((unsigned)TG_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tg_fence_before();
+    __syncthreads();
+    tg_fence_after();
+    const unsigned tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------------------
+        if (lane == 0) {
+            unsigned it = 0;
+            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+                const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    const unsigned st = it % TG_STAGES, use = it / TG_STAGES;
+                    if (use > 0 && !tg_wait(tg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
+                    const unsigned bar = tg_smem_u32(&sh->full[st]);
+                    tg_mbar_expect_tx(bar, TG_STAGE_BYTES);
+                    const unsigned a_dst = tg_smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
+                    const unsigned b_dst = a_dst + TG_A_BYTES;
+#pragma unroll
+                    for (int i = 0; i < TG_BM / 32; ++i)
+                        tg_tma_load_2d(a_dst + i * TG_BOX_BYTES, &map_d, bar, tm * TG_BM + i * 32, ks * TG_BK);
+#pragma unroll
+                    for (int i = 0; i < TG_BN / 32; ++i)
+                        tg_tma_load_2d(b_dst + i * TG_BOX_BYTES, &map_a, bar, tn * TG_BN + i * 32, ks * TG_BK);
+                }
+                if (sh->abort_flag) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer --------------------------------------------
+        if (lane == 0) {
+            const unsigned idesc = tg_make_idesc(TG_BM, TG_BN);
+            unsigned it = 0, tile_i = 0;
+            for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_i) {
+                const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
+                if (ab_use > 0 && !tg_wait(tg_smem_u32(&sh->tmem_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
+                tg_fence_after();
+                const unsigned d_tmem = tmem_base + ab * (unsigned)TG_BN;
+                bool ok = true;
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    const unsigned st = it % TG_STAGES, use = it / TG_STAGES;
+                    if (!tg_wait(tg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    tg_fence_after();
+                    const unsigned a_addr = tg_smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
+                    const unsigned b_addr = a_addr + TG_A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < TG_BK / 8; ++kk) {      // eight samples per instruction
+                        const unsigned long long da = tg_make_desc(a_addr + kk * 1024, TG_BOX_BYTES);
+                        const unsigned long long db = tg_make_desc(b_addr + kk * 1024, TG_BOX_BYTES);
+                        tg_mma_tf32(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tg_commit(tg_smem_u32(&sh->empty[st]));      // the stage may be refilled once these are done
+                }
+                if (!ok) break;
+                tg_commit(tg_smem_u32(&sh->tmem_full[ab]));      // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (warps 2..5) ---------------------------------
+        const int quad = warp & 3;                 // the TMEM lane quadrant this warp may read
+        unsigned tile_i = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_i) {
+            const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
+            const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
+            if (!tg_wait(tg_smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
+            tg_fence_after();
+            const int row = tm * TG_BM + quad * 32 + lane;
+            float* out = P.gw + (size_t)row * P.N + (size_t)tn * TG_BN;
+#pragma unroll 1
+            for (int cchunk = 0; cchunk < TG_BN / 32; ++cchunk) {
+                unsigned r[32];
+                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TG_BN + cchunk * 32, r);
+                const int col0 = tn * TG_BN + cchunk * 32;
+                if (row < P.N) {
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        if (col0 + 4 * v < P.N)
+                            __stcs(reinterpret_cast<float4*>(out + cchunk * 32 + 4 * v),
+                                   make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                               __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+                    }
+                }
+            }
+            tg_fence_before();
+            tg_mbar_arrive(tg_smem_u32(&sh->tmem_empty[ab]));
+        }
+    }
+
+    tg_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tg_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)TG_TMEM_COLS)
+                     : "memory");
+    }
+}
+
+typedef CUresult (*tg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+tg_encode_fn tg_get_encode()
+{
+    static tg_encode_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<tg_encode_fn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// [B][N] fp32 matrix as a 2-D tensor map with 32-float x 32-row boxes, 128-byte swizzle of 32-byte atoms.
+bool tg_encode_operand(CUtensorMap* m, const float* base, int N, int B)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)B};
+    cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)TG_BK};
+    cuuint32_t estr[2] = {1, 1};
+    return tg_get_encode()(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool lf_tf32_supported(const lf_ctx* c)
+{
+    if (c->B < 2) return false;
+    if ((size_t)c->smem_optin < TG_SMEM_BYTES) return false;
+    if (!tg_get_encode()) return false;
+    // opt in to the large dynamic shared memory once per device (not during a stream capture)
+    static int attr_dev = -1;
+    if (attr_dev != c->device) {
+        if (cudaFuncSetAttribute(k_gw_gemm_tf32, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)TG_SMEM_BYTES) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        attr_dev = c->device;
+    }
+    return true;
+}
+
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, cudaStream_t s,
+                    int* launches)
+{
+    alignas(64) CUtensorMap map_d, map_a;
+    if (!tg_encode_operand(&map_d, delta_l, c->N, c->B) || !tg_encode_operand(&map_a, a_prev, c->N, c->B)) {
+        c->last_cuda_error = (int)cudaErrorInvalidValue;
+        return LF_ECUDA;
+    }
+    TgParams P;
+    P.N = c->N; P.B = c->B;
+    P.tiles_m = (c->N + TG_BM - 1) / TG_BM;
+    P.tiles_n = (c->N + TG_BN - 1) / TG_BN;
+    P.gw = gw_l;
+    P.status = c->status_dev;
+    P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
+    const int tiles = P.tiles_m * P.tiles_n;
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    k_gw_gemm_tf32<<<grid, TG_THREADS, TG_SMEM_BYTES, s>>>(map_d, map_a, P);
+    LF_CUDA_TRY(c, cudaGetLastError());
+    *launches += 1;
+    return LF_OK;
+}
+
 void lf_tf32_release(lf_ctx*) {}
