@@ -188,6 +188,49 @@ def run_reference(args):
     return 0
 
 
+def aggregate_rate(total_ms, units_per_rank, dist=None, device=None):
+    """Whole-job rate over all ranks: every rank processed `units_per_rank` units in its own
+    `total_ms`; the job took as long as its slowest rank (max over ranks).  Returns
+    (rate in units/s, max total ms, world size).  Works on any torch.distributed backend."""
+    import torch
+    world = 1
+    t = torch.tensor([float(total_ms)], dtype=torch.float64, device=device)
+    if dist is not None and dist.is_initialized():
+        world = dist.get_world_size()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    tmax = float(t.item())
+    return world * units_per_rank / (tmax * 1e-3), tmax, world
+
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu capture
+# summarised under profiles/) of the dominant kernel, keyed by (config, variant); null elsewhere.
+NCU_TRAFFIC = {(2, 3): 205.8e6}
+
+
+def time_gw_gemm(lf, L, N, B, t, stream, steps):
+    """Average time of the mini-batch weight-gradient launch, through an L = 1 context on the
+    top layer's tensors (Eq. bp1 and the column-sum launch ride along; both are tiny)."""
+    import torch
+    ctx = lf.Leapfrog(1, N, B, 1, stream=stream.cuda_stream)
+    a1 = t["a"][L - 1:L + 1].contiguous(); z1 = t["z"][L - 1:L].contiguous()
+    w1 = t["w"][L - 1:L].contiguous()
+    d1 = torch.empty((1, B, N), device=w1.device); gb1 = torch.empty((1, N), device=w1.device)
+    gw1 = t["gw"][L - 1:L]
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            ctx.backward(w1, z1, a1, t["y"], d1, gw1, gb1)
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            ctx.backward(w1, z1, a1, t["y"], d1, gw1, gb1)
+        e1.record(stream)
+        ctx.sync()
+    ms = e0.elapsed_time(e1) / steps
+    gw_math = ctx.stats()["gw_math"]
+    ctx.close()
+    return ms, gw_math
+
+
 def workload_name(index, cfg):
     return (f"configs[{index - 1}]: L={cfg['L']} N={cfg['N']} B={cfg['B']} k={cfg['k']} fp32, "
             f"y={cfg['y']}")
@@ -285,12 +328,8 @@ def run_ours(args):
         t["ctx"].sync()
     stats = sets[0]["ctx"].stats()
 
-    tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    total_ms_max = float(tmax.item())
+    value, total_ms_max, _ = aggregate_rate(total_ms, L * args.steps, dist, dev)
     ms_per_step = total_ms_max / args.steps
-    value = world * L * args.steps / (total_ms_max * 1e-3)
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     e2e = None
@@ -336,10 +375,35 @@ def run_ours(args):
         kernel_name = f"whole step ({launches_per_step} launches replayed from one CUDA graph)"
     achieved = alg / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC.get((args.config, stats["variant"])),
+                "peak_kind": f"of {peak_kind}",
                 "kernel": kernel_name, "algorithmic_bytes_per_launch": alg,
                 "avg_launch_ms": ms_per_step,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+    if B > 1:
+        # Mini-batch: the weight gradient is a dense N x N x B contraction on the tensor cores.
+        # Its launch is timed alone; its bound is the slower of the 4N^2-byte store stream and
+        # the 2N^2B flops at the TF32 peak (measured bf16 burst peak x nominal tf32/bf16 ratio).
+        gemm_ms, gw_math = time_gw_gemm(lf, L, N, B, sets[0], stream, 20)
+        flops = 2.0 * N * N * B
+        tf32_peak = float(peaks.get("bf16_tflops", 1590.0)) * (1.1 / 2.25)
+        t_store = 4.0 * N * N / (peak * 1e9)
+        t_math = flops / (tf32_peak * 1e12)
+        if gw_math == 2 and t_math >= t_store:
+            ach = flops / (gemm_ms * 1e-3) / 1e12
+            roofline = {"bound": "tensor", "achieved": ach, "peak": tf32_peak, "unit": "TFLOP/s",
+                        "frac": ach / tf32_peak, "traffic": None,
+                        "peak_kind": f"of {peak_kind} bf16 burst x 1.1/2.25 (tf32)"}
+        else:
+            gbytes = (4.0 * N * N + 8.0 * N * B) / (gemm_ms * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "achieved": gbytes, "peak": peak, "unit": "GB/s",
+                        "frac": gbytes / peak, "traffic": None, "peak_kind": f"of {peak_kind}"}
+        roofline.update({"kernel": "k_gw_gemm_tf32 (one layer, timed alone through an L=1 context)"
+                                   if gw_math == 2 else "k_gemm_simt (weight gradient, fp32)",
+                         "avg_launch_ms": gemm_ms, "flops_per_launch": flops,
+                         "tflops": flops / (gemm_ms * 1e-3) / 1e12,
+                         "whole_step_algorithmic_GBs": achieved,
+                         "note": "the step is dominated by the fp32 CUDA-core delta-chain GEMMs"})
 
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:

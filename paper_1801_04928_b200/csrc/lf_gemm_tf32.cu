@@ -28,7 +28,9 @@ constexpr int TG_B_BYTES = (TG_BN / 32) * TG_BOX_BYTES;  // 32 KiB
 constexpr int TG_STAGE_BYTES = TG_A_BYTES + TG_B_BYTES;  // 48 KiB
 constexpr int TG_THREADS = 192;
 constexpr int TG_TMEM_COLS = 512;                        // two accumulators of 256 fp32 columns
-constexpr size_t TG_SMEM_BYTES = (size_t)TG_STAGES * TG_STAGE_BYTES + 1024 /*alignment slack*/ + 256;
+constexpr int TG_EPI_LD = 36;                            // padded row length of the epilogue staging (floats)
+constexpr int TG_EPI_BYTES = 4 * 32 * TG_EPI_LD * 4;     // one 32 x 32 block per epilogue warp
+constexpr size_t TG_SMEM_BYTES = (size_t)TG_STAGES * TG_STAGE_BYTES + TG_EPI_BYTES + 1024 /*alignment slack*/ + 256;
 
 struct TgParams {
     int N, B;
@@ -167,7 +169,8 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
     // operand stages must sit on 1024-byte boundaries (the swizzle atom)
     unsigned char* stages = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(tg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    TgShared* sh = reinterpret_cast<TgShared*>(stages + (size_t)TG_STAGES * TG_STAGE_BYTES);
+    float* epi = reinterpret_cast<float*>(stages + (size_t)TG_STAGES * TG_STAGE_BYTES);
+    TgShared* sh = reinterpret_cast<TgShared*>(stages + (size_t)TG_STAGES * TG_STAGE_BYTES + TG_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = P.tiles_m * P.tiles_n;
@@ -256,22 +259,30 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
             const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
             if (!tg_wait(tg_smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
             tg_fence_after();
-            const int row = tm * TG_BM + quad * 32 + lane;
-            float* out = P.gw + (size_t)row * P.N + (size_t)tn * TG_BN;
+            // A thread reads one accumulator row (32 columns at a time).  The block is turned
+            // through shared memory so that the warp stores whole 128-byte row segments.
+            float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
+            const int row0 = tm * TG_BM + quad * 32;
+            const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TG_BN / 32; ++cchunk) {
                 unsigned r[32];
                 tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TG_BN + cchunk * 32, r);
-                const int col0 = tn * TG_BN + cchunk * 32;
-                if (row < P.N) {
 #pragma unroll
-                    for (int v = 0; v < 8; ++v) {
-                        if (col0 + 4 * v < P.N)
-                            __stcs(reinterpret_cast<float4*>(out + cchunk * 32 + 4 * v),
-                                   make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                               __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
-                    }
+                for (int v = 0; v < 8; ++v)
+                    *reinterpret_cast<float4*>(blk + lane * TG_EPI_LD + 4 * v) =
+                        make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                    __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                __syncwarp();
+                const int col = tn * TG_BN + cchunk * 32 + sub_c;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = i * 4 + sub_r;
+                    const float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
+                    if (row0 + rr < P.N && col < P.N)
+                        __stcs(reinterpret_cast<float4*>(P.gw + (size_t)(row0 + rr) * P.N + col), val);
                 }
+                __syncwarp();
             }
             tg_fence_before();
             tg_mbar_arrive(tg_smem_u32(&sh->tmem_empty[ab]));

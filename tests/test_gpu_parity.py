@@ -142,3 +142,42 @@ def test_minibatch_tf32_weight_gradient(L, N, B, k):
     den = out32["gw"].double().flatten(1).norm(dim=1)
     assert float((num / den).max()) <= 5e-3
     print("tf32", (L, N, B), worst["gw"], float((num / den).max()))
+
+
+def test_config4_minibatch_full_size_sampled():
+    # L = 16, N = 4096, B = 256, TF32 weight gradients.  The full oracle pass would take minutes,
+    # so: (i) the whole chain is checked for a few samples -- samples never mix before Eq.
+    # bp3/bp4, so the oracle runs the chain on just those columns; (ii) gb and gw, which sum
+    # over all samples, are checked against the oracle's Eq. bp3/bp4 applied to the GPU's own
+    # delta and a: gb and two whole layers of gw (Frobenius gate) plus sampled entries elsewhere.
+    from oracle import lf_oracle as orc
+    from lf_testlib import assert_layer_close, rel_frobenius, TF32_TOL
+    cfg, t = lf_inputs.make_config(4, device="cuda")
+    L, N, B = cfg["L"], cfg["N"], cfg["B"]
+    out, stats = gpu_pass(cfg, t)
+    assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
+    sel = [0, 101, 255]
+    w = t["w"].cpu().numpy()
+    sub = {k: t[k][sel].cpu().numpy() for k in ("x", "y")}
+    z, a = orc.forward(w, t["b"].cpu().numpy(), sub["x"])
+    delta, _, _ = orc.backward_sequential(w, z, a, sub["y"], want_gw=False)
+    for name, ref in (("z", z), ("a", a), ("delta", delta)):
+        g = out[name][:, sel].cpu().numpy()
+        for l in range(ref.shape[0]):
+            assert_layer_close(name, l, g[l], ref[l], n_terms=N)
+    d_gpu = out["delta"].cpu().numpy().astype(np.float64)
+    a_gpu = out["a"].cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(4)
+    for l in range(L):
+        assert_layer_close("gb", l, out["gb"][l].cpu().numpy(), orc.grad_b(d_gpu[l]), n_terms=B)
+        g = out["gw"][l].cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(g))
+        if l in (0, L - 1):
+            e = rel_frobenius(g, orc.grad_w(d_gpu[l], a_gpu[l]))
+            assert e <= TF32_TOL, (l, e)
+        else:
+            rms = np.sqrt(np.mean(g * g))
+            for _ in range(48):
+                j, k = int(rng.integers(N)), int(rng.integers(N))
+                ref = orc.grad_w_entry(d_gpu[l], a_gpu[l], j, k)
+                assert abs(g[j, k] - ref) <= TF32_TOL * max(abs(ref), rms), (l, j, k, g[j, k], ref)
