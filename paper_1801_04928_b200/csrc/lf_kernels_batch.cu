@@ -106,15 +106,32 @@ k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __
     }
 }
 
-// Eq. bp3 for a mini-batch: gb_j = sum_b delta_bj, samples added in index order.
-__global__ void k_grad_b_colsum(const float* __restrict__ delta_l, float* __restrict__ gb_l, int N,
-                                int B)
+// Eq. bp3 for a mini-batch: gb_j = sum_b delta_bj.  A CTA owns 32 columns; warp w adds the
+// samples w, w+8, ... (lanes = columns, 128-byte rows), then the eight warp sums are added in
+// warp order, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256)
+k_grad_b_colsum(const float* __restrict__ delta_l, float* __restrict__ gb_l, int N, int B)
 {
-    int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= N) return;
-    float s = 0.f;
-    for (int b = 0; b < B; ++b) s += delta_l[(size_t)b * N + j];
-    gb_l[j] = s;
+    __shared__ float part[8][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j = blockIdx.x * 32 + lane;
+    float s0 = 0.f, s1 = 0.f;
+    if (j < N) {
+        int b = warp;
+        for (; b + 8 < B; b += 16) {
+            s0 += delta_l[(size_t)b * N + j];
+            s1 += delta_l[(size_t)(b + 8) * N + j];
+        }
+        if (b < B) s0 += delta_l[(size_t)b * N + j];
+    }
+    part[warp][lane] = s0 + s1;
+    __syncthreads();
+    if (warp == 0 && j < N) {
+        float s = part[0][lane];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) s += part[q][lane];
+        gb_l[j] = s;
+    }
 }
 
 inline dim3 gemm_grid(int M, int Nn) { return dim3((Nn + BN - 1) / BN, (M + BM - 1) / BM); }
@@ -150,6 +167,6 @@ cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* g
 
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s)
 {
-    k_grad_b_colsum<<<(N + 127) / 128, 128, 0, s>>>(delta_l, gb_l, N, B);
+    k_grad_b_colsum<<<(N + 31) / 32, 256, 0, s>>>(delta_l, gb_l, N, B);
     return cudaGetLastError();
 }

@@ -1,0 +1,108 @@
+"""Sweep of the backward pass over width, batch, leapfrog workers and variant.
+
+    python -m paper_1801_04928_b200.sweep [--L 48] [--out sweep.jsonl] [--quick]
+
+For every point of the grid (L fixed; N in {256, 1024, 4096, 8192}; B in {1, 16, 128, 1024};
+k in {1, 2, 4, 8, 16}) the backward pass is timed with CUDA events for each variant that
+exists at that point: for B = 1 the stream schedule, the persistent leapfrog CTA groups and
+the fused pass; for B > 1 the stream schedule with the fp32 and the TF32 weight gradient.
+One JSON object per line is written, and a table of the fastest variant per (N, B) is printed.
+Inputs are the seeded synthetic tensors of ``lf_inputs`` drawn on the GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def time_point(lf, torch, t, L, N, B, k, variant, gw_math, steps, warmup):
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream) as ctx:
+        ctx.set_option(lf.LF_OPT_VARIANT, variant)
+        ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+            e1.record(stream)
+            ctx.sync()
+        st = ctx.stats()
+    return e0.elapsed_time(e1) / steps, st
+
+
+def main():
+    import torch
+    import lf_inputs
+    import paper_1801_04928_b200 as lf
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--L", type=int, default=lf_inputs.SWEEP["L"])
+    ap.add_argument("--out", default="sweep.jsonl")
+    ap.add_argument("--quick", action="store_true", help="k in {1, 4} only")
+    ap.add_argument("--N", type=int, nargs="*", default=list(lf_inputs.SWEEP["N"]))
+    ap.add_argument("--B", type=int, nargs="*", default=list(lf_inputs.SWEEP["B"]))
+    args = ap.parse_args()
+    ks = (1, 4) if args.quick else lf_inputs.SWEEP["k"]
+    L = args.L
+    names = {1: "streams", 2: "persistent", 3: "fused"}
+    rows = []
+    with open(args.out, "w") as f:
+        for N in args.N:
+            for B in args.B:
+                y_kind = "uniform" if B == 1 else "onehot"
+                t = lf_inputs.make_inputs(L, N, B, y_kind, lf_inputs.SEED_BASE + lf_inputs.SWEEP_CONFIG_INDEX,
+                                          "cuda")
+                t["z"] = torch.empty((L, B, N), device="cuda"); t["a"] = torch.empty((L + 1, B, N), device="cuda")
+                t["delta"] = torch.empty((L, B, N), device="cuda")
+                t["gw"] = torch.empty((L, N, N), device="cuda"); t["gb"] = torch.empty((L, N), device="cuda")
+                with lf.Leapfrog(L, N, B, 1) as ctx:
+                    ctx.forward(t["w"], t["b"], t["x"], t["z"], t["a"])
+                    ctx.sync()
+                flops = 2.0 * N * N * B
+                slow = flops * L > 2e12            # seconds per step on the fp32 chain
+                steps, warmup = (2, 1) if slow else ((5, 2) if N >= 4096 or B > 1 else (50, 5))
+                points = []
+                if B == 1:
+                    for k in ks:
+                        points += [(k, 1, lf.LF_GW_MATH_AUTO), (k, 2, lf.LF_GW_MATH_AUTO)]
+                    points.append((1, 3, lf.LF_GW_MATH_AUTO))   # the fused pass has no k
+                else:
+                    for k in ks:
+                        points.append((k, 1, lf.LF_GW_MATH_TF32))
+                    points.append((ks[-1] if len(ks) < 3 else 4, 1, lf.LF_GW_MATH_FP32))
+                for (k, variant, gw_math) in points:
+                    ms, st = time_point(lf, torch, t, L, N, B, k, variant, gw_math, steps, warmup)
+                    alg = 4.0 * N * N * (2 * L - 1) + 12.0 * N * B * L
+                    row = dict(L=L, N=N, B=B, k=k, variant=names[st["variant"]], requested=names[variant],
+                               gw_math={1: "fp32", 2: "tf32"}[st["gw_math"]], ms=ms,
+                               layers_per_s=L / (ms * 1e-3), alg_GBs=alg / (ms * 1e-3) / 1e9,
+                               chain_ctas=st["chain_ctas"], worker_ctas=st["worker_ctas"])
+                    rows.append(row)
+                    f.write(json.dumps(row) + "\n"); f.flush()
+                    print(json.dumps(row), flush=True)
+                del t
+                torch.cuda.empty_cache()
+    print("\n| N | B | fastest | k | ms | layers/s | algorithmic GB/s |")
+    print("|---|---|---|---|---|---|---|")
+    for N in args.N:
+        for B in args.B:
+            cand = [r for r in rows if r["N"] == N and r["B"] == B]
+            if not cand:
+                continue
+            b = min(cand, key=lambda r: r["ms"])
+            print(f"| {N} | {B} | {b['variant']}/{b['gw_math']} | {b['k']} | {b['ms']:.4f} | "
+                  f"{b['layers_per_s']:.0f} | {b['alg_GBs']:.0f} |")
+
+
+if __name__ == "__main__":
+    main()
