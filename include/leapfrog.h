@@ -63,11 +63,20 @@ enum lf_gw_math {
     LF_GW_MATH_TF32 = 2  /* inputs rounded to TF32, fp32 accumulation in tensor memory        */
 };
 
+/* Arithmetic of the B > 1 delta recurrence (Eq. bp2 as an N x N x B contraction). */
+enum lf_delta_math {
+    LF_DELTA_MATH_AUTO = 0,  /* tensor cores when B > 1 and the device supports it               */
+    LF_DELTA_MATH_FP32 = 1,  /* fp32 FMA on the CUDA cores                                        */
+    LF_DELTA_MATH_3XTF32 = 2 /* tensor cores; every operand split into two TF32 numbers, three
+                                products per term, fp32 accumulation: fp32-level accuracy        */
+};
+
 enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
     LF_OPT_WAIT_BUDGET_US = 3,/* upper bound of any device-side wait, microseconds (>= 1)     */
     LF_OPT_USE_GRAPH = 4,     /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
+    LF_OPT_DELTA_MATH = 6,    /* enum lf_delta_math                                           */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -85,6 +94,7 @@ typedef struct lf_stats {
     int launches_backward;    /* kernels launched by the last lf_backward                     */
     unsigned int device_status; /* status word read by the last lf_sync (0 = clean)           */
     long long workspace_bytes;  /* device memory owned by the context                         */
+    int delta_math;           /* arithmetic the last lf_backward used for Eq. bp2 (B > 1)     */
 } lf_stats;
 
 /*

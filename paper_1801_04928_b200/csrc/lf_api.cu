@@ -57,6 +57,12 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
     return LF_OK;
 }
 
+int resolve_delta_math(const lf_ctx* c)
+{
+    if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
+    return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
+}
+
 // One delta-chain step on stream s: Eq. bp1 for l = L, Eq. bp2 below.
 int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const float* y,
                        float* delta, float* gb, cudaStream_t s, int* launches)
@@ -72,7 +78,11 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
         const float* d_up = delta + (size_t)l * slab(c);
         if (B == 1)
             LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, N, s));
-        else
+        else if (c->stats.delta_math == LF_DELTA_MATH_3XTF32) {
+            int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, s, launches);
+            if (rc != LF_OK) return rc;
+            return LF_OK;
+        } else
             LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, N, B, s));
     }
     *launches += 1;
@@ -122,7 +132,7 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
         c->stats.launches_backward = launches;
         return rc;
     }
-    lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math};
+    lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math};
     if (!(c->graph_valid && c->graph_key == key)) {
         drop_graph(c);
         LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -209,6 +219,8 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
     ok = ok && cudaMalloc(&c->sync_words, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
     ws += c->sync_words_count * sizeof(unsigned);
     ok = ok && cudaMalloc(&c->status_dev, sizeof(unsigned)) == cudaSuccess; ws += sizeof(unsigned);
+    const size_t dg_bytes = lf_delta_tc_scratch_bytes(c);
+    if (dg_bytes) { ok = ok && cudaMalloc(&c->dg_partial, dg_bytes) == cudaSuccess; ws += dg_bytes; }
     ok = ok && cudaMallocHost(&c->status_host, sizeof(unsigned)) == cudaSuccess;
     if (ok) {
         ok = ok && cudaMemset(c->counters, 0, counter_bytes) == cudaSuccess;
@@ -267,6 +279,10 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value < 1 || value > 60000000LL) return LF_EINVAL;
             ctx->wait_budget_us = value;
             return LF_OK;
+        case LF_OPT_DELTA_MATH:
+            if (value < LF_DELTA_MATH_AUTO || value > LF_DELTA_MATH_3XTF32) return LF_EINVAL;
+            ctx->opt_delta_math = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -320,6 +336,7 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
         variant = LF_VARIANT_STREAMS;
     ctx->stats.variant = variant;
     ctx->stats.gw_math = gw_math;
+    ctx->stats.delta_math = resolve_delta_math(ctx);
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
@@ -424,6 +441,7 @@ int lf_destroy(lf_ctx* ctx)
     if (ctx->counters) cudaFree(ctx->counters);
     if (ctx->sync_words) cudaFree(ctx->sync_words);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
+    if (ctx->dg_partial) cudaFree(ctx->dg_partial);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     if (ctx->stage) cudaFree(ctx->stage);
     lf_persistent_release(ctx);

@@ -1,0 +1,479 @@
+// Mini-batch delta recurrence (Eq. bp2 for B > 1) on the tensor cores at fp32 accuracy:
+//     T[b][n] = sum_j D[b][j] * W[j][n],   delta^l[b][n] = T[b][n] * a^l[b][n] (1 - a^l[b][n])
+// with D = delta^{l+1} [B][N] and W = w^{l+1} [N][N] (row j, column n).
+//
+// A TF32 product keeps 11 significant bits, far too few for the 1e-5 gate on delta, so every
+// operand x is split in shared memory into hi = tf32(x) (round to nearest) and lo = x - hi
+// (exact in fp32) and three products are accumulated in fp32: lo*hi + hi*lo + hi*hi; the
+// dropped lo*lo term and the truncation of lo are of relative size 2^-22.  The tensor core
+// adds into its fp32 accumulator by truncation, which biases long accumulations (about 1e-5
+// relative after 768 instructions); therefore an accumulator in tensor memory only ever holds
+// the 12 instructions of one 32-wide K stage (small terms first), and the stage results are
+// added in registers with round-to-nearest (two accumulators in TMEM, used alternately, so
+// the adding overlaps the next stage's instructions).
+//
+// Work unit = (128 samples) x (128 columns n) x (one K split of the j range); one CTA per unit,
+// units dealt round-robin.  Warp 0: TMA producer (D as K-major 128-byte-swizzled rows, W as
+// MN-major boxes in the 128-byte swizzle with 32-byte atoms).  Warps 2-5: split each stage in
+// place (hi overwrites the raw tile, lo goes beside it), then act as the epilogue.  Warp 1:
+// issues the tcgen05.mma kind::tf32 instructions (M = 128, N = 128, K = 8), accumulator in TMEM.
+// Partial results of the K splits go to scratch; k_delta_finish adds them in split order and
+// applies sigma'.  All waits are bounded; on expiry the status word is raised.
+#include <cuda.h>
+
+#include "lf_internal.h"
+
+namespace {
+
+constexpr int DG_BM = 128, DG_BN = 128, DG_BK = 32;
+constexpr int DG_STAGES = 3;
+constexpr int DG_A_BYTES = DG_BM * DG_BK * 4;            // 16 KiB: 128 rows of 128 bytes
+constexpr int DG_BOX_BYTES = 32 * DG_BK * 4;             // 4 KiB: 32 columns x 32 rows of W
+constexpr int DG_B_BYTES = (DG_BN / 32) * DG_BOX_BYTES;  // 16 KiB
+constexpr int DG_RAW_BYTES = DG_A_BYTES + DG_B_BYTES;    // what TMA delivers per stage
+constexpr int DG_STAGE_BYTES = 2 * DG_RAW_BYTES;         // hi (in place) + lo
+constexpr int DG_THREADS = 192;
+constexpr int DG_TMEM_COLS = 256;                        // two stage accumulators of 128 columns
+constexpr int DG_EPI_LD = 36;
+constexpr int DG_EPI_BYTES = 4 * 32 * DG_EPI_LD * 4;
+constexpr size_t DG_SMEM_BYTES = (size_t)DG_STAGES * DG_STAGE_BYTES + DG_EPI_BYTES + 1024 + 256;
+
+struct DgParams {
+    int N, B;
+    int tiles_m, tiles_n, splits;
+    int k_per_split;          // j range of one split (multiple of DG_BK)
+    float* partial;           // [splits][B][N]
+    unsigned* status;
+    unsigned long long budget_ns;
+};
+
+struct DgShared {
+    unsigned long long full[DG_STAGES];    // TMA landed
+    unsigned long long split_done[DG_STAGES];  // hi/lo written (128 arrivals)
+    unsigned long long empty[DG_STAGES];   // MMAs that read the stage are done
+    unsigned long long acc_full[2], acc_empty[2];   // stage accumulator p holds a finished stage / is drained
+    unsigned tmem_base;
+    volatile unsigned abort_flag;
+};
+
+__device__ __forceinline__ unsigned dg_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long dg_timer()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void dg_mbar_init(unsigned bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void dg_mbar_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void dg_mbar_arrive(unsigned bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool dg_mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool dg_wait(unsigned bar, unsigned parity, const DgParams& P, DgShared* sh)
+{
+    if (dg_mbar_try_wait(bar, parity)) return true;
+    if (sh->abort_flag) return false;
+    const unsigned long long t0 = dg_timer();
+    unsigned spins = 0;
+    while (!dg_mbar_try_wait(bar, parity)) {
+        if ((++spins & 15u) == 0u) {
+            if (sh->abort_flag) return false;
+            if (dg_timer() - t0 > P.budget_ns) {
+                atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
+                sh->abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void dg_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// K-major operand, 128-byte swizzle: rows of 128 bytes (32 floats along K), eight rows per
+// 1024-byte atom (SBO); one instruction consumes 32 bytes of every row.
+__device__ __forceinline__ unsigned long long dg_desc_kmajor(unsigned smem_addr)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (unsigned long long)1 << 16;                                // LBO: not used by swizzled K-major
+    d |= (unsigned long long)((1024u >> 4) & 0x3FFFu) << 32;         // SBO: next group of eight rows
+    d |= 1ull << 46;
+    d |= 2ull << 61;                                                 // 128-byte swizzle
+    return d;
+}
+// MN-major 32-bit operand, 128-byte swizzle with 32-byte atoms: 32 floats along N per row,
+// four K rows per 512-byte atom (SBO), next 32 columns 4 KiB further (LBO).
+__device__ __forceinline__ unsigned long long dg_desc_mnmajor(unsigned smem_addr)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (unsigned long long)((DG_BOX_BYTES >> 4) & 0x3FFFu) << 16;
+    d |= (unsigned long long)((512u >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= 1ull << 61;
+    return d;
+}
+__device__ __forceinline__ unsigned dg_idesc()
+{
+    unsigned d = 0;
+    d |= 1u << 4;                             // fp32 accumulator
+    d |= 2u << 7;                             // A: TF32
+    d |= 2u << 10;                            // B: TF32
+    d |= 0u << 15;                            // A is K-major
+    d |= 1u << 16;                            // B is MN-major
+    d |= (unsigned)(DG_BN >> 3) << 17;
+    d |= (unsigned)(DG_BM >> 4) << 24;
+    return d;
+}
+__device__ __forceinline__ void dg_mma(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                       unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void dg_commit(unsigned bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void dg_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void dg_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ float dg_tf32_rn(float x)
+{
+    unsigned r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ void dg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(DG_THREADS, 1)
+k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_w,
+                const DgParams P)
+{
+    extern __shared__ unsigned char dg_smem_raw[];
+    unsigned char* stages = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(dg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    float* epi = reinterpret_cast<float*>(stages + (size_t)DG_STAGES * DG_STAGE_BYTES);
+    DgShared* sh = reinterpret_cast<DgShared*>(stages + (size_t)DG_STAGES * DG_STAGE_BYTES + DG_EPI_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_units = P.tiles_m * P.tiles_n * P.splits;
+    const int n_k = P.k_per_split / DG_BK;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < DG_STAGES; ++i) {
+            dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 128);
+            dg_mbar_init(dg_smem_u32(&sh->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            dg_mbar_init(dg_smem_u32(&sh->acc_full[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->acc_empty[i]), 128);
+        }
+        sh->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(dg_smem_u32(&sh->tmem_base)), "r"((unsigned)DG_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    dg_fence_before();
+    __syncthreads();
+    dg_fence_after();
+    const unsigned tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------------------
+        if (lane == 0) {
+            unsigned it = 0;
+            for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+                const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
+                const int j0 = sp * P.k_per_split;
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
+                    if (use > 0 && !dg_wait(dg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
+                    const unsigned bar = dg_smem_u32(&sh->full[st]);
+                    dg_mbar_expect_tx(bar, DG_RAW_BYTES);
+                    const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
+                    dg_tma_load_2d(a_dst, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM);
+#pragma unroll
+                    for (int i = 0; i < DG_BN / 32; ++i)
+                        dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
+                                       j0 + ks * DG_BK);
+                }
+                if (sh->abort_flag) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer --------------------------------------------
+        if (lane == 0) {
+            const unsigned idesc = dg_idesc();
+            unsigned it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
+                    const unsigned p = it & 1u, p_use = it >> 1;
+                    if (!dg_wait(dg_smem_u32(&sh->split_done[st]), use & 1u, P, sh)) { ok = false; break; }
+                    if (p_use > 0 && !dg_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
+                    dg_fence_after();
+                    const unsigned hi = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
+                    const unsigned lo = hi + DG_RAW_BYTES;
+                    const unsigned d_tmem = tmem_base + p * (unsigned)DG_BN;
+                    // the eight small products first, then the four large ones
+#pragma unroll
+                    for (int kk = 0; kk < DG_BK / 8; ++kk) {
+                        dg_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_mnmajor(hi + DG_A_BYTES + kk * 1024), idesc,
+                               kk > 0 ? 1u : 0u);
+                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_mnmajor(lo + DG_A_BYTES + kk * 1024), idesc, 1u);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < DG_BK / 8; ++kk)
+                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_mnmajor(hi + DG_A_BYTES + kk * 1024), idesc, 1u);
+                    dg_commit(dg_smem_u32(&sh->empty[st]));
+                    dg_commit(dg_smem_u32(&sh->acc_full[p]));
+                }
+            }
+        }
+    } else {
+        // ---------------- operand split (hi/lo) and epilogue: warps 2..5 ----------------------
+        const int tt = threadIdx.x - 64;
+        const int quad = warp & 3;
+        unsigned it = 0;
+        bool ok = true;
+        float acc[DG_BN];      // this thread's output row (sample), all 128 columns of the tile
+        // add the finished stage `j` (accumulator j & 1) into the registers; first == overwrite
+        auto drain = [&](unsigned j, bool first) -> bool {
+            const unsigned p = j & 1u;
+            if (!dg_wait(dg_smem_u32(&sh->acc_full[p]), (j >> 1) & 1u, P, sh)) return false;
+            dg_fence_after();
+#pragma unroll
+            for (int cchunk = 0; cchunk < DG_BN / 32; ++cchunk) {
+                unsigned r[32];
+                dg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DG_BN + cchunk * 32, r);
+#pragma unroll
+                for (int v = 0; v < 32; ++v)
+                    acc[cchunk * 32 + v] = first ? __uint_as_float(r[v]) : acc[cchunk * 32 + v] + __uint_as_float(r[v]);
+            }
+            dg_fence_before();
+            dg_mbar_arrive(dg_smem_u32(&sh->acc_empty[p]));
+            return true;
+        };
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
+            for (int ks = 0; ks < n_k; ++ks, ++it) {
+                const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
+                if (!dg_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DG_STAGE_BYTES);
+                float4* lo = reinterpret_cast<float4*>(stages + (size_t)st * DG_STAGE_BYTES + DG_RAW_BYTES);
+#pragma unroll 4
+                for (int i = 0; i < DG_RAW_BYTES / 16 / 128; ++i) {
+                    const int idx = tt + i * 128;
+                    const float4 v = raw[idx];
+                    const float4 h = make_float4(dg_tf32_rn(v.x), dg_tf32_rn(v.y), dg_tf32_rn(v.z), dg_tf32_rn(v.w));
+                    raw[idx] = h;
+                    lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+                }
+                // the tensor core reads shared memory through the async proxy
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                dg_mbar_arrive(dg_smem_u32(&sh->split_done[st]));
+                if (ks > 0 && !drain(it - 1, ks == 1)) { ok = false; break; }
+            }
+            if (!ok) break;
+            if (!drain(it - 1, n_k == 1)) { ok = false; break; }
+            float* blk = epi + (warp - 2) * 32 * DG_EPI_LD;
+            const int row0 = tm * DG_BM + quad * 32;
+            const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
+            float* out = P.partial + (size_t)sp * P.B * P.N;
+#pragma unroll
+            for (int cchunk = 0; cchunk < DG_BN / 32; ++cchunk) {
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    *reinterpret_cast<float4*>(blk + lane * DG_EPI_LD + 4 * v) =
+                        make_float4(acc[cchunk * 32 + 4 * v], acc[cchunk * 32 + 4 * v + 1],
+                                    acc[cchunk * 32 + 4 * v + 2], acc[cchunk * 32 + 4 * v + 3]);
+                __syncwarp();
+                const int col = tn * DG_BN + cchunk * 32 + sub_c;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = i * 4 + sub_r;
+                    const float4 val = *reinterpret_cast<const float4*>(blk + rr * DG_EPI_LD + sub_c);
+                    if (row0 + rr < P.B && col < P.N)
+                        *reinterpret_cast<float4*>(out + (size_t)(row0 + rr) * P.N + col) = val;
+                }
+                __syncwarp();
+            }
+        }
+    }
+
+    dg_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        dg_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DG_TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// delta^l = (sum over the K splits, in split order) * sigma'(z^l), sigma' = a (1 - a)
+__global__ void __launch_bounds__(256)
+k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
+               size_t n4, int splits)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 s = reinterpret_cast<const float4*>(partial)[i];
+    for (int sp = 1; sp < splits; ++sp) {
+        const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
+        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+    const float4 av = reinterpret_cast<const float4*>(a_l)[i];
+    reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * (av.x * (1.0f - av.x)), s.y * (av.y * (1.0f - av.y)),
+                                                        s.z * (av.z * (1.0f - av.z)), s.w * (av.w * (1.0f - av.w)));
+}
+
+typedef CUresult (*dg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+dg_encode_fn dg_get_encode()
+{
+    static dg_encode_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<dg_encode_fn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+struct DgPlan { int tiles_m, tiles_n, splits, k_per_split; };
+
+DgPlan dg_plan(const lf_ctx* c)
+{
+    DgPlan p;
+    p.tiles_m = (c->B + DG_BM - 1) / DG_BM;
+    p.tiles_n = (c->N + DG_BN - 1) / DG_BN;
+    int s = c->sm_count / (p.tiles_m * p.tiles_n);
+    if (s < 1) s = 1;
+    if (s > 8) s = 8;
+    const int kb = (c->N + DG_BK - 1) / DG_BK;            // K blocks in all
+    if (s > kb) s = kb;
+    const int kb_per = (kb + s - 1) / s;
+    p.splits = (kb + kb_per - 1) / kb_per;                 // no empty split
+    p.k_per_split = kb_per * DG_BK;
+    return p;
+}
+
+}  // namespace
+
+size_t lf_delta_tc_scratch_bytes(const lf_ctx* c)
+{
+    if (c->B < 2) return 0;
+    DgPlan p = dg_plan(c);
+    return (size_t)p.splits * c->B * c->N * sizeof(float);
+}
+
+bool lf_delta_tc_supported(const lf_ctx* c)
+{
+    if (c->B < 2 || !c->dg_partial) return false;
+    if ((size_t)c->smem_optin < DG_SMEM_BYTES) return false;
+    if (!dg_get_encode()) return false;
+    static int attr_dev = -1;
+    if (attr_dev != c->device) {
+        if (cudaFuncSetAttribute(k_delta_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)DG_SMEM_BYTES) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        attr_dev = c->device;
+    }
+    return true;
+}
+
+int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
+                     cudaStream_t s, int* launches)
+{
+    alignas(64) CUtensorMap map_d, map_w;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)c->N, (cuuint64_t)c->B};
+        cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
+        cuuint32_t box[2] = {32, (cuuint32_t)DG_BM};
+        cuuint32_t estr[2] = {1, 1};
+        if (dg_get_encode()(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(delta_up), dims, strides,
+                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            c->last_cuda_error = (int)cudaErrorInvalidValue;
+            return LF_ECUDA;
+        }
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)c->N, (cuuint64_t)c->N};
+        cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
+        cuuint32_t box[2] = {32, (cuuint32_t)DG_BK};
+        cuuint32_t estr[2] = {1, 1};
+        if (dg_get_encode()(&map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(w_up), dims, strides, box,
+                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            c->last_cuda_error = (int)cudaErrorInvalidValue;
+            return LF_ECUDA;
+        }
+    }
+    const DgPlan pl = dg_plan(c);
+    DgParams P;
+    P.N = c->N; P.B = c->B;
+    P.tiles_m = pl.tiles_m; P.tiles_n = pl.tiles_n; P.splits = pl.splits; P.k_per_split = pl.k_per_split;
+    P.partial = c->dg_partial;
+    P.status = c->status_dev;
+    P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
+    const int units = pl.tiles_m * pl.tiles_n * pl.splits;
+    const int grid = units < c->sm_count ? units : c->sm_count;
+    k_delta_gemm_tc<<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);
+    LF_CUDA_TRY(c, cudaGetLastError());
+    const size_t n4 = (size_t)c->B * c->N / 4;
+    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, pl.splits);
+    LF_CUDA_TRY(c, cudaGetLastError());
+    *launches += 2;
+    return LF_OK;
+}

@@ -35,6 +35,7 @@ struct lf_ctx {
     int opt_gw_math;
     long long wait_budget_us;
     int use_graph;
+    int opt_delta_math;      // enum lf_delta_math
     int withhold;            // test hook: one chain CTA withholds its published delta values
 
     // workspace (device)
@@ -44,7 +45,7 @@ struct lf_ctx {
     size_t sync_words_count;
     unsigned* status_dev;    // device status word
     unsigned* status_host;   // pinned mirror
-    float* tf32_scratch;     // reserved for operand repacking of the tensor-core path
+    float* dg_partial;       // B > 1: K-split partial sums of the tensor-core delta GEMM
 
     // leapfrog workers as streams
     cudaStream_t* wstreams;  // keff streams
@@ -122,3 +123,9 @@ bool lf_tf32_supported(const lf_ctx* c);
 int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l,
                     cudaStream_t s, int* launches);
 void lf_tf32_release(lf_ctx* c);
+
+// ---- 3xTF32 tensor-core delta recurrence (B > 1) ----------------------------------------------
+size_t lf_delta_tc_scratch_bytes(const lf_ctx* c);
+bool lf_delta_tc_supported(const lf_ctx* c);
+int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
+                     cudaStream_t s, int* launches);

@@ -37,13 +37,17 @@ def test_single_sample_parity(L, N, k, variant):
     assert torch.equal(out["gb"], out["delta"][:, 0])  # Eq. bp3, single sample
 
 
+@pytest.mark.parametrize("delta_math", [lf.LF_DELTA_MATH_FP32, lf.LF_DELTA_MATH_3XTF32])
 @pytest.mark.parametrize("L,N,B,k", [(2, 8, 2, 1), (3, 68, 3, 2), (3, 256, 16, 4),
-                                     (4, 132, 70, 3), (2, 320, 129, 2)])
-def test_minibatch_fp32_parity(L, N, B, k):
+                                     (4, 132, 70, 3), (2, 320, 129, 2), (5, 1028, 260, 2)])
+def test_minibatch_fp32_parity(L, N, B, k, delta_math):
+    # fp32 gate (1e-5 per tensor per layer) for both forms of the delta recurrence: fp32 on
+    # the CUDA cores, and the tensor cores with every operand split into two TF32 numbers.
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=N + B)
-    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32)
-    assert stats["gw_math"] == lf.LF_GW_MATH_FP32
+    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math)
+    assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == delta_math
+    assert stats["device_status"] == 0
     ref = oracle_pass(t, want_gw=True)
     compare_all(cfg, out, ref)
 
