@@ -416,6 +416,9 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         }
         chain_sync();
 
+        // With one column block and at most 32 columns to finish per CTA the four chain warps
+        // send their partial sums straight to the finishing CTA (recv then holds C*4 rows of 32).
+        const bool direct = nCB == 1 && P.slice <= 32;
         int it = 0;
         for (int s = L; s >= 2; --s) {
             PK_STAMP(0);
@@ -423,8 +426,11 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             const float* dr = d_rows + p * PK_DROWS;
             float* recv_p = recv + p * PK_MAX_CLUSTER * PK_MAX_SLICE;
             const float a_mine_next = (finisher && s >= 3) ? P.a[(size_t)(s - 2) * N + my_col] : 0.f;
-            // this step's partial sums for my slice: C CTAs x slice floats will be credited
-            if (tid == 0) mbar_expect_tx(smem_u32(&sh->part_ready[p]), (unsigned)(C * P.slice * sizeof(float)));
+            // this step's partial sums for my slice will be credited: slice floats from every
+            // CTA of the cluster (from each of its four chain warps on the direct path)
+            if (tid == 0)
+                mbar_expect_tx(smem_u32(&sh->part_ready[p]),
+                               (unsigned)(C * P.slice * sizeof(float)) * (direct ? PK_CHAIN_WARPS : 1));
 
 #pragma unroll
             for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
@@ -456,13 +462,24 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                             acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off);
                             acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
                         }
-                        if (lane < WC4) red_p[warp * 32 + lane] = acc;
+                        if (direct) {
+                            // narrow strip: every warp hands its own partial sums to the finishing CTA
+                            if (lane < WC4) {
+                                const int cs = lane * 4;
+                                const int owner = cs / P.slice, off = cs - owner * P.slice;
+                                st_async_f32x4(map_to_cta(smem_u32(recv_p + (c * PK_CHAIN_WARPS + warp) * 32 + off),
+                                                          (unsigned)owner),
+                                               acc, map_to_cta(smem_u32(&sh->part_ready[p]), (unsigned)owner));
+                            }
+                        } else if (lane < WC4) {
+                            red_p[warp * 32 + lane] = acc;
+                        }
                     }
                     chain_sync();   // the stage is free again (and red_p is complete)
                     if (tid == 0 && is_it < total && !sh->abort_flag) issue_next();
                 }
                 if (cb == 0) PK_STAMP(2);
-                if (tid < WC4) {
+                if (!direct && tid < WC4) {
                     // add the warps' entries in order; warps (tid>>5), +wpr, ... hold my columns
                     const int l5 = tid & 31;
                     int wq = tid >> 5;
@@ -484,7 +501,10 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             PK_STAMP(4);
             if (tid < P.slice) {
                 float v = recv_p[tid];
-                for (int cc = 1; cc < C; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
+                if (direct)
+                    for (int cc = 1; cc < C * PK_CHAIN_WARPS; ++cc) v += recv_p[cc * 32 + tid];
+                else
+                    for (int cc = 1; cc < C; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
                 if (my_col < N) {
                     const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
                     if (!(P.withhold && blockIdx.x == 0)) st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
@@ -504,22 +524,46 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 const unsigned long long* slots = P.xch + (size_t)(s - 2) * N;
                 for (int r0 = 0; r0 < Hr_pad; r0 += 4 * PK_CHAIN_THREADS) {
                     unsigned long long v[4];
-                    bool want[4];
+                    bool pend[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {      // four polls in flight per thread
+                    for (int u = 0; u < 4; ++u) {      // up to four polls in flight per thread
                         const int r = r0 + u * PK_CHAIN_THREADS + tid;
-                        want[u] = r < Hr && row_base + r < N;
-                        v[u] = want[u] ? ld_slot(slots + row_base + r) : 0ull;
+                        pend[u] = r < Hr && row_base + r < N;
+                        v[u] = pend[u] ? ld_slot(slots + row_base + r) : 0ull;
+                    }
+                    // poll whatever is still missing, all of it together, until it is there
+                    unsigned long long t0 = 0;
+                    unsigned rounds = 0;
+                    for (;;) {
+                        bool any = false;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (pend[u]) {
+                                if ((unsigned)(v[u] >> 32) == P.epoch) pend[u] = false;
+                                else { v[u] = ld_slot(slots + row_base + r0 + u * PK_CHAIN_THREADS + tid); any = true; }
+                            }
+                        }
+                        if (!any) break;
+                        bool give_up = sh->abort_flag != 0u;
+                        if (!give_up && (++rounds & 15u) == 0u) {
+                            const unsigned long long now = globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            if (now - t0 > P.budget_ns || *((volatile unsigned*)P.status) != 0u) {
+                                raise_timeout(P, sh, LF_DEV_TIMEOUT_FLAG);
+                                give_up = true;
+                            }
+                        }
+                        if (give_up) {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (pend[u]) v[u] = 0ull;
+                            break;
+                        }
                     }
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const int r = r0 + u * PK_CHAIN_THREADS + tid;
-                        if (r >= Hr_pad) continue;
-                        float d = 0.f;
-                        if (want[u])
-                            d = ((unsigned)(v[u] >> 32) == P.epoch) ? __uint_as_float((unsigned)v[u])
-                                                                   : wait_slot(slots + row_base + r, P, sh);
-                        dn[r] = d;
+                        if (r < Hr_pad) dn[r] = __uint_as_float((unsigned)v[u]);
                     }
                 }
                 mbar_arrive(smem_u32(&sh->d_ready[pn]));
