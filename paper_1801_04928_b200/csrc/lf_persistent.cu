@@ -500,11 +500,17 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             wait_bar<true>(smem_u32(&sh->part_ready[p]), (unsigned)(((L - s) >> 1) & 1), P, sh);
             PK_STAMP(4);
             if (tid < P.slice) {
-                float v = recv_p[tid];
-                if (direct)
-                    for (int cc = 1; cc < C * PK_CHAIN_WARPS; ++cc) v += recv_p[cc * 32 + tid];
-                else
-                    for (int cc = 1; cc < C; ++cc) v += recv_p[cc * PK_MAX_SLICE + tid];
+                // add the partial sums in a fixed order (loads issued together, adds in sequence)
+                const int n_src = direct ? C * PK_CHAIN_WARPS : C;
+                const int src_ld = direct ? 32 : PK_MAX_SLICE;
+                float part[PK_MAX_CLUSTER * PK_CHAIN_WARPS];
+#pragma unroll
+                for (int cc = 0; cc < PK_MAX_CLUSTER * PK_CHAIN_WARPS; ++cc)
+                    part[cc] = cc < n_src ? recv_p[cc * src_ld + tid] : 0.f;
+                float v = part[0];
+#pragma unroll
+                for (int cc = 1; cc < PK_MAX_CLUSTER * PK_CHAIN_WARPS; ++cc)
+                    if (cc < n_src) v += part[cc];
                 if (my_col < N) {
                     const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
                     if (!(P.withhold && blockIdx.x == 0)) st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
