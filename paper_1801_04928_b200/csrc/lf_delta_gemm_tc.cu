@@ -238,6 +238,14 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                 }
                 if (sh->abort_flag) break;
             }
+            // after giving up: do not let the CTA exit under loads that are still landing
+            if (sh->abort_flag) {
+                const unsigned long long t0 = dg_timer();
+                for (unsigned j = it > DG_STAGES ? it - DG_STAGES : 0; j < it; ++j) {
+                    const unsigned bar = dg_smem_u32(&sh->full[j % DG_STAGES]);
+                    while (!dg_mbar_try_wait(bar, (j / DG_STAGES) & 1u) && dg_timer() - t0 < 50000000ull) { }
+                }
+            }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------------------

@@ -220,6 +220,14 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                 }
                 if (sh->abort_flag) break;
             }
+            // after giving up: do not let the CTA exit under loads that are still landing
+            if (sh->abort_flag) {
+                const unsigned long long t0 = tg_timer();
+                for (unsigned j = it > TG_STAGES ? it - TG_STAGES : 0; j < it; ++j) {
+                    const unsigned bar = tg_smem_u32(&sh->full[j % TG_STAGES]);
+                    while (!tg_mbar_try_wait(bar, (j / TG_STAGES) & 1u) && tg_timer() - t0 < 50000000ull) { }
+                }
+            }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------------------

@@ -418,7 +418,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
 
         // With one column block and at most 32 columns to finish per CTA the four chain warps
         // send their partial sums straight to the finishing CTA (recv then holds C*4 rows of 32).
-        const bool direct = nCB == 1 && P.slice <= 32;
+        const bool direct = nCB == 1 && WC4 <= 32 && P.slice <= 32;   // (every warp must span the whole strip)
         int it = 0;
         for (int s = L; s >= 2; --s) {
             PK_STAMP(0);
@@ -576,6 +576,16 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             }
             chain_sync();
             PK_STAMP(6);
+        }
+        // A CTA that gave up waiting gets here with weight tiles possibly still on their way into
+        // its shared memory; it must not exit under them.  Wait for the last loads, with a limit.
+        if (tid == 0 && sh->abort_flag) {
+            const unsigned long long t0 = globaltimer_ns();
+            for (int j = is_it > PK_STAGES ? is_it - PK_STAGES : 0; j < is_it; ++j) {
+                const unsigned bar = smem_u32(&sh->full[j % PK_STAGES]);
+                const unsigned parity = (unsigned)((j / PK_STAGES) & 1);
+                while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < 50000000ull) { }
+            }
         }
     }
     __syncthreads();

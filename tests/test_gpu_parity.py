@@ -21,7 +21,7 @@ def _inputs(L, N, B, y="uniform", seed=1):
 # sizes: below one tile, exactly one strip, several strips with a ragged tail, N not a
 # multiple of 128, L < k, L = 1.
 SMALL_B1 = [(1, 4, 1), (2, 8, 3), (3, 64, 2), (5, 260, 4), (4, 516, 16), (6, 1024, 3),
-            (3, 1156, 2), (2, 2052, 1)]
+            (3, 1156, 2), (2, 2052, 1), (3, 3072, 2)]   # 3072: 256-column strips, 32 columns per finisher
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
