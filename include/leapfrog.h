@@ -140,10 +140,14 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
                 float* delta, float* gw, float* gb);
 
 /*
- * The same backward pass on HOST buffers (pageable or pinned; same layouts): copies w, z, a,
- * y to device staging owned by the context (allocated on first use, counted in
- * workspace_bytes), runs lf_backward, copies delta, gw, gb back, all on the context's
- * stream.  The host buffers must stay valid until lf_sync() returns.
+ * The same backward pass on HOST buffers (pageable or pinned; same layouts): w, z, a, y are
+ * copied to device staging owned by the context (allocated on first use, counted in
+ * workspace_bytes), delta, gw, gb are copied back.  The copies are pipelined with the per-layer
+ * schedule (LF_VARIANT_STREAMS): weights arrive top layer first on a copy stream, layer l is
+ * processed as soon as w^{l+1} is there, and gw^l is sent back as soon as its worker has
+ * written it, so both PCIe directions are busy at once (use pinned memory for that).  All work
+ * is joined back into the context's stream.  The host buffers must stay valid until
+ * lf_sync() returns.
  */
 int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a,
                      const float* y, float* delta, float* gw, float* gb);

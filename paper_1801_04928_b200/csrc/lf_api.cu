@@ -372,16 +372,62 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     float* d_d = d_y + n_y;
     float* d_gw = d_d + n_d;
     float* d_gb = d_gw + n_gw;
-    cudaStream_t s = ctx->stream;
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w, w, n_w * sizeof(float), cudaMemcpyHostToDevice, s));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_z, z, n_z * sizeof(float), cudaMemcpyHostToDevice, s));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, s));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, s));
-    int rc = lf_backward(ctx, d_w, d_z, d_a, d_y, d_d, d_gw, d_gb);
-    if (rc != LF_OK) return rc;
+    // copy stream and per-layer arrival events (created on first use)
+    if (!ctx->h2d_stream) {
+        LF_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking));
+        ctx->w_ready_ev = new (std::nothrow) cudaEvent_t[ctx->L]();
+        if (!ctx->w_ready_ev) return LF_ENOMEM;
+        for (int l = 0; l < ctx->L; ++l)
+            LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->w_ready_ev[l], cudaEventDisableTiming));
+        LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->small_ev, cudaEventDisableTiming));
+        LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->h2d_done_ev, cudaEventDisableTiming));
+    }
+    // The copies are pipelined with the per-layer schedule: the weights arrive top layer
+    // first on a copy stream, the chain step of layer l starts as soon as w^{l+1} is there,
+    // and the worker that finishes gw^l sends it back at once, so the two PCIe directions
+    // are busy at the same time.
+    cudaStream_t s = ctx->stream, hs = ctx->h2d_stream;
+    const int Li = ctx->L;
+    const int gw_math = resolve_gw_math(ctx);
+    ctx->stats.variant = LF_VARIANT_STREAMS;
+    ctx->stats.gw_math = gw_math;
+    ctx->stats.delta_math = resolve_delta_math(ctx);
+    int launches = 0;
+    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
+    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(hs, ctx->fork_ev, 0));
+    for (int j = 0; j < ctx->keff; ++j) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->wstreams[j], ctx->fork_ev, 0));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_z, z, n_z * sizeof(float), cudaMemcpyHostToDevice, hs));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, hs));
+    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, hs));
+    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, hs));
+    for (int l = Li; l >= 1; --l) {
+        LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w + (size_t)(l - 1) * M, w + (size_t)(l - 1) * M, M * sizeof(float),
+                                         cudaMemcpyHostToDevice, hs));
+        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->w_ready_ev[l - 1], hs));
+    }
+    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->h2d_done_ev, hs));
+    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->small_ev, 0));
+    for (int l = Li; l >= 1; --l) {
+        if (l < Li) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0));   // w^{l+1}
+        int rc = enqueue_chain_step(ctx, l, d_w, d_a, d_y, d_d, d_gb, s, &launches);
+        if (rc != LF_OK) return rc;
+        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->ready_ev[l - 1], s));
+        const int j = (Li - l) % ctx->keff;
+        cudaStream_t wsj = ctx->wstreams[j];
+        LF_CUDA_TRY(ctx, cudaStreamWaitEvent(wsj, ctx->ready_ev[l - 1], 0));
+        rc = enqueue_gradients(ctx, l, d_a, d_d, d_gw, d_gb, gw_math, wsj, &launches);
+        if (rc != LF_OK) return rc;
+        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw + (size_t)(l - 1) * M, d_gw + (size_t)(l - 1) * M, M * sizeof(float),
+                                         cudaMemcpyDeviceToHost, wsj));
+    }
+    for (int j = 0; j < ctx->keff; ++j) {
+        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->done_ev[j], ctx->wstreams[j]));
+        LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->done_ev[j], 0));
+    }
+    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->h2d_done_ev, 0));
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(delta, d_d, n_d * sizeof(float), cudaMemcpyDeviceToHost, s));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw, d_gw, n_gw * sizeof(float), cudaMemcpyDeviceToHost, s));
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, s));
+    ctx->stats.launches_backward = launches;
     return LF_OK;
 }
 
@@ -444,6 +490,14 @@ int lf_destroy(lf_ctx* ctx)
     if (ctx->dg_partial) cudaFree(ctx->dg_partial);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->h2d_stream) { cudaStreamSynchronize(ctx->h2d_stream); cudaStreamDestroy(ctx->h2d_stream); }
+    if (ctx->w_ready_ev) {
+        for (int l = 0; l < ctx->L; ++l)
+            if (ctx->w_ready_ev[l]) cudaEventDestroy(ctx->w_ready_ev[l]);
+        delete[] ctx->w_ready_ev;
+    }
+    if (ctx->small_ev) cudaEventDestroy(ctx->small_ev);
+    if (ctx->h2d_done_ev) cudaEventDestroy(ctx->h2d_done_ev);
     lf_persistent_release(ctx);
     lf_tf32_release(ctx);
     delete ctx;

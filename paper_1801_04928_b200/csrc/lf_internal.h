@@ -72,6 +72,9 @@ struct lf_ctx {
     // host-buffer entry point staging
     float* stage;            // one allocation holding w, z, a, y, delta, gw, gb
     size_t stage_bytes;
+    cudaStream_t h2d_stream; // host -> device copies of the host entry point
+    cudaEvent_t* w_ready_ev; // L events: w^l has arrived in staging
+    cudaEvent_t small_ev, h2d_done_ev;
 
     int last_cuda_error;
     lf_stats stats;

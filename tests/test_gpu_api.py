@@ -73,7 +73,7 @@ def test_host_buffer_entry_point_matches_device_path():
     L, N = 4, 516
     cfg = dict(L=L, N=N, B=1, k=2)
     t = _buffers(L, N)
-    out, _ = gpu_pass(cfg, t)
+    out, _ = gpu_pass(cfg, t, variant=lf.LF_VARIANT_STREAMS)   # the host entry pipelines the per-layer schedule
     host = {k: out[k].cpu() if k in ("z", "a") else t[k].cpu() for k in ("w", "z", "a", "y")}
     res = {k: torch.empty_like(out[k], device="cpu").pin_memory() for k in ("delta", "gw", "gb")}
     with lf.Leapfrog(L, N, 1, 2) as ctx:
@@ -82,3 +82,5 @@ def test_host_buffer_entry_point_matches_device_path():
         assert ctx.stats()["workspace_bytes"] > 4 * 2 * L * N * N
     for k in ("delta", "gw", "gb"):
         assert torch.equal(res[k], out[k].cpu())
+    ref = oracle_pass(t)
+    compare_all(cfg, dict(z=out["z"], a=out["a"], **{k: v.cuda() for k, v in res.items()}), ref)
