@@ -63,7 +63,8 @@ enum lf_gw_math {
     LF_GW_MATH_TF32 = 2  /* inputs rounded to TF32, fp32 accumulation in tensor memory        */
 };
 
-/* Arithmetic of the B > 1 delta recurrence (Eq. bp2 as an N x N x B contraction). */
+/* Arithmetic of the B > 1 delta recurrence and forward pass (Eq. bp2 and Eq. z as N x N x B
+ * contractions). */
 enum lf_delta_math {
     LF_DELTA_MATH_AUTO = 0,  /* tensor cores when B > 1 and the device supports it               */
     LF_DELTA_MATH_FP32 = 1,  /* fp32 FMA on the CUDA cores                                        */

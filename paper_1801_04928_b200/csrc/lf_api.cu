@@ -313,11 +313,16 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
         const float* a_prev = a + (size_t)(l - 1) * slab(ctx);
         float* z_l = z + (size_t)(l - 1) * slab(ctx);
         float* a_l = a + (size_t)l * slab(ctx);
-        if (B == 1)
+        if (B == 1) {
             LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, N, s));
-        else
+            ++launches;
+        } else if (resolve_delta_math(ctx) == LF_DELTA_MATH_3XTF32) {
+            int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, s, &launches);
+            if (rc2 != LF_OK) return rc2;
+        } else {
             LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, N, B, s));
-        ++launches;
+            ++launches;
+        }
     }
     ctx->stats.launches_forward = launches;
     return LF_OK;

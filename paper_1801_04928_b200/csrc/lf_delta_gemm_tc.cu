@@ -1,6 +1,8 @@
 // Mini-batch delta recurrence (Eq. bp2 for B > 1) on the tensor cores at fp32 accuracy:
 //     T[b][n] = sum_j D[b][j] * W[j][n],   delta^l[b][n] = T[b][n] * a^l[b][n] (1 - a^l[b][n])
-// with D = delta^{l+1} [B][N] and W = w^{l+1} [N][N] (row j, column n).
+// with D = delta^{l+1} [B][N] and W = w^{l+1} [N][N] (row j, column n).  The same kernel, with
+// the W operand read K-major instead, does the mini-batch forward contraction (Eq. z):
+//     Z[b][n] = sum_j A[b][j] * W[n][j] + bias[n],   A = a^{l-1}, W = w^l.
 //
 // A TF32 product keeps 11 significant bits, far too few for the 1e-5 gate on delta, so every
 // operand x is split in shared memory into hi = tf32(x) (round to nearest) and lo = x - hi
@@ -133,14 +135,20 @@ __device__ __forceinline__ unsigned long long dg_desc_mnmajor(unsigned smem_addr
     d |= 1ull << 61;
     return d;
 }
-__device__ __forceinline__ unsigned dg_idesc()
+// descriptor of the W tile for K step kk (eight values of the contraction index)
+template <bool W_KMAJOR>
+__device__ __forceinline__ unsigned long long dg_desc_w(unsigned tile_addr, int kk)
+{
+    return W_KMAJOR ? dg_desc_kmajor(tile_addr + kk * 32) : dg_desc_mnmajor(tile_addr + kk * 1024);
+}
+__device__ __forceinline__ unsigned dg_idesc(bool w_kmajor)
 {
     unsigned d = 0;
     d |= 1u << 4;                             // fp32 accumulator
     d |= 2u << 7;                             // A: TF32
     d |= 2u << 10;                            // B: TF32
     d |= 0u << 15;                            // A is K-major
-    d |= 1u << 16;                            // B is MN-major
+    d |= (w_kmajor ? 0u : 1u) << 16;          // B operand: K-major or MN-major
     d |= (unsigned)(DG_BN >> 3) << 17;
     d |= (unsigned)(DG_BM >> 4) << 24;
     return d;
@@ -180,6 +188,9 @@ __device__ __forceinline__ void dg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// W_KMAJOR = false: T = D * W   (Eq. bp2: w^{l+1}[j][n], contraction over its rows j; MN-major operand)
+// W_KMAJOR = true : T = D * W^T (Eq. z:  w^l[n][j],     contraction over its columns j; K-major operand)
+template <bool W_KMAJOR>
 __global__ void __launch_bounds__(DG_THREADS, 1)
 k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_w,
                 const DgParams P)
@@ -231,10 +242,14 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                     dg_mbar_expect_tx(bar, DG_RAW_BYTES);
                     const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
                     dg_tma_load_2d(a_dst, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM);
+                    if (W_KMAJOR) {
+                        dg_tma_load_2d(a_dst + DG_A_BYTES, &map_w, bar, j0 + ks * DG_BK, tn * DG_BN);
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < DG_BN / 32; ++i)
-                        dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
-                                       j0 + ks * DG_BK);
+                        for (int i = 0; i < DG_BN / 32; ++i)
+                            dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
+                                           j0 + ks * DG_BK);
+                    }
                 }
                 if (sh->abort_flag) break;
             }
@@ -250,7 +265,7 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------------------
         if (lane == 0) {
-            const unsigned idesc = dg_idesc();
+            const unsigned idesc = dg_idesc(W_KMAJOR);
             unsigned it = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
@@ -266,13 +281,13 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                     // the eight small products first, then the four large ones
 #pragma unroll
                     for (int kk = 0; kk < DG_BK / 8; ++kk) {
-                        dg_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_mnmajor(hi + DG_A_BYTES + kk * 1024), idesc,
+                        dg_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
                                kk > 0 ? 1u : 0u);
-                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_mnmajor(lo + DG_A_BYTES + kk * 1024), idesc, 1u);
+                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
                     }
 #pragma unroll
                     for (int kk = 0; kk < DG_BK / 8; ++kk)
-                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_mnmajor(hi + DG_A_BYTES + kk * 1024), idesc, 1u);
+                        dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
                     dg_commit(dg_smem_u32(&sh->empty[st]));
                     dg_commit(dg_smem_u32(&sh->acc_full[p]));
                 }
@@ -375,6 +390,25 @@ k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l,
                                                         s.z * (av.z * (1.0f - av.z)), s.w * (av.w * (1.0f - av.w)));
 }
 
+// forward: z^l = (sum over the K splits) + b^l ; a^l = sigma(z^l)
+__global__ void __launch_bounds__(256)
+k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_l, float* __restrict__ z_l,
+                 float* __restrict__ a_l, size_t n4, int n4_row, int splits)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 s = reinterpret_cast<const float4*>(partial)[i];
+    for (int sp = 1; sp < splits; ++sp) {
+        const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
+        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+    const float4 bb = reinterpret_cast<const float4*>(b_l)[i % n4_row];
+    s.x += bb.x; s.y += bb.y; s.z += bb.z; s.w += bb.w;
+    reinterpret_cast<float4*>(z_l)[i] = s;
+    reinterpret_cast<float4*>(a_l)[i] = make_float4(1.0f / (1.0f + expf(-s.x)), 1.0f / (1.0f + expf(-s.y)),
+                                                    1.0f / (1.0f + expf(-s.z)), 1.0f / (1.0f + expf(-s.w)));
+}
+
 typedef CUresult (*dg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -430,7 +464,9 @@ bool lf_delta_tc_supported(const lf_ctx* c)
     if (!dg_get_encode()) return false;
     static int attr_dev = -1;
     if (attr_dev != c->device) {
-        if (cudaFuncSetAttribute(k_delta_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(k_delta_gemm_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)DG_SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(k_delta_gemm_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)DG_SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return false;
@@ -440,8 +476,8 @@ bool lf_delta_tc_supported(const lf_ctx* c)
     return true;
 }
 
-int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
-                     cudaStream_t s, int* launches)
+// Encode the two operand maps and launch one contraction into c->dg_partial.
+static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kmajor, cudaStream_t s, DgPlan* plan_out)
 {
     alignas(64) CUtensorMap map_d, map_w;
     {
@@ -449,7 +485,7 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
         cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
         cuuint32_t box[2] = {32, (cuuint32_t)DG_BM};
         cuuint32_t estr[2] = {1, 1};
-        if (dg_get_encode()(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(delta_up), dims, strides,
+        if (dg_get_encode()(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(lhs), dims, strides,
                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
             c->last_cuda_error = (int)cudaErrorInvalidValue;
@@ -459,10 +495,12 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     {
         cuuint64_t dims[2] = {(cuuint64_t)c->N, (cuuint64_t)c->N};
         cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
-        cuuint32_t box[2] = {32, (cuuint32_t)DG_BK};
+        cuuint32_t box_mn[2] = {32, (cuuint32_t)DG_BK};      // 32 columns n x 32 rows j
+        cuuint32_t box_k[2] = {32, (cuuint32_t)DG_BN};       // 32 values of j x 128 rows n
         cuuint32_t estr[2] = {1, 1};
-        if (dg_get_encode()(&map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(w_up), dims, strides, box,
-                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+        if (dg_get_encode()(&map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(w_mat), dims, strides,
+                            w_kmajor ? box_k : box_mn, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            w_kmajor ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
             c->last_cuda_error = (int)cudaErrorInvalidValue;
             return LF_ECUDA;
@@ -477,10 +515,37 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     const int units = pl.tiles_m * pl.tiles_n * pl.splits;
     const int grid = units < c->sm_count ? units : c->sm_count;
-    k_delta_gemm_tc<<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);
+    if (w_kmajor)
+        k_delta_gemm_tc<true><<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);
+    else
+        k_delta_gemm_tc<false><<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);
     LF_CUDA_TRY(c, cudaGetLastError());
+    *plan_out = pl;
+    return LF_OK;
+}
+
+int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
+                     cudaStream_t s, int* launches)
+{
+    DgPlan pl;
+    int rc = dg_launch(c, delta_up, w_up, false, s, &pl);
+    if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * c->N / 4;
     k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, pl.splits);
+    LF_CUDA_TRY(c, cudaGetLastError());
+    *launches += 2;
+    return LF_OK;
+}
+
+int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const float* a_prev, float* z_l, float* a_l,
+                       cudaStream_t s, int* launches)
+{
+    DgPlan pl;
+    int rc = dg_launch(c, a_prev, w_l, true, s, &pl);
+    if (rc != LF_OK) return rc;
+    const size_t n4 = (size_t)c->B * c->N / 4;
+    k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, c->N / 4,
+                                                                  pl.splits);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
