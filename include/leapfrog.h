@@ -47,7 +47,10 @@ enum lf_status {
     LF_ECAPACITY = -8  /* size is beyond the fixed capacity of an allocation-free entry point */
 };
 
-/* How lf_backward schedules Eq. bp4 (the weight gradients) against the delta chain. */
+/* How lf_backward schedules Eq. bp4 (the weight gradients) against the delta chain.  The two
+ * persistent variants exist for B = 1 and N <= 16384; elsewhere, and when the device cannot
+ * keep the grid co-resident, lf_backward uses LF_VARIANT_STREAMS instead -- lf_get_stats()
+ * reports the variant that actually ran. */
 enum lf_variant {
     LF_VARIANT_AUTO = 0,       /* pick from the built-in per-(N,B) table of measurements      */
     LF_VARIANT_STREAMS = 1,    /* one launch per layer; the k leapfrog workers are k streams  */
