@@ -32,6 +32,7 @@ METRIC = "backward_layers_per_sec"
 UNIT = "layers/s"
 HBM_FALLBACK_GBS = 6650.0  # used only if MEASURED_PEAKS.json is absent
 VARIANT_NAMES = {"auto": 0, "streams": 1, "persistent": 2, "fused": 3}
+TC_TILING_NAMES = {"auto": 0, "one_sm": 1, "two_sm": 2}
 
 
 def parse_args():
@@ -43,6 +44,10 @@ def parse_args():
     p.add_argument("--config", type=int, default=2)
     p.add_argument("--variant", default="auto", choices=sorted(VARIANT_NAMES))
     p.add_argument("--k", type=int, default=0, help="leapfrog workers (0 = the config's k)")
+    p.add_argument("--tc-tiling", default="auto", choices=["auto", "one_sm", "two_sm"],
+                   help="tiling of the tensor-core contractions (B > 1)")
+    p.add_argument("--layers", type=int, default=0,
+                   help="override the config's L (a smaller case of the same kernels, for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=5)
     p.add_argument("--cpu-seconds", type=float, default=10.0)
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -162,7 +167,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     import lf_inputs
-    cfg, cpu = lf_inputs.make_config(args.config)
+    cfg, cpu = lf_inputs.make_config(args.config, **({"L": args.layers} if args.layers else {}))
     if args.k:
         cfg["k"] = args.k
     per_step = max(1.0, min(15.0, 90.0 / max(1, args.steps + args.warmup)))
@@ -207,11 +212,12 @@ def aggregate_rate(total_ms, units_per_rank, dist=None, device=None):
 NCU_TRAFFIC = {(2, 3): 205.7e6}
 
 
-def time_gw_gemm(lf, L, N, B, t, stream, steps):
+def time_gw_gemm(lf, L, N, B, t, stream, steps, gw_tiling=0):
     """Average time of the mini-batch weight-gradient launch, through an L = 1 context on the
     top layer's tensors (Eq. bp1 and the column-sum launch ride along; both are tiny)."""
     import torch
     ctx = lf.Leapfrog(1, N, B, 1, stream=stream.cuda_stream)
+    ctx.set_option(lf.LF_OPT_TC_TILING, gw_tiling)
     a1 = t["a"][L - 1:L + 1].contiguous(); z1 = t["z"][L - 1:L].contiguous()
     w1 = t["w"][L - 1:L].contiguous()
     d1 = torch.empty((1, B, N), device=w1.device); gb1 = torch.empty((1, N), device=w1.device)
@@ -226,9 +232,9 @@ def time_gw_gemm(lf, L, N, B, t, stream, steps):
         e1.record(stream)
         ctx.sync()
     ms = e0.elapsed_time(e1) / steps
-    gw_math = ctx.stats()["gw_math"]
+    st = ctx.stats()
     ctx.close()
-    return ms, gw_math
+    return ms, st["gw_math"], st["gw_tiling"]
 
 
 def workload_name(index, cfg):
@@ -254,7 +260,7 @@ def run_ours(args):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg, cpu = lf_inputs.make_config(args.config)
+    cfg, cpu = lf_inputs.make_config(args.config, **({"L": args.layers} if args.layers else {}))
     if args.k:
         cfg["k"] = args.k
     L, N, B, k = cfg["L"], cfg["N"], cfg["B"], cfg["k"]
@@ -278,6 +284,7 @@ def run_ours(args):
         t["gb"] = torch.empty((L, N), dtype=torch.float32, device=dev)
         ctx = lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream)
         ctx.set_option(lf.LF_OPT_VARIANT, variant)
+        ctx.set_option(lf.LF_OPT_TC_TILING, TC_TILING_NAMES[args.tc_tiling])
         t["ctx"] = ctx
         sets.append(t)
     torch.cuda.synchronize(dev)
@@ -384,7 +391,8 @@ def run_ours(args):
         # Mini-batch: the weight gradient is a dense N x N x B contraction on the tensor cores.
         # Its launch is timed alone; its bound is the slower of the 4N^2-byte store stream and
         # the 2N^2B flops at the TF32 peak (measured bf16 burst peak x nominal tf32/bf16 ratio).
-        gemm_ms, gw_math = time_gw_gemm(lf, L, N, B, sets[0], stream, 20)
+        gemm_ms, gw_math, gw_tiling = time_gw_gemm(lf, L, N, B, sets[0], stream, 20,
+                                                   TC_TILING_NAMES[args.tc_tiling])
         flops = 2.0 * N * N * B
         tf32_peak = float(peaks.get("bf16_tflops", 1590.0)) * (1.1 / 2.25)
         t_store = 4.0 * N * N / (peak * 1e9)
@@ -398,12 +406,14 @@ def run_ours(args):
             gbytes = (4.0 * N * N + 8.0 * N * B) / (gemm_ms * 1e-3) / 1e9
             roofline = {"bound": "hbm", "achieved": gbytes, "peak": peak, "unit": "GB/s",
                         "frac": gbytes / peak, "traffic": None, "peak_kind": f"of {peak_kind}"}
-        roofline.update({"kernel": "k_gw_gemm_tf32 (one layer, timed alone through an L=1 context)"
+        tf32_kernel = "k_gw_gemm_tf32_pair" if gw_tiling == 2 else "k_gw_gemm_tf32"
+        roofline.update({"kernel": f"{tf32_kernel} (one layer, timed alone through an L=1 context)"
                                    if gw_math == 2 else "k_gemm_simt (weight gradient, fp32)",
                          "avg_launch_ms": gemm_ms, "flops_per_launch": flops,
                          "tflops": flops / (gemm_ms * 1e-3) / 1e12,
                          "whole_step_algorithmic_GBs": achieved,
-                         "note": "the step is dominated by the fp32 CUDA-core delta-chain GEMMs"})
+                         "note": "the step also holds the 3xTF32 delta-chain contractions "
+                                 "(three tensor-core products per term)"})
 
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:

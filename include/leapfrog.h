@@ -75,12 +75,23 @@ enum lf_delta_math {
                                 products per term, fp32 accumulation: fp32-level accuracy        */
 };
 
+/* Tiling of the tensor-core contractions (B > 1): one CTA per tile, or a pair of CTAs (two
+ * multiprocessors) per tile, which share one operand and halve the traffic per multiply-add. */
+enum lf_tc_tiling {
+    LF_TC_TILING_AUTO = 0,   /* CTA pairs where they apply and the device can co-schedule them  */
+    LF_TC_TILING_ONE_SM = 1, /* one CTA per tile                                                */
+    LF_TC_TILING_TWO_SM = 2  /* CTA pairs: Eq. bp4 for B <= 256 (the delta operand of a row
+                                block stays in shared memory), Eq. bp2 / Eq. z for B > 128;
+                                other sizes use ONE_SM                                          */
+};
+
 enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
     LF_OPT_WAIT_BUDGET_US = 3,/* upper bound of any device-side wait, microseconds (>= 1)     */
     LF_OPT_USE_GRAPH = 4,     /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
     LF_OPT_DELTA_MATH = 6,    /* enum lf_delta_math                                           */
+    LF_OPT_TC_TILING = 7,     /* enum lf_tc_tiling                                            */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -99,6 +110,9 @@ typedef struct lf_stats {
     unsigned int device_status; /* status word read by the last lf_sync (0 = clean)           */
     long long workspace_bytes;  /* device memory owned by the context                         */
     int delta_math;           /* arithmetic the last lf_backward used for Eq. bp2 (B > 1)     */
+    int gw_tiling;            /* tiling of the last TF32 weight-gradient launch (enum lf_tc_tiling,
+                                 ONE_SM or TWO_SM; 0 if none ran)                             */
+    int delta_tiling;         /* the same for the last tensor-core Eq. bp2 / Eq. z launch     */
 } lf_stats;
 
 /*

@@ -20,6 +20,8 @@ LF_VARIANT_AUTO, LF_VARIANT_STREAMS, LF_VARIANT_PERSISTENT, LF_VARIANT_FUSED = 0
 LF_GW_MATH_AUTO, LF_GW_MATH_FP32, LF_GW_MATH_TF32 = 0, 1, 2
 LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH, LF_OPT_WITHHOLD = 1, 2, 3, 4, 5
 LF_OPT_DELTA_MATH = 6
+LF_OPT_TC_TILING = 7
+LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
 LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
 
 EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
@@ -34,7 +36,7 @@ class lf_stats(ctypes.Structure):
                 ("chain_ctas", ctypes.c_int), ("worker_ctas", ctypes.c_int),
                 ("launches_forward", ctypes.c_int), ("launches_backward", ctypes.c_int),
                 ("device_status", ctypes.c_uint), ("workspace_bytes", ctypes.c_longlong),
-                ("delta_math", ctypes.c_int)]
+                ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:

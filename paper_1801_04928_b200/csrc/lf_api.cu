@@ -207,6 +207,7 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
     c->opt_gw_math = LF_GW_MATH_AUTO;
     c->wait_budget_us = 2000000;
     c->use_graph = 1;
+    c->tc_pair_kernels = 1;
 
     bool ok = true;
     size_t ws = 0;
@@ -282,6 +283,11 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
         case LF_OPT_DELTA_MATH:
             if (value < LF_DELTA_MATH_AUTO || value > LF_DELTA_MATH_3XTF32) return LF_EINVAL;
             ctx->opt_delta_math = (int)value;
+            return LF_OK;
+        case LF_OPT_TC_TILING:
+            if (value < LF_TC_TILING_AUTO || value > LF_TC_TILING_TWO_SM) return LF_EINVAL;
+            ctx->tc_pair_kernels = value != LF_TC_TILING_ONE_SM;
+            drop_graph(ctx);
             return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;

@@ -373,6 +373,358 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
     }
 }
 
+// ================================================================================================
+// Two-SM form (more than 128 samples): a pair of CTAs (one thread-block cluster) works on
+// 256 samples x 256 columns with tcgen05.mma.cta_group::2 (M = 256, N = 256, K = 8).  Each CTA
+// loads and splits only HALF of the W tile (128 columns), which the tensor cores of both CTAs
+// read, so the shared-memory traffic per multiply-add falls; and the three jobs that share one
+// set of warps in the kernel above -- splitting a stage, issuing its products, adding the
+// finished stage into the running sums -- have warps of their own here, so they overlap:
+//   warp 0       TMA producer: this CTA's 128 samples of D and its 128 columns of W per stage;
+//   warp 1       leader CTA (cluster rank 0) only: issues the products for both CTAs;
+//   warps 4-7    split this CTA's stage into hi/lo (in place + beside it);
+//   warps 8-15   running sums of this CTA's 128 samples: a thread holds one sample and 128 of
+//                the 256 columns in registers.  They need about 200 registers per thread and the
+//                other warps few, so the warpgroups re-divide the register file at the start
+//                (setmaxnreg: 2 x 128 threads x 48 + 2 x 128 threads x 208 = 512 x 128).
+// Hand-offs across the pair: the splitting warps of both CTAs arrive on the leader's "split done"
+// barrier, the leader's tcgen05.commit reaches the "stage free" and "accumulator full" barriers
+// of both CTAs, the summing warps of both arrive on the leader's "accumulator drained" barrier.
+// Arithmetic and summation order per output element are those of the one-SM kernel above.
+constexpr int DP_BN = 256;                               // columns of a pair tile (128 loaded per CTA)
+constexpr int DP_BNH = DP_BN / 2;
+constexpr int DP_STAGES = 3;
+constexpr int DP_B_BYTES = (DP_BNH / 32) * DG_BOX_BYTES; // 16 KiB (either operand form)
+constexpr int DP_RAW_BYTES = DG_A_BYTES + DP_B_BYTES;    // 32 KiB per CTA and stage from TMA
+constexpr int DP_STAGE_BYTES = 2 * DP_RAW_BYTES;         // hi (in place) + lo
+constexpr int DP_THREADS = 512;                          // four warpgroups
+constexpr int DP_SPLITTERS = 128;                        // warps 4-7
+constexpr int DP_REGS_LAUNCH = 128, DP_REGS_SMALL = 48, DP_REGS_SUM = 208;
+static_assert(2 * 128 * DP_REGS_SMALL + 2 * 128 * DP_REGS_SUM <= DP_THREADS * DP_REGS_LAUNCH,
+              "the warpgroups' register shares must fit into what the CTA is launched with");
+constexpr int DP_TMEM_COLS = 512;                        // two stage accumulators of 256 columns
+constexpr int DP_EPI_LD = 20;                            // 16 columns + padding
+constexpr int DP_EPI_BYTES = 8 * 32 * DP_EPI_LD * 4;
+constexpr size_t DP_SMEM_BYTES = (size_t)DP_STAGES * DP_STAGE_BYTES + DP_EPI_BYTES + 1024 + 256;
+
+struct DpShared {
+    unsigned long long full[DP_STAGES];        // this CTA's TMA data of the stage has landed
+    unsigned long long split_done[DP_STAGES];  // leader: hi/lo of both CTAs written (8 warp arrivals)
+    unsigned long long empty[DP_STAGES];       // both: the multiplications that read the stage are done
+    unsigned long long acc_full[2];            // both: stage accumulator p holds a finished stage
+    unsigned long long acc_empty[2];           // leader: accumulator p drained by both CTAs (16 warp arrivals)
+    unsigned tmem_base;
+    volatile unsigned abort_flag;
+};
+
+__device__ __forceinline__ unsigned dp_cluster_rank()
+{
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ unsigned dp_map_to_rank(unsigned local_addr, unsigned rank)
+{
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void dp_cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void dp_mma(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                       unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrive on the barrier at this offset in both CTAs once the tensor-core work issued so far is done
+__device__ __forceinline__ void dp_commit_both(unsigned bar)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void dp_arrive_cluster(unsigned cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool dp_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool dp_wait(unsigned bar, unsigned parity, const DgParams& P, DpShared* sh)
+{
+    if (dp_try_wait(bar, parity)) return true;
+    if (sh->abort_flag) return false;
+    const unsigned long long t0 = dg_timer();
+    unsigned spins = 0;
+    while (!dp_try_wait(bar, parity)) {
+        if ((++spins & 15u) == 0u) {
+            if (sh->abort_flag) return false;
+            if (dg_timer() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
+                atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
+                sh->abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ unsigned dp_idesc(bool w_kmajor)
+{
+    unsigned d = 0;
+    d |= 1u << 4;                             // fp32 accumulator
+    d |= 2u << 7;                             // A: TF32
+    d |= 2u << 10;                            // B: TF32
+    d |= 0u << 15;                            // A is K-major
+    d |= (w_kmajor ? 0u : 1u) << 16;          // B operand: K-major or MN-major
+    d |= (unsigned)(DP_BN >> 3) << 17;
+    d |= (unsigned)((2 * DG_BM) >> 4) << 24;
+    return d;
+}
+// 32 lanes x 64 consecutive fp32 columns of tensor memory as two loads in flight together
+__device__ __forceinline__ void dp_tmem_ld64(unsigned taddr, unsigned (&r)[64])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+          "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]),
+          "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+          "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr + 32u) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+template <bool W_KMAJOR>
+__global__ void __launch_bounds__(DP_THREADS, 1)
+k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_w,
+                     const DgParams P)
+{
+    extern __shared__ unsigned char dg_smem_raw[];
+    // the same offsets in both CTAs: one descriptor addresses the shared memory of both
+    unsigned char* stages = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(dg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    float* epi = reinterpret_cast<float*>(stages + (size_t)DP_STAGES * DP_STAGE_BYTES);
+    DpShared* sh = reinterpret_cast<DpShared*>(stages + (size_t)DP_STAGES * DP_STAGE_BYTES + DP_EPI_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned rank = dp_cluster_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int n_units = P.tiles_m * P.tiles_n * P.splits;     // tiles_m: 256-sample blocks, tiles_n: 256-column blocks
+    const int n_k = P.k_per_split / DG_BK;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < DP_STAGES; ++i) {
+            dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 8);
+            dg_mbar_init(dg_smem_u32(&sh->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            dg_mbar_init(dg_smem_u32(&sh->acc_full[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->acc_empty[i]), 16);
+        }
+        sh->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(dg_smem_u32(&sh->tmem_base)), "r"((unsigned)DP_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    dg_fence_before();
+    __syncthreads();
+    dp_cluster_sync();   // the peer's barriers exist before anything can arrive on them
+    dg_fence_after();
+    const unsigned tmem_base = sh->tmem_base;
+
+    if (warp < 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(DP_REGS_SMALL));
+        if (warp == 0) {
+            // ------------------------------ TMA producer (each CTA, its own halves) ------------
+            if (lane == 0) {
+                unsigned it = 0;
+                bool ok = true;
+                for (int u = pair; u < n_units && ok; u += n_pairs) {
+                    const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
+                    const int j0 = sp * P.k_per_split;
+                    const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM;       // my samples
+                    const int col0 = tn * DP_BN + (int)rank * DP_BNH;          // my columns of W
+                    for (int ks = 0; ks < n_k; ++ks, ++it) {
+                        const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
+                        if (use > 0 && !dp_wait(dg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                        const unsigned bar = dg_smem_u32(&sh->full[st]);
+                        dg_mbar_expect_tx(bar, DP_RAW_BYTES);
+                        const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DP_STAGE_BYTES);
+                        dg_tma_load_2d(a_dst, &map_d, bar, j0 + ks * DG_BK, row0);
+                        if (W_KMAJOR) {
+                            dg_tma_load_2d(a_dst + DG_A_BYTES, &map_w, bar, j0 + ks * DG_BK, col0);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < DP_BNH / 32; ++i)
+                                dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, col0 + i * 32,
+                                               j0 + ks * DG_BK);
+                        }
+                    }
+                }
+                // after giving up: do not let the CTA exit under loads that are still landing
+                if (sh->abort_flag) {
+                    const unsigned long long t0 = dg_timer();
+                    for (unsigned j = it > DP_STAGES ? it - DP_STAGES : 0; j < it; ++j) {
+                        const unsigned bar = dg_smem_u32(&sh->full[j % DP_STAGES]);
+                        while (!dg_mbar_try_wait(bar, (j / DP_STAGES) & 1u) && dg_timer() - t0 < 50000000ull) { }
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            // ------------------------------ MMA issuer (leader CTA only) -----------------------
+            if (lane == 0 && rank == 0) {
+                const unsigned idesc = dp_idesc(W_KMAJOR);
+                unsigned it = 0;
+                bool ok = true;
+                for (int u = pair; u < n_units && ok; u += n_pairs) {
+                    for (int ks = 0; ks < n_k; ++ks, ++it) {
+                        const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
+                        const unsigned p = it & 1u, p_use = it >> 1;
+                        if (!dp_wait(dg_smem_u32(&sh->split_done[st]), use & 1u, P, sh)) { ok = false; break; }
+                        if (p_use > 0 && !dp_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
+                        dg_fence_after();
+                        const unsigned hi = dg_smem_u32(stages + (size_t)st * DP_STAGE_BYTES);
+                        const unsigned lo = hi + DP_RAW_BYTES;
+                        const unsigned d_tmem = tmem_base + p * (unsigned)DP_BN;
+                        // the eight small products first, then the four large ones
+#pragma unroll
+                        for (int kk = 0; kk < DG_BK / 8; ++kk) {
+                            dp_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
+                                   kk > 0 ? 1u : 0u);
+                            dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < DG_BK / 8; ++kk)
+                            dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
+                        dp_commit_both(dg_smem_u32(&sh->empty[st]));
+                        dp_commit_both(dg_smem_u32(&sh->acc_full[p]));
+                    }
+                }
+            }
+        } else if (warp >= 4) {
+            // ------------------------------ operand split (hi/lo): warps 4..7 ------------------
+            const int tt = threadIdx.x - 128;
+            const unsigned leader_split_done0 = dp_map_to_rank(dg_smem_u32(&sh->split_done[0]), 0);
+            unsigned it = 0;
+            bool ok = true;
+            for (int u = pair; u < n_units && ok; u += n_pairs) {
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
+                    if (!dp_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES);
+                    float4* lo = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES + DP_RAW_BYTES);
+#pragma unroll 4
+                    for (int i = 0; i < DP_RAW_BYTES / 16 / DP_SPLITTERS; ++i) {
+                        const int idx = tt + i * DP_SPLITTERS;
+                        const float4 v = raw[idx];
+                        const float4 h = make_float4(dg_tf32_rn(v.x), dg_tf32_rn(v.y), dg_tf32_rn(v.z), dg_tf32_rn(v.w));
+                        raw[idx] = h;
+                        lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+                    }
+                    // the tensor cores (of both CTAs) read this shared memory through the async proxy
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) dp_arrive_cluster(leader_split_done0 + st * (unsigned)sizeof(unsigned long long));
+                }
+            }
+        }
+    } else {
+        // ------------------------------ running sums and output: warps 8..15 -------------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(DP_REGS_SUM));
+        const int quad = warp & 3;               // the TMEM lane quadrant this warp may read
+        const int half = (warp - 8) >> 2;        // which 128 of the 256 accumulator columns
+        const unsigned leader_acc_empty0 = dp_map_to_rank(dg_smem_u32(&sh->acc_empty[0]), 0);
+        unsigned it = 0;
+        bool ok = true;
+        float acc[DP_BNH];     // this thread's sample, its 128 columns of the tile
+        for (int u = pair; u < n_units && ok; u += n_pairs) {
+            const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
+#pragma unroll
+            for (int v = 0; v < DP_BNH; ++v) acc[v] = 0.f;
+            for (int ks = 0; ks < n_k; ++ks, ++it) {
+                // add the finished stage (accumulator it & 1) into the registers
+                const unsigned p = it & 1u;
+                if (!dp_wait(dg_smem_u32(&sh->acc_full[p]), (it >> 1) & 1u, P, sh)) { ok = false; break; }
+                dg_fence_after();
+#pragma unroll
+                for (int cchunk = 0; cchunk < DP_BNH / 32; ++cchunk) {
+                    unsigned r[32];
+                    dg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DP_BN + half * DP_BNH + cchunk * 32, r);
+#pragma unroll
+                    for (int v = 0; v < 32; ++v)
+                        acc[cchunk * 32 + v] += __uint_as_float(r[v]);
+                }
+                dg_fence_before();
+                __syncwarp();
+                if (lane == 0) dp_arrive_cluster(leader_acc_empty0 + p * (unsigned)sizeof(unsigned long long));
+            }
+            if (!ok) break;
+            float* blk = epi + (warp - 8) * 32 * DP_EPI_LD;
+            const int sub_r = lane >> 2, sub_c = (lane & 3) * 4;
+            const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM + quad * 32 + sub_r;
+            const int col0 = tn * DP_BN + half * DP_BNH + sub_c;
+            // four rows per lane (row0 + 8 i), 16 columns per pass; constant offsets from one pointer per row
+            float* out_row = P.partial + (size_t)sp * P.B * P.N + (size_t)row0 * P.N + col0;
+            const size_t row_step = (size_t)8 * P.N;
+#pragma unroll
+            for (int cchunk = 0; cchunk < DP_BNH / 16; ++cchunk) {
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    *reinterpret_cast<float4*>(blk + lane * DP_EPI_LD + 4 * v) =
+                        make_float4(acc[cchunk * 16 + 4 * v], acc[cchunk * 16 + 4 * v + 1],
+                                    acc[cchunk * 16 + 4 * v + 2], acc[cchunk * 16 + 4 * v + 3]);
+                __syncwarp();
+                if (col0 + cchunk * 16 < P.N) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 val = *reinterpret_cast<const float4*>(blk + (i * 8 + sub_r) * DP_EPI_LD + sub_c);
+                        if (row0 + i * 8 < P.B)
+                            *reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 16) = val;
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    }
+
+    // neither CTA may leave, or free tensor memory, while the other can still reach it
+    dg_fence_before();
+    __syncthreads();
+    dp_cluster_sync();
+    if (warp == 1) {
+        dg_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DP_TMEM_COLS)
+                     : "memory");
+    }
+}
+
 // delta^l = (sum over the K splits, in split order) * sigma'(z^l), sigma' = a (1 - a)
 __global__ void __launch_bounds__(256)
 k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
@@ -448,13 +800,65 @@ DgPlan dg_plan(const lf_ctx* c)
     return p;
 }
 
+// Largest number of CTA pairs of the two-SM kernels that can be resident at once (0: unusable).
+// Queried once per device; also opts the kernels in to their dynamic shared memory.
+int dp_max_pairs(const lf_ctx* c)
+{
+    static int cached_dev = -1, cached = 0;
+    if (cached_dev == c->device) return cached;
+    int n = 0;
+    if ((size_t)c->smem_optin >= DP_SMEM_BYTES &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        cfg.gridDim = dim3(2 * 16); cfg.blockDim = dim3(DP_THREADS); cfg.dynamicSmemBytes = DP_SMEM_BYTES;
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int n0 = 0, n1 = 0;
+        if (cudaOccupancyMaxActiveClusters(&n0, k_delta_gemm_tc_pair<false>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n1, k_delta_gemm_tc_pair<true>, &cfg) == cudaSuccess)
+            n = n0 < n1 ? n0 : n1;
+    }
+    cudaGetLastError();
+    cached_dev = c->device; cached = n;
+    return n;
+}
+
+// The two-SM kernels pay off once a pair's 256 samples are more than half filled.
+bool dp_use_pairs(const lf_ctx* c) { return c->tc_pair_kernels && c->B > DG_BM && dp_max_pairs(c) > 0; }
+
+DgPlan dp_plan(const lf_ctx* c, int pairs)
+{
+    DgPlan p;
+    p.tiles_m = (c->B + 2 * DG_BM - 1) / (2 * DG_BM);
+    p.tiles_n = (c->N + DP_BN - 1) / DP_BN;
+    int s = pairs / (p.tiles_m * p.tiles_n);
+    if (s < 1) s = 1;
+    if (s > 8) s = 8;
+    const int kb = (c->N + DG_BK - 1) / DG_BK;
+    if (s > kb) s = kb;
+    const int kb_per = (kb + s - 1) / s;
+    p.splits = (kb + kb_per - 1) / kb_per;
+    p.k_per_split = kb_per * DG_BK;
+    return p;
+}
+
 }  // namespace
 
 size_t lf_delta_tc_scratch_bytes(const lf_ctx* c)
 {
     if (c->B < 2) return 0;
-    DgPlan p = dg_plan(c);
-    return (size_t)p.splits * c->B * c->N * sizeof(float);
+    // K-split partial sums [splits][B][N] of whichever tiling has more splits
+    int splits = dg_plan(c).splits;
+    if (c->B > DG_BM && dp_max_pairs(c) > 0) {
+        const int s2 = dp_plan(c, dp_max_pairs(c)).splits;
+        if (s2 > splits) splits = s2;
+    }
+    return (size_t)splits * c->B * c->N * sizeof(float);
 }
 
 bool lf_delta_tc_supported(const lf_ctx* c)
@@ -473,6 +877,7 @@ bool lf_delta_tc_supported(const lf_ctx* c)
         }
         attr_dev = c->device;
     }
+    dp_max_pairs(c);
     return true;
 }
 
@@ -506,7 +911,9 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
             return LF_ECUDA;
         }
     }
-    const DgPlan pl = dg_plan(c);
+    const bool pairs = dp_use_pairs(c);
+    const int max_pairs = pairs ? dp_max_pairs(c) : 0;
+    const DgPlan pl = pairs ? dp_plan(c, max_pairs) : dg_plan(c);
     DgParams P;
     P.N = c->N; P.B = c->B;
     P.tiles_m = pl.tiles_m; P.tiles_n = pl.tiles_n; P.splits = pl.splits; P.k_per_split = pl.k_per_split;
@@ -514,6 +921,23 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     const int units = pl.tiles_m * pl.tiles_n * pl.splits;
+    if (pairs) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        cfg.gridDim = dim3(2 * (units < max_pairs ? units : max_pairs));
+        cfg.blockDim = dim3(DP_THREADS); cfg.dynamicSmemBytes = DP_SMEM_BYTES; cfg.stream = s;
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        if (w_kmajor)
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true>, map_d, map_w, P));
+        else
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false>, map_d, map_w, P));
+        c->stats.delta_tiling = LF_TC_TILING_TWO_SM;
+        *plan_out = pl;
+        return LF_OK;
+    }
+    c->stats.delta_tiling = LF_TC_TILING_ONE_SM;
     const int grid = units < c->sm_count ? units : c->sm_count;
     if (w_kmajor)
         k_delta_gemm_tc<true><<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);

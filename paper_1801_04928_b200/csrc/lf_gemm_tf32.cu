@@ -306,6 +306,301 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
     }
 }
 
+// ================================================================================================
+// Two-SM form for batches of at most 256 samples: a pair of CTAs (one thread-block cluster) works
+// on 256 rows of gw at a time with tcgen05.mma.cta_group::2 (M = 256, N = 128, K = 8).
+//   * The delta operand of the pair's 256 rows -- every sample of it, at most 128 KiB per CTA --
+//     is loaded ONCE per row block and stays in shared memory while the pair walks along the
+//     row block; only the activation operand streams (64 columns x 32 samples = 8 KiB per CTA
+//     and stage), and the two CTAs read each other's half of it.  Per 64 KiB of gradient a CTA
+//     stores it then loads 64 KiB of operands, against 192 KiB in the one-SM kernel above, whose
+//     speed is set by exactly those loads.
+//   * 256 x 128 pair tiles, each pair a contiguous run of them in row-major order (a run crosses
+//     a row-block boundary at most once when N <= 256 * pairs); four accumulators of 128 columns
+//     in tensor memory, so the epilogue of a tile overlaps the next tiles' multiplications.
+// Hand-offs between the two CTAs: both producers credit their loads to the LEADER's (rank 0)
+// "full" barriers; the leader's tcgen05.commit reaches the "empty" / "accumulator full" barriers
+// of both CTAs at once; the epilogue warps of both CTAs arrive on the leader's "accumulator
+// empty" barrier.  All waits are bounded as above.
+constexpr int TP_BM = 128;                               // rows of gw per CTA (256 per pair)
+constexpr int TP_BN = 128;                               // columns of a pair tile (64 loaded per CTA)
+constexpr int TP_MAX_KS = 8;                             // at most 8 x 32 = 256 samples
+constexpr int TP_STAGES = 8;
+constexpr int TP_ACC = 4;                                // accumulators of TP_BN columns
+constexpr int TP_A_STAGE_BYTES = (TP_BM / 32) * TG_BOX_BYTES;        // 16 KiB: 128 rows x 32 samples
+constexpr int TP_B_STAGE_BYTES = (TP_BN / 2 / 32) * TG_BOX_BYTES;    //  8 KiB:  64 columns x 32 samples
+constexpr int TP_A_BYTES = TP_MAX_KS * TP_A_STAGE_BYTES;             // 128 KiB
+constexpr int TP_THREADS = 192;
+constexpr size_t TP_SMEM_BYTES = (size_t)TP_A_BYTES + (size_t)TP_STAGES * TP_B_STAGE_BYTES + TG_EPI_BYTES +
+                                 1024 /*alignment slack*/ + 512;
+
+struct TpShared {
+    unsigned long long a_full[TP_MAX_KS];   // leader: delta operand chunk ks of both CTAs has landed
+    unsigned long long a_empty;             // both: the resident delta operand may be replaced
+    unsigned long long b_full[TP_STAGES];   // leader: stage of both CTAs has landed
+    unsigned long long b_empty[TP_STAGES];  // both: stage may be refilled
+    unsigned long long acc_full[TP_ACC];    // both: accumulator complete
+    unsigned long long acc_empty[TP_ACC];   // leader: accumulator drained by both CTAs
+    unsigned tmem_base;
+    volatile unsigned abort_flag;
+};
+
+__device__ __forceinline__ unsigned tp_cluster_rank()
+{
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ unsigned tp_map_to_rank(unsigned local_addr, unsigned rank)
+{
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void tp_cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are credited to an mbarrier that may sit in
+// the other CTA of the pair (`bar` is a shared::cluster address).
+__device__ __forceinline__ void tp_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tp_mma_tf32(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                            unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once every
+// tensor-core operation issued so far has completed
+__device__ __forceinline__ void tp_commit_both(unsigned bar)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tp_arrive_remote(unsigned cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool tp_try_wait_cluster(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait on a barrier of this CTA; returns false once this CTA has given up.
+__device__ __forceinline__ bool tp_wait(unsigned bar, unsigned parity, const TgParams& P, TpShared* sh)
+{
+    if (tp_try_wait_cluster(bar, parity)) return true;
+    if (sh->abort_flag) return false;
+    const unsigned long long t0 = tg_timer();
+    unsigned spins = 0;
+    while (!tp_try_wait_cluster(bar, parity)) {
+        if ((++spins & 15u) == 0u) {
+            if (sh->abort_flag) return false;
+            if (tg_timer() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
+                atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
+                sh->abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(TP_THREADS, 1)
+k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_a,
+                    const TgParams P)
+{
+    extern __shared__ unsigned char tg_smem_raw[];
+    // Both CTAs of the pair must use the same offsets (the tensor core applies one descriptor to
+    // both); the dynamic shared memory starts at the same address in every CTA of a launch.
+    unsigned char* a_res = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(tg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    unsigned char* b_ring = a_res + TP_A_BYTES;
+    float* epi = reinterpret_cast<float*>(b_ring + (size_t)TP_STAGES * TP_B_STAGE_BYTES);
+    TpShared* sh = reinterpret_cast<TpShared*>(reinterpret_cast<unsigned char*>(epi) + TG_EPI_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned rank = tp_cluster_rank();          // 0 = leader (issues the multiplications)
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int n_k = (P.B + TG_BK - 1) / TG_BK;        // <= TP_MAX_KS
+    const int n_tiles = P.tiles_m * P.tiles_n;        // tiles_m counts 256-row blocks here
+    const int t_begin = (int)(((long long)n_tiles * pair) / n_pairs);
+    const int t_end = (int)(((long long)n_tiles * (pair + 1)) / n_pairs);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < TP_MAX_KS; ++i) tg_mbar_init(tg_smem_u32(&sh->a_full[i]), 1);
+        tg_mbar_init(tg_smem_u32(&sh->a_empty), 1);
+        for (int i = 0; i < TP_STAGES; ++i) {
+            tg_mbar_init(tg_smem_u32(&sh->b_full[i]), 1);
+            tg_mbar_init(tg_smem_u32(&sh->b_empty[i]), 1);
+        }
+        for (int i = 0; i < TP_ACC; ++i) {
+            tg_mbar_init(tg_smem_u32(&sh->acc_full[i]), 1);
+            tg_mbar_init(tg_smem_u32(&sh->acc_empty[i]), 8);   // four epilogue warps of each CTA
+        }
+        sh->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // tensor memory for the accumulators, the same columns in both CTAs
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tg_smem_u32(&sh->tmem_base)), "r"((unsigned)(TP_ACC * TP_BN)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tg_fence_before();
+    __syncthreads();
+    tp_cluster_sync();   // the peer's barriers exist before anything can arrive on them
+    tg_fence_after();
+    const unsigned tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer (each CTA, its own halves) ----------------
+        if (lane == 0) {
+            unsigned it = 0, a_loads = 0;
+            int cur_rb = -1;
+            const int my_row0 = (int)rank * TP_BM;
+            const int my_col0 = (int)rank * (TP_BN / 2);
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int rb = t / P.tiles_n, tn = t - rb * P.tiles_n;
+                const bool new_rb = rb != cur_rb;
+                if (new_rb) {
+                    // the resident delta operand changes: wait until every multiplication that
+                    // reads the old one is done
+                    if (a_loads > 0 && !tp_wait(tg_smem_u32(&sh->a_empty), (a_loads - 1) & 1u, P, sh)) break;
+                    cur_rb = rb;
+                    ++a_loads;
+                }
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    if (new_rb) {
+                        const unsigned lbar = tg_smem_u32(&sh->a_full[ks]);
+                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_A_STAGE_BYTES);
+                        const unsigned bar = tp_map_to_rank(lbar, 0);
+                        const unsigned dst = tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES);
+#pragma unroll
+                        for (int i = 0; i < TP_BM / 32; ++i)
+                            tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
+                                           ks * TG_BK);
+                    }
+                    const unsigned st = it % TP_STAGES, use = it / TP_STAGES;
+                    if (use > 0 && !tp_wait(tg_smem_u32(&sh->b_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                    const unsigned lbar = tg_smem_u32(&sh->b_full[st]);
+                    if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
+                    const unsigned bar = tp_map_to_rank(lbar, 0);
+                    const unsigned dst = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
+#pragma unroll
+                    for (int i = 0; i < TP_BN / 2 / 32; ++i)
+                        tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (leader CTA only) ---------------------------
+        if (lane == 0 && rank == 0) {
+            const unsigned idesc = tg_make_idesc(2 * TP_BM, TP_BN);
+            unsigned it = 0, tile_i = 0, a_loads = 0;
+            int cur_rb = -1;
+            for (int t = t_begin; t < t_end; ++t, ++tile_i) {
+                const int rb = t / P.tiles_n;
+                const bool new_rb = rb != cur_rb;
+                if (new_rb) { cur_rb = rb; ++a_loads; }
+                const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
+                if (ab_use > 0 && !tp_wait(tg_smem_u32(&sh->acc_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
+                tg_fence_after();
+                const unsigned d_tmem = tmem_base + ab * (unsigned)TP_BN;
+                bool ok = true;
+                for (int ks = 0; ks < n_k; ++ks, ++it) {
+                    if (new_rb && !tp_wait(tg_smem_u32(&sh->a_full[ks]), (a_loads - 1) & 1u, P, sh)) { ok = false; break; }
+                    const unsigned st = it % TP_STAGES, use = it / TP_STAGES;
+                    if (!tp_wait(tg_smem_u32(&sh->b_full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    tg_fence_after();
+                    const unsigned a_addr = tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES);
+                    const unsigned b_addr = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < TG_BK / 8; ++kk) {      // eight samples per instruction
+                        const unsigned long long da = tg_make_desc(a_addr + kk * 1024, TG_BOX_BYTES);
+                        const unsigned long long db = tg_make_desc(b_addr + kk * 1024, TG_BOX_BYTES);
+                        tp_mma_tf32(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tp_commit_both(tg_smem_u32(&sh->b_empty[st]));
+                }
+                if (!ok) break;
+                // the last tile of a row block frees the resident operand for the next one
+                if (t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(tg_smem_u32(&sh->a_empty));
+                tp_commit_both(tg_smem_u32(&sh->acc_full[ab]));
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (warps 2..5 of both CTAs) ---------------------
+        const int quad = warp & 3;                 // the TMEM lane quadrant this warp may read
+        const unsigned leader_acc_empty0 = tp_map_to_rank(tg_smem_u32(&sh->acc_empty[0]), 0);
+        unsigned tile_i = 0;
+        for (int t = t_begin; t < t_end; ++t, ++tile_i) {
+            const int rb = t / P.tiles_n, tn = t - rb * P.tiles_n;
+            const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
+            if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
+            tg_fence_after();
+            float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
+            const int row0 = rb * 2 * TP_BM + (int)rank * TP_BM + quad * 32;
+            const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
+#pragma unroll 1
+            for (int cchunk = 0; cchunk < TP_BN / 32; ++cchunk) {
+                unsigned r[32];
+                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + cchunk * 32, r);
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    *reinterpret_cast<float4*>(blk + lane * TG_EPI_LD + 4 * v) =
+                        make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                    __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                __syncwarp();
+                const int col = tn * TP_BN + cchunk * 32 + sub_c;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = i * 4 + sub_r;
+                    const float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
+                    if (row0 + rr < P.N && col < P.N)
+                        __stcs(reinterpret_cast<float4*>(P.gw + (size_t)(row0 + rr) * P.N + col), val);
+                }
+                __syncwarp();
+            }
+            tg_fence_before();
+            __syncwarp();
+            if (lane == 0) tp_arrive_remote(leader_acc_empty0 + ab * (unsigned)sizeof(unsigned long long));
+        }
+    }
+
+    // Neither CTA may leave (or free tensor memory) while the other can still reach it: the
+    // leader's multiplications read the peer's shared memory and write the peer's tensor
+    // memory, and its commits arrive on the peer's barriers.
+    tg_fence_before();
+    __syncthreads();
+    if (sh->abort_flag && threadIdx.x == 0 && rank == 0) {
+        // after giving up: let loads that are still landing finish (bounded)
+        const unsigned long long t0 = tg_timer();
+        while (tg_timer() - t0 < 200000ull) { }
+    }
+    tp_cluster_sync();
+    if (warp == 1) {
+        tg_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((unsigned)(TP_ACC * TP_BN)) : "memory");
+    }
+}
+
+
 typedef CUresult (*tg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -341,6 +636,29 @@ bool tg_encode_operand(CUtensorMap* m, const float* base, int N, int B)
 
 }  // namespace
 
+// Largest number of CTA pairs of the two-SM kernel that can be resident at once (0: unusable).
+// Queried once per device; also opts the kernel in to its dynamic shared memory.
+static int tp_max_pairs(const lf_ctx* c)
+{
+    static int cached_dev = -1, cached = 0;
+    if (cached_dev == c->device) return cached;
+    int n = 0;
+    if ((size_t)c->smem_optin >= TP_SMEM_BYTES &&
+        cudaFuncSetAttribute(k_gw_gemm_tf32_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)TP_SMEM_BYTES) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        cfg.gridDim = dim3(2 * 16); cfg.blockDim = dim3(TP_THREADS); cfg.dynamicSmemBytes = TP_SMEM_BYTES;
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, k_gw_gemm_tf32_pair, &cfg) != cudaSuccess) n = 0;
+    }
+    cudaGetLastError();
+    cached_dev = c->device; cached = n;
+    return n;
+}
+
 bool lf_tf32_supported(const lf_ctx* c)
 {
     if (c->B < 2) return false;
@@ -356,6 +674,7 @@ bool lf_tf32_supported(const lf_ctx* c)
         }
         attr_dev = c->device;
     }
+    tp_max_pairs(c);
     return true;
 }
 
@@ -369,15 +688,35 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
     }
     TgParams P;
     P.N = c->N; P.B = c->B;
-    P.tiles_m = (c->N + TG_BM - 1) / TG_BM;
-    P.tiles_n = (c->N + TG_BN - 1) / TG_BN;
     P.gw = gw_l;
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
+    const int max_pairs = c->tc_pair_kernels && c->B <= TP_MAX_KS * TG_BK ? tp_max_pairs(c) : 0;
+    if (max_pairs > 0) {
+        // two-SM kernel: the delta operand of a 256-row block stays in shared memory
+        P.tiles_m = (c->N + 2 * TP_BM - 1) / (2 * TP_BM);
+        P.tiles_n = (c->N + TP_BN - 1) / TP_BN;
+        const int tiles = P.tiles_m * P.tiles_n;
+        const int pairs = tiles < max_pairs ? tiles : max_pairs;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(TP_THREADS); cfg.dynamicSmemBytes = TP_SMEM_BYTES;
+        cfg.stream = s;
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_gw_gemm_tf32_pair, map_d, map_a, P));
+        c->stats.gw_tiling = LF_TC_TILING_TWO_SM;
+        *launches += 1;
+        return LF_OK;
+    }
+    P.tiles_m = (c->N + TG_BM - 1) / TG_BM;
+    P.tiles_n = (c->N + TG_BN - 1) / TG_BN;
     const int tiles = P.tiles_m * P.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     k_gw_gemm_tf32<<<grid, TG_THREADS, TG_SMEM_BYTES, s>>>(map_d, map_a, P);
     LF_CUDA_TRY(c, cudaGetLastError());
+    c->stats.gw_tiling = LF_TC_TILING_ONE_SM;
     *launches += 1;
     return LF_OK;
 }

@@ -36,6 +36,7 @@ struct lf_ctx {
     long long wait_budget_us;
     int use_graph;
     int opt_delta_math;      // enum lf_delta_math
+    int tc_pair_kernels;     // 1: the tensor-core contractions may use the two-SM (CTA pair) kernels
     int withhold;            // test hook: one chain CTA withholds its published delta values
 
     // workspace (device)

@@ -37,17 +37,26 @@ def test_single_sample_parity(L, N, k, variant):
     assert torch.equal(out["gb"], out["delta"][:, 0])  # Eq. bp3, single sample
 
 
-@pytest.mark.parametrize("delta_math", [lf.LF_DELTA_MATH_FP32, lf.LF_DELTA_MATH_3XTF32])
+@pytest.mark.parametrize("delta_math,tiling", [(lf.LF_DELTA_MATH_FP32, lf.LF_TC_TILING_AUTO),
+                                               (lf.LF_DELTA_MATH_3XTF32, lf.LF_TC_TILING_ONE_SM),
+                                               (lf.LF_DELTA_MATH_3XTF32, lf.LF_TC_TILING_TWO_SM)])
 @pytest.mark.parametrize("L,N,B,k", [(2, 8, 2, 1), (3, 68, 3, 2), (3, 256, 16, 4),
-                                     (4, 132, 70, 3), (2, 320, 129, 2), (5, 1028, 260, 2)])
-def test_minibatch_fp32_parity(L, N, B, k, delta_math):
-    # fp32 gate (1e-5 per tensor per layer) for both forms of the delta recurrence: fp32 on
-    # the CUDA cores, and the tensor cores with every operand split into two TF32 numbers.
+                                     (4, 132, 70, 3), (2, 320, 129, 2), (5, 1028, 260, 2),
+                                     (3, 772, 256, 1), (2, 2052, 515, 2)])
+def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
+    # fp32 gate (1e-5 per tensor per layer) for every form of the delta recurrence (and of the
+    # forward pass, which shares its kernels): fp32 on the CUDA cores, and the tensor cores with
+    # every operand split into two TF32 numbers, one CTA per tile or a CTA pair per tile (pairs
+    # take over above 128 samples: B = 129 and 260 leave a pair's second half nearly empty,
+    # B = 515 needs three 256-sample blocks, N = 2052 several K splits with a ragged last one).
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=N + B)
-    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math)
+    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math, tc_tiling=tiling)
     assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == delta_math
     assert stats["device_status"] == 0
+    if delta_math == lf.LF_DELTA_MATH_3XTF32 and L > 1:
+        want = lf.LF_TC_TILING_TWO_SM if (tiling == lf.LF_TC_TILING_TWO_SM and B > 128) else lf.LF_TC_TILING_ONE_SM
+        assert stats["delta_tiling"] == want
     ref = oracle_pass(t, want_gw=True)
     compare_all(cfg, out, ref)
 
@@ -129,15 +138,19 @@ def test_config3_parity_long_chain():
         assert torch.equal(out["gw"][l], torch.outer(out["delta"][l, 0], out["a"][l, 0]))
 
 
+@pytest.mark.parametrize("tiling", [lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM])
 @pytest.mark.parametrize("L,N,B,k", [(2, 256, 32, 1), (3, 512, 256, 2), (2, 388, 70, 2), (2, 132, 16, 1),
-                                     (2, 1028, 129, 3), (2, 64, 8, 1)])
-def test_minibatch_tf32_weight_gradient(L, N, B, k):
+                                     (2, 1028, 129, 3), (2, 64, 8, 1), (2, 2308, 96, 2)])
+def test_minibatch_tf32_weight_gradient(L, N, B, k, tiling):
     # Eq. bp4 on the tensor cores: relative Frobenius error per layer <= 5e-3 against the
-    # float64 oracle; everything else on the path stays fp32 and keeps the 1e-5 gate.
+    # float64 oracle; everything else on the path stays fp32 and keeps the 1e-5 gate.  Both
+    # tilings: one CTA per tile, and CTA pairs with the delta operand resident (N = 2308 gives
+    # pairs runs of several tiles that cross a row-block boundary, with ragged last tiles).
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=3 * N + B)
-    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_TF32)
+    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_TF32, tc_tiling=tiling)
     assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
+    assert stats["gw_tiling"] == tiling
     ref = oracle_pass(t, want_gw=True)
     worst = compare_all(cfg, out, ref, gw_tf32=True)
     # and against the fp32 CUDA-core contraction of the same delta and a
@@ -146,6 +159,31 @@ def test_minibatch_tf32_weight_gradient(L, N, B, k):
     den = out32["gw"].double().flatten(1).norm(dim=1)
     assert float((num / den).max()) <= 5e-3
     print("tf32", (L, N, B), worst["gw"], float((num / den).max()))
+
+
+def test_tf32_pair_kernel_long_runs():
+    # N = 6148, B = 64: about sixteen 256 x 128 tiles per CTA pair, so every accumulator in tensor
+    # memory and every barrier is reused several times and every run crosses row blocks.  One
+    # layer; the oracle's Eq. bp4 is applied to the GPU's own delta and activations.
+    from oracle import lf_oracle as orc
+    from lf_testlib import rel_frobenius, TF32_TOL
+    L, N, B = 1, 6148, 64
+    cfg = dict(L=L, N=N, B=B, k=1)
+    t = _inputs(L, N, B, y="onehot", seed=77)
+    outs = {}
+    for tiling in (lf.LF_TC_TILING_TWO_SM, lf.LF_TC_TILING_ONE_SM):
+        out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_TF32, tc_tiling=tiling, repeat=2)
+        assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
+        assert stats["gw_tiling"] == tiling
+        outs[tiling] = out["gw"][0].cpu().numpy()
+    ref = orc.grad_w(out["delta"][0].cpu().numpy().astype(np.float64),
+                     out["a"][0].cpu().numpy().astype(np.float64))
+    for tiling, g in outs.items():
+        assert np.all(np.isfinite(g))
+        e = rel_frobenius(g, ref)
+        assert e <= TF32_TOL, (tiling, e)
+    # the two tilings multiply the same truncated operands and add the samples in the same order
+    assert np.array_equal(outs[lf.LF_TC_TILING_TWO_SM], outs[lf.LF_TC_TILING_ONE_SM])
 
 
 def test_config4_minibatch_full_size_sampled():
