@@ -382,7 +382,7 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 // finished stage into the running sums -- have warps of their own here, so they overlap:
 //   warp 0       TMA producer: this CTA's 128 samples of D and its 128 columns of W per stage;
 //   warp 1       leader CTA (cluster rank 0) only: issues the products for both CTAs;
-//   warps 4-7    split this CTA's stage into hi/lo (in place + beside it);
+//   warps 2-7    split this CTA's stage into hi/lo (in place + beside it);
 //   warps 8-15   running sums of this CTA's 128 samples: a thread holds one sample and 128 of
 //                the 256 columns in registers.  They need about 200 registers per thread and the
 //                other warps few, so the warpgroups re-divide the register file at the start
@@ -398,7 +398,7 @@ constexpr int DP_B_BYTES = (DP_BNH / 32) * DG_BOX_BYTES; // 16 KiB (either opera
 constexpr int DP_RAW_BYTES = DG_A_BYTES + DP_B_BYTES;    // 32 KiB per CTA and stage from TMA
 constexpr int DP_STAGE_BYTES = 2 * DP_RAW_BYTES;         // hi (in place) + lo
 constexpr int DP_THREADS = 512;                          // four warpgroups
-constexpr int DP_SPLITTERS = 128;                        // warps 4-7
+constexpr int DP_SPLITTERS = 192;                        // warps 2-7
 constexpr int DP_REGS_LAUNCH = 128, DP_REGS_SMALL = 48, DP_REGS_SUM = 208;
 static_assert(2 * 128 * DP_REGS_SMALL + 2 * 128 * DP_REGS_SUM <= DP_THREADS * DP_REGS_LAUNCH,
               "the warpgroups' register shares must fit into what the CTA is launched with");
@@ -409,7 +409,7 @@ constexpr size_t DP_SMEM_BYTES = (size_t)DP_STAGES * DP_STAGE_BYTES + DP_EPI_BYT
 
 struct DpShared {
     unsigned long long full[DP_STAGES];        // this CTA's TMA data of the stage has landed
-    unsigned long long split_done[DP_STAGES];  // leader: hi/lo of both CTAs written (8 warp arrivals)
+    unsigned long long split_done[DP_STAGES];  // leader: hi/lo of both CTAs written (12 warp arrivals)
     unsigned long long empty[DP_STAGES];       // both: the multiplications that read the stage are done
     unsigned long long acc_full[2];            // both: stage accumulator p holds a finished stage
     unsigned long long acc_empty[2];           // leader: accumulator p drained by both CTAs (16 warp arrivals)
@@ -538,7 +538,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     if (threadIdx.x == 0) {
         for (int i = 0; i < DP_STAGES; ++i) {
             dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
-            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 8);
+            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 2 * DP_SPLITTERS / 32);
             dg_mbar_init(dg_smem_u32(&sh->empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -628,9 +628,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     }
                 }
             }
-        } else if (warp >= 4) {
-            // ------------------------------ operand split (hi/lo): warps 4..7 ------------------
-            const int tt = threadIdx.x - 128;
+        } else {
+            // ------------------------------ operand split (hi/lo): warps 2..7 ------------------
+            const int tt = threadIdx.x - 64;
             const unsigned leader_split_done0 = dp_map_to_rank(dg_smem_u32(&sh->split_done[0]), 0);
             unsigned it = 0;
             bool ok = true;
@@ -641,8 +641,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES);
                     float4* lo = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES + DP_RAW_BYTES);
 #pragma unroll 4
-                    for (int i = 0; i < DP_RAW_BYTES / 16 / DP_SPLITTERS; ++i) {
+                    for (int i = 0; i < (DP_RAW_BYTES / 16 + DP_SPLITTERS - 1) / DP_SPLITTERS; ++i) {
                         const int idx = tt + i * DP_SPLITTERS;
+                        if (idx >= DP_RAW_BYTES / 16) break;
                         const float4 v = raw[idx];
                         const float4 h = make_float4(dg_tf32_rn(v.x), dg_tf32_rn(v.y), dg_tf32_rn(v.z), dg_tf32_rn(v.w));
                         raw[idx] = h;
@@ -674,12 +675,12 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 if (!dp_wait(dg_smem_u32(&sh->acc_full[p]), (it >> 1) & 1u, P, sh)) { ok = false; break; }
                 dg_fence_after();
 #pragma unroll
-                for (int cchunk = 0; cchunk < DP_BNH / 32; ++cchunk) {
-                    unsigned r[32];
-                    dg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DP_BN + half * DP_BNH + cchunk * 32, r);
+                for (int cchunk = 0; cchunk < DP_BNH / 64; ++cchunk) {
+                    unsigned r[64];
+                    dp_tmem_ld64(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DP_BN + half * DP_BNH + cchunk * 64, r);
 #pragma unroll
-                    for (int v = 0; v < 32; ++v)
-                        acc[cchunk * 32 + v] += __uint_as_float(r[v]);
+                    for (int v = 0; v < 64; ++v)
+                        acc[cchunk * 64 + v] += __uint_as_float(r[v]);
                 }
                 dg_fence_before();
                 __syncwarp();

@@ -161,6 +161,18 @@ __device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 32 lanes x 16 consecutive fp32 columns of tensor memory -> 16 registers per thread
+__device__ __forceinline__ void tg_tmem_ld16(unsigned taddr, unsigned (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(TG_THREADS, 1)
 k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_a,
                const TgParams P)
@@ -308,30 +320,32 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
 
 // ================================================================================================
 // Two-SM form for batches of at most 256 samples: a pair of CTAs (one thread-block cluster) works
-// on 256 rows of gw at a time with tcgen05.mma.cta_group::2 (M = 256, N = 128, K = 8).
+// on 256 rows of gw at a time with tcgen05.mma.cta_group::2 (M = 256, N = 256, K = 8; an
+// instruction of this kind takes about as long for 128 columns as for 256, so tiles are 256 wide).
 //   * The delta operand of the pair's 256 rows -- every sample of it, at most 128 KiB per CTA --
 //     is loaded ONCE per row block and stays in shared memory while the pair walks along the
-//     row block; only the activation operand streams (64 columns x 32 samples = 8 KiB per CTA
-//     and stage), and the two CTAs read each other's half of it.  Per 64 KiB of gradient a CTA
-//     stores it then loads 64 KiB of operands, against 192 KiB in the one-SM kernel above, whose
-//     speed is set by exactly those loads.
-//   * 256 x 128 pair tiles, each pair a contiguous run of them in row-major order (a run crosses
-//     a row-block boundary at most once when N <= 256 * pairs); four accumulators of 128 columns
-//     in tensor memory, so the epilogue of a tile overlaps the next tiles' multiplications.
+//     row block; only the activation operand streams (128 columns x 32 samples = 16 KiB per CTA
+//     and stage), and the two CTAs read each other's half of it.  Per 128 KiB of gradient a CTA
+//     stores it then loads 128 KiB of operands, against 384 KiB in the one-SM kernel above,
+//     which waits for those loads (a multiprocessor takes in about 32 bytes per clock from L2).
+//   * 256 x 256 pair tiles, each pair a contiguous run of them in row-major order; two
+//     accumulators of 256 columns in tensor memory, so the epilogue of a tile overlaps the
+//     next tile's multiplications.
 // Hand-offs between the two CTAs: both producers credit their loads to the LEADER's (rank 0)
 // "full" barriers; the leader's tcgen05.commit reaches the "empty" / "accumulator full" barriers
 // of both CTAs at once; the epilogue warps of both CTAs arrive on the leader's "accumulator
 // empty" barrier.  All waits are bounded as above.
 constexpr int TP_BM = 128;                               // rows of gw per CTA (256 per pair)
-constexpr int TP_BN = 128;                               // columns of a pair tile (64 loaded per CTA)
+constexpr int TP_BN = 256;                               // columns of a pair tile (128 loaded per CTA)
 constexpr int TP_MAX_KS = 8;                             // at most 8 x 32 = 256 samples
-constexpr int TP_STAGES = 8;
-constexpr int TP_ACC = 4;                                // accumulators of TP_BN columns
+constexpr int TP_STAGES = 3;
+constexpr int TP_ACC = 2;                                // accumulators of TP_BN columns
 constexpr int TP_A_STAGE_BYTES = (TP_BM / 32) * TG_BOX_BYTES;        // 16 KiB: 128 rows x 32 samples
-constexpr int TP_B_STAGE_BYTES = (TP_BN / 2 / 32) * TG_BOX_BYTES;    //  8 KiB:  64 columns x 32 samples
+constexpr int TP_B_STAGE_BYTES = (TP_BN / 2 / 32) * TG_BOX_BYTES;    // 16 KiB: 128 columns x 32 samples
 constexpr int TP_A_BYTES = TP_MAX_KS * TP_A_STAGE_BYTES;             // 128 KiB
-constexpr int TP_THREADS = 192;
-constexpr size_t TP_SMEM_BYTES = (size_t)TP_A_BYTES + (size_t)TP_STAGES * TP_B_STAGE_BYTES + TG_EPI_BYTES +
+constexpr int TP_THREADS = 320;                          // producer, issuer, eight epilogue warps
+constexpr int TP_EPI_BYTES = 8 * 32 * TG_EPI_LD * 4;    // one 32 x 32 block per epilogue warp
+constexpr size_t TP_SMEM_BYTES = (size_t)TP_A_BYTES + (size_t)TP_STAGES * TP_B_STAGE_BYTES + TP_EPI_BYTES +
                                  1024 /*alignment slack*/ + 512;
 
 struct TpShared {
@@ -431,7 +445,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
         (reinterpret_cast<uintptr_t>(tg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
     unsigned char* b_ring = a_res + TP_A_BYTES;
     float* epi = reinterpret_cast<float*>(b_ring + (size_t)TP_STAGES * TP_B_STAGE_BYTES);
-    TpShared* sh = reinterpret_cast<TpShared*>(reinterpret_cast<unsigned char*>(epi) + TG_EPI_BYTES);
+    TpShared* sh = reinterpret_cast<TpShared*>(reinterpret_cast<unsigned char*>(epi) + TP_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned rank = tp_cluster_rank();          // 0 = leader (issues the multiplications)
@@ -450,7 +464,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
         }
         for (int i = 0; i < TP_ACC; ++i) {
             tg_mbar_init(tg_smem_u32(&sh->acc_full[i]), 1);
-            tg_mbar_init(tg_smem_u32(&sh->acc_empty[i]), 8);   // four epilogue warps of each CTA
+            tg_mbar_init(tg_smem_u32(&sh->acc_empty[i]), 16);  // eight epilogue warps of each CTA
         }
         sh->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -544,35 +558,41 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             }
         }
     } else {
-        // ------------------------------ epilogue (warps 2..5 of both CTAs) ---------------------
+        // ------------------------------ epilogue (warps 2..9 of both CTAs) ---------------------
+        // Two warps per TMEM lane quadrant, each taking 128 of the tile's 256 columns in blocks
+        // of 32 x 32 that are turned through shared memory, so that a warp stores whole 128-byte
+        // row segments.
         const int quad = warp & 3;                 // the TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;
         const unsigned leader_acc_empty0 = tp_map_to_rank(tg_smem_u32(&sh->acc_empty[0]), 0);
+        float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
+        const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
         unsigned tile_i = 0;
         for (int t = t_begin; t < t_end; ++t, ++tile_i) {
             const int rb = t / P.tiles_n, tn = t - rb * P.tiles_n;
             const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
             if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
             tg_fence_after();
-            float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
-            const int row0 = rb * 2 * TP_BM + (int)rank * TP_BM + quad * 32;
-            const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
+            const int row0 = rb * 2 * TP_BM + (int)rank * TP_BM + quad * 32 + sub_r;
+            const int col0 = tn * TP_BN + half * (TP_BN / 2) + sub_c;
+            float* out_row = P.gw + (size_t)row0 * P.N + col0;
+            const size_t row_step = (size_t)4 * P.N;
 #pragma unroll 1
-            for (int cchunk = 0; cchunk < TP_BN / 32; ++cchunk) {
+            for (int cchunk = 0; cchunk < TP_BN / 2 / 32; ++cchunk) {
                 unsigned r[32];
-                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + cchunk * 32, r);
+                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + half * (TP_BN / 2) + cchunk * 32, r);
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
                     *reinterpret_cast<float4*>(blk + lane * TG_EPI_LD + 4 * v) =
                         make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
                                     __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
                 __syncwarp();
-                const int col = tn * TP_BN + cchunk * 32 + sub_c;
+                if (col0 + cchunk * 32 < P.N) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int rr = i * 4 + sub_r;
-                    const float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
-                    if (row0 + rr < P.N && col < P.N)
-                        __stcs(reinterpret_cast<float4*>(P.gw + (size_t)(row0 + rr) * P.N + col), val);
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 val = *reinterpret_cast<const float4*>(blk + (i * 4 + sub_r) * TG_EPI_LD + sub_c);
+                        if (row0 + i * 4 < P.N) __stcs(reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 32), val);
+                    }
                 }
                 __syncwarp();
             }

@@ -162,7 +162,7 @@ def test_minibatch_tf32_weight_gradient(L, N, B, k, tiling):
 
 
 def test_tf32_pair_kernel_long_runs():
-    # N = 6148, B = 64: about sixteen 256 x 128 tiles per CTA pair, so every accumulator in tensor
+    # N = 6148, B = 64: about eight 256 x 256 tiles per CTA pair, so every accumulator in tensor
     # memory and every barrier is reused several times and every run crosses row blocks.  One
     # layer; the oracle's Eq. bp4 is applied to the GPU's own delta and activations.
     from oracle import lf_oracle as orc
