@@ -44,6 +44,8 @@ struct DgParams {
     int N, B;
     int tiles_m, tiles_n, splits;
     int k_per_split;          // j range of one split (multiple of DG_BK)
+    int kb_per_tile;          // two-SM kernel: K blocks (of DG_BK) of one tile
+    int g_total;              // two-SM kernel: tiles * kb_per_tile, dealt to the pairs in contiguous runs
     float* partial;           // [splits][B][N]
     unsigned* status;
     unsigned long long budget_ns;
@@ -390,7 +392,12 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 // Hand-offs across the pair: the splitting warps of both CTAs arrive on the leader's "split done"
 // barrier, the leader's tcgen05.commit reaches the "stage free" and "accumulator full" barriers
 // of both CTAs, the summing warps of both arrive on the leader's "accumulator drained" barrier.
-// Arithmetic and summation order per output element are those of the one-SM kernel above.
+// Work is dealt by K block, not by tile: the tiles x K-blocks sequence is cut into one contiguous
+// run per pair (runs differ by at most one block), so a pair may finish one tile's tail and
+// start the next tile.  Every run segment inside a tile writes its partial sums to the slot
+// given by its position among the segments of that tile; k_delta_finish / k_forward_finish add
+// a tile's slots in that order, so the result does not depend on timing.
+// Arithmetic per output element is that of the one-SM kernel above.
 constexpr int DP_BN = 256;                               // columns of a pair tile (128 loaded per CTA)
 constexpr int DP_BNH = DP_BN / 2;
 constexpr int DP_STAGES = 3;
@@ -481,6 +488,30 @@ __device__ __forceinline__ bool dp_wait(unsigned bar, unsigned parity, const DgP
     }
     return true;
 }
+// The pair whose run contains block g when g_total blocks are cut into n_pairs runs
+// [p * g_total / n_pairs, (p + 1) * g_total / n_pairs).
+// (g_total * (n_pairs + 1) stays below 2^31: checked by the host before this tiling is chosen.)
+__host__ __device__ __forceinline__ int dp_owner(int g, int g_total, int n_pairs)
+{
+    return ((g + 1) * n_pairs - 1) / g_total;
+}
+struct DpSegment {
+    int tile;       // tm * tiles_n + tn
+    int kb0, kb1;   // K blocks [kb0, kb1) of that tile
+    int slot;       // which partial-sum slot of the tile this segment writes
+};
+// Next segment of the run [g, g1): advances g.  Every role of the kernel walks the same sequence.
+__device__ __forceinline__ bool dp_next_segment(int& g, int g1, const DgParams& P, int pair, int n_pairs, DpSegment& sg)
+{
+    if (g >= g1) return false;
+    sg.tile = g / P.kb_per_tile;
+    sg.kb0 = g - sg.tile * P.kb_per_tile;
+    const int left = g1 - g;
+    sg.kb1 = left < P.kb_per_tile - sg.kb0 ? sg.kb0 + left : P.kb_per_tile;
+    sg.slot = pair - dp_owner(sg.tile * P.kb_per_tile, P.g_total, n_pairs);
+    g += sg.kb1 - sg.kb0;
+    return true;
+}
 __device__ __forceinline__ unsigned dp_idesc(bool w_kmajor)
 {
     unsigned d = 0;
@@ -532,8 +563,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned rank = dp_cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_units = P.tiles_m * P.tiles_n * P.splits;     // tiles_m: 256-sample blocks, tiles_n: 256-column blocks
-    const int n_k = P.k_per_split / DG_BK;
+    const int g_begin = (int)((long long)P.g_total * pair / n_pairs), g_end = (int)((long long)P.g_total * (pair + 1) / n_pairs);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < DP_STAGES; ++i) {
@@ -566,9 +596,10 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             if (lane == 0) {
                 unsigned it = 0;
                 bool ok = true;
-                for (int u = pair; u < n_units && ok; u += n_pairs) {
-                    const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
-                    const int j0 = sp * P.k_per_split;
+                DpSegment sg;
+                for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
+                    const int tn = sg.tile % P.tiles_n, tm = sg.tile / P.tiles_n;
+                    const int j0 = sg.kb0 * DG_BK, n_k = sg.kb1 - sg.kb0;
                     const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM;       // my samples
                     const int col0 = tn * DP_BN + (int)rank * DP_BNH;          // my columns of W
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
@@ -603,7 +634,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 const unsigned idesc = dp_idesc(W_KMAJOR);
                 unsigned it = 0;
                 bool ok = true;
-                for (int u = pair; u < n_units && ok; u += n_pairs) {
+                DpSegment sg;
+                for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
+                    const int n_k = sg.kb1 - sg.kb0;
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
                         const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
                         const unsigned p = it & 1u, p_use = it >> 1;
@@ -634,7 +667,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             const unsigned leader_split_done0 = dp_map_to_rank(dg_smem_u32(&sh->split_done[0]), 0);
             unsigned it = 0;
             bool ok = true;
-            for (int u = pair; u < n_units && ok; u += n_pairs) {
+            DpSegment sg;
+            for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
+                const int n_k = sg.kb1 - sg.kb0;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
                     if (!dp_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
@@ -665,8 +700,10 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
         unsigned it = 0;
         bool ok = true;
         float acc[DP_BNH];     // this thread's sample, its 128 columns of the tile
-        for (int u = pair; u < n_units && ok; u += n_pairs) {
-            const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
+        DpSegment sg;
+        for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
+            const int tn = sg.tile % P.tiles_n, tm = sg.tile / P.tiles_n, sp = sg.slot;
+            const int n_k = sg.kb1 - sg.kb0;
 #pragma unroll
             for (int v = 0; v < DP_BNH; ++v) acc[v] = 0.f;
             for (int ks = 0; ks < n_k; ++ks, ++it) {
@@ -726,13 +763,30 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     }
 }
 
-// delta^l = (sum over the K splits, in split order) * sigma'(z^l), sigma' = a (1 - a)
+// How many partial-sum slots hold a contribution to output element i (float4 index into [B][N]).
+// One-SM kernel: the same number of K splits everywhere.  Two-SM kernel (n_pairs > 0): as many as
+// there are run segments in the element's tile.
+struct DgSlots {
+    int splits;
+    int n_pairs, tiles_n, kb_per_tile, row4;   // row4 = N / 4
+    int g_total;
+};
+__device__ __forceinline__ int dg_slot_count(const DgSlots& S, size_t i)
+{
+    if (S.n_pairs == 0) return S.splits;
+    const int b = (int)(i / (size_t)S.row4), n = (int)(i % (size_t)S.row4) * 4;
+    const int g0 = ((b / (2 * DG_BM)) * S.tiles_n + n / DP_BN) * S.kb_per_tile;
+    return dp_owner(g0 + S.kb_per_tile - 1, S.g_total, S.n_pairs) - dp_owner(g0, S.g_total, S.n_pairs) + 1;
+}
+
+// delta^l = (sum over the partial-sum slots, in slot order) * sigma'(z^l), sigma' = a (1 - a)
 __global__ void __launch_bounds__(256)
 k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
-               size_t n4, int splits)
+               size_t n4, const DgSlots S)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
+    const int splits = dg_slot_count(S, i);
     float4 s = reinterpret_cast<const float4*>(partial)[i];
     for (int sp = 1; sp < splits; ++sp) {
         const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
@@ -743,13 +797,14 @@ k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l,
                                                         s.z * (av.z * (1.0f - av.z)), s.w * (av.w * (1.0f - av.w)));
 }
 
-// forward: z^l = (sum over the K splits) + b^l ; a^l = sigma(z^l)
+// forward: z^l = (sum over the partial-sum slots) + b^l ; a^l = sigma(z^l)
 __global__ void __launch_bounds__(256)
 k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_l, float* __restrict__ z_l,
-                 float* __restrict__ a_l, size_t n4, int n4_row, int splits)
+                 float* __restrict__ a_l, size_t n4, int n4_row, const DgSlots S)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
+    const int splits = dg_slot_count(S, i);
     float4 s = reinterpret_cast<const float4*>(partial)[i];
     for (int sp = 1; sp < splits; ++sp) {
         const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
@@ -783,11 +838,15 @@ dg_encode_fn dg_get_encode()
     return fn;
 }
 
-struct DgPlan { int tiles_m, tiles_n, splits, k_per_split; };
+struct DgPlan {
+    int tiles_m, tiles_n, splits, k_per_split;
+    int pairs, kb_per_tile;      // two-SM kernel (pairs > 0): launched pairs and K blocks per tile
+    int g_total;
+};
 
 DgPlan dg_plan(const lf_ctx* c)
 {
-    DgPlan p;
+    DgPlan p = {};
     p.tiles_m = (c->B + DG_BM - 1) / DG_BM;
     p.tiles_n = (c->N + DG_BN - 1) / DG_BN;
     int s = c->sm_count / (p.tiles_m * p.tiles_n);
@@ -830,22 +889,34 @@ int dp_max_pairs(const lf_ctx* c)
 }
 
 // The two-SM kernels pay off once a pair's 256 samples are more than half filled.
-bool dp_use_pairs(const lf_ctx* c) { return c->tc_pair_kernels && c->B > DG_BM && dp_max_pairs(c) > 0; }
+bool dp_use_pairs(const lf_ctx* c);
 
-DgPlan dp_plan(const lf_ctx* c, int pairs)
+// Two-SM kernel: tiles x K-blocks cut into one contiguous run per pair; `splits` becomes the
+// largest number of run segments (= partial-sum slots) any tile has.
+DgPlan dp_plan(const lf_ctx* c, int max_pairs)
 {
-    DgPlan p;
+    DgPlan p = {};
     p.tiles_m = (c->B + 2 * DG_BM - 1) / (2 * DG_BM);
     p.tiles_n = (c->N + DP_BN - 1) / DP_BN;
-    int s = pairs / (p.tiles_m * p.tiles_n);
-    if (s < 1) s = 1;
-    if (s > 8) s = 8;
-    const int kb = (c->N + DG_BK - 1) / DG_BK;
-    if (s > kb) s = kb;
-    const int kb_per = (kb + s - 1) / s;
-    p.splits = (kb + kb_per - 1) / kb_per;
-    p.k_per_split = kb_per * DG_BK;
+    p.kb_per_tile = (c->N + DG_BK - 1) / DG_BK;
+    p.k_per_split = p.kb_per_tile * DG_BK;
+    const int tiles = p.tiles_m * p.tiles_n;
+    const long long g_total = (long long)tiles * p.kb_per_tile;
+    if (g_total * (max_pairs + 1) >= (1ll << 31)) return p;      // pairs == 0: not usable at this size
+    p.g_total = (int)g_total;
+    p.pairs = p.g_total < max_pairs ? p.g_total : max_pairs;
+    p.splits = 1;
+    for (int t = 0; t < tiles; ++t) {
+        const int g0 = t * p.kb_per_tile;
+        const int n = dp_owner(g0 + p.kb_per_tile - 1, p.g_total, p.pairs) - dp_owner(g0, p.g_total, p.pairs) + 1;
+        if (n > p.splits) p.splits = n;
+    }
     return p;
+}
+
+bool dp_use_pairs(const lf_ctx* c)
+{
+    return c->tc_pair_kernels && c->B > DG_BM && dp_max_pairs(c) > 0 && dp_plan(c, dp_max_pairs(c)).pairs > 0;
 }
 
 }  // namespace
@@ -880,6 +951,14 @@ bool lf_delta_tc_supported(const lf_ctx* c)
     }
     dp_max_pairs(c);
     return true;
+}
+
+static DgSlots dg_slots(const lf_ctx* c, const DgPlan& pl)
+{
+    DgSlots S = {};
+    S.splits = pl.splits; S.n_pairs = pl.pairs; S.tiles_n = pl.tiles_n; S.kb_per_tile = pl.kb_per_tile;
+    S.row4 = c->N / 4; S.g_total = pl.g_total;
+    return S;
 }
 
 // Encode the two operand maps and launch one contraction into c->dg_partial.
@@ -918,6 +997,7 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
     DgParams P;
     P.N = c->N; P.B = c->B;
     P.tiles_m = pl.tiles_m; P.tiles_n = pl.tiles_n; P.splits = pl.splits; P.k_per_split = pl.k_per_split;
+    P.kb_per_tile = pl.kb_per_tile; P.g_total = pl.g_total;
     P.partial = c->dg_partial;
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
@@ -925,7 +1005,7 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
     if (pairs) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
-        cfg.gridDim = dim3(2 * (units < max_pairs ? units : max_pairs));
+        cfg.gridDim = dim3(2 * pl.pairs);
         cfg.blockDim = dim3(DP_THREADS); cfg.dynamicSmemBytes = DP_SMEM_BYTES; cfg.stream = s;
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -956,7 +1036,7 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     int rc = dg_launch(c, delta_up, w_up, false, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * c->N / 4;
-    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, pl.splits);
+    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(c, pl));
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
@@ -970,7 +1050,7 @@ int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const floa
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * c->N / 4;
     k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, c->N / 4,
-                                                                  pl.splits);
+                                                                  dg_slots(c, pl));
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;

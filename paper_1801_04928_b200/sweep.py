@@ -86,7 +86,8 @@ def main():
                     row = dict(L=L, N=N, B=B, k=k, variant=names[st["variant"]], requested=names[variant],
                                gw_math={1: "fp32", 2: "tf32"}[st["gw_math"]], ms=ms,
                                layers_per_s=L / (ms * 1e-3), alg_GBs=alg / (ms * 1e-3) / 1e9,
-                               chain_ctas=st["chain_ctas"], worker_ctas=st["worker_ctas"])
+                               chain_ctas=st["chain_ctas"], worker_ctas=st["worker_ctas"],
+                               gw_tiling=st["gw_tiling"], delta_tiling=st["delta_tiling"])
                     rows.append(row)
                     f.write(json.dumps(row) + "\n"); f.flush()
                     print(json.dumps(row), flush=True)
