@@ -16,6 +16,8 @@
  *   Section 2, Eq. bp3 : dC/db^l_j = delta^l_j
  *   Section 2, Eq. bp4 : dC/dw^l_jk = a^{l-1}_k delta^l_j
  *   Section 3, Algorithm 1 : the leapfrog schedule with k threads (lfo_backward_leapfrog)
+ *   (not in the paper)     : the gradient-descent step that consumes Eq. bp4, w - eta dC/dw
+ *                            (lfo_sgd_step); the paper ends with the gradients of one pass
  *
  * Readings taken where the paper is silent or garbled:
  *   - Eq. z prints no bias although b^l is defined and Eq. bp3 differentiates by it: the
@@ -308,4 +310,15 @@ int lfo_backward_leapfrog(int L, int N, int B, int k, const lfo_w_t *w, const do
     if (!writer) free(wr);
     if (!writes) free(ws);
     return 0;
+}
+
+/* One step of plain gradient descent on every weight matrix: w_new = w - eta * gw, with gw the
+ * Eq. bp4 gradients of a pass.  The paper has no counterpart (it ends with the gradients of
+ * one pass); this is the textbook definition of the step that consumes them, element by
+ * element in float64, so that a fused "gradient + update" kernel has something to be checked
+ * against.  Biases are left to the caller. */
+void lfo_sgd_step(int L, int N, const lfo_w_t *w, const double *gw, double eta, double *w_new)
+{
+    const size_t n = (size_t)L * N * N;
+    for (size_t i = 0; i < n; ++i) w_new[i] = (double)w[i] - eta * gw[i];
 }

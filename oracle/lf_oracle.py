@@ -78,6 +78,8 @@ def _lib(tag: str) -> ctypes.CDLL:
             lib.lfo_backward_leapfrog.argtypes = [i, i, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp,
                                                   _c_dp, _c_dp, _c_ip, _c_ip,
                                                   ctypes.POINTER(ctypes.c_longlong), i]
+            lib.lfo_sgd_step.restype = None
+            lib.lfo_sgd_step.argtypes = [i, i, wp, _c_dp, ctypes.c_double, _c_dp]
             assert lib.lfo_weight_bytes() == (8 if tag == "f64" else 4)
             _LIBS[tag] = lib
         return _LIBS[tag]
@@ -189,6 +191,16 @@ def backward_sequential(w, z, a, y, want_gw: bool = True):
     lib.lfo_backward_sequential(L, N, B, wp, _p(z), _p(a), _p(y), _p(delta),
                                 _p(gw) if want_gw else None, _p(gb))
     return delta, gw, gb
+
+
+def sgd_step(w, gw, eta: float):
+    """w - eta * gw for all L weight matrices (float64); not in the paper, see the C file."""
+    lib, w, wp = _w(w)
+    L, N, _ = w.shape
+    gw = _d(gw)
+    out = np.empty((L, N, N), dtype=np.float64)
+    lib.lfo_sgd_step(L, N, wp, _p(gw), float(eta), _p(out))
+    return out
 
 
 def backward_leapfrog(w, z, a, y, k: int, want_gw: bool = True, threads: bool = True):

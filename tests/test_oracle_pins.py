@@ -345,3 +345,56 @@ def test_leapfrog_recomputes_the_chain_in_every_thread():
             expect += k
             jj += k
     assert bp2 == expect and bp2 > L - 1
+
+
+# ---- the gradient-descent step that consumes Eq. bp4 (not in the paper) -------------------------
+def test_sgd_step_lowers_the_cost_by_eta_times_gradient_norm():
+    # First-order check of sign and scale, against the cost itself: for a small step
+    # C(w - eta g) - C(w) = -eta |g|^2 + O(eta^2).  A wrong sign gives +eta |g|^2, a missing
+    # eta or a step along something other than dC/dw changes the ratio.
+    L, N, B = 3, 6, 2
+    w, b, x, y = _net(L, N, B, seed=21)
+    z, a = orc.forward(w, b, x)
+    _, gw, _ = orc.backward_sequential(w, z, a, y)
+    c0 = orc.cost(a, y)
+    g2 = float(np.sum(gw * gw))
+    for eta in (1e-3, 1e-4):
+        w1 = orc.sgd_step(w, gw, eta)
+        _, a1 = orc.forward(w1, b, x)
+        drop = orc.cost(a1, y) - c0
+        assert drop < 0
+        assert abs(drop / (-eta * g2) - 1.0) < 50 * eta      # second-order remainder shrinks with eta
+
+
+def test_sgd_step_is_affine_in_eta_and_leaves_w_alone_at_zero():
+    L, N = 2, 5
+    w, b, x, y = _net(L, N, 1, seed=22)
+    z, a = orc.forward(w, b, x)
+    _, gw, _ = orc.backward_sequential(w, z, a, y)
+    assert np.array_equal(orc.sgd_step(w, gw, 0.0), w)
+    s1 = orc.sgd_step(w, gw, 0.25) - w
+    s2 = orc.sgd_step(w, gw, 0.5) - w
+    np.testing.assert_allclose(s2, 2.0 * s1, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(s1, -0.25 * gw, rtol=1e-12, atol=1e-15)
+
+
+def test_sgd_step_closed_form_on_the_zero_network():
+    # w = 0, b = 0: a = 1/2 everywhere, delta^L = (1/2 - y)/4 and the lower deltas vanish, so
+    # only the top matrix moves: w_new^L[j][k] = -eta (1/2 - y_j) / 8.
+    L, N, eta = 3, 4, 0.7
+    w = np.zeros((L, N, N)); b = np.zeros((L, N))
+    x = np.linspace(0.1, 0.9, N)[None, :]
+    y = np.array([[1.0, 0.0, 0.25, 0.5]])
+    z, a = orc.forward(w, b, x)
+    _, gw, _ = orc.backward_sequential(w, z, a, y)
+    w1 = orc.sgd_step(w, gw, eta)
+    assert np.all(w1[: L - 1] == 0.0)
+    want = np.repeat((-eta * (0.5 - y[0]) / 8.0)[:, None], N, axis=1)
+    np.testing.assert_allclose(w1[L - 1], want, rtol=1e-13, atol=1e-16)
+
+
+def test_sgd_step_float_weight_flavour_promotes_exactly():
+    rng = np.random.default_rng(23)
+    w32 = rng.standard_normal((2, 4, 4)).astype(np.float32)
+    gw = rng.standard_normal((2, 4, 4))
+    assert np.array_equal(orc.sgd_step(w32, gw, 0.3), orc.sgd_step(w32.astype(np.float64), gw, 0.3))
