@@ -81,8 +81,8 @@ enum lf_tc_tiling {
     LF_TC_TILING_AUTO = 0,   /* CTA pairs where they apply and the device can co-schedule them  */
     LF_TC_TILING_ONE_SM = 1, /* one CTA per tile                                                */
     LF_TC_TILING_TWO_SM = 2  /* CTA pairs: Eq. bp4 for B <= 256 (the delta operand of a row
-                                block stays in shared memory), Eq. bp2 / Eq. z for B > 128;
-                                other sizes use ONE_SM                                          */
+                                block stays in shared memory), Eq. bp2 / Eq. z for B > 128 and
+                                N >= 512; other sizes use ONE_SM                                */
 };
 
 enum lf_option {
@@ -156,6 +156,23 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
  */
 int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
                 float* delta, float* gw, float* gb);
+
+/*
+ * Backward pass fused with one step of gradient descent on the weights.  (The paper has no
+ * counterpart: it ends with the gradients of one pass.  This is the step that follows, folded
+ * into the gradient writer so that gw is never stored and read back.)  As lf_backward, except
+ * that in place of gw^l the call writes
+ *     w_new^l = w^l - eta * gw^l,        l = 1..L,   w_new laid out like w ([L][N][N]),
+ * every element of it, gw^l being the Eq. bp4 gradient of this pass (fp32, or TF32 products
+ * for B > 1 under LF_GW_MATH_TF32).  Each element is one fused multiply-add of the fp32
+ * gradient, fma(-eta, gw, w), i.e. one rounding.  w is only read; w_new must not overlap w
+ * (the delta chain still reads w^{l+1} after w_new^{l+1} has been written).  delta and gb are
+ * written as by lf_backward; the bias update b - eta * gb is left to the caller (N values per
+ * layer).
+ * Errors: as lf_backward; LF_EINVAL if eta is not finite or w_new overlaps w.
+ */
+int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                    float eta, float* delta, float* w_new, float* gb);
 
 /*
  * The same backward pass on HOST buffers (pageable or pinned; same layouts): w, z, a, y are

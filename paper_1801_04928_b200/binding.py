@@ -25,7 +25,7 @@ LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
 LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
 
 EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
-           "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
+           "lf_backward_sgd", "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
            "lf_strerror", "lf_version", "lf_destroy", "lf_delta_step_static")
 
 
@@ -52,6 +52,7 @@ def _load() -> ctypes.CDLL:
     lib.lf_forward.argtypes = [vp] * 6
     lib.lf_backward.argtypes = [vp] * 8
     lib.lf_backward_host.argtypes = [vp] * 8
+    lib.lf_backward_sgd.argtypes = [vp] * 5 + [ctypes.c_float] + [vp] * 3
     lib.lf_sync.argtypes = [vp]
     lib.lf_owner.argtypes = [vp, i]
     lib.lf_get_stats.argtypes = [vp, ctypes.POINTER(lf_stats)]
@@ -120,6 +121,11 @@ def lf_forward(ctx, w, b, x, z, a) -> int:
 def lf_backward(ctx, w, z, a, y, delta, gw, gb) -> int:
     return _lib.lf_backward(ctx, _ptr(w), _ptr(z), _ptr(a), _ptr(y), _ptr(delta), _ptr(gw),
                             _ptr(gb))
+
+
+def lf_backward_sgd(ctx, w, z, a, y, eta: float, delta, w_new, gb) -> int:
+    return _lib.lf_backward_sgd(ctx, _ptr(w), _ptr(z), _ptr(a), _ptr(y), ctypes.c_float(eta), _ptr(delta),
+                                _ptr(w_new), _ptr(gb))
 
 
 def lf_backward_host(ctx, w, z, a, y, delta, gw, gb) -> int:
@@ -191,6 +197,9 @@ class Leapfrog:
 
     def backward(self, w, z, a, y, delta, gw, gb):
         self._check(lf_backward(self._h, w, z, a, y, delta, gw, gb), "lf_backward")
+
+    def backward_sgd(self, w, z, a, y, eta, delta, w_new, gb):
+        self._check(lf_backward_sgd(self._h, w, z, a, y, eta, delta, w_new, gb), "lf_backward_sgd")
 
     def backward_host(self, w, z, a, y, delta, gw, gb):
         self._check(lf_backward_host(self._h, w, z, a, y, delta, gw, gb), "lf_backward_host")

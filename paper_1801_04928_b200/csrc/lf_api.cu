@@ -40,15 +40,17 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
     const float* d_l = delta + (size_t)(l - 1) * slab(c);
     const float* a_prev = a + (size_t)(l - 1) * slab(c);
     float* gw_l = gw + (size_t)(l - 1) * mat(c);
+    lf_sgd sgd = {nullptr, 0.f};
+    if (c->sgd_on) { sgd.w_sub = c->sgd_w + (size_t)(l - 1) * mat(c); sgd.eta = c->sgd_eta; }
     if (c->B == 1) {
-        LF_CUDA_TRY(c, lfk_gw_rank1(d_l, a_prev, gw_l, c->N, s));
+        LF_CUDA_TRY(c, lfk_gw_rank1(d_l, a_prev, gw_l, c->N, sgd, s));
         *launches += 1;
     } else {
         if (gw_math == LF_GW_MATH_TF32) {
-            int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, s, launches);
+            int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, sgd, s, launches);
             if (rc != LF_OK) return rc;
         } else {
-            LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, c->N, c->B, s));
+            LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, c->N, c->B, sgd, s));
             *launches += 1;
         }
         LF_CUDA_TRY(c, lfk_grad_b_colsum(d_l, gb + (size_t)(l - 1) * c->N, c->N, c->B, s));
@@ -132,7 +134,8 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
         c->stats.launches_backward = launches;
         return rc;
     }
-    lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math};
+    lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math,
+                     c->sgd_on, c->sgd_eta};
     if (!(c->graph_valid && c->graph_key == key)) {
         drop_graph(c);
         LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -351,6 +354,22 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
+}
+
+int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                    float eta, float* delta, float* w_new, float* gb)
+{
+    if (!ctx) return LF_ENULL;
+    if (!w || !w_new) return LF_ENULL;
+    if (!(eta == eta) || eta - eta != 0.f) return LF_EINVAL;          // NaN or infinite
+    const size_t bytes = (size_t)ctx->L * mat(ctx) * sizeof(float);
+    const char* lo = reinterpret_cast<const char*>(w);
+    const char* out = reinterpret_cast<const char*>(w_new);
+    if (out < lo + bytes && lo < out + bytes) return LF_EINVAL;        // w_new overlaps w
+    ctx->sgd_on = 1; ctx->sgd_eta = eta; ctx->sgd_w = w;
+    const int rc = lf_backward(ctx, w, z, a, y, delta, w_new, gb);
+    ctx->sgd_on = 0; ctx->sgd_w = nullptr;
+    return rc;
 }
 
 int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,

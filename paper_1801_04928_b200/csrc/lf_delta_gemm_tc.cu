@@ -904,7 +904,9 @@ DgPlan dp_plan(const lf_ctx* c, int max_pairs)
     const long long g_total = (long long)tiles * p.kb_per_tile;
     if (g_total * (max_pairs + 1) >= (1ll << 31)) return p;      // pairs == 0: not usable at this size
     p.g_total = (int)g_total;
-    p.pairs = p.g_total < max_pairs ? p.g_total : max_pairs;
+    // no run shorter than four K blocks: below that the per-run set-up and output outweigh the balance
+    const int by_length = p.g_total / 4 > 0 ? p.g_total / 4 : 1;
+    p.pairs = by_length < max_pairs ? by_length : max_pairs;
     p.splits = 1;
     for (int t = 0; t < tiles; ++t) {
         const int g0 = t * p.kb_per_tile;
@@ -916,7 +918,9 @@ DgPlan dp_plan(const lf_ctx* c, int max_pairs)
 
 bool dp_use_pairs(const lf_ctx* c)
 {
-    return c->tc_pair_kernels && c->B > DG_BM && dp_max_pairs(c) > 0 && dp_plan(c, dp_max_pairs(c)).pairs > 0;
+    // (narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there)
+    return c->tc_pair_kernels && c->B > DG_BM && c->N >= 512 && dp_max_pairs(c) > 0 &&
+           dp_plan(c, dp_max_pairs(c)).pairs > 0;
 }
 
 }  // namespace
@@ -926,7 +930,7 @@ size_t lf_delta_tc_scratch_bytes(const lf_ctx* c)
     if (c->B < 2) return 0;
     // K-split partial sums [splits][B][N] of whichever tiling has more splits
     int splits = dg_plan(c).splits;
-    if (c->B > DG_BM && dp_max_pairs(c) > 0) {
+    if (c->B > DG_BM && c->N >= 512 && dp_max_pairs(c) > 0) {
         const int s2 = dp_plan(c, dp_max_pairs(c)).splits;
         if (s2 > splits) splits = s2;
     }

@@ -35,6 +35,7 @@ constexpr size_t TG_SMEM_BYTES = (size_t)TG_STAGES * TG_STAGE_BYTES + TG_EPI_BYT
 struct TgParams {
     int N, B;
     int tiles_m, tiles_n;
+    lf_sgd sgd;               // w_sub != nullptr: store w_sub - eta * (the contraction) instead
     float* gw;
     unsigned* status;
     unsigned long long budget_ns;
@@ -157,18 +158,6 @@ __device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// 32 lanes x 16 consecutive fp32 columns of tensor memory -> 16 registers per thread
-__device__ __forceinline__ void tg_tmem_ld16(unsigned taddr, unsigned (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -298,9 +287,13 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int rr = i * 4 + sub_r;
-                    const float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
-                    if (row0 + rr < P.N && col < P.N)
-                        __stcs(reinterpret_cast<float4*>(P.gw + (size_t)(row0 + rr) * P.N + col), val);
+                    float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
+                    if (row0 + rr < P.N && col < P.N) {
+                        const size_t off = (size_t)(row0 + rr) * P.N + col;
+                        if (P.sgd.w_sub)
+                            val = lf_sgd_apply4(P.sgd.eta, __ldcs(reinterpret_cast<const float4*>(P.sgd.w_sub + off)), val);
+                        __stcs(reinterpret_cast<float4*>(P.gw + off), val);
+                    }
                 }
                 __syncwarp();
             }
@@ -575,7 +568,9 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             tg_fence_after();
             const int row0 = rb * 2 * TP_BM + (int)rank * TP_BM + quad * 32 + sub_r;
             const int col0 = tn * TP_BN + half * (TP_BN / 2) + sub_c;
-            float* out_row = P.gw + (size_t)row0 * P.N + col0;
+            const size_t out_off = (size_t)row0 * P.N + col0;
+            float* out_row = P.gw + out_off;
+            const float* w_row = P.sgd.w_sub ? P.sgd.w_sub + out_off : nullptr;
             const size_t row_step = (size_t)4 * P.N;
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TP_BN / 2 / 32; ++cchunk) {
@@ -590,8 +585,12 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 if (col0 + cchunk * 32 < P.N) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const float4 val = *reinterpret_cast<const float4*>(blk + (i * 4 + sub_r) * TG_EPI_LD + sub_c);
-                        if (row0 + i * 4 < P.N) __stcs(reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 32), val);
+                        float4 val = *reinterpret_cast<const float4*>(blk + (i * 4 + sub_r) * TG_EPI_LD + sub_c);
+                        if (row0 + i * 4 < P.N) {
+                            if (w_row)
+                                val = lf_sgd_apply4(P.sgd.eta, __ldcs(reinterpret_cast<const float4*>(w_row + i * row_step + cchunk * 32)), val);
+                            __stcs(reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 32), val);
+                        }
                     }
                 }
                 __syncwarp();
@@ -698,7 +697,7 @@ bool lf_tf32_supported(const lf_ctx* c)
     return true;
 }
 
-int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, cudaStream_t s,
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, lf_sgd sgd, cudaStream_t s,
                     int* launches)
 {
     alignas(64) CUtensorMap map_d, map_a;
@@ -709,6 +708,7 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
     TgParams P;
     P.N = c->N; P.B = c->B;
     P.gw = gw_l;
+    P.sgd = sgd;
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     const int max_pairs = c->tc_pair_kernels && c->B <= TP_MAX_KS * TG_BK ? tp_max_pairs(c) : 0;

@@ -17,11 +17,28 @@ struct lf_graph_key {
     const void *w, *z, *a, *y;
     void *delta, *gw, *gb;
     int variant, gw_math;
+    int sgd;        // 1: the graph writes w - eta * gw instead of gw
+    float eta;
     bool operator==(const lf_graph_key& o) const {
         return w == o.w && z == o.z && a == o.a && y == o.y && delta == o.delta &&
-               gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math;
+               gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math &&
+               sgd == o.sgd && (!sgd || eta == o.eta);
     }
 };
+
+// Fused weight update of the gradient writers: w_sub == nullptr -> store the gradient g itself,
+// else store w_sub[...] - eta * g (w_sub is the weight matrix of the same layer).
+struct lf_sgd {
+    const float* w_sub;
+    float eta;
+};
+#ifdef __CUDACC__
+// one rounding: fma(-eta, g, w)
+__device__ __forceinline__ float4 lf_sgd_apply4(float eta, float4 w, float4 g)
+{
+    return make_float4(fmaf(-eta, g.x, w.x), fmaf(-eta, g.y, w.y), fmaf(-eta, g.z, w.z), fmaf(-eta, g.w, w.w));
+}
+#endif
 
 struct lf_ctx {
     int L, N, B, k, keff;
@@ -37,6 +54,9 @@ struct lf_ctx {
     int use_graph;
     int opt_delta_math;      // enum lf_delta_math
     int tc_pair_kernels;     // 1: the tensor-core contractions may use the two-SM (CTA pair) kernels
+    int sgd_on;              // the current backward call is lf_backward_sgd
+    float sgd_eta;
+    const float* sgd_w;      // its weights (what the update is subtracted from)
     int withhold;            // test hook: one chain CTA withholds its published delta values
 
     // workspace (device)
@@ -103,7 +123,7 @@ cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const flo
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,
                              int N, cudaStream_t s);
 cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
-                         cudaStream_t s);
+                         lf_sgd sgd, cudaStream_t s);
 
 // B > 1 kernels (fp32 on the CUDA cores)
 cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
@@ -111,7 +131,7 @@ cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
                            float* delta_l, int N, int B, cudaStream_t s);
 cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
-                             int B, cudaStream_t s);
+                             int B, lf_sgd sgd, cudaStream_t s);
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s);
 
 // ---- persistent single-launch backward (B = 1) ---------------------------------------------
@@ -124,7 +144,7 @@ void lf_persistent_release(lf_ctx* c);
 
 // ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------
 bool lf_tf32_supported(const lf_ctx* c);
-int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l,
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, lf_sgd sgd,
                     cudaStream_t s, int* launches);
 void lf_tf32_release(lf_ctx* c);
 

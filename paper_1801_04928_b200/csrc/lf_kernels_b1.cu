@@ -163,7 +163,7 @@ constexpr int GW1_THREADS = 256;
 
 __global__ void __launch_bounds__(GW1_THREADS)
 k_gw_rank1(const float* __restrict__ delta_l, const float* __restrict__ a_prev,
-           float* __restrict__ gw_l, int N)
+           float* __restrict__ gw_l, int N, const lf_sgd sgd)
 {
     const int n4 = N >> 2;
     const size_t total4 = (size_t)N * n4;
@@ -175,7 +175,10 @@ k_gw_rank1(const float* __restrict__ delta_l, const float* __restrict__ a_prev,
         int c = (int)(i - (size_t)j * n4);
         float d = delta_l[j];
         float4 a4 = av[c];
-        __stcs(out + i, make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w));
+        float4 g = make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w);
+        if (sgd.w_sub)   // fused update: w - eta * g, the weights streamed through once
+            g = lf_sgd_apply4(sgd.eta, ld_stream(reinterpret_cast<const float4*>(sgd.w_sub) + i), g);
+        __stcs(out + i, g);
     }
 }
 
@@ -224,13 +227,13 @@ cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const flo
 }
 
 cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
-                         cudaStream_t s)
+                         lf_sgd sgd, cudaStream_t s)
 {
     size_t total4 = (size_t)N * (N >> 2);
     size_t want = (total4 + GW1_THREADS - 1) / GW1_THREADS;
     int grid = (int)(want < (size_t)148 * 16 ? want : (size_t)148 * 16);
     if (grid < 1) grid = 1;
-    k_gw_rank1<<<grid, GW1_THREADS, 0, s>>>(delta_l, a_prev, gw_l, N);
+    k_gw_rank1<<<grid, GW1_THREADS, 0, s>>>(delta_l, a_prev, gw_l, N, sgd);
     return cudaGetLastError();
 }
 

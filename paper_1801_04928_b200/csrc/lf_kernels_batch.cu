@@ -23,7 +23,7 @@ template <bool A_KMAJOR, bool B_KMAJOR, int EPI>
 __global__ void __launch_bounds__(256)
 k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __restrict__ C,
             float* __restrict__ C2, const float* __restrict__ aux, int M, int Nn, int K, int lda,
-            int ldb, int ldc)
+            int ldb, int ldc, float eta)
 {
     __shared__ __align__(16) float As[BK][BM + PAD];
     __shared__ __align__(16) float Bs[BK][BN + PAD];
@@ -101,6 +101,8 @@ k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __
             r.z *= av.z * (1.0f - av.z); r.w *= av.w * (1.0f - av.w);
             *reinterpret_cast<float4*>(C + off) = r;
         } else {
+            // EPI_PLAIN: the contraction itself, or (aux = the weight matrix) aux - eta * it
+            if (aux) r = lf_sgd_apply4(eta, *reinterpret_cast<const float4*>(aux + off), r);
             *reinterpret_cast<float4*>(C + off) = r;
         }
     }
@@ -143,7 +145,7 @@ cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_
 {
     // M = B (samples), Nn = N (neuron j), K = N (neuron k of the layer below)
     k_gemm_simt<true, true, EPI_FORWARD><<<gemm_grid(B, N), 256, 0, s>>>(
-        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N);
+        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N, 0.f);
     return cudaGetLastError();
 }
 
@@ -152,16 +154,16 @@ cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float
 {
     // M = B, Nn = N (neuron k of layer l), K = N (neuron j of layer l+1); w_up[j][k] is n-contiguous
     k_gemm_simt<true, false, EPI_DELTA><<<gemm_grid(B, N), 256, 0, s>>>(
-        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N);
+        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N, 0.f);
     return cudaGetLastError();
 }
 
 cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
-                             int B, cudaStream_t s)
+                             int B, lf_sgd sgd, cudaStream_t s)
 {
     // M = N (j), Nn = N (k), K = B; both operands are contiguous along their M / N index
     k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(N, N), 256, 0, s>>>(
-        delta_l, a_prev, gw_l, nullptr, nullptr, N, N, B, N, N, N);
+        delta_l, a_prev, gw_l, nullptr, sgd.w_sub, N, N, B, N, N, N, sgd.eta);
     return cudaGetLastError();
 }
 

@@ -59,6 +59,8 @@ struct PkParams {
     unsigned long long budget_ns;
     const float* a;
     const float* y;
+    const float* w_sub;       // fused weight update: store w_sub - eta * gw in place of gw (null: plain gw)
+    float eta;
     float* delta;
     float* gw;
     float* gb;
@@ -256,12 +258,17 @@ __device__ void worker_store_rows(const PkParams& P, int l, int row0, int row1, 
     for (int r = row0 + tid; r < row1; r += PK_THREADS) d_rows[r - row0] = wait_slot(slots + r, P, sh);
     __syncthreads();
     float* gw_l = P.gw + (size_t)(l - 1) * N * N;
+    const float* w_l = P.w_sub ? P.w_sub + (size_t)(l - 1) * N * N : nullptr;
     for (int r = row0 + warp; r < row1; r += PK_THREADS / 32) {
         const float d = d_rows[r - row0];
         float* out = gw_l + (size_t)r * N;
+        const float* w_row = w_l ? w_l + (size_t)r * N : nullptr;
+#pragma unroll 4
         for (int c = lane; c < n4; c += 32) {
             float4 a4 = reinterpret_cast<const float4*>(a_sm)[c];
-            st_stream4(out + 4 * c, make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w));
+            float4 g = make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w);
+            if (w_row) g = lf_sgd_apply4(P.eta, __ldcg(reinterpret_cast<const float4*>(w_row) + c), g);
+            st_stream4(out + 4 * c, g);
         }
     }
     __syncthreads();
@@ -356,10 +363,24 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                     const float4 av = a4[cb];
                     float* out = gw_s + (size_t)row_base * N + col;
                     const int rows = row_end - row_base;
+                    if (P.w_sub) {
+                        // fused update: the tile of w^s was fetched for the chain a moment ago, so
+                        // this second read is served by L2 (layer 1, which the chain never reads,
+                        // comes from memory)
+                        const float* w_in = P.w_sub + (size_t)(s - 1) * N * N + (size_t)row_base * N + col;
 #pragma unroll 4
-                    for (int rr = trow; rr < rows; rr += RG) {
-                        const float d = dr[rr];
-                        st_stream4(out + (size_t)rr * N, make_float4(d * av.x, d * av.y, d * av.z, d * av.w));
+                        for (int rr = trow; rr < rows; rr += RG) {
+                            const float d = dr[rr];
+                            const float4 wv = __ldcg(reinterpret_cast<const float4*>(w_in + (size_t)rr * N));
+                            st_stream4(out + (size_t)rr * N,
+                                       lf_sgd_apply4(P.eta, wv, make_float4(d * av.x, d * av.y, d * av.z, d * av.w)));
+                        }
+                    } else {
+#pragma unroll 4
+                        for (int rr = trow; rr < rows; rr += RG) {
+                            const float d = dr[rr];
+                            st_stream4(out + (size_t)rr * N, make_float4(d * av.x, d * av.y, d * av.z, d * av.w));
+                        }
                     }
                 }
                 mbar_arrive(smem_u32(&sh->d_free[p]));
@@ -757,6 +778,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
+    P.w_sub = c->sgd_on ? c->sgd_w : nullptr; P.eta = c->sgd_eta;
     P.xch = reinterpret_cast<unsigned long long*>(c->sync_words);
     P.status = c->status_dev;
 #ifdef LF_PK_TRACE

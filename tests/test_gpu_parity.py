@@ -47,15 +47,16 @@ def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
     # fp32 gate (1e-5 per tensor per layer) for every form of the delta recurrence (and of the
     # forward pass, which shares its kernels): fp32 on the CUDA cores, and the tensor cores with
     # every operand split into two TF32 numbers, one CTA per tile or a CTA pair per tile (pairs
-    # take over above 128 samples: B = 129 and 260 leave a pair's second half nearly empty,
-    # B = 515 needs three 256-sample blocks, N = 2052 several K splits with a ragged last one).
+    # take over above 128 samples and from 512 columns: B = 260 leaves a pair's second half nearly
+    # empty, B = 515 needs three 256-sample blocks, N = 2052 gives runs that end inside a tile).
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=N + B)
     out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math, tc_tiling=tiling)
     assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == delta_math
     assert stats["device_status"] == 0
     if delta_math == lf.LF_DELTA_MATH_3XTF32 and L > 1:
-        want = lf.LF_TC_TILING_TWO_SM if (tiling == lf.LF_TC_TILING_TWO_SM and B > 128) else lf.LF_TC_TILING_ONE_SM
+        pairs = tiling == lf.LF_TC_TILING_TWO_SM and B > 128 and N >= 512   # the library's rule for CTA pairs
+        want = lf.LF_TC_TILING_TWO_SM if pairs else lf.LF_TC_TILING_ONE_SM
         assert stats["delta_tiling"] == want
     ref = oracle_pass(t, want_gw=True)
     compare_all(cfg, out, ref)
