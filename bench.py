@@ -46,6 +46,9 @@ def parse_args():
     p.add_argument("--k", type=int, default=0, help="leapfrog workers (0 = the config's k)")
     p.add_argument("--tc-tiling", default="auto", choices=["auto", "one_sm", "two_sm"],
                    help="tiling of the tensor-core contractions (B > 1)")
+    p.add_argument("--sgd", type=float, default=None, metavar="ETA",
+                   help="time lf_backward_sgd (gradient + weight update in one pass) with this step size "
+                        "instead of lf_backward; not the headline metric")
     p.add_argument("--layers", type=int, default=0,
                    help="override the config's L (a smaller case of the same kernels, for profiler captures)")
     p.add_argument("--e2e-steps", type=int, default=5)
@@ -294,7 +297,10 @@ def run_ours(args):
 
     def step(i):
         t = sets[i % n_sets]
-        t["ctx"].backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+        if args.sgd is not None:   # gw receives the updated weights
+            t["ctx"].backward_sgd(t["w"], t["z"], t["a"], t["y"], args.sgd, t["delta"], t["gw"], t["gb"])
+        else:
+            t["ctx"].backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
 
     def barrier():
         torch.cuda.synchronize(dev)
@@ -375,6 +381,8 @@ def run_ours(args):
 
     peak, peak_kind, peaks = measured_peaks()
     alg = algorithmic_bytes(L, N, B)
+    if args.sgd is not None:
+        alg += 4 * N * N          # the update also reads w^1, which the plain pass never touches
     launches_per_step = stats["launches_backward"]
     if launches_per_step == 1:
         kernel_name = "persistent backward kernel (one launch per step)"
@@ -425,6 +433,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(args.config, cfg), "L": L, "N": N, "B": B, "k": k,
                    "variant": stats["variant"], "gw_math": stats["gw_math"],
+                   **({"fused_sgd_eta": args.sgd} if args.sgd is not None else {}),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2_policy": f"{n_sets} rotating buffer sets of {set_bytes >> 20} MiB (w + gw); "
                                 "inputs larger than the 126 MB L2"},
