@@ -26,7 +26,8 @@
  *     the input as layer 1, so paper layer p is l = p - 1 here and the paper's L is L + 1.
  *   - All layers, input and output included, are N wide.
  *   - C is the quadratic cost C = 1/2 sum_b ||a^L_b - y_b||^2 (a SUM over the B samples,
- *     no 1/B), hence grad_a C = a^L - y.
+ *     no 1/B), hence grad_a C = a^L - y.  (The *_cross_entropy functions are the same pass
+ *     under a second cost, see there.)
  *   - Mini-batch (B > 1) is an extension: every sample is an independent column; bp3 and
  *     bp4 are summed over the samples.
  *   - Algorithm 1 never applies bp3/bp4 at the top layer L; that is an omission.  The
@@ -186,6 +187,20 @@ static void lfo_emit_layer(int l, int N, int B, const double *delta_l, const dou
         lfo_grad_w(N, B, delta_l, a + (size_t)(l - 1) * slab, gw + (size_t)(l - 1) * N * N);
 }
 
+/* Everything below Eq. bp1: the caller has put delta^L into the top slab of `delta`; bp2
+ * downwards, bp3/bp4 at every layer (L included). */
+void lfo_backward_below_top(int L, int N, int B, const lfo_w_t *w, const double *z,
+                            const double *a, double *delta, double *gw, double *gb)
+{
+    size_t slab = (size_t)B * (size_t)N;
+    lfo_emit_layer(L, N, B, delta + (size_t)(L - 1) * slab, a, gw, gb);
+    for (int l = L - 1; l >= 1; --l) {
+        lfo_delta_step(N, B, w + (size_t)l * N * N, delta + (size_t)l * slab,
+                       z + (size_t)(l - 1) * slab, delta + (size_t)(l - 1) * slab);
+        lfo_emit_layer(l, N, B, delta + (size_t)(l - 1) * slab, a, gw, gb);
+    }
+}
+
 /* Plain sequential backpropagation: bp1 at L, then bp2 downwards, bp3/bp4 everywhere. */
 void lfo_backward_sequential(int L, int N, int B, const lfo_w_t *w, const double *z,
                              const double *a, const double *y, double *delta, double *gw,
@@ -194,12 +209,42 @@ void lfo_backward_sequential(int L, int N, int B, const lfo_w_t *w, const double
     size_t slab = (size_t)B * (size_t)N;
     lfo_output_error(N, B, a + (size_t)L * slab, y, z + (size_t)(L - 1) * slab,
                      delta + (size_t)(L - 1) * slab);
-    lfo_emit_layer(L, N, B, delta + (size_t)(L - 1) * slab, a, gw, gb);
-    for (int l = L - 1; l >= 1; --l) {
-        lfo_delta_step(N, B, w + (size_t)l * N * N, delta + (size_t)l * slab,
-                       z + (size_t)(l - 1) * slab, delta + (size_t)(l - 1) * slab);
-        lfo_emit_layer(l, N, B, delta + (size_t)(l - 1) * slab, a, gw, gb);
+    lfo_backward_below_top(L, N, B, w, z, a, delta, gw, gb);
+}
+
+/* ---- a second cost function: cross-entropy ------------------------------------------------
+ * Section 2 leaves C open ("the cost function"; Eq. bp1 only needs grad_a C).  Besides the
+ * quadratic cost this oracle knows the cross-entropy of sigmoid outputs,
+ *     C = - sum_b sum_j [ y_bj ln a^L_bj + (1 - y_bj) ln(1 - a^L_bj) ]      (a sum, no 1/B),
+ * whose gradient by the activations is grad_a C = (a - y) / (a (1 - a)).  Eq. bp1 is applied
+ * as printed, grad_a C (.) sigma'(z^L); nothing is simplified here (that the product collapses
+ * to a - y is what an implementation may use and what the tests then confirm). */
+double lfo_cost_cross_entropy(int L, int N, int B, const double *a, const double *y)
+{
+    const double *aL = a + (size_t)L * B * N;
+    double c = 0.0;
+    for (size_t i = 0; i < (size_t)B * N; ++i)
+        c -= y[i] * log(aL[i]) + (1.0 - y[i]) * log(1.0 - aL[i]);
+    return c;
+}
+
+void lfo_output_error_cross_entropy(int N, int B, const double *aL, const double *y, const double *zL,
+                                    double *deltaL)
+{
+    for (size_t i = 0; i < (size_t)B * N; ++i) {
+        double grad_a = (aL[i] - y[i]) / (aL[i] * (1.0 - aL[i]));
+        deltaL[i] = grad_a * lfo_sigmoid_prime(zL[i]);                 /* Eq. bp1 */
     }
+}
+
+void lfo_backward_sequential_cross_entropy(int L, int N, int B, const lfo_w_t *w, const double *z,
+                                           const double *a, const double *y, double *delta,
+                                           double *gw, double *gb)
+{
+    size_t slab = (size_t)B * (size_t)N;
+    lfo_output_error_cross_entropy(N, B, a + (size_t)L * slab, y, z + (size_t)(L - 1) * slab,
+                                   delta + (size_t)(L - 1) * slab);
+    lfo_backward_below_top(L, N, B, w, z, a, delta, gw, gb);
 }
 
 /* ---- Algorithm 1, taken literally ------------------------------------------------------ */

@@ -78,6 +78,13 @@ def _lib(tag: str) -> ctypes.CDLL:
             lib.lfo_backward_leapfrog.argtypes = [i, i, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp,
                                                   _c_dp, _c_dp, _c_ip, _c_ip,
                                                   ctypes.POINTER(ctypes.c_longlong), i]
+            lib.lfo_cost_cross_entropy.restype = ctypes.c_double
+            lib.lfo_cost_cross_entropy.argtypes = [i, i, i, _c_dp, _c_dp]
+            lib.lfo_output_error_cross_entropy.restype = None
+            lib.lfo_output_error_cross_entropy.argtypes = [i, i, _c_dp, _c_dp, _c_dp, _c_dp]
+            lib.lfo_backward_sequential_cross_entropy.restype = None
+            lib.lfo_backward_sequential_cross_entropy.argtypes = [i, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp,
+                                                                  _c_dp, _c_dp]
             lib.lfo_sgd_step.restype = None
             lib.lfo_sgd_step.argtypes = [i, i, wp, _c_dp, ctypes.c_double, _c_dp]
             assert lib.lfo_weight_bytes() == (8 if tag == "f64" else 4)
@@ -126,20 +133,23 @@ def forward(w, b, x):
     return z, a
 
 
-def cost(a, y) -> float:
-    """C = 1/2 sum_b ||a^L_b - y_b||^2 from the activations of a forward pass."""
+def cost(a, y, cross_entropy: bool = False) -> float:
+    """C from the activations of a forward pass: 1/2 sum_b ||a^L_b - y_b||^2, or the
+    cross-entropy of the sigmoid outputs."""
     a = _d(a)
     Lp1, B, N = a.shape
     y = _d(y).reshape(B, N)
-    return _lib("f64").lfo_cost(Lp1 - 1, N, B, _p(a), _p(y))
+    fn = _lib("f64").lfo_cost_cross_entropy if cross_entropy else _lib("f64").lfo_cost
+    return fn(Lp1 - 1, N, B, _p(a), _p(y))
 
 
-def output_error(aL, y, zL):
-    """Eq. bp1."""
+def output_error(aL, y, zL, cross_entropy: bool = False):
+    """Eq. bp1 under either cost."""
     aL, y, zL = _d(aL), _d(y), _d(zL)
     B, N = aL.shape
     out = np.empty((B, N), dtype=np.float64)
-    _lib("f64").lfo_output_error(N, B, _p(aL), _p(y), _p(zL), _p(out))
+    fn = _lib("f64").lfo_output_error_cross_entropy if cross_entropy else _lib("f64").lfo_output_error
+    fn(N, B, _p(aL), _p(y), _p(zL), _p(out))
     return out
 
 
@@ -178,8 +188,9 @@ def grad_w_entry(delta_l, a_prev, j: int, k: int) -> float:
     return _lib("f64").lfo_grad_w_entry(N, B, _p(delta_l), _p(a_prev), int(j), int(k))
 
 
-def backward_sequential(w, z, a, y, want_gw: bool = True):
-    """Plain backpropagation.  Returns delta[L,B,N], gw[L,N,N] (or None), gb[L,N]."""
+def backward_sequential(w, z, a, y, want_gw: bool = True, cross_entropy: bool = False):
+    """Plain backpropagation under the quadratic (default) or the cross-entropy cost.
+    Returns delta[L,B,N], gw[L,N,N] (or None), gb[L,N]."""
     lib, w, wp = _w(w)
     L, N, _ = w.shape
     z, a = _d(z), _d(a)
@@ -188,8 +199,8 @@ def backward_sequential(w, z, a, y, want_gw: bool = True):
     delta = np.empty((L, B, N), dtype=np.float64)
     gb = np.empty((L, N), dtype=np.float64)
     gw = np.empty((L, N, N), dtype=np.float64) if want_gw else None
-    lib.lfo_backward_sequential(L, N, B, wp, _p(z), _p(a), _p(y), _p(delta),
-                                _p(gw) if want_gw else None, _p(gb))
+    fn = lib.lfo_backward_sequential_cross_entropy if cross_entropy else lib.lfo_backward_sequential
+    fn(L, N, B, wp, _p(z), _p(a), _p(y), _p(delta), _p(gw) if want_gw else None, _p(gb))
     return delta, gw, gb
 
 

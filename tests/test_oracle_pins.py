@@ -398,3 +398,57 @@ def test_sgd_step_float_weight_flavour_promotes_exactly():
     w32 = rng.standard_normal((2, 4, 4)).astype(np.float32)
     gw = rng.standard_normal((2, 4, 4))
     assert np.array_equal(orc.sgd_step(w32, gw, 0.3), orc.sgd_step(w32.astype(np.float64), gw, 0.3))
+
+
+# ---- the second cost function: cross-entropy of the sigmoid outputs -----------------------------
+def _cost_ce(w, b, x, y):
+    _, a = orc.forward(w, b, x)
+    return orc.cost(a, y, cross_entropy=True)
+
+
+def test_cross_entropy_cost_definition():
+    # one layer, zero weights and biases: a = 1/2, so C = N ln 2 per sample whatever y is
+    N = 5
+    w = np.zeros((1, N, N)); b = np.zeros((1, N))
+    x = np.full((2, N), 0.3); y = np.array([[1, 0, 0.25, 0.5, 0.75], [0, 1, 1, 0, 0.1]], dtype=float)
+    _, a = orc.forward(w, b, x)
+    assert abs(orc.cost(a, y, cross_entropy=True) - 2 * N * np.log(2.0)) < 1e-13
+    # and against the formula written out with numpy on a random net
+    w, b, x, y = _net(2, 4, 3, seed=31)
+    _, a = orc.forward(w, b, x)
+    want = -np.sum(y * np.log(a[-1]) + (1 - y) * np.log(1 - a[-1]))
+    assert abs(orc.cost(a, y, cross_entropy=True) - want) < 1e-12 * abs(want)
+
+
+@pytest.mark.parametrize("L,N,B,y_kind", [(1, 3, 1, "uniform"), (3, 5, 3, "uniform"), (4, 6, 2, "onehot")])
+def test_cross_entropy_gradients_match_central_differences(L, N, B, y_kind):
+    # Eq. bp1 with grad_a C of the cross-entropy, then the same bp2-bp4: every dC/dw and dC/db
+    # against central differences of the cross-entropy cost itself.
+    w, b, x, y = _net(L, N, B, seed=500 + 100 * L + 10 * N + B, y_kind=y_kind)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y, cross_entropy=True)
+    h = 1e-5
+    for l in range(L):
+        fd_w = np.empty((N, N)); fd_b = np.empty((N,))
+        for j in range(N):
+            for k in range(N):
+                wp = w.copy(); wp[l, j, k] += h
+                wm = w.copy(); wm[l, j, k] -= h
+                fd_w[j, k] = (_cost_ce(wp, b, x, y) - _cost_ce(wm, b, x, y)) / (2 * h)
+            bp = b.copy(); bp[l, j] += h
+            bm = b.copy(); bm[l, j] -= h
+            fd_b[j] = (_cost_ce(w, bp, x, y) - _cost_ce(w, bm, x, y)) / (2 * h)
+        assert np.max(np.abs(gw[l] - fd_w)) <= 2e-7 * np.max(np.abs(fd_w)) + 1e-12
+        assert np.max(np.abs(gb[l] - fd_b)) <= 2e-7 * np.max(np.abs(fd_b)) + 1e-12
+
+
+def test_cross_entropy_output_error_collapses_to_a_minus_y():
+    # grad_a C (.) sigma'(z) = (a - y)/(a(1-a)) * a(1-a) = a - y: the closed form an implementation
+    # may use; below the top layer the two costs share Eq. bp2-bp4, so their deltas differ exactly
+    # by what the top deltas differ.
+    w, b, x, y = _net(3, 6, 2, seed=33)
+    z, a = orc.forward(w, b, x)
+    d_top = orc.output_error(a[-1], y, z[-1], cross_entropy=True)
+    np.testing.assert_allclose(d_top, a[-1] - y, rtol=1e-12, atol=1e-15)
+    d_ce, _, _ = orc.backward_sequential(w, z, a, y, cross_entropy=True)
+    np.testing.assert_allclose(d_ce[1], orc.delta_step(w[2], d_top, z[1]), rtol=1e-13, atol=0)
