@@ -85,6 +85,14 @@ enum lf_tc_tiling {
                                 N >= 512; other sizes use ONE_SM                                */
 };
 
+/* The cost function C of Eq. bp1, delta^L = grad_a C (.) sigma'(z^L); Section 2 leaves it open
+ * ("the cost function").  Both are sums over the B samples (no 1/B). */
+enum lf_cost {
+    LF_COST_QUADRATIC = 0,     /* C = 1/2 sum ||a^L - y||^2: delta^L = (a^L - y) (.) sigma'(z^L)  */
+    LF_COST_CROSS_ENTROPY = 1  /* C = -sum [y ln a^L + (1-y) ln(1-a^L)] on the sigmoid outputs:
+                                  grad_a C = (a^L - y) / (a^L (1 - a^L)), so delta^L = a^L - y   */
+};
+
 enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
@@ -92,6 +100,7 @@ enum lf_option {
     LF_OPT_USE_GRAPH = 4,     /* 0/1: replay the STREAMS variant from a captured CUDA graph   */
     LF_OPT_DELTA_MATH = 6,    /* enum lf_delta_math                                           */
     LF_OPT_TC_TILING = 7,     /* enum lf_tc_tiling                                            */
+    LF_OPT_COST = 8,          /* enum lf_cost (default LF_COST_QUADRATIC)                     */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -113,6 +122,7 @@ typedef struct lf_stats {
     int gw_tiling;            /* tiling of the last TF32 weight-gradient launch (enum lf_tc_tiling,
                                  ONE_SM or TWO_SM; 0 if none ran)                             */
     int delta_tiling;         /* the same for the last tensor-core Eq. bp2 / Eq. z launch     */
+    int cost;                 /* cost function the last lf_backward used (enum lf_cost)       */
 } lf_stats;
 
 /*
@@ -142,7 +152,9 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
                float* a);
 
 /*
- * Backward pass under the quadratic cost C = 1/2 sum_b ||a^L_b - y_b||^2:
+ * Backward pass under the quadratic cost C = 1/2 sum_b ||a^L_b - y_b||^2 (or, with
+ * LF_OPT_COST = LF_COST_CROSS_ENTROPY, the cross-entropy cost, for which Eq. bp1 reads
+ * delta^L = a^L - y):
  *   Eq. bp1  delta^L = (a^L - y) (.) sigma'(z^L)
  *   Eq. bp2  delta^l = ((w^{l+1})^T delta^{l+1}) (.) sigma'(z^l),  l = L-1 .. 1
  *   Eq. bp3  gb^l = sum_b delta^l_b
@@ -156,6 +168,15 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
  */
 int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
                 float* delta, float* gw, float* gb);
+
+/*
+ * Eq. bp4 alone, for one layer:  gw_l = sum_b delta_l[b] (a_prev[b])^T  with delta_l = delta^l and
+ * a_prev = a^{l-1}, both [B][N]; gw_l receives all N x N entries.  The same kernel, arithmetic
+ * (LF_OPT_GW_MATH) and tiling as inside lf_backward, enqueued on the context's stream; the
+ * result is bitwise what lf_backward writes into that layer's slab of gw.  Device pointers,
+ * 16-byte aligned, owned by the caller.
+ */
+int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_l);
 
 /*
  * Backward pass fused with one step of gradient descent on the weights.  (The paper has no

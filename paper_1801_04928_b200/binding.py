@@ -21,11 +21,13 @@ LF_GW_MATH_AUTO, LF_GW_MATH_FP32, LF_GW_MATH_TF32 = 0, 1, 2
 LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH, LF_OPT_WITHHOLD = 1, 2, 3, 4, 5
 LF_OPT_DELTA_MATH = 6
 LF_OPT_TC_TILING = 7
+LF_OPT_COST = 8
+LF_COST_QUADRATIC, LF_COST_CROSS_ENTROPY = 0, 1
 LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
 LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
 
 EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
-           "lf_backward_sgd", "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
+           "lf_backward_sgd", "lf_grad_w", "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
            "lf_strerror", "lf_version", "lf_destroy", "lf_delta_step_static")
 
 
@@ -36,7 +38,7 @@ class lf_stats(ctypes.Structure):
                 ("chain_ctas", ctypes.c_int), ("worker_ctas", ctypes.c_int),
                 ("launches_forward", ctypes.c_int), ("launches_backward", ctypes.c_int),
                 ("device_status", ctypes.c_uint), ("workspace_bytes", ctypes.c_longlong),
-                ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int)]
+                ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int), ("cost", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -52,6 +54,7 @@ def _load() -> ctypes.CDLL:
     lib.lf_forward.argtypes = [vp] * 6
     lib.lf_backward.argtypes = [vp] * 8
     lib.lf_backward_host.argtypes = [vp] * 8
+    lib.lf_grad_w.argtypes = [vp] * 4
     lib.lf_backward_sgd.argtypes = [vp] * 5 + [ctypes.c_float] + [vp] * 3
     lib.lf_sync.argtypes = [vp]
     lib.lf_owner.argtypes = [vp, i]
@@ -121,6 +124,10 @@ def lf_forward(ctx, w, b, x, z, a) -> int:
 def lf_backward(ctx, w, z, a, y, delta, gw, gb) -> int:
     return _lib.lf_backward(ctx, _ptr(w), _ptr(z), _ptr(a), _ptr(y), _ptr(delta), _ptr(gw),
                             _ptr(gb))
+
+
+def lf_grad_w(ctx, delta_l, a_prev, gw_l) -> int:
+    return _lib.lf_grad_w(ctx, _ptr(delta_l), _ptr(a_prev), _ptr(gw_l))
 
 
 def lf_backward_sgd(ctx, w, z, a, y, eta: float, delta, w_new, gb) -> int:
@@ -197,6 +204,9 @@ class Leapfrog:
 
     def backward(self, w, z, a, y, delta, gw, gb):
         self._check(lf_backward(self._h, w, z, a, y, delta, gw, gb), "lf_backward")
+
+    def grad_w(self, delta_l, a_prev, gw_l):
+        self._check(lf_grad_w(self._h, delta_l, a_prev, gw_l), "lf_grad_w")
 
     def backward_sgd(self, w, z, a, y, eta, delta, w_new, gb):
         self._check(lf_backward_sgd(self._h, w, z, a, y, eta, delta, w_new, gb), "lf_backward_sgd")

@@ -74,7 +74,7 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
     const float* a_l = a + (size_t)l * slab(c);
     float* gb_l = gb + (size_t)(l - 1) * N;
     if (l == L) {
-        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, s));
+        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, c->opt_cost, s));
     } else {
         const float* w_up = w + (size_t)l * mat(c);  // w^{l+1}
         const float* d_up = delta + (size_t)l * slab(c);
@@ -135,7 +135,7 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
         return rc;
     }
     lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math,
-                     c->sgd_on, c->sgd_eta};
+                     c->sgd_on, c->sgd_eta, c->opt_cost};
     if (!(c->graph_valid && c->graph_key == key)) {
         drop_graph(c);
         LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -292,6 +292,10 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             ctx->tc_pair_kernels = value != LF_TC_TILING_ONE_SM;
             drop_graph(ctx);
             return LF_OK;
+        case LF_OPT_COST:
+            if (value != LF_COST_QUADRATIC && value != LF_COST_CROSS_ENTROPY) return LF_EINVAL;
+            ctx->opt_cost = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -351,9 +355,29 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     ctx->stats.variant = variant;
     ctx->stats.gw_math = gw_math;
     ctx->stats.delta_math = resolve_delta_math(ctx);
+    ctx->stats.cost = ctx->opt_cost;
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
+}
+
+int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_l)
+{
+    if (!ctx) return LF_ENULL;
+    const void* ps[] = {delta_l, a_prev, gw_l};
+    int rc = check_ptrs(ps, 3);
+    if (rc != LF_OK) return rc;
+    const int gw_math = resolve_gw_math(ctx);
+    ctx->stats.gw_math = gw_math;
+    const lf_sgd plain = {nullptr, 0.f};
+    int launches = 0;
+    if (ctx->B == 1)
+        LF_CUDA_TRY(ctx, lfk_gw_rank1(delta_l, a_prev, gw_l, ctx->N, plain, ctx->stream));
+    else if (gw_math == LF_GW_MATH_TF32)
+        return lf_gw_gemm_tf32(ctx, delta_l, a_prev, gw_l, plain, ctx->stream, &launches);
+    else
+        LF_CUDA_TRY(ctx, lfk_gw_gemm_fp32(delta_l, a_prev, gw_l, ctx->N, ctx->B, plain, ctx->stream));
+    return LF_OK;
 }
 
 int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
@@ -422,6 +446,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     ctx->stats.variant = LF_VARIANT_STREAMS;
     ctx->stats.gw_math = gw_math;
     ctx->stats.delta_math = resolve_delta_math(ctx);
+    ctx->stats.cost = ctx->opt_cost;
     int launches = 0;
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
     LF_CUDA_TRY(ctx, cudaStreamWaitEvent(hs, ctx->fork_ev, 0));

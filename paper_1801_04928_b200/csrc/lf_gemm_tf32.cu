@@ -162,6 +162,18 @@ __device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Fused weight update: ask L2 for the part of the w tile this warp will subtract from (32 rows x
+// `cols` columns starting at row_first, col_first), one 128-byte line per request, while the
+// tile is still being multiplied.
+__device__ __forceinline__ void tg_prefetch_w(const float* w, int N, int row_first, int col_first, int cols, int lane)
+{
+    const int row = row_first + lane;
+    if (row >= N) return;
+    const float* p = w + (size_t)row * N + col_first;
+    for (int c = 0; c < cols && col_first + c < N; c += 32)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p + c));
+}
+
 __global__ void __launch_bounds__(TG_THREADS, 1)
 k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_a,
                const TgParams P)
@@ -266,6 +278,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
         for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_i) {
             const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
             const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
+            if (P.sgd.w_sub) tg_prefetch_w(P.sgd.w_sub, P.N, tm * TG_BM + quad * 32, tn * TG_BN, TG_BN, lane);
             if (!tg_wait(tg_smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
             tg_fence_after();
             // A thread reads one accumulator row (32 columns at a time).  The block is turned
@@ -275,6 +288,15 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
             const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TG_BN / 32; ++cchunk) {
+                // fused weight update: the loads of w go out before the accumulator is fetched
+                float4 wv[8];
+                const int col_w = tn * TG_BN + cchunk * 32 + sub_c;
+                if (P.sgd.w_sub && col_w < P.N) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (row0 + i * 4 + sub_r < P.N)
+                            wv[i] = __ldcs(reinterpret_cast<const float4*>(P.sgd.w_sub + (size_t)(row0 + i * 4 + sub_r) * P.N + col_w));
+                }
                 unsigned r[32];
                 tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TG_BN + cchunk * 32, r);
 #pragma unroll
@@ -290,8 +312,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                     float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
                     if (row0 + rr < P.N && col < P.N) {
                         const size_t off = (size_t)(row0 + rr) * P.N + col;
-                        if (P.sgd.w_sub)
-                            val = lf_sgd_apply4(P.sgd.eta, __ldcs(reinterpret_cast<const float4*>(P.sgd.w_sub + off)), val);
+                        if (P.sgd.w_sub) val = lf_sgd_apply4(P.sgd.eta, wv[i], val);
                         __stcs(reinterpret_cast<float4*>(P.gw + off), val);
                     }
                 }
@@ -564,16 +585,26 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
         for (int t = t_begin; t < t_end; ++t, ++tile_i) {
             const int rb = t / P.tiles_n, tn = t - rb * P.tiles_n;
             const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
-            if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
-            tg_fence_after();
             const int row0 = rb * 2 * TP_BM + (int)rank * TP_BM + quad * 32 + sub_r;
             const int col0 = tn * TP_BN + half * (TP_BN / 2) + sub_c;
             const size_t out_off = (size_t)row0 * P.N + col0;
             float* out_row = P.gw + out_off;
             const float* w_row = P.sgd.w_sub ? P.sgd.w_sub + out_off : nullptr;
             const size_t row_step = (size_t)4 * P.N;
+            if (w_row)
+                tg_prefetch_w(P.sgd.w_sub, P.N, row0 - sub_r, tn * TP_BN + half * (TP_BN / 2), TP_BN / 2, lane);
+            if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
+            tg_fence_after();
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TP_BN / 2 / 32; ++cchunk) {
+                // fused weight update: the loads of w go out before the accumulator is fetched
+                float4 wv[8];
+                if (w_row && col0 + cchunk * 32 < P.N) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (row0 + i * 4 < P.N)
+                            wv[i] = __ldcs(reinterpret_cast<const float4*>(w_row + i * row_step + cchunk * 32));
+                }
                 unsigned r[32];
                 tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + half * (TP_BN / 2) + cchunk * 32, r);
 #pragma unroll
@@ -587,8 +618,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                     for (int i = 0; i < 8; ++i) {
                         float4 val = *reinterpret_cast<const float4*>(blk + (i * 4 + sub_r) * TG_EPI_LD + sub_c);
                         if (row0 + i * 4 < P.N) {
-                            if (w_row)
-                                val = lf_sgd_apply4(P.sgd.eta, __ldcs(reinterpret_cast<const float4*>(w_row + i * row_step + cchunk * 32)), val);
+                            if (w_row) val = lf_sgd_apply4(P.sgd.eta, wv[i], val);
                             __stcs(reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 32), val);
                         }
                     }

@@ -19,10 +19,11 @@ struct lf_graph_key {
     int variant, gw_math;
     int sgd;        // 1: the graph writes w - eta * gw instead of gw
     float eta;
+    int cost;       // enum lf_cost baked into the Eq. bp1 kernel
     bool operator==(const lf_graph_key& o) const {
         return w == o.w && z == o.z && a == o.a && y == o.y && delta == o.delta &&
                gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math &&
-               sgd == o.sgd && (!sgd || eta == o.eta);
+               sgd == o.sgd && (!sgd || eta == o.eta) && cost == o.cost;
     }
 };
 
@@ -54,6 +55,7 @@ struct lf_ctx {
     int use_graph;
     int opt_delta_math;      // enum lf_delta_math
     int tc_pair_kernels;     // 1: the tensor-core contractions may use the two-SM (CTA pair) kernels
+    int opt_cost;            // enum lf_cost
     int sgd_on;              // the current backward call is lf_backward_sgd
     float sgd_eta;
     const float* sgd_w;      // its weights (what the update is subtracted from)
@@ -117,7 +119,7 @@ cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* 
                                float* z_l, float* a_l, int N, cudaStream_t s);
 cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s);
 cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
-                             int B, cudaStream_t s);
+                             int B, int cost, cudaStream_t s);
 int lfk_delta_row_chunks(int N);  // number of row chunks the delta matvec splits N rows into
 cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,

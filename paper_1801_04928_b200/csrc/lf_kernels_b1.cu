@@ -56,14 +56,17 @@ k_forward_matvec(const float* __restrict__ w, const float* __restrict__ b,
     }
 }
 
-// ---- Eq. bp1 : delta^L = (a^L - y) (.) sigma'(z^L), sigma' = a (1 - a) --------------------------
+// ---- Eq. bp1 : delta^L = grad_a C (.) sigma'(z^L), sigma' = a (1 - a) ---------------------------
+// quadratic cost: grad_a C = a^L - y;  cross-entropy: grad_a C = (a^L - y) / (a^L (1 - a^L)), which
+// the factor sigma' cancels, leaving delta^L = a^L - y
 __global__ void k_output_error(const float* __restrict__ aL, const float* __restrict__ y,
-                               float* __restrict__ deltaL, float* __restrict__ gbL, size_t n)
+                               float* __restrict__ deltaL, float* __restrict__ gbL, size_t n, int cost)
 {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float av = aL[i];
-    float d = (av - y[i]) * (av * (1.0f - av));
+    float d = av - y[i];
+    if (cost == LF_COST_QUADRATIC) d *= av * (1.0f - av);
     deltaL[i] = d;
     if (gbL) gbL[i] = d;  // Eq. bp3 for a single sample
 }
@@ -198,11 +201,11 @@ cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s)
 }
 
 cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
-                             int B, cudaStream_t s)
+                             int B, int cost, cudaStream_t s)
 {
     size_t n = (size_t)N * B;
     int grid = (int)((n + 255) / 256);
-    k_output_error<<<grid, 256, 0, s>>>(aL, y, deltaL, B == 1 ? gbL : nullptr, n);
+    k_output_error<<<grid, 256, 0, s>>>(aL, y, deltaL, B == 1 ? gbL : nullptr, n, cost);
     return cudaGetLastError();
 }
 

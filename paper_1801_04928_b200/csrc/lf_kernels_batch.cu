@@ -36,6 +36,14 @@ k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    // EPI_PLAIN with a weight matrix to update: fetch its values now, they are needed last
+    float4 wsub[4];
+    if (EPI == EPI_PLAIN && aux && n0 + tx * 4 < Nn) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (m0 + ty * 4 + i < M)
+                wsub[i] = *reinterpret_cast<const float4*>(aux + (size_t)(m0 + ty * 4 + i) * ldc + n0 + tx * 4);
+    }
 
     for (int k0 = 0; k0 < K; k0 += BK) {
         // ---- stage the A tile as As[k][m]
@@ -102,7 +110,7 @@ k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __
             *reinterpret_cast<float4*>(C + off) = r;
         } else {
             // EPI_PLAIN: the contraction itself, or (aux = the weight matrix) aux - eta * it
-            if (aux) r = lf_sgd_apply4(eta, *reinterpret_cast<const float4*>(aux + off), r);
+            if (aux) r = lf_sgd_apply4(eta, wsub[i], r);
             *reinterpret_cast<float4*>(C + off) = r;
         }
     }

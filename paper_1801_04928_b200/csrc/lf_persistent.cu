@@ -38,6 +38,7 @@ constexpr int PK_STAGE_FLOATS = 8192;   // 32 KiB per pipeline stage
 constexpr int PK_STAGES = 6;
 constexpr int PK_MAX_NCB = 4;           // column blocks per strip (strip width <= 4 * 256)
 constexpr int PK_MAX_SLICE = 128;       // strip columns finished per CTA (strip / C)
+constexpr int PK_SGD_BATCH = 16;        // fused weight update: loads of w a thread keeps in flight
 constexpr int PK_DROWS = 2176;          // floats of delta held per CTA and buffer (tile rows, padded)
 
 struct PkParams {
@@ -55,6 +56,7 @@ struct PkParams {
     int slice;     // Ws / C
     int keff;      // effective leapfrog workers
     int withhold;  // test hook: chain CTA 0 publishes nothing (the others' waits must expire)
+    int cost;      // enum lf_cost: which grad_a C enters Eq. bp1
     unsigned epoch;
     unsigned long long budget_ns;
     const float* a;
@@ -193,6 +195,7 @@ struct PkShared {
     unsigned long long part_ready[2];    // partial sums of a step have landed here (by step parity)
     unsigned long long d_ready[2];       // chain warps filled delta buffer p
     unsigned long long d_free[2];        // store warps are done with delta buffer p
+    unsigned long long st_done[PK_STAGES];   // fused weight update: store warps have read the stage
     volatile unsigned abort_flag;        // set once a wait of this CTA has run out
 };
 
@@ -246,6 +249,7 @@ __device__ __forceinline__ void wait_bar(unsigned bar, unsigned parity, const Pk
 }
 
 // Eq. bp4 for the rows [row0, row1) and all N columns: the leapfrog worker's store stream.
+template <bool UPDATE>
 __device__ void worker_store_rows(const PkParams& P, int l, int row0, int row1, float* d_rows,
                                   float* a_sm, PkShared* sh)
 {
@@ -258,22 +262,71 @@ __device__ void worker_store_rows(const PkParams& P, int l, int row0, int row1, 
     for (int r = row0 + tid; r < row1; r += PK_THREADS) d_rows[r - row0] = wait_slot(slots + r, P, sh);
     __syncthreads();
     float* gw_l = P.gw + (size_t)(l - 1) * N * N;
-    const float* w_l = P.w_sub ? P.w_sub + (size_t)(l - 1) * N * N : nullptr;
+    const float* w_l = UPDATE ? P.w_sub + (size_t)(l - 1) * N * N : nullptr;
     for (int r = row0 + warp; r < row1; r += PK_THREADS / 32) {
         const float d = d_rows[r - row0];
         float* out = gw_l + (size_t)r * N;
-        const float* w_row = w_l ? w_l + (size_t)r * N : nullptr;
+        if (UPDATE) {
+            const float4* w_row = reinterpret_cast<const float4*>(w_l + (size_t)r * N);
+            for (int c0 = lane; c0 < n4; c0 += 32 * PK_SGD_BATCH) {
+                float4 wv[PK_SGD_BATCH];
+#pragma unroll
+                for (int u = 0; u < PK_SGD_BATCH; ++u)
+                    if (c0 + 32 * u < n4) wv[u] = __ldcg(w_row + c0 + 32 * u);
+#pragma unroll
+                for (int u = 0; u < PK_SGD_BATCH; ++u) {
+                    const int c = c0 + 32 * u;
+                    if (c < n4) {
+                        const float4 a4 = reinterpret_cast<const float4*>(a_sm)[c];
+                        st_stream4(out + 4 * c, lf_sgd_apply4(P.eta, wv[u], make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w)));
+                    }
+                }
+            }
+        } else {
 #pragma unroll 4
-        for (int c = lane; c < n4; c += 32) {
-            float4 a4 = reinterpret_cast<const float4*>(a_sm)[c];
-            float4 g = make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w);
-            if (w_row) g = lf_sgd_apply4(P.eta, __ldcg(reinterpret_cast<const float4*>(w_row) + c), g);
-            st_stream4(out + 4 * c, g);
+            for (int c = lane; c < n4; c += 32) {
+                float4 a4 = reinterpret_cast<const float4*>(a_sm)[c];
+                st_stream4(out + 4 * c, make_float4(d * a4.x, d * a4.y, d * a4.z, d * a4.w));
+            }
         }
     }
     __syncthreads();
 }
 
+// Fused weight update of one column block of a CTA's tile (store warps of the fused variant):
+// out[rr][0..3] = w_in[rr][0..3] - eta * d[rr] * av for this thread's rows rr = trow, trow + RG, ...
+// A load costs a round trip that a store does not: every thread keeps PK_SGD_BATCH loads of w in
+// flight (a rotating queue in registers: use the oldest, then reissue its slot) so that the reads
+// keep up with the store stream.  Used for layer 1, which the chain never reads (the other layers
+// take w from the chain's shared-memory stages).
+// Not inlined: the queue would otherwise be live across the caller's unrolled column blocks.
+__device__ __noinline__ void store_tile_updated(const float* __restrict__ w_in, float* __restrict__ out,
+                                                const float* dr, float4 av, int rows, int trow, int RG, int N,
+                                                float eta)
+{
+    const int n_mine = rows > trow ? (rows - trow + RG - 1) / RG : 0;   // rows of this thread
+    float4 wq[PK_SGD_BATCH];
+#pragma unroll
+    for (int u = 0; u < PK_SGD_BATCH; ++u)
+        if (u < n_mine) wq[u] = __ldcg(reinterpret_cast<const float4*>(w_in + (size_t)(trow + u * RG) * N));
+    for (int base = 0; base < n_mine; base += PK_SGD_BATCH) {
+#pragma unroll
+        for (int u = 0; u < PK_SGD_BATCH; ++u) {
+            const int idx = base + u;
+            if (idx < n_mine) {
+                const int rr = trow + idx * RG;
+                const float d = dr[rr];
+                st_stream4(out + (size_t)rr * N, lf_sgd_apply4(eta, wq[u], make_float4(d * av.x, d * av.y, d * av.z, d * av.w)));
+                if (idx + PK_SGD_BATCH < n_mine)
+                    wq[u] = __ldcg(reinterpret_cast<const float4*>(w_in + (size_t)(rr + PK_SGD_BATCH * RG) * N));
+            }
+        }
+    }
+}
+
+// UPDATE = true: the instance behind lf_backward_sgd (P.w_sub set); the plain instance carries
+// none of its code.
+template <bool UPDATE>
 __global__ void __launch_bounds__(PK_THREADS, 1)
 k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams P)
 {
@@ -291,7 +344,10 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
     const bool is_chain_cluster = cluster_id < P.Qc;
 
     if (tid == 0) {
-        for (int i = 0; i < PK_STAGES; ++i) mbar_init(smem_u32(&sh->full[i]), 1);
+        for (int i = 0; i < PK_STAGES; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->st_done[i]), PK_THREADS - PK_CHAIN_THREADS);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh->part_ready[i]), 1);
             mbar_init(smem_u32(&sh->d_ready[i]), PK_CHAIN_THREADS);
@@ -316,7 +372,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         float* dr = stages + 16384;                   // up to N floats
         for (int l = L; l >= 1; --l) {
             if ((((L - l) % P.keff) % G) != g) continue;   // not a layer of my group
-            if (row0 < row1) worker_store_rows(P, l, row0, row1, dr, a_sm, sh);
+            if (row0 < row1) worker_store_rows<UPDATE>(P, l, row0, row1, dr, a_sm, sh);
         }
         cluster_sync_all();   // the cluster's CTAs leave together
         return;
@@ -348,6 +404,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 }
             };
             load_a4(L - 1, a4);
+            int it_store = 0;   // running sub-tile index, the chain warps' `it`
             for (int s = L; s >= 1; --s) {
                 const int p = s & 1;
                 const unsigned use = (unsigned)((L - s) >> 1);      // how often buffer p was used before
@@ -355,6 +412,42 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 wait_bar<false>(smem_u32(&sh->d_ready[p]), use & 1u, P, sh);
                 const float* dr = d_rows + p * PK_DROWS;
                 float* gw_s = P.gw + (size_t)(s - 1) * N * N;
+                if (UPDATE && s >= 2) {
+                    // Fused weight update, layers the chain reads: the sub-tiles of w^s pass through
+                    // this CTA's shared memory for the chain anyway, so the store warps take w from
+                    // there (the same stage, the same element mapping as the chain warps) -- no second
+                    // read of w from memory -- and tell the producer when they are done with a stage.
+                    const int rows = row_end - row_base;
+#pragma unroll
+                    for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
+                        if (cb >= nCB) break;
+                        const int col = col_base + cb * Wc + tcol * 4;
+                        const float4 av = a4[cb];
+                        float* out = gw_s + (size_t)row_base * N + col;
+                        for (int rb = 0; rb < nRB; ++rb, ++it_store) {
+                            const int st = it_store % PK_STAGES;
+                            wait_bar<false>(smem_u32(&sh->full[st]), (unsigned)((it_store / PK_STAGES) & 1), P, sh);
+                            const float4* tile = reinterpret_cast<const float4*>(stages + (size_t)st * PK_STAGE_FLOATS);
+                            if (col < N) {
+#pragma unroll 8
+                                for (int i = 0; i < 16; ++i) {
+                                    const int rr = rb * R + trow + i * RG;
+                                    if (rr < rows) {
+                                        const float d = dr[rr];
+                                        st_stream4(out + (size_t)rr * N,
+                                                   lf_sgd_apply4(P.eta, tile[ht + i * PK_CHAIN_THREADS],
+                                                                 make_float4(d * av.x, d * av.y, d * av.z, d * av.w)));
+                                    }
+                                }
+                            }
+                            mbar_arrive(smem_u32(&sh->st_done[st]));
+                        }
+                    }
+                    mbar_arrive(smem_u32(&sh->d_free[p]));
+#pragma unroll
+                    for (int cb = 0; cb < PK_MAX_NCB; ++cb) a4[cb] = a4_next[cb];
+                    continue;
+                }
 #pragma unroll
                 for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
                     if (cb >= nCB) break;
@@ -363,18 +456,10 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                     const float4 av = a4[cb];
                     float* out = gw_s + (size_t)row_base * N + col;
                     const int rows = row_end - row_base;
-                    if (P.w_sub) {
-                        // fused update: the tile of w^s was fetched for the chain a moment ago, so
-                        // this second read is served by L2 (layer 1, which the chain never reads,
-                        // comes from memory)
-                        const float* w_in = P.w_sub + (size_t)(s - 1) * N * N + (size_t)row_base * N + col;
-#pragma unroll 4
-                        for (int rr = trow; rr < rows; rr += RG) {
-                            const float d = dr[rr];
-                            const float4 wv = __ldcg(reinterpret_cast<const float4*>(w_in + (size_t)rr * N));
-                            st_stream4(out + (size_t)rr * N,
-                                       lf_sgd_apply4(P.eta, wv, make_float4(d * av.x, d * av.y, d * av.z, d * av.w)));
-                        }
+                    if (UPDATE) {
+                        // fused update of layer 1, which the chain never reads: w^1 comes from memory
+                        store_tile_updated(P.w_sub + (size_t)(s - 1) * N * N + (size_t)row_base * N + col, out, dr, av,
+                                           rows, trow, RG, N, P.eta);
                     } else {
 #pragma unroll 4
                         for (int rr = trow; rr < rows; rr += RG) {
@@ -406,6 +491,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             ++is_it;
             if (++is_rb == nRB) { is_rb = 0; if (++is_cb == nCB) { is_cb = 0; --is_s; } }
         };
+        const bool stores_read_stages = UPDATE && P.fused;
         if (tid == 0) {
             const int pre = total < PK_STAGES ? total : PK_STAGES;
             for (int i = 0; i < pre; ++i) issue_next();
@@ -424,7 +510,8 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 float d = 0.f;
                 if (r < Hr && row < N) {
                     const float av = aL[row];
-                    d = (av - P.y[row]) * (av * (1.0f - av));
+                    d = av - P.y[row];
+                    if (P.cost == LF_COST_QUADRATIC) d *= av * (1.0f - av);   // cross-entropy: sigma' cancels
                     if (q == 0) {
                         P.delta[(size_t)(L - 1) * N + row] = d;
                         P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
@@ -496,8 +583,19 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                             red_p[warp * 32 + lane] = acc;
                         }
                     }
-                    chain_sync();   // the stage is free again (and red_p is complete)
-                    if (tid == 0 && is_it < total && !sh->abort_flag) issue_next();
+                    chain_sync();   // the chain warps are done with the stage (and red_p is complete)
+                    if (tid == 0 && !sh->abort_flag) {
+                        if (!stores_read_stages) {
+                            if (is_it < total) issue_next();
+                        } else if (it >= 1 && is_it < total) {
+                            // fused weight update: the store warps read the stages too.  Refill the
+                            // stage of the sub-tile before this one, which they have had a whole
+                            // sub-tile's time to finish, rather than stall the chain on this one.
+                            wait_bar<false>(smem_u32(&sh->st_done[(it - 1) % PK_STAGES]),
+                                            (unsigned)(((it - 1) / PK_STAGES) & 1), P, sh);
+                            issue_next();
+                        }
+                    }
                 }
                 if (cb == 0) PK_STAMP(2);
                 if (!direct && tid < WC4) {
@@ -636,7 +734,8 @@ encode_tiled_fn get_encode_fn()
 }
 
 constexpr size_t PK_SMEM_BYTES = (size_t)PK_STAGES * PK_STAGE_FLOATS * 4 + (size_t)2 * PK_DROWS * 4 +
-                                 2 * PK_CHAIN_THREADS * 16 + 2 * PK_MAX_CLUSTER * PK_MAX_SLICE * 4 + 128;
+                                 2 * PK_CHAIN_THREADS * 16 + 2 * PK_MAX_CLUSTER * PK_MAX_SLICE * 4 + 256;
+static_assert(sizeof(PkShared) <= 256, "the barrier block must fit into the space reserved for it");
 
 struct PkPlan {
     bool ok;
@@ -664,11 +763,18 @@ int max_active_clusters(const lf_ctx* c, int C)
     }
     if (cached[C] >= 0) return cached[C];
     int n = 0;
-    if (cudaFuncSetAttribute(k_backward_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(k_backward_persistent<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)PK_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_backward_persistent<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)PK_SMEM_BYTES) == cudaSuccess) {
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[1];
         cluster_launch_config(&cfg, at, C, 16);
-        if (cudaOccupancyMaxActiveClusters(&n, k_backward_persistent, &cfg) != cudaSuccess) n = 0;
+        int n_upd = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_backward_persistent<false>, &cfg) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n_upd, k_backward_persistent<true>, &cfg) != cudaSuccess)
+            n = 0;
+        else if (n_upd < n)
+            n = n_upd;
     }
     cudaGetLastError();
     cached[C] = n;
@@ -739,9 +845,17 @@ bool lf_persistent_supported(const lf_ctx* c, int variant)
     return make_plan(c, variant).ok;
 }
 
+// LF_VARIANT_AUTO for one sample: fused pass or leapfrog CTA groups, from measurement (B200, L = 32,
+// buffers rotated so that nothing is found in L2; k = 1..8).  The groups variant gives the chain
+// half of the clusters; where that leaves it strips of exactly 32 or 64 columns (N <= 512 and
+// 896..1152) its shorter delta hand-off wins by 3-12 %, at the other widths the fused pass is
+// equal or ahead (from N = 3072 by 5-8 %).
 int lf_auto_variant(const lf_ctx* c)
 {
     if (c->B != 1) return LF_VARIANT_STREAMS;
+    const int N = c->N;
+    const bool groups_faster = N <= 576 || (N >= 832 && N <= 1216);
+    if (groups_faster && make_plan(c, LF_VARIANT_PERSISTENT).ok) return LF_VARIANT_PERSISTENT;
     return make_plan(c, LF_VARIANT_FUSED).ok ? LF_VARIANT_FUSED : LF_VARIANT_STREAMS;
 }
 
@@ -776,6 +890,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
+    P.cost = c->opt_cost;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
     P.w_sub = c->sgd_on ? c->sgd_w : nullptr; P.eta = c->sgd_eta;
@@ -787,13 +902,18 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.trace = c->trace_dev;
 #endif
 
-    LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_persistent<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)PK_SMEM_BYTES));
+    LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_persistent<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)PK_SMEM_BYTES));
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[1];
     cluster_launch_config(&cfg, at, pl.C, pl.Qc + pl.Qw);
     cfg.stream = c->stream;
     const CUtensorMap* mp = reinterpret_cast<const CUtensorMap*>(c->w_map_storage);
-    LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_persistent, *mp, P));
+    if (P.w_sub)
+        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_persistent<true>, *mp, P));
+    else
+        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_persistent<false>, *mp, P));
     c->stats.launches_backward = 1;
     c->stats.chain_ctas = pl.Qc * pl.C;
     c->stats.worker_ctas = pl.Qw * pl.C;

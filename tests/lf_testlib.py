@@ -14,7 +14,7 @@ DENORMAL = 2.0 ** -149
 
 
 def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=None,
-             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0):
+             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0):
     """lf_forward + lf_backward on device tensors t (w,b,x,y).  Returns dict of device tensors
     and the stats of the context."""
     L, N, B = cfg["L"], cfg["N"], cfg["B"]
@@ -32,6 +32,7 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
         ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
         ctx.set_option(lf.LF_OPT_DELTA_MATH, delta_math)
         ctx.set_option(lf.LF_OPT_TC_TILING, tc_tiling)
+        ctx.set_option(lf.LF_OPT_COST, cost)
         ctx.set_option(lf.LF_OPT_USE_GRAPH, 1 if use_graph else 0)
         ctx.forward(t["w"], t["b"], t["x"], z, a)
         for _ in range(repeat):
@@ -43,14 +44,14 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
     return dict(z=z, a=a, delta=delta, gw=gw, gb=gb), stats
 
 
-def oracle_pass(t, want_gw=False):
+def oracle_pass(t, want_gw=False, cross_entropy=False):
     """Forward + sequential backward of the oracle on host copies (fp32 weights promoted)."""
     w = t["w"].detach().cpu().numpy()
     b = t["b"].detach().cpu().numpy()
     x = t["x"].detach().cpu().numpy()
     y = t["y"].detach().cpu().numpy()
     z, a = orc.forward(w, b, x)
-    delta, gw, gb = orc.backward_sequential(w, z, a, y, want_gw=want_gw)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y, want_gw=want_gw, cross_entropy=cross_entropy)
     return dict(z=z, a=a, delta=delta, gw=gw, gb=gb)
 
 

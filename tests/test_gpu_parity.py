@@ -224,3 +224,35 @@ def test_config4_minibatch_full_size_sampled():
                 j, k = int(rng.integers(N)), int(rng.integers(N))
                 ref = orc.grad_w_entry(d_gpu[l], a_gpu[l], j, k)
                 assert abs(g[j, k] - ref) <= TF32_TOL * max(abs(ref), rms), (l, j, k, g[j, k], ref)
+
+
+@pytest.mark.parametrize("L,N,B,gw_math", [(3, 516, 1, lf.LF_GW_MATH_AUTO), (2, 388, 70, lf.LF_GW_MATH_FP32),
+                                           (3, 772, 256, lf.LF_GW_MATH_TF32), (2, 1028, 300, lf.LF_GW_MATH_TF32)])
+def test_grad_w_alone_is_the_layer_slab_of_backward(L, N, B, gw_math):
+    # lf_grad_w (Eq. bp4 of one layer as a call of its own) must give bitwise what lf_backward
+    # writes for that layer, and so inherits its parity with the oracle.
+    cfg = dict(L=L, N=N, B=B, k=2)
+    t = _inputs(L, N, B, y="uniform" if B == 1 else "onehot", seed=17 * N + B)
+    out, stats = gpu_pass(cfg, t, variant=lf.LF_VARIANT_STREAMS, gw_math=gw_math)
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with lf.Leapfrog(L, N, B, 2, stream=st.cuda_stream) as ctx:
+        ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
+        for l in range(L):
+            g = torch.full((N, N), float("nan"), device="cuda")
+            ctx.grad_w(out["delta"][l], out["a"][l], g)
+            ctx.sync()
+            assert torch.equal(g, out["gw"][l]), l
+        assert ctx.stats()["gw_math"] == stats["gw_math"]
+
+
+@pytest.mark.parametrize("N,want", [(512, lf.LF_VARIANT_PERSISTENT), (768, lf.LF_VARIANT_FUSED),
+                                    (1024, lf.LF_VARIANT_PERSISTENT), (2052, lf.LF_VARIANT_FUSED)])
+def test_auto_variant_follows_the_measured_table(N, want):
+    # LF_VARIANT_AUTO for one sample: leapfrog CTA groups at the widths where they were measured
+    # faster than the fused pass, the fused pass elsewhere; the result passes parity either way.
+    cfg = dict(L=3, N=N, B=1, k=2)
+    t = _inputs(3, N, 1, seed=N)
+    out, stats = gpu_pass(cfg, t)
+    assert stats["variant"] == want and stats["device_status"] == 0
+    compare_all(cfg, out, oracle_pass(t))
