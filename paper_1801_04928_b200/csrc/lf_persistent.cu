@@ -812,8 +812,10 @@ PkPlan plan_for_cluster(const lf_ctx* c, int variant, int C)
     return p;
 }
 
-// Pick the cluster size that puts the most CTAs (SMs) to work; ties go to the larger cluster,
-// whose strips are wider.
+// Pick the cluster size that puts the most CTAs (SMs) on the delta chain -- the chain sets the pace
+// (measured for the leapfrog groups at N = 256..2048: the cluster size with the most chain CTAs was
+// the fastest or within 2 % of it, however many workers it left); ties go to the larger cluster,
+// whose CTAs hold fewer rows each.
 PkPlan make_plan(const lf_ctx* c, int variant)
 {
     PkPlan best = {};
@@ -824,7 +826,7 @@ PkPlan make_plan(const lf_ctx* c, int variant)
     for (int C = PK_MAX_CLUSTER; C >= 2; C >>= 1) {
         PkPlan p = plan_for_cluster(c, variant, C);
         if (!p.ok) continue;
-        const int ctas = (p.Qc + p.Qw) * C;
+        const int ctas = p.Qc * C;
         if (ctas > best_ctas) { best = p; best_ctas = ctas; }
     }
     return best;
@@ -846,15 +848,17 @@ bool lf_persistent_supported(const lf_ctx* c, int variant)
 }
 
 // LF_VARIANT_AUTO for one sample: fused pass or leapfrog CTA groups, from measurement (B200, L = 32,
-// buffers rotated so that nothing is found in L2; k = 1..8).  The groups variant gives the chain
-// half of the clusters; where that leaves it strips of exactly 32 or 64 columns (N <= 512 and
-// 896..1152) its shorter delta hand-off wins by 3-12 %, at the other widths the fused pass is
-// equal or ahead (from N = 3072 by 5-8 %).
+// buffers rotated so that nothing is found in L2, N = 256..4096, k = 1..8).  Up to N = 2048 the pass
+// is bound by the delta hand-off, and the groups variant -- whose chain has half of the clusters,
+// hence wider strips and fewer CTAs to wait for -- is 1-12 % ahead with up to four workers; with
+// more workers (fewer CTAs per layer) only at the widths listed.  From N = 2560 the pass is
+// bandwidth-bound and the fused pass, which leaves no SM without a share of the weights, is 4-8 %
+// ahead.
 int lf_auto_variant(const lf_ctx* c)
 {
     if (c->B != 1) return LF_VARIANT_STREAMS;
     const int N = c->N;
-    const bool groups_faster = N <= 576 || (N >= 832 && N <= 1216);
+    const bool groups_faster = c->keff <= 4 ? N <= 2048 : (N <= 576 || (N >= 832 && N <= 1280));
     if (groups_faster && make_plan(c, LF_VARIANT_PERSISTENT).ok) return LF_VARIANT_PERSISTENT;
     return make_plan(c, LF_VARIANT_FUSED).ok ? LF_VARIANT_FUSED : LF_VARIANT_STREAMS;
 }
