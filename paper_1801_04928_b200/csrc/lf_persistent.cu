@@ -30,7 +30,9 @@
 
 namespace {
 
-constexpr int PK_THREADS = 256;
+constexpr int PK_THREADS = 256;          // chain warps 0-3 and store warps 4-7
+constexpr int PK_LAUNCH_THREADS = 288;   // + warp 8, whose lane 0 is the TMA producer of a chain CTA
+constexpr int PK_PRODUCER_WARP = 8;
 constexpr int PK_CHAIN_THREADS = 128;   // warps 0-3
 constexpr int PK_CHAIN_WARPS = 4;
 constexpr int PK_MAX_CLUSTER = 8;       // cluster sizes 2, 4 and 8 are used
@@ -196,6 +198,7 @@ struct PkShared {
     unsigned long long d_ready[2];       // chain warps filled delta buffer p
     unsigned long long d_free[2];        // store warps are done with delta buffer p
     unsigned long long st_done[PK_STAGES];   // fused weight update: store warps have read the stage
+    unsigned long long empty[PK_STAGES];     // the four chain warps have read the stage
     volatile unsigned abort_flag;        // set once a wait of this CTA has run out
 };
 
@@ -256,14 +259,16 @@ __device__ void worker_store_rows(const PkParams& P, int l, int row0, int row1, 
     const int N = P.N, n4 = N >> 2;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const float* a_prev = P.a + (size_t)(l - 1) * N;
-    for (int c = tid; c < n4; c += PK_THREADS)
-        reinterpret_cast<float4*>(a_sm)[c] = reinterpret_cast<const float4*>(a_prev)[c];
-    const unsigned long long* slots = P.xch + (size_t)(l - 1) * N;
-    for (int r = row0 + tid; r < row1; r += PK_THREADS) d_rows[r - row0] = wait_slot(slots + r, P, sh);
+    if (tid < PK_THREADS) {   // (the ninth warp has no part in a worker CTA; it only keeps the barriers whole)
+        for (int c = tid; c < n4; c += PK_THREADS)
+            reinterpret_cast<float4*>(a_sm)[c] = reinterpret_cast<const float4*>(a_prev)[c];
+        const unsigned long long* slots = P.xch + (size_t)(l - 1) * N;
+        for (int r = row0 + tid; r < row1; r += PK_THREADS) d_rows[r - row0] = wait_slot(slots + r, P, sh);
+    }
     __syncthreads();
     float* gw_l = P.gw + (size_t)(l - 1) * N * N;
     const float* w_l = UPDATE ? P.w_sub + (size_t)(l - 1) * N * N : nullptr;
-    for (int r = row0 + warp; r < row1; r += PK_THREADS / 32) {
+    for (int r = row0 + warp; warp < PK_THREADS / 32 && r < row1; r += PK_THREADS / 32) {
         const float d = d_rows[r - row0];
         float* out = gw_l + (size_t)r * N;
         if (UPDATE) {
@@ -327,7 +332,7 @@ __device__ __noinline__ void store_tile_updated(const float* __restrict__ w_in, 
 // UPDATE = true: the instance behind lf_backward_sgd (P.w_sub set); the plain instance carries
 // none of its code.
 template <bool UPDATE>
-__global__ void __launch_bounds__(PK_THREADS, 1)
+__global__ void __launch_bounds__(PK_LAUNCH_THREADS, 1)
 k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams P)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -347,6 +352,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         for (int i = 0; i < PK_STAGES; ++i) {
             mbar_init(smem_u32(&sh->full[i]), 1);
             mbar_init(smem_u32(&sh->st_done[i]), PK_THREADS - PK_CHAIN_THREADS);
+            mbar_init(smem_u32(&sh->empty[i]), PK_CHAIN_WARPS);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh->part_ready[i]), 1);
@@ -390,7 +396,43 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
     const int col_base = q * Ws;
     const int Hr_pad = nRB * R;
 
-    if (warp >= PK_CHAIN_WARPS) {
+    if (warp == PK_PRODUCER_WARP) {
+        // ------------------------- producer: weight sub-tiles by TMA, ahead of the chain ---------
+        // Issuing a tensor copy costs its thread several hundred cycles; on a thread of the chain
+        // warps that was a sixth of every layer step.  Here it costs nothing: lane 0 waits until
+        // the chain warps (and, under the fused weight update, the store warps) are done with a
+        // stage and refills it.
+        if (lane == 0) {
+            const int nSub = nCB * nRB;
+            const int total = (L - 1) * nSub;
+            const unsigned stage_bytes = (unsigned)(R * Wc * sizeof(float));
+            int is_s = L, is_cb = 0, is_rb = 0, is_it = 0;   // the next sub-tile: layer, column block, row block
+            for (; is_it < total; ++is_it) {
+                const int st = is_it % PK_STAGES;
+                if (is_it >= PK_STAGES) {
+                    const unsigned parity = (unsigned)(((is_it / PK_STAGES) - 1) & 1);
+                    wait_bar<false>(smem_u32(&sh->empty[st]), parity, P, sh);
+                    if (UPDATE && P.fused) wait_bar<false>(smem_u32(&sh->st_done[st]), parity, P, sh);
+                    if (sh->abort_flag) break;
+                }
+                const unsigned bar = smem_u32(&sh->full[st]);
+                mbar_expect_tx(bar, stage_bytes);
+                tma_load_3d(smem_u32(stages + (size_t)st * PK_STAGE_FLOATS), &w_map, bar,
+                            col_base + is_cb * Wc, row_base + is_rb * R, is_s - 1);
+                if (++is_rb == nRB) { is_rb = 0; if (++is_cb == nCB) { is_cb = 0; --is_s; } }
+            }
+            // A CTA that gave up waiting may still have weight tiles on their way into its shared
+            // memory; it must not exit under them.  Wait for the last loads, with a limit.
+            if (sh->abort_flag) {
+                const unsigned long long t0 = globaltimer_ns();
+                for (int j = is_it > PK_STAGES ? is_it - PK_STAGES : 0; j < is_it; ++j) {
+                    const unsigned bar = smem_u32(&sh->full[j % PK_STAGES]);
+                    const unsigned parity = (unsigned)((j / PK_STAGES) & 1);
+                    while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < 50000000ull) { }
+                }
+            }
+        }
+    } else if (warp >= PK_CHAIN_WARPS) {
         // ------------------------- store warps: gw^s = delta^s (x) a^{s-1} ---------------------
         if (P.fused) {
             float4 a4[PK_MAX_NCB], a4_next[PK_MAX_NCB];
@@ -475,27 +517,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         }
     } else {
         // ------------------------- chain warps --------------------------------------------------
-        const int nSub = nCB * nRB;
-        const int total = (L - 1) * nSub;
-        const unsigned stage_bytes = (unsigned)(R * Wc * sizeof(float));
         const int wpr = WC4 > 32 ? WC4 / 32 : 1;   // warps that share one tile row
-
-        // producer state (thread 0): the next sub-tile to fetch, as (layer, column block, row block)
-        int is_s = L, is_cb = 0, is_rb = 0, is_it = 0;
-        auto issue_next = [&]() {
-            const int st = is_it % PK_STAGES;
-            const unsigned bar = smem_u32(&sh->full[st]);
-            mbar_expect_tx(bar, stage_bytes);
-            tma_load_3d(smem_u32(stages + (size_t)st * PK_STAGE_FLOATS), &w_map, bar,
-                        col_base + is_cb * Wc, row_base + is_rb * R, is_s - 1);
-            ++is_it;
-            if (++is_rb == nRB) { is_rb = 0; if (++is_cb == nCB) { is_cb = 0; --is_s; } }
-        };
-        const bool stores_read_stages = UPDATE && P.fused;
-        if (tid == 0) {
-            const int pre = total < PK_STAGES ? total : PK_STAGES;
-            for (int i = 0; i < pre; ++i) issue_next();
-        }
 
         const int my_col = col_base + c * P.slice + tid;   // the column this thread finishes (tid < slice)
         const bool finisher = tid < P.slice && my_col < N;
@@ -583,19 +605,11 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                             red_p[warp * 32 + lane] = acc;
                         }
                     }
-                    chain_sync();   // the chain warps are done with the stage (and red_p is complete)
-                    if (tid == 0 && !sh->abort_flag) {
-                        if (!stores_read_stages) {
-                            if (is_it < total) issue_next();
-                        } else if (it >= 1 && is_it < total) {
-                            // fused weight update: the store warps read the stages too.  Refill the
-                            // stage of the sub-tile before this one, which they have had a whole
-                            // sub-tile's time to finish, rather than stall the chain on this one.
-                            wait_bar<false>(smem_u32(&sh->st_done[(it - 1) % PK_STAGES]),
-                                            (unsigned)(((it - 1) / PK_STAGES) & 1), P, sh);
-                            issue_next();
-                        }
-                    }
+                    // this warp is done with the stage: tell the producer (no CTA-wide barrier per
+                    // sub-tile; only the entries in red_p need one, at the end of a column block)
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->empty[st]));
+                    if (rb == nRB - 1 && !direct) chain_sync();   // red_p is complete
                 }
                 if (cb == 0) PK_STAMP(2);
                 if (!direct && tid < WC4) {
@@ -696,16 +710,6 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             chain_sync();
             PK_STAMP(6);
         }
-        // A CTA that gave up waiting gets here with weight tiles possibly still on their way into
-        // its shared memory; it must not exit under them.  Wait for the last loads, with a limit.
-        if (tid == 0 && sh->abort_flag) {
-            const unsigned long long t0 = globaltimer_ns();
-            for (int j = is_it > PK_STAGES ? is_it - PK_STAGES : 0; j < is_it; ++j) {
-                const unsigned bar = smem_u32(&sh->full[j % PK_STAGES]);
-                const unsigned parity = (unsigned)((j / PK_STAGES) & 1);
-                while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < 50000000ull) { }
-            }
-        }
     }
     __syncthreads();
     cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory
@@ -746,7 +750,7 @@ void cluster_launch_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int
 {
     *cfg = cudaLaunchConfig_t{};
     cfg->gridDim = dim3(C * clusters);
-    cfg->blockDim = dim3(PK_THREADS);
+    cfg->blockDim = dim3(PK_LAUNCH_THREADS);
     cfg->dynamicSmemBytes = PK_SMEM_BYTES;
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
