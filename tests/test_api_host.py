@@ -51,6 +51,8 @@ def test_null_context_is_an_error_not_a_crash():
     assert lf.lf_forward(None, 16, 16, 16, 16, 16) == lf.LF_ENULL
     assert lf.lf_backward(None, 16, 16, 16, 16, 16, 16, 16) == lf.LF_ENULL
     assert lf.lf_owner(None, 1) == -1
+    assert lf.lf_grad_w(None, 16, 16, 16) == lf.LF_ENULL
+    assert lf.lf_backward_sgd(None, 16, 16, 16, 16, 0.1, 16, 32, 16) == lf.LF_ENULL
 
 
 def test_no_device_means_an_error_not_a_fallback():

@@ -258,3 +258,19 @@ def test_auto_variant_follows_the_measured_table(N, k, want):
     out, stats = gpu_pass(cfg, t)
     assert stats["variant"] == want and stats["device_status"] == 0
     compare_all(cfg, out, oracle_pass(t))
+
+
+def test_width_beyond_the_persistent_kernels_falls_back_to_streams():
+    # N = 16388 is wider than any strip plan of the persistent kernel (and past its documented
+    # limit of 16384): AUTO, and an explicit request for the fused pass, must run the stream
+    # variant instead, say so in the stats, and still pass parity.
+    L, N = 2, 16388
+    cfg = dict(L=L, N=N, B=1, k=2)
+    t = _inputs(L, N, 1, seed=4)
+    ref = oracle_pass(t)
+    for variant in (lf.LF_VARIANT_AUTO, lf.LF_VARIANT_FUSED):
+        out, stats = gpu_pass(cfg, t, variant=variant)
+        assert stats["variant"] == lf.LF_VARIANT_STREAMS and stats["device_status"] == 0
+        compare_all(cfg, out, ref)
+        del out
+        torch.cuda.empty_cache()
