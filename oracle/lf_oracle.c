@@ -10,7 +10,7 @@
  * What it follows (arXiv 1801.04928, "Leapfrogging for parallelism in deep neural networks"):
  *   Section 2, Eq. x   : a^0 = x                      (the paper's "layer 1" is the input)
  *   Section 2, Eq. z   : z^l = w^l a^{l-1} + b^l      (bias reading, see below)
- *   Section 2, Eq. a   : a^l = sigma(z^l)
+ *   Section 2, Eq. a   : a^l = sigma(z^l)             (sigmoid by default; lfo_set_activation)
  *   Section 2, Eq. bp1 : delta^L = grad_a C (.) sigma'(z^L)
  *   Section 2, Eq. bp2 : delta^l = ((w^{l+1})^T delta^{l+1}) (.) sigma'(z^l)
  *   Section 2, Eq. bp3 : dC/db^l_j = delta^l_j
@@ -83,6 +83,39 @@ static double lfo_sigmoid_prime(double t)
 double lfo_sigma(double t) { return lfo_sigmoid(t); }
 double lfo_sigma_prime(double t) { return lfo_sigmoid_prime(t); }
 
+/* The activation function of Eq. a and its derivative in Eq. bp1 / bp2.  The paper writes sigma
+ * for it and says its equations hold generally; the sigmoid is the default and what every
+ * workload of the paper's kind uses.  Two more are offered so that an implementation's choice of
+ * activation can be checked: tanh, and the rectifier max(t, 0) with derivative [t > 0] (taken as
+ * 0 at t = 0).  The choice is a property of the whole pass, so it is a setting of this library
+ * instance rather than an argument of every function. */
+enum { LFO_ACT_SIGMOID = 0, LFO_ACT_TANH = 1, LFO_ACT_RELU = 2 };
+static int lfo_activation = LFO_ACT_SIGMOID;
+
+int lfo_set_activation(int kind)
+{
+    if (kind < LFO_ACT_SIGMOID || kind > LFO_ACT_RELU) return -1;
+    lfo_activation = kind;
+    return 0;
+}
+
+static double lfo_act(double t)
+{
+    if (lfo_activation == LFO_ACT_TANH) return tanh(t);
+    if (lfo_activation == LFO_ACT_RELU) return t > 0.0 ? t : 0.0;
+    return lfo_sigmoid(t);
+}
+
+static double lfo_act_prime(double t)
+{
+    if (lfo_activation == LFO_ACT_TANH) {
+        double h = tanh(t);
+        return 1.0 - h * h;
+    }
+    if (lfo_activation == LFO_ACT_RELU) return t > 0.0 ? 1.0 : 0.0;
+    return lfo_sigmoid_prime(t);
+}
+
 /* Eq. x, Eq. z, Eq. a: the forward pass.  a has L+1 slabs of B*N, a[0] := x. */
 void lfo_forward(int L, int N, int B, const lfo_w_t *w, const double *b, const double *x,
                  double *z, double *a)
@@ -101,7 +134,7 @@ void lfo_forward(int L, int N, int B, const lfo_w_t *w, const double *b, const d
                 for (int k = 0; k < N; ++k)
                     acc += (double)wl[IDX2(j, k, N)] * aprev[IDX2(s, k, N)];
                 zl[IDX2(s, j, N)] = acc + bl[j];                          /* Eq. z */
-                al[IDX2(s, j, N)] = lfo_sigmoid(zl[IDX2(s, j, N)]);       /* Eq. a */
+                al[IDX2(s, j, N)] = lfo_act(zl[IDX2(s, j, N)]);           /* Eq. a */
             }
         }
     }
@@ -124,7 +157,7 @@ void lfo_output_error(int N, int B, const double *aL, const double *y, const dou
                       double *deltaL)
 {
     for (size_t i = 0; i < (size_t)B * N; ++i)
-        deltaL[i] = (aL[i] - y[i]) * lfo_sigmoid_prime(zL[i]);
+        deltaL[i] = (aL[i] - y[i]) * lfo_act_prime(zL[i]);
 }
 
 /* Eq. bp2 at one layer: delta^l = ((w^{l+1})^T delta^{l+1}) (.) sigma'(z^l).
@@ -137,7 +170,7 @@ void lfo_delta_step(int N, int B, const lfo_w_t *w_up, const double *delta_up,
             double acc = 0.0;
             for (int j = 0; j < N; ++j)                    /* ((w^{l+1})^T delta^{l+1})_k */
                 acc += (double)w_up[IDX2(j, k, N)] * delta_up[IDX2(s, j, N)];
-            delta_l[IDX2(s, k, N)] = acc * lfo_sigmoid_prime(z_l[IDX2(s, k, N)]);
+            delta_l[IDX2(s, k, N)] = acc * lfo_act_prime(z_l[IDX2(s, k, N)]);
         }
     }
 }
@@ -233,7 +266,7 @@ void lfo_output_error_cross_entropy(int N, int B, const double *aL, const double
 {
     for (size_t i = 0; i < (size_t)B * N; ++i) {
         double grad_a = (aL[i] - y[i]) / (aL[i] * (1.0 - aL[i]));
-        deltaL[i] = grad_a * lfo_sigmoid_prime(zL[i]);                 /* Eq. bp1 */
+        deltaL[i] = grad_a * lfo_act_prime(zL[i]);                     /* Eq. bp1 */
     }
 }
 

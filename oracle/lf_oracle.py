@@ -85,11 +85,41 @@ def _lib(tag: str) -> ctypes.CDLL:
             lib.lfo_backward_sequential_cross_entropy.restype = None
             lib.lfo_backward_sequential_cross_entropy.argtypes = [i, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp,
                                                                   _c_dp, _c_dp]
+            lib.lfo_set_activation.restype = i
+            lib.lfo_set_activation.argtypes = [i]
+            lib.lfo_set_activation(_ACTIVATION)
             lib.lfo_sgd_step.restype = None
             lib.lfo_sgd_step.argtypes = [i, i, wp, _c_dp, ctypes.c_double, _c_dp]
             assert lib.lfo_weight_bytes() == (8 if tag == "f64" else 4)
             _LIBS[tag] = lib
         return _LIBS[tag]
+
+
+ACTIVATIONS = {"sigmoid": 0, "tanh": 1, "relu": 2}
+_ACTIVATION = 0
+
+
+def set_activation(name: str) -> None:
+    """Choose the activation function of every later pass (both compiled flavours)."""
+    global _ACTIVATION
+    _ACTIVATION = ACTIVATIONS[name]
+    for tag in ("f64", "f32"):
+        if _lib(tag).lfo_set_activation(_ACTIVATION) != 0:
+            raise ValueError(name)
+
+
+class activation:
+    """``with activation("tanh"): ...`` -- the sigmoid is restored afterwards."""
+
+    def __init__(self, name: str):
+        self.name = name
+
+    def __enter__(self):
+        set_activation(self.name)
+        return self
+
+    def __exit__(self, *exc):
+        set_activation("sigmoid")
 
 
 def _w(w: np.ndarray):

@@ -452,3 +452,49 @@ def test_cross_entropy_output_error_collapses_to_a_minus_y():
     np.testing.assert_allclose(d_top, a[-1] - y, rtol=1e-12, atol=1e-15)
     d_ce, _, _ = orc.backward_sequential(w, z, a, y, cross_entropy=True)
     np.testing.assert_allclose(d_ce[1], orc.delta_step(w[2], d_top, z[1]), rtol=1e-13, atol=0)
+
+
+# ---- other activation functions (the paper's equations are stated for a general sigma) ---------
+@pytest.mark.parametrize("act", ["tanh", "relu"])
+@pytest.mark.parametrize("L,N,B", [(1, 3, 1), (3, 5, 3), (4, 6, 2)])
+def test_other_activations_match_central_differences(act, L, N, B):
+    # The same finite-difference pin as for the sigmoid.  The rectifier is not differentiable where
+    # z = 0; with these seeds no pre-activation comes within 1e-3 of it (checked), so a step of
+    # 1e-5 never crosses the kink.
+    w, b, x, y = _net(L, N, B, seed=700 + 100 * L + 10 * N + B)
+    with orc.activation(act):
+        z, a = orc.forward(w, b, x)
+        if act == "relu":
+            assert np.min(np.abs(z)) > 1e-3
+        delta, gw, gb = orc.backward_sequential(w, z, a, y)
+        h = 1e-5
+        for l in range(L):
+            fd_w = np.empty((N, N)); fd_b = np.empty((N,))
+            for j in range(N):
+                for k in range(N):
+                    wp = w.copy(); wp[l, j, k] += h
+                    wm = w.copy(); wm[l, j, k] -= h
+                    fd_w[j, k] = (_cost(wp, b, x, y) - _cost(wm, b, x, y)) / (2 * h)
+                bp = b.copy(); bp[l, j] += h
+                bm = b.copy(); bm[l, j] -= h
+                fd_b[j] = (_cost(w, bp, x, y) - _cost(w, bm, x, y)) / (2 * h)
+            assert np.max(np.abs(gw[l] - fd_w)) <= 2e-7 * max(np.max(np.abs(fd_w)), 1e-3) + 1e-12
+            assert np.max(np.abs(gb[l] - fd_b)) <= 2e-7 * max(np.max(np.abs(fd_b)), 1e-3) + 1e-12
+    # and the setting does not leak
+    assert abs(orc.forward(np.zeros((1, 2, 2)), np.zeros((1, 2)), np.ones((1, 2)))[1][1, 0, 0] - 0.5) < 1e-15
+
+
+def test_activation_values_and_closed_forms():
+    w = np.zeros((1, 3, 3)); b = np.array([[-2.0, 0.0, 1.5]]); x = np.ones((1, 3)); y = np.zeros((1, 3))
+    with orc.activation("tanh"):
+        z, a = orc.forward(w, b, x)
+        np.testing.assert_allclose(a[1, 0], np.tanh(b[0]), rtol=1e-15)
+        d, _, _ = orc.backward_sequential(w, z, a, y)
+        np.testing.assert_allclose(d[0, 0], np.tanh(b[0]) * (1 - np.tanh(b[0]) ** 2), rtol=1e-14)
+    with orc.activation("relu"):
+        z, a = orc.forward(w, b, x)
+        assert np.array_equal(a[1, 0], [0.0, 0.0, 1.5])
+        d, _, _ = orc.backward_sequential(w, z, a, y)
+        assert np.array_equal(d[0, 0], [0.0, 0.0, 1.5])           # (a - y) * [z > 0], 0 at z = 0
+    with pytest.raises(KeyError):
+        orc.set_activation("softplus")
