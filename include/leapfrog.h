@@ -93,6 +93,14 @@ enum lf_cost {
                                   grad_a C = (a^L - y) / (a^L (1 - a^L)), so delta^L = a^L - y   */
 };
 
+/* The activation function sigma of Eq. a (and sigma' of Eq. bp1 / bp2, taken from the stored
+ * activations).  The paper writes a general sigma; the sigmoid is the default. */
+enum lf_activation {
+    LF_ACT_SIGMOID = 0, /* sigma(t) = 1 / (1 + e^{-t}),  sigma' = a (1 - a)                        */
+    LF_ACT_TANH = 1,    /* sigma(t) = tanh t,             sigma' = 1 - a^2                         */
+    LF_ACT_RELU = 2     /* sigma(t) = max(t, 0),          sigma' = [a > 0]  (0 where t <= 0)       */
+};
+
 enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
@@ -101,6 +109,10 @@ enum lf_option {
     LF_OPT_DELTA_MATH = 6,    /* enum lf_delta_math                                           */
     LF_OPT_TC_TILING = 7,     /* enum lf_tc_tiling                                            */
     LF_OPT_COST = 8,          /* enum lf_cost (default LF_COST_QUADRATIC)                     */
+    LF_OPT_ACTIVATION = 9,    /* enum lf_activation (default LF_ACT_SIGMOID); applies to
+                                 lf_forward and lf_backward alike, so set it before both.
+                                 LF_COST_CROSS_ENTROPY needs the sigmoid: lf_backward returns
+                                 LF_EINVAL for any other pairing                              */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -123,6 +135,7 @@ typedef struct lf_stats {
                                  ONE_SM or TWO_SM; 0 if none ran)                             */
     int delta_tiling;         /* the same for the last tensor-core Eq. bp2 / Eq. z launch     */
     int cost;                 /* cost function the last lf_backward used (enum lf_cost)       */
+    int activation;           /* activation the last lf_forward / lf_backward used            */
 } lf_stats;
 
 /*

@@ -22,6 +22,8 @@ LF_OPT_VARIANT, LF_OPT_GW_MATH, LF_OPT_WAIT_BUDGET_US, LF_OPT_USE_GRAPH, LF_OPT_
 LF_OPT_DELTA_MATH = 6
 LF_OPT_TC_TILING = 7
 LF_OPT_COST = 8
+LF_OPT_ACTIVATION = 9
+LF_ACT_SIGMOID, LF_ACT_TANH, LF_ACT_RELU = 0, 1, 2
 LF_COST_QUADRATIC, LF_COST_CROSS_ENTROPY = 0, 1
 LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
 LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
@@ -38,7 +40,7 @@ class lf_stats(ctypes.Structure):
                 ("chain_ctas", ctypes.c_int), ("worker_ctas", ctypes.c_int),
                 ("launches_forward", ctypes.c_int), ("launches_backward", ctypes.c_int),
                 ("device_status", ctypes.c_uint), ("workspace_bytes", ctypes.c_longlong),
-                ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int), ("cost", ctypes.c_int)]
+                ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int), ("cost", ctypes.c_int), ("activation", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:

@@ -74,18 +74,18 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
     const float* a_l = a + (size_t)l * slab(c);
     float* gb_l = gb + (size_t)(l - 1) * N;
     if (l == L) {
-        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, c->opt_cost, s));
+        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, c->opt_cost, c->opt_act, s));
     } else {
         const float* w_up = w + (size_t)l * mat(c);  // w^{l+1}
         const float* d_up = delta + (size_t)l * slab(c);
         if (B == 1)
-            LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, N, s));
+            LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, N, c->opt_act, s));
         else if (c->stats.delta_math == LF_DELTA_MATH_3XTF32) {
             int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, s, launches);
             if (rc != LF_OK) return rc;
             return LF_OK;
         } else
-            LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, N, B, s));
+            LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, N, B, c->opt_act, s));
     }
     *launches += 1;
     return LF_OK;
@@ -135,7 +135,7 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
         return rc;
     }
     lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math,
-                     c->sgd_on, c->sgd_eta, c->opt_cost};
+                     c->sgd_on, c->sgd_eta, c->opt_cost, c->opt_act};
     if (!(c->graph_valid && c->graph_key == key)) {
         drop_graph(c);
         LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -296,6 +296,10 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value != LF_COST_QUADRATIC && value != LF_COST_CROSS_ENTROPY) return LF_EINVAL;
             ctx->opt_cost = (int)value;
             return LF_OK;
+        case LF_OPT_ACTIVATION:
+            if (value < LF_ACT_SIGMOID || value > LF_ACT_RELU) return LF_EINVAL;
+            ctx->opt_act = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -327,17 +331,18 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
         float* z_l = z + (size_t)(l - 1) * slab(ctx);
         float* a_l = a + (size_t)l * slab(ctx);
         if (B == 1) {
-            LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, N, s));
+            LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, N, ctx->opt_act, s));
             ++launches;
         } else if (resolve_delta_math(ctx) == LF_DELTA_MATH_3XTF32) {
             int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, s, &launches);
             if (rc2 != LF_OK) return rc2;
         } else {
-            LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, N, B, s));
+            LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, N, B, ctx->opt_act, s));
             ++launches;
         }
     }
     ctx->stats.launches_forward = launches;
+    ctx->stats.activation = ctx->opt_act;
     return LF_OK;
 }
 
@@ -348,6 +353,7 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     const void* ps[] = {w, z, a, y, delta, gw, gb};
     int rc = check_ptrs(ps, 7);
     if (rc != LF_OK) return rc;
+    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
     int variant = resolve_variant(ctx);
     const int gw_math = resolve_gw_math(ctx);
     if (variant != LF_VARIANT_STREAMS && !lf_persistent_supported(ctx, variant))
@@ -356,6 +362,7 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     ctx->stats.gw_math = gw_math;
     ctx->stats.delta_math = resolve_delta_math(ctx);
     ctx->stats.cost = ctx->opt_cost;
+    ctx->stats.activation = ctx->opt_act;
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
@@ -447,6 +454,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     ctx->stats.gw_math = gw_math;
     ctx->stats.delta_math = resolve_delta_math(ctx);
     ctx->stats.cost = ctx->opt_cost;
+    ctx->stats.activation = ctx->opt_act;
     int launches = 0;
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
     LF_CUDA_TRY(ctx, cudaStreamWaitEvent(hs, ctx->fork_ev, 0));
@@ -466,6 +474,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
         if (l < Li) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0));   // w^{l+1}
         int rc = enqueue_chain_step(ctx, l, d_w, d_a, d_y, d_d, d_gb, s, &launches);
         if (rc != LF_OK) return rc;
+    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
         LF_CUDA_TRY(ctx, cudaEventRecord(ctx->ready_ev[l - 1], s));
         const int j = (Li - l) % ctx->keff;
         cudaStream_t wsj = ctx->wstreams[j];

@@ -782,7 +782,7 @@ __device__ __forceinline__ int dg_slot_count(const DgSlots& S, size_t i)
 // delta^l = (sum over the partial-sum slots, in slot order) * sigma'(z^l), sigma' = a (1 - a)
 __global__ void __launch_bounds__(256)
 k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
-               size_t n4, const DgSlots S)
+               size_t n4, const DgSlots S, int act)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
@@ -793,14 +793,14 @@ k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l,
         s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
     }
     const float4 av = reinterpret_cast<const float4*>(a_l)[i];
-    reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * (av.x * (1.0f - av.x)), s.y * (av.y * (1.0f - av.y)),
-                                                        s.z * (av.z * (1.0f - av.z)), s.w * (av.w * (1.0f - av.w)));
+    reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * lf_act_prime(av.x, act), s.y * lf_act_prime(av.y, act),
+                                                        s.z * lf_act_prime(av.z, act), s.w * lf_act_prime(av.w, act));
 }
 
 // forward: z^l = (sum over the partial-sum slots) + b^l ; a^l = sigma(z^l)
 __global__ void __launch_bounds__(256)
 k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_l, float* __restrict__ z_l,
-                 float* __restrict__ a_l, size_t n4, int n4_row, const DgSlots S)
+                 float* __restrict__ a_l, size_t n4, int n4_row, const DgSlots S, int act)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
@@ -813,8 +813,7 @@ k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_
     const float4 bb = reinterpret_cast<const float4*>(b_l)[i % n4_row];
     s.x += bb.x; s.y += bb.y; s.z += bb.z; s.w += bb.w;
     reinterpret_cast<float4*>(z_l)[i] = s;
-    reinterpret_cast<float4*>(a_l)[i] = make_float4(1.0f / (1.0f + expf(-s.x)), 1.0f / (1.0f + expf(-s.y)),
-                                                    1.0f / (1.0f + expf(-s.z)), 1.0f / (1.0f + expf(-s.w)));
+    reinterpret_cast<float4*>(a_l)[i] = make_float4(lf_act(s.x, act), lf_act(s.y, act), lf_act(s.z, act), lf_act(s.w, act));
 }
 
 typedef CUresult (*dg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1040,7 +1039,7 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     int rc = dg_launch(c, delta_up, w_up, false, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * c->N / 4;
-    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(c, pl));
+    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(c, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
@@ -1054,7 +1053,7 @@ int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const floa
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * c->N / 4;
     k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, c->N / 4,
-                                                                  dg_slots(c, pl));
+                                                                  dg_slots(c, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;

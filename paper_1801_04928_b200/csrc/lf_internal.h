@@ -20,10 +20,11 @@ struct lf_graph_key {
     int sgd;        // 1: the graph writes w - eta * gw instead of gw
     float eta;
     int cost;       // enum lf_cost baked into the Eq. bp1 kernel
+    int act;        // enum lf_activation baked into the kernels
     bool operator==(const lf_graph_key& o) const {
         return w == o.w && z == o.z && a == o.a && y == o.y && delta == o.delta &&
                gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math &&
-               sgd == o.sgd && (!sgd || eta == o.eta) && cost == o.cost;
+               sgd == o.sgd && (!sgd || eta == o.eta) && cost == o.cost && act == o.act;
     }
 };
 
@@ -34,6 +35,19 @@ struct lf_sgd {
     float eta;
 };
 #ifdef __CUDACC__
+// Eq. a and the derivative used by Eq. bp1 / bp2, the latter from the stored activation a = sigma(z)
+__device__ __forceinline__ float lf_act(float t, int kind)
+{
+    if (kind == LF_ACT_TANH) return tanhf(t);
+    if (kind == LF_ACT_RELU) return fmaxf(t, 0.0f);
+    return 1.0f / (1.0f + expf(-t));
+}
+__device__ __forceinline__ float lf_act_prime(float a, int kind)
+{
+    if (kind == LF_ACT_TANH) return 1.0f - a * a;
+    if (kind == LF_ACT_RELU) return a > 0.0f ? 1.0f : 0.0f;
+    return a * (1.0f - a);
+}
 // one rounding: fma(-eta, g, w)
 __device__ __forceinline__ float4 lf_sgd_apply4(float eta, float4 w, float4 g)
 {
@@ -56,6 +70,7 @@ struct lf_ctx {
     int opt_delta_math;      // enum lf_delta_math
     int tc_pair_kernels;     // 1: the tensor-core contractions may use the two-SM (CTA pair) kernels
     int opt_cost;            // enum lf_cost
+    int opt_act;             // enum lf_activation
     int sgd_on;              // the current backward call is lf_backward_sgd
     float sgd_eta;
     const float* sgd_w;      // its weights (what the update is subtracted from)
@@ -116,22 +131,22 @@ struct lf_ctx {
 
 // B = 1 kernels
 cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* a_prev,
-                               float* z_l, float* a_l, int N, cudaStream_t s);
+                               float* z_l, float* a_l, int N, int act, cudaStream_t s);
 cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s);
 cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
-                             int B, int cost, cudaStream_t s);
+                             int B, int cost, int act, cudaStream_t s);
 int lfk_delta_row_chunks(int N);  // number of row chunks the delta matvec splits N rows into
 cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,
-                             int N, cudaStream_t s);
+                             int N, int act, cudaStream_t s);
 cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
                          lf_sgd sgd, cudaStream_t s);
 
 // B > 1 kernels (fp32 on the CUDA cores)
 cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
-                             float* z_l, float* a_l, int N, int B, cudaStream_t s);
+                             float* z_l, float* a_l, int N, int B, int act, cudaStream_t s);
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
-                           float* delta_l, int N, int B, cudaStream_t s);
+                           float* delta_l, int N, int B, int act, cudaStream_t s);
 cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
                              int B, lf_sgd sgd, cudaStream_t s);
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s);

@@ -8,8 +8,6 @@
 
 namespace {
 
-__device__ __forceinline__ float lf_sigmoid(float t) { return 1.0f / (1.0f + expf(-t)); }
-
 __device__ __forceinline__ float4 ld_stream(const float4* p)
 {
     // Weights are read once per pass: keep them from displacing the vectors in L1.
@@ -22,7 +20,7 @@ constexpr int FWD_WARPS = 8;
 __global__ void __launch_bounds__(FWD_WARPS * 32)
 k_forward_matvec(const float* __restrict__ w, const float* __restrict__ b,
                  const float* __restrict__ a_prev, float* __restrict__ z,
-                 float* __restrict__ a, int N)
+                 float* __restrict__ a, int N, int act)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = blockIdx.x * FWD_WARPS + warp;
@@ -52,7 +50,7 @@ k_forward_matvec(const float* __restrict__ w, const float* __restrict__ b,
     if (lane == 0) {
         float zz = acc + b[j];
         z[j] = zz;
-        a[j] = lf_sigmoid(zz);
+        a[j] = lf_act(zz, act);
     }
 }
 
@@ -60,13 +58,13 @@ k_forward_matvec(const float* __restrict__ w, const float* __restrict__ b,
 // quadratic cost: grad_a C = a^L - y;  cross-entropy: grad_a C = (a^L - y) / (a^L (1 - a^L)), which
 // the factor sigma' cancels, leaving delta^L = a^L - y
 __global__ void k_output_error(const float* __restrict__ aL, const float* __restrict__ y,
-                               float* __restrict__ deltaL, float* __restrict__ gbL, size_t n, int cost)
+                               float* __restrict__ deltaL, float* __restrict__ gbL, size_t n, int cost, int act)
 {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     float av = aL[i];
     float d = av - y[i];
-    if (cost == LF_COST_QUADRATIC) d *= av * (1.0f - av);
+    if (cost == LF_COST_QUADRATIC) d *= lf_act_prime(av, act);
     deltaL[i] = d;
     if (gbL) gbL[i] = d;  // Eq. bp3 for a single sample
 }
@@ -86,7 +84,7 @@ __global__ void __launch_bounds__(DMV_WARPS * 32)
 k_delta_matvec(const float* __restrict__ w_up, const float* __restrict__ delta_up,
                const float* __restrict__ a_l, float* __restrict__ delta_l,
                float* __restrict__ gb_l, float* __restrict__ partial,
-               unsigned* __restrict__ counters, int N, int rows_per_chunk, int chunks)
+               unsigned* __restrict__ counters, int N, int rows_per_chunk, int chunks, int act)
 {
     __shared__ float4 red[DMV_WARPS][DMV_STRIP4];
     __shared__ bool is_last;
@@ -151,10 +149,10 @@ k_delta_matvec(const float* __restrict__ w_up, const float* __restrict__ delta_u
         }
         float4 av = reinterpret_cast<const float4*>(a_l)[c4];
         float4 d;
-        d.x = t0.x * (av.x * (1.0f - av.x));
-        d.y = t0.y * (av.y * (1.0f - av.y));
-        d.z = t0.z * (av.z * (1.0f - av.z));
-        d.w = t0.w * (av.w * (1.0f - av.w));
+        d.x = t0.x * lf_act_prime(av.x, act);
+        d.y = t0.y * lf_act_prime(av.y, act);
+        d.z = t0.z * lf_act_prime(av.z, act);
+        d.w = t0.w * lf_act_prime(av.w, act);
         reinterpret_cast<float4*>(delta_l)[c4] = d;
         if (gb_l) reinterpret_cast<float4*>(gb_l)[c4] = d;  // Eq. bp3
     }
@@ -188,10 +186,10 @@ k_gw_rank1(const float* __restrict__ delta_l, const float* __restrict__ a_prev,
 }  // namespace
 
 cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* a_prev,
-                               float* z_l, float* a_l, int N, cudaStream_t s)
+                               float* z_l, float* a_l, int N, int act, cudaStream_t s)
 {
     int grid = (N + FWD_WARPS - 1) / FWD_WARPS;
-    k_forward_matvec<<<grid, FWD_WARPS * 32, 0, s>>>(w_l, b_l, a_prev, z_l, a_l, N);
+    k_forward_matvec<<<grid, FWD_WARPS * 32, 0, s>>>(w_l, b_l, a_prev, z_l, a_l, N, act);
     return cudaGetLastError();
 }
 
@@ -201,11 +199,11 @@ cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s)
 }
 
 cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
-                             int B, int cost, cudaStream_t s)
+                             int B, int cost, int act, cudaStream_t s)
 {
     size_t n = (size_t)N * B;
     int grid = (int)((n + 255) / 256);
-    k_output_error<<<grid, 256, 0, s>>>(aL, y, deltaL, B == 1 ? gbL : nullptr, n, cost);
+    k_output_error<<<grid, 256, 0, s>>>(aL, y, deltaL, B == 1 ? gbL : nullptr, n, cost, act);
     return cudaGetLastError();
 }
 
@@ -217,7 +215,7 @@ int lfk_delta_row_chunks(int N)
 
 cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,
-                             int N, cudaStream_t s)
+                             int N, int act, cudaStream_t s)
 {
     int n4 = N >> 2;
     int strips = (n4 + DMV_STRIP4 - 1) / DMV_STRIP4;
@@ -225,7 +223,7 @@ cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const flo
     int chunks = (N + rows - 1) / rows;
     dim3 grid(strips, chunks);
     k_delta_matvec<<<grid, DMV_WARPS * 32, 0, s>>>(w_up, delta_up, a_l, delta_l, gb_l, partial,
-                                                  counters, N, rows, chunks);
+                                                  counters, N, rows, chunks, act);
     return cudaGetLastError();
 }
 
@@ -307,6 +305,6 @@ extern "C" int lf_delta_step_static(const float* w_up, const float* delta_up, co
         return LF_ECUDA;
     dim3 grid(strips, chunks);
     k_delta_matvec<<<grid, DMV_WARPS * 32, 0, s>>>(w_up, delta_up, a_l, delta_l, nullptr, partial,
-                                                  counters, N, rows, chunks);
+                                                  counters, N, rows, chunks, LF_ACT_SIGMOID);
     return cudaGetLastError() == cudaSuccess ? LF_OK : LF_ECUDA;
 }

@@ -9,8 +9,6 @@
 
 namespace {
 
-__device__ __forceinline__ float lf_sigmoid(float t) { return 1.0f / (1.0f + expf(-t)); }
-
 constexpr int BM = 64, BN = 64, BK = 16, PAD = 4;
 
 enum { EPI_PLAIN = 0, EPI_FORWARD = 1, EPI_DELTA = 2 };
@@ -23,7 +21,7 @@ template <bool A_KMAJOR, bool B_KMAJOR, int EPI>
 __global__ void __launch_bounds__(256)
 k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __restrict__ C,
             float* __restrict__ C2, const float* __restrict__ aux, int M, int Nn, int K, int lda,
-            int ldb, int ldc, float eta)
+            int ldb, int ldc, float eta, int act)
 {
     __shared__ __align__(16) float As[BK][BM + PAD];
     __shared__ __align__(16) float Bs[BK][BN + PAD];
@@ -101,12 +99,12 @@ k_gemm_simt(const float* __restrict__ A, const float* __restrict__ Bm, float* __
             float4 bb = *reinterpret_cast<const float4*>(aux + n);
             r.x += bb.x; r.y += bb.y; r.z += bb.z; r.w += bb.w;
             *reinterpret_cast<float4*>(C + off) = r;                       // z
-            *reinterpret_cast<float4*>(C2 + off) = make_float4(lf_sigmoid(r.x), lf_sigmoid(r.y),
-                                                               lf_sigmoid(r.z), lf_sigmoid(r.w));
+            *reinterpret_cast<float4*>(C2 + off) = make_float4(lf_act(r.x, act), lf_act(r.y, act),
+                                                               lf_act(r.z, act), lf_act(r.w, act));
         } else if (EPI == EPI_DELTA) {
             float4 av = *reinterpret_cast<const float4*>(aux + off);
-            r.x *= av.x * (1.0f - av.x); r.y *= av.y * (1.0f - av.y);
-            r.z *= av.z * (1.0f - av.z); r.w *= av.w * (1.0f - av.w);
+            r.x *= lf_act_prime(av.x, act); r.y *= lf_act_prime(av.y, act);
+            r.z *= lf_act_prime(av.z, act); r.w *= lf_act_prime(av.w, act);
             *reinterpret_cast<float4*>(C + off) = r;
         } else {
             // EPI_PLAIN: the contraction itself, or (aux = the weight matrix) aux - eta * it
@@ -149,20 +147,20 @@ inline dim3 gemm_grid(int M, int Nn) { return dim3((Nn + BN - 1) / BN, (M + BM -
 }  // namespace
 
 cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
-                             float* z_l, float* a_l, int N, int B, cudaStream_t s)
+                             float* z_l, float* a_l, int N, int B, int act, cudaStream_t s)
 {
     // M = B (samples), Nn = N (neuron j), K = N (neuron k of the layer below)
     k_gemm_simt<true, true, EPI_FORWARD><<<gemm_grid(B, N), 256, 0, s>>>(
-        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N, 0.f);
+        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N, 0.f, act);
     return cudaGetLastError();
 }
 
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
-                           float* delta_l, int N, int B, cudaStream_t s)
+                           float* delta_l, int N, int B, int act, cudaStream_t s)
 {
     // M = B, Nn = N (neuron k of layer l), K = N (neuron j of layer l+1); w_up[j][k] is n-contiguous
     k_gemm_simt<true, false, EPI_DELTA><<<gemm_grid(B, N), 256, 0, s>>>(
-        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N, 0.f);
+        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N, 0.f, act);
     return cudaGetLastError();
 }
 
@@ -171,7 +169,7 @@ cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* g
 {
     // M = N (j), Nn = N (k), K = B; both operands are contiguous along their M / N index
     k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(N, N), 256, 0, s>>>(
-        delta_l, a_prev, gw_l, nullptr, sgd.w_sub, N, N, B, N, N, N, sgd.eta);
+        delta_l, a_prev, gw_l, nullptr, sgd.w_sub, N, N, B, N, N, N, sgd.eta, LF_ACT_SIGMOID);
     return cudaGetLastError();
 }
 

@@ -59,6 +59,7 @@ struct PkParams {
     int keff;      // effective leapfrog workers
     int withhold;  // test hook: chain CTA 0 publishes nothing (the others' waits must expire)
     int cost;      // enum lf_cost: which grad_a C enters Eq. bp1
+    int act;       // enum lf_activation: sigma' from the stored activations
     unsigned epoch;
     unsigned long long budget_ns;
     const float* a;
@@ -533,7 +534,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 if (r < Hr && row < N) {
                     const float av = aL[row];
                     d = av - P.y[row];
-                    if (P.cost == LF_COST_QUADRATIC) d *= av * (1.0f - av);   // cross-entropy: sigma' cancels
+                    if (P.cost == LF_COST_QUADRATIC) d *= lf_act_prime(av, P.act);   // cross-entropy: sigma' cancels
                     if (q == 0) {
                         P.delta[(size_t)(L - 1) * N + row] = d;
                         P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
@@ -645,7 +646,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 for (int cc = 1; cc < PK_MAX_CLUSTER * PK_CHAIN_WARPS; ++cc)
                     if (cc < n_src) v += part[cc];
                 if (my_col < N) {
-                    const float d = v * (a_mine * (1.0f - a_mine));   // Eq. bp2
+                    const float d = v * lf_act_prime(a_mine, P.act);   // Eq. bp2
                     if (!(P.withhold && blockIdx.x == 0)) st_slot(P.xch + (size_t)(s - 2) * N + my_col, d, P.epoch);
                     P.delta[(size_t)(s - 2) * N + my_col] = d;
                     P.gb[(size_t)(s - 2) * N + my_col] = d;           // Eq. bp3
@@ -898,7 +899,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
-    P.cost = c->opt_cost;
+    P.cost = c->opt_cost; P.act = c->opt_act;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
     P.w_sub = c->sgd_on ? c->sgd_w : nullptr; P.eta = c->sgd_eta;

@@ -14,7 +14,7 @@ DENORMAL = 2.0 ** -149
 
 
 def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=None,
-             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0):
+             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0, act=0):
     """lf_forward + lf_backward on device tensors t (w,b,x,y).  Returns dict of device tensors
     and the stats of the context."""
     L, N, B = cfg["L"], cfg["N"], cfg["B"]
@@ -33,6 +33,7 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
         ctx.set_option(lf.LF_OPT_DELTA_MATH, delta_math)
         ctx.set_option(lf.LF_OPT_TC_TILING, tc_tiling)
         ctx.set_option(lf.LF_OPT_COST, cost)
+        ctx.set_option(lf.LF_OPT_ACTIVATION, act)
         ctx.set_option(lf.LF_OPT_USE_GRAPH, 1 if use_graph else 0)
         ctx.forward(t["w"], t["b"], t["x"], z, a)
         for _ in range(repeat):
