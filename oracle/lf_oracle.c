@@ -400,3 +400,99 @@ void lfo_sgd_step(int L, int N, const lfo_w_t *w, const double *gw, double eta, 
     const size_t n = (size_t)L * N * N;
     for (size_t i = 0; i < n; ++i) w_new[i] = (double)w[i] - eta * gw[i];
 }
+
+/* ---- layers of different widths ----------------------------------------------------------
+ * Section 2 gives the hidden layers one width N "for simplicity" and notes that the equations
+ * hold generally.  Here they are written out once more for widths n_0 .. n_L (n_0 the input,
+ * n_L the output): w^l is n_l x n_{l-1}, every per-layer array is the concatenation of its
+ * layers' blocks in layer order without padding,
+ *     w, gw : block l = [n_l][n_{l-1}]      b, gb : block l = [n_l]
+ *     z, delta : block l = [B][n_l]         a : block l = [B][n_l], l = 0..L, block 0 = x
+ * Same equations, same order of operations as the functions above; only the index ranges of
+ * the sums follow the layer.  cross_entropy != 0 selects the second cost in Eq. bp1. */
+void lfo_forward_widths(int L, const int *n, int B, const lfo_w_t *w, const double *b,
+                        const double *x, double *z, double *a)
+{
+    memcpy(a, x, (size_t)B * (size_t)n[0] * sizeof(double));             /* Eq. x */
+    const lfo_w_t *wl = w;
+    const double *bl = b, *aprev = a;
+    double *zl = z;
+    for (int l = 1; l <= L; ++l) {
+        int rows = n[l], cols = n[l - 1];
+        double *al = (double *)aprev + (size_t)B * cols;
+        for (int s = 0; s < B; ++s) {
+            for (int j = 0; j < rows; ++j) {
+                double acc = 0.0;
+                for (int k = 0; k < cols; ++k)
+                    acc += (double)wl[IDX2(j, k, cols)] * aprev[IDX2(s, k, cols)];
+                zl[IDX2(s, j, rows)] = acc + bl[j];                       /* Eq. z */
+                al[IDX2(s, j, rows)] = lfo_act(zl[IDX2(s, j, rows)]);     /* Eq. a */
+            }
+        }
+        wl += (size_t)rows * cols;
+        bl += rows;
+        zl += (size_t)B * rows;
+        aprev = al;
+    }
+}
+
+void lfo_backward_widths(int L, const int *n, int B, int cross_entropy, const lfo_w_t *w,
+                         const double *z, const double *a, const double *y, double *delta,
+                         double *gw, double *gb)
+{
+    /* where each layer's block starts (index l = 1..L; a also has l = 0) */
+    size_t *ow = (size_t *)malloc(((size_t)L + 2) * sizeof(size_t));
+    size_t *oh = (size_t *)malloc(((size_t)L + 2) * sizeof(size_t));
+    size_t *oa = (size_t *)malloc(((size_t)L + 2) * sizeof(size_t));
+    ow[1] = 0; oh[1] = 0; oa[0] = 0;
+    for (int l = 1; l <= L; ++l) {
+        ow[l + 1] = ow[l] + (size_t)n[l] * (size_t)n[l - 1];
+        oh[l + 1] = oh[l] + (size_t)n[l];
+        oa[l] = oa[l - 1] + (size_t)n[l - 1];
+    }
+    for (int l = L; l >= 1; --l) {
+        int rows = n[l], cols = n[l - 1];
+        double *dl = delta + (size_t)B * oh[l];
+        const double *zl = z + (size_t)B * oh[l];
+        if (l == L) {                                                     /* Eq. bp1 */
+            const double *aL = a + (size_t)B * oa[L];
+            for (size_t i = 0; i < (size_t)B * rows; ++i) {
+                double grad_a = cross_entropy ? (aL[i] - y[i]) / (aL[i] * (1.0 - aL[i]))
+                                              : aL[i] - y[i];
+                dl[i] = grad_a * lfo_act_prime(zl[i]);
+            }
+        } else {                                                          /* Eq. bp2 */
+            int up = n[l + 1];
+            const lfo_w_t *wu = w + ow[l + 1];                            /* w^{l+1}: up x rows */
+            const double *du = delta + (size_t)B * oh[l + 1];
+            for (int s = 0; s < B; ++s) {
+                for (int k = 0; k < rows; ++k) {
+                    double acc = 0.0;
+                    for (int j = 0; j < up; ++j)
+                        acc += (double)wu[IDX2(j, k, rows)] * du[IDX2(s, j, up)];
+                    dl[IDX2(s, k, rows)] = acc * lfo_act_prime(zl[IDX2(s, k, rows)]);
+                }
+            }
+        }
+        for (int j = 0; j < rows; ++j) {                                  /* Eq. bp3 */
+            double acc = 0.0;
+            for (int s = 0; s < B; ++s) acc += dl[IDX2(s, j, rows)];
+            gb[oh[l] + j] = acc;
+        }
+        if (gw) {                                                         /* Eq. bp4 */
+            const double *ap = a + (size_t)B * oa[l - 1];
+            double *gl = gw + ow[l];
+            for (int j = 0; j < rows; ++j) {
+                for (int k = 0; k < cols; ++k) {
+                    double acc = 0.0;
+                    for (int s = 0; s < B; ++s)
+                        acc += ap[IDX2(s, k, cols)] * dl[IDX2(s, j, rows)];
+                    gl[IDX2(j, k, cols)] = acc;
+                }
+            }
+        }
+    }
+    free(ow);
+    free(oh);
+    free(oa);
+}

@@ -88,6 +88,10 @@ def _lib(tag: str) -> ctypes.CDLL:
             lib.lfo_set_activation.restype = i
             lib.lfo_set_activation.argtypes = [i]
             lib.lfo_set_activation(_ACTIVATION)
+            lib.lfo_forward_widths.restype = None
+            lib.lfo_forward_widths.argtypes = [i, _c_ip, i, wp, _c_dp, _c_dp, _c_dp, _c_dp]
+            lib.lfo_backward_widths.restype = None
+            lib.lfo_backward_widths.argtypes = [i, _c_ip, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp]
             lib.lfo_sgd_step.restype = None
             lib.lfo_sgd_step.argtypes = [i, i, wp, _c_dp, ctypes.c_double, _c_dp]
             assert lib.lfo_weight_bytes() == (8 if tag == "f64" else 4)
@@ -268,3 +272,66 @@ def backward_leapfrog(w, z, a, y, k: int, want_gw: bool = True, threads: bool = 
     if rc != 0:
         raise ValueError("lfo_backward_leapfrog: invalid sizes")
     return delta, gw, gb, writer, writes, total.value
+
+
+# ---- layers of different widths -----------------------------------------------------------------
+# Arrays are flat: each is the concatenation of its per-layer blocks (see the C file).  `widths`
+# is [n_0, ..., n_L]; `split` cuts a flat array back into per-layer views.
+
+def _widths(widths):
+    n = np.ascontiguousarray(widths, dtype=np.int32)
+    if n.ndim != 1 or n.size < 2 or (n < 1).any():
+        raise ValueError("widths must be [n_0, ..., n_L], all >= 1")
+    return n, n.ctypes.data_as(_c_ip)
+
+
+def sizes_widths(widths, B: int) -> dict[str, int]:
+    """Element counts of the flat arrays of a network with these widths."""
+    n = [int(v) for v in widths]
+    hidden = sum(n[1:])
+    return {"w": sum(n[l] * n[l - 1] for l in range(1, len(n))), "b": hidden, "z": B * hidden,
+            "a": B * sum(n), "x": B * n[0], "y": B * n[-1]}
+
+
+def split(flat, widths, kind: str, B: int = 1):
+    """Per-layer views of a flat array: kind 'w' -> [n_l, n_{l-1}], 'b' -> [n_l], 'z' -> [B, n_l]
+    (l = 1..L), 'a' -> [B, n_l] (l = 0..L)."""
+    n = [int(v) for v in widths]
+    out, pos = [], 0
+    for l in range(0 if kind == "a" else 1, len(n)):
+        shape = {"w": (n[l], n[l - 1]) if l else None, "b": (n[l],), "z": (B, n[l]), "a": (B, n[l])}[kind]
+        cnt = int(np.prod(shape))
+        out.append(flat[pos:pos + cnt].reshape(shape))
+        pos += cnt
+    assert pos == flat.size
+    return out
+
+
+def forward_widths(widths, w, b, x):
+    """Eq. x, z, a for layer widths n_0..n_L; flat w, b, x in, flat float64 z, a out."""
+    n, npnt = _widths(widths)
+    lib, w, wp = _w(w)
+    B = np.asarray(x).size // int(n[0])
+    sz = sizes_widths(n, B)
+    assert w.size == sz["w"] and np.asarray(b).size == sz["b"] and np.asarray(x).size == sz["x"]
+    b, x = _d(b).ravel(), _d(x).ravel()
+    z = np.empty(sz["z"], dtype=np.float64)
+    a = np.empty(sz["a"], dtype=np.float64)
+    lib.lfo_forward_widths(n.size - 1, npnt, B, wp, _p(b), _p(x), _p(z), _p(a))
+    return z, a
+
+
+def backward_widths(widths, w, z, a, y, want_gw: bool = True, cross_entropy: bool = False):
+    """Eq. bp1-bp4 for layer widths n_0..n_L; flat arrays; returns flat delta, gw (or None), gb."""
+    n, npnt = _widths(widths)
+    lib, w, wp = _w(w)
+    B = np.asarray(y).size // int(n[-1])
+    sz = sizes_widths(n, B)
+    z, a, y = _d(z).ravel(), _d(a).ravel(), _d(y).ravel()
+    assert w.size == sz["w"] and z.size == sz["z"] and a.size == sz["a"] and y.size == sz["y"]
+    delta = np.empty(sz["z"], dtype=np.float64)
+    gb = np.empty(sz["b"], dtype=np.float64)
+    gw = np.empty(sz["w"], dtype=np.float64) if want_gw else None
+    lib.lfo_backward_widths(n.size - 1, npnt, B, 1 if cross_entropy else 0, wp, _p(z), _p(a), _p(y),
+                            _p(delta), _p(gw) if want_gw else None, _p(gb))
+    return delta, gw, gb

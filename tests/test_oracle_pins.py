@@ -498,3 +498,98 @@ def test_activation_values_and_closed_forms():
         assert np.array_equal(d[0, 0], [0.0, 0.0, 1.5])           # (a - y) * [z > 0], 0 at z = 0
     with pytest.raises(KeyError):
         orc.set_activation("softplus")
+
+
+# ---- layers of different widths ------------------------------------------------------------------
+def _net_widths(widths, B, seed):
+    r = np.random.default_rng(seed)
+    sz = orc.sizes_widths(widths, B)
+    w = np.concatenate([r.normal(0.0, 1.0 / np.sqrt(widths[l - 1]), size=widths[l] * widths[l - 1])
+                        for l in range(1, len(widths))])
+    b = r.normal(0.0, 1.0, size=sz["b"])
+    x = r.uniform(0.0, 1.0, size=sz["x"])
+    y = r.uniform(0.0, 1.0, size=sz["y"])
+    return w, b, x, y
+
+
+def _cost_widths(widths, w, b, x, y, B, cross_entropy=False):
+    _, a = orc.forward_widths(widths, w, b, x)
+    aL = orc.split(a, widths, "a", B)[-1]
+    return orc.cost(aL[None], y.reshape(B, -1), cross_entropy=cross_entropy)
+
+
+@pytest.mark.parametrize("act,cross_entropy", [("sigmoid", False), ("sigmoid", True), ("tanh", False)])
+@pytest.mark.parametrize("widths,B", [([3, 5, 2], 1), ([4, 2, 6, 3], 3), ([2, 7, 7, 1, 5], 2)])
+def test_widths_gradients_match_central_differences(widths, B, act, cross_entropy):
+    # Every dC/dw and dC/db of a network whose layers differ in width, against central differences
+    # of the cost (forward pass only).  Catches a block offset or a row length taken from the wrong
+    # layer: with n_l != n_{l-1} either one reads another layer's numbers.
+    w, b, x, y = _net_widths(widths, B, seed=900 + sum(widths) + B)
+    with orc.activation(act):
+        z, a = orc.forward_widths(widths, w, b, x)
+        delta, gw, gb = orc.backward_widths(widths, w, z, a, y, cross_entropy=cross_entropy)
+        h = 1e-5
+        fd_w = np.empty_like(w); fd_b = np.empty_like(b)
+        for i in range(w.size):
+            wp = w.copy(); wp[i] += h
+            wm = w.copy(); wm[i] -= h
+            fd_w[i] = (_cost_widths(widths, wp, b, x, y, B, cross_entropy) -
+                       _cost_widths(widths, wm, b, x, y, B, cross_entropy)) / (2 * h)
+        for i in range(b.size):
+            bp = b.copy(); bp[i] += h
+            bm = b.copy(); bm[i] -= h
+            fd_b[i] = (_cost_widths(widths, w, bp, x, y, B, cross_entropy) -
+                       _cost_widths(widths, w, bm, x, y, B, cross_entropy)) / (2 * h)
+    for g, f in zip(orc.split(gw, widths, "w"), orc.split(fd_w, widths, "w")):
+        assert np.max(np.abs(g - f)) <= 3e-7 * np.max(np.abs(f)) + 1e-12
+    for g, f in zip(orc.split(gb, widths, "b"), orc.split(fd_b, widths, "b")):
+        assert np.max(np.abs(g - f)) <= 3e-7 * np.max(np.abs(f)) + 1e-12
+    # Eq. bp3 for one sample: gb is delta itself
+    if B == 1:
+        assert np.array_equal(gb, delta)
+
+
+def test_widths_with_one_common_width_is_the_uniform_oracle_bitwise():
+    L, N, B = 4, 6, 3
+    w, b, x, y = _net(L, N, B, seed=77)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    widths = [N] * (L + 1)
+    z2, a2 = orc.forward_widths(widths, w.ravel(), b.ravel(), x.ravel())
+    d2, gw2, gb2 = orc.backward_widths(widths, w.ravel(), z2, a2, y.ravel())
+    assert np.array_equal(z2, z.ravel()) and np.array_equal(a2, a.ravel())
+    assert np.array_equal(d2, delta.ravel()) and np.array_equal(gw2, gw.ravel()) and np.array_equal(gb2, gb.ravel())
+    dce, _, _ = orc.backward_sequential(w, z, a, y, cross_entropy=True)
+    d3, _, _ = orc.backward_widths(widths, w.ravel(), z2, a2, y.ravel(), cross_entropy=True)
+    assert np.array_equal(d3, dce.ravel())
+
+
+def test_widths_network_is_the_zero_padded_uniform_network():
+    # Embed widths [4, 7, 3, 5] into the uniform network of width 7 with zero weights to and from the
+    # padding neurons.  The padding neurons fire (sigma(b) != 0) but nothing reads them, and adding
+    # exact zeros changes no sum: the real entries must come out bitwise equal, the gradients by the
+    # padding weights that leave real neurons (rows of padding neurons) need not vanish, those into
+    # padding columns of layer 1 multiply x-padding = 0.
+    widths, B = [4, 7, 3, 5], 2
+    L, N = len(widths) - 1, max(widths)
+    w, b, x, y = _net_widths(widths, B, seed=5)
+    W = np.zeros((L, N, N)); Bv = np.zeros((L, N)); X = np.zeros((B, N)); Y = np.zeros((B, N))
+    for l, (wl, bl) in enumerate(zip(orc.split(w, widths, "w"), orc.split(b, widths, "b")), start=1):
+        W[l - 1, :widths[l], :widths[l - 1]] = wl
+        Bv[l - 1, :widths[l]] = bl
+    X[:, :widths[0]] = x.reshape(B, -1)
+    Y[:, :widths[-1]] = y.reshape(B, -1)
+    Z, A = orc.forward(W, Bv, X)
+    # the padded outputs must not contribute to delta^L: give them the target they already hit
+    Y[:, widths[-1]:] = A[-1][:, widths[-1]:]
+    D, GW, GB = orc.backward_sequential(W, Z, A, Y)
+    z, a = orc.forward_widths(widths, w, b, x)
+    d, gw, gb = orc.backward_widths(widths, w, z, a, y)
+    for l, (zl, dl, gwl, gbl) in enumerate(zip(orc.split(z, widths, "z", B), orc.split(d, widths, "z", B),
+                                               orc.split(gw, widths, "w"), orc.split(gb, widths, "b")), start=1):
+        assert np.array_equal(zl, Z[l - 1][:, :widths[l]])
+        assert np.array_equal(dl, D[l - 1][:, :widths[l]])
+        assert np.array_equal(gwl, GW[l - 1][:widths[l], :widths[l - 1]])
+        assert np.array_equal(gbl, GB[l - 1][:widths[l]])
+    for l, al in enumerate(orc.split(a, widths, "a", B)):
+        assert np.array_equal(al, A[l][:, :widths[l]])
