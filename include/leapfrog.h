@@ -148,6 +148,31 @@ typedef struct lf_stats {
 int lf_create(lf_ctx** out, int L, int N, int B, int k);
 
 /*
+ * The same for a network whose layers differ in width (Section 2 gives only the hidden layers
+ * a common width N and says the equations hold generally): widths is a HOST array of L + 1
+ * ints, widths[0] = n_0 the width of the input x, widths[l] = n_l the number of neurons of
+ * weight layer l, widths[L] = n_L the width of the output and of y.  Every width must be
+ * >= 1 and a multiple of 4.  The array is copied; the caller may free it on return.
+ *
+ * Layouts: each array is the concatenation of its per-layer blocks, in layer order, with no
+ * padding (all block starts stay 16-byte aligned because the widths are multiples of 4):
+ *     w, gw    block l = [n_l][n_{l-1}] row-major, l = 1..L   (w^l_jk: neuron k below -> neuron j)
+ *     b, gb    block l = [n_l]
+ *     z, delta block l = [B][n_l]
+ *     a        block l = [B][n_l], l = 0..L, a block 0 = x
+ *     x [B][n_0],  y [B][n_L]
+ * With all widths equal this is lf_create(L, widths[0], B, k) exactly, layouts included.
+ * Otherwise the context runs one launch per layer with the k workers as streams
+ * (LF_VARIANT_STREAMS) and fp32 arithmetic throughout -- the single-launch and the
+ * tensor-core kernels are written for one common width; options asking for them are accepted
+ * and lf_get_stats() reports what ran, with N = the widest layer.  lf_forward, lf_backward,
+ * lf_backward_sgd and lf_backward_host take such a context; lf_grad_w, which names no layer,
+ * returns LF_EINVAL for it.
+ * Errors: LF_ENULL (out, widths), LF_EINVAL (sizes), LF_ECUDA, LF_ENOMEM.
+ */
+int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k);
+
+/*
  * Use `cuda_stream` (a cudaStream_t, borrowed, must outlive the work enqueued on it) for
  * all subsequent calls.  NULL selects the legacy default stream (the initial setting).
  */

@@ -60,3 +60,28 @@ def make_config(index: int, device: str | torch.device = "cpu", **override):
     cfg.update(override)
     t = make_inputs(cfg["L"], cfg["N"], cfg["B"], cfg["y"], SEED_BASE + index, device)
     return cfg, t
+
+
+def make_inputs_widths(widths, B: int, y: str = "uniform", seed: int = SEED_BASE,
+                       device: str | torch.device = "cpu") -> dict[str, torch.Tensor]:
+    """The same distributions for a network whose layers have widths n_0..n_L (w^l is
+    n_l x n_{l-1} with std 1/sqrt(n_{l-1})).  Every tensor is flat: the per-layer blocks one after
+    the other, in layer order (w: [n_l][n_{l-1}] row-major; b: [n_l]; x: [B][n_0]; y: [B][n_L])."""
+    if y not in ("onehot", "uniform"):
+        raise ValueError("y must be 'onehot' or 'uniform'")
+    n = [int(v) for v in widths]
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(seed))
+    w = torch.cat([torch.empty(n[l] * n[l - 1], dtype=torch.float32, device=dev)
+                   .normal_(0.0, 1.0, generator=g).mul_(float(n[l - 1]) ** -0.5) for l in range(1, len(n))])
+    b = torch.empty(sum(n[1:]), dtype=torch.float32, device=dev).normal_(0.0, 1.0, generator=g)
+    x = torch.empty(B * n[0], dtype=torch.float32, device=dev).uniform_(0.0, 1.0, generator=g)
+    if y == "uniform":
+        yt = torch.empty(B * n[-1], dtype=torch.float32, device=dev).uniform_(0.0, 1.0, generator=g)
+    else:
+        idx = torch.randint(0, n[-1], (B,), generator=g, device=dev)
+        yt = torch.zeros((B, n[-1]), dtype=torch.float32, device=dev)
+        yt[torch.arange(B, device=dev), idx] = 1.0
+        yt = yt.reshape(-1)
+    return dict(w=w, b=b, x=x, y=yt)

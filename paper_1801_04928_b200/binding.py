@@ -28,7 +28,7 @@ LF_COST_QUADRATIC, LF_COST_CROSS_ENTROPY = 0, 1
 LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
 LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
 
-EXPORTS = ("lf_create", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
+EXPORTS = ("lf_create", "lf_create_widths", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
            "lf_backward_sgd", "lf_grad_w", "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",
            "lf_strerror", "lf_version", "lf_destroy", "lf_delta_step_static")
 
@@ -51,6 +51,7 @@ def _load() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     vp, i, ll = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong
     lib.lf_create.argtypes = [ctypes.POINTER(vp), i, i, i, i]
+    lib.lf_create_widths.argtypes = [ctypes.POINTER(vp), i, ctypes.POINTER(ctypes.c_int), i, i]
     lib.lf_set_stream.argtypes = [vp, vp]
     lib.lf_set_option.argtypes = [vp, i, ll]
     lib.lf_forward.argtypes = [vp] * 6
@@ -108,6 +109,15 @@ def lf_create(L: int, N: int, B: int, k: int):
     """Returns (status, handle)."""
     h = ctypes.c_void_p(None)
     rc = _lib.lf_create(ctypes.byref(h), int(L), int(N), int(B), int(k))
+    return rc, h
+
+
+def lf_create_widths(widths, B: int, k: int):
+    """``widths`` = [n_0, ..., n_L] (host ints).  Returns (status, handle)."""
+    h = ctypes.c_void_p(None)
+    n = [int(v) for v in widths]
+    arr = (ctypes.c_int * len(n))(*n)
+    rc = _lib.lf_create_widths(ctypes.byref(h), len(n) - 1, arr, int(B), int(k))
     return rc, h
 
 
@@ -182,11 +192,16 @@ def lf_delta_step_static(w_up, delta_up, a_l, delta_l, N: int, cuda_stream: int 
 class Leapfrog:
     """Owns one ``lf_ctx``; raises :class:`LeapfrogError` on any non-zero status."""
 
-    def __init__(self, L: int, N: int, B: int = 1, k: int = 1, stream: int | None = None):
-        rc, self._h = lf_create(L, N, B, k)
+    def __init__(self, L: int, N: int, B: int = 1, k: int = 1, stream: int | None = None, widths=None):
+        """``widths`` = [n_0, ..., n_L] selects lf_create_widths (L and N are then taken from it)."""
+        if widths is not None:
+            rc, self._h = lf_create_widths(widths, B, k)
+            L, N = len(widths) - 1, max(int(v) for v in widths)
+        else:
+            rc, self._h = lf_create(L, N, B, k)
         if rc != LF_OK:
             self._h = None
-            raise LeapfrogError(rc, "lf_create")
+            raise LeapfrogError(rc, "lf_create_widths" if widths is not None else "lf_create")
         self.L, self.N, self.B, self.k = L, N, B, k
         if stream is not None:
             self.set_stream(stream)

@@ -17,18 +17,24 @@ int check_ptrs(const void* const* ps, int n)
     return LF_OK;
 }
 
-inline size_t slab(const lf_ctx* c) { return (size_t)c->B * (size_t)c->N; }
-inline size_t mat(const lf_ctx* c) { return (size_t)c->N * (size_t)c->N; }
+// Where layer l's block starts inside the caller's arrays (floats).
+inline size_t w_at(const lf_ctx* c, int l) { return c->off_w[l - 1]; }                      // w, gw: l = 1..L
+inline size_t v_at(const lf_ctx* c, int l) { return c->off_h[l - 1]; }                      // b, gb
+inline size_t h_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_h[l - 1]; }       // z, delta
+inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; }           // a: l = 0..L
 
+// Contexts with per-layer widths run one launch per layer with the fp32 kernels; the persistent
+// and the tensor-core kernels are written for one common width.
 int resolve_variant(const lf_ctx* c)
 {
+    if (!c->uniform) return LF_VARIANT_STREAMS;
     if (c->opt_variant != LF_VARIANT_AUTO) return c->opt_variant;
     return lf_auto_variant(c);
 }
 
 int resolve_gw_math(const lf_ctx* c)
 {
-    if (c->B == 1) return LF_GW_MATH_FP32;  // rank-1: one multiply per element, nothing to contract
+    if (c->B == 1 || !c->uniform) return LF_GW_MATH_FP32;  // B = 1 is rank-1: one multiply per element, nothing to contract
     if (c->opt_gw_math == LF_GW_MATH_FP32) return LF_GW_MATH_FP32;
     return lf_tf32_supported(c) ? LF_GW_MATH_TF32 : LF_GW_MATH_FP32;
 }
@@ -37,23 +43,24 @@ int resolve_gw_math(const lf_ctx* c)
 int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, float* gw, float* gb,
                       int gw_math, cudaStream_t s, int* launches)
 {
-    const float* d_l = delta + (size_t)(l - 1) * slab(c);
-    const float* a_prev = a + (size_t)(l - 1) * slab(c);
-    float* gw_l = gw + (size_t)(l - 1) * mat(c);
+    const float* d_l = delta + h_at(c, l);
+    const float* a_prev = a + a_at(c, l - 1);
+    float* gw_l = gw + w_at(c, l);
+    const int n_out = c->width[l], n_in = c->width[l - 1];
     lf_sgd sgd = {nullptr, 0.f};
-    if (c->sgd_on) { sgd.w_sub = c->sgd_w + (size_t)(l - 1) * mat(c); sgd.eta = c->sgd_eta; }
+    if (c->sgd_on) { sgd.w_sub = c->sgd_w + w_at(c, l); sgd.eta = c->sgd_eta; }
     if (c->B == 1) {
-        LF_CUDA_TRY(c, lfk_gw_rank1(d_l, a_prev, gw_l, c->N, sgd, s));
+        LF_CUDA_TRY(c, lfk_gw_rank1(d_l, a_prev, gw_l, n_out, n_in, sgd, s));
         *launches += 1;
     } else {
         if (gw_math == LF_GW_MATH_TF32) {
             int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, sgd, s, launches);
             if (rc != LF_OK) return rc;
         } else {
-            LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, c->N, c->B, sgd, s));
+            LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, n_out, n_in, c->B, sgd, s));
             *launches += 1;
         }
-        LF_CUDA_TRY(c, lfk_grad_b_colsum(d_l, gb + (size_t)(l - 1) * c->N, c->N, c->B, s));
+        LF_CUDA_TRY(c, lfk_grad_b_colsum(d_l, gb + v_at(c, l), n_out, c->B, s));
         *launches += 1;
     }
     return LF_OK;
@@ -61,7 +68,7 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
 
 int resolve_delta_math(const lf_ctx* c)
 {
-    if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
+    if (c->B == 1 || !c->uniform || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
     return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
 }
 
@@ -69,23 +76,25 @@ int resolve_delta_math(const lf_ctx* c)
 int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const float* y,
                        float* delta, float* gb, cudaStream_t s, int* launches)
 {
-    const int L = c->L, N = c->N, B = c->B;
-    float* d_l = delta + (size_t)(l - 1) * slab(c);
-    const float* a_l = a + (size_t)l * slab(c);
-    float* gb_l = gb + (size_t)(l - 1) * N;
+    const int L = c->L, B = c->B, n_l = c->width[l];
+    float* d_l = delta + h_at(c, l);
+    const float* a_l = a + a_at(c, l);
+    float* gb_l = gb + v_at(c, l);
     if (l == L) {
-        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, N, B, c->opt_cost, c->opt_act, s));
+        LF_CUDA_TRY(c, lfk_output_error(a_l, y, d_l, gb_l, n_l, B, c->opt_cost, c->opt_act, s));
     } else {
-        const float* w_up = w + (size_t)l * mat(c);  // w^{l+1}
-        const float* d_up = delta + (size_t)l * slab(c);
+        const float* w_up = w + w_at(c, l + 1);  // w^{l+1}: n_{l+1} x n_l
+        const float* d_up = delta + h_at(c, l + 1);
+        const int n_up = c->width[l + 1];
         if (B == 1)
-            LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, N, c->opt_act, s));
+            LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, n_up, n_l,
+                                            c->opt_act, s));
         else if (c->stats.delta_math == LF_DELTA_MATH_3XTF32) {
             int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, s, launches);
             if (rc != LF_OK) return rc;
             return LF_OK;
         } else
-            LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, N, B, c->opt_act, s));
+            LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, n_up, n_l, B, c->opt_act, s));
     }
     *launches += 1;
     return LF_OK;
@@ -193,6 +202,27 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
     if (!out) return LF_ENULL;
     *out = nullptr;
     if (L < 1 || N < 1 || B < 1 || k < 1 || (N & 3) != 0) return LF_EINVAL;
+    int* widths = new (std::nothrow) int[(size_t)L + 1];
+    if (!widths) return LF_ENOMEM;
+    for (int l = 0; l <= L; ++l) widths[l] = N;
+    const int rc = lf_create_widths(out, L, widths, B, k);
+    delete[] widths;
+    return rc;
+}
+
+int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
+{
+    if (!out) return LF_ENULL;
+    *out = nullptr;
+    if (!widths) return LF_ENULL;
+    if (L < 1 || B < 1 || k < 1) return LF_EINVAL;
+    int N = 0;            // the widest layer
+    bool uniform = true;
+    for (int l = 0; l <= L; ++l) {
+        if (widths[l] < 1 || (widths[l] & 3) != 0) return LF_EINVAL;
+        if (widths[l] > N) N = widths[l];
+        if (widths[l] != widths[0]) uniform = false;
+    }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return LF_ECUDA;
     cudaDeviceProp prop;
@@ -202,6 +232,24 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
     if (!c) return LF_ENOMEM;
     memset(c, 0, sizeof(*c));
     c->L = L; c->N = N; c->B = B; c->k = k; c->keff = k < L ? k : L;
+    c->uniform = uniform;
+    c->width = new (std::nothrow) int[(size_t)L + 1];
+    c->off_w = new (std::nothrow) size_t[(size_t)L + 1];
+    c->off_h = new (std::nothrow) size_t[(size_t)L + 1];
+    c->off_a = new (std::nothrow) size_t[(size_t)L + 2];
+    if (!c->width || !c->off_w || !c->off_h || !c->off_a) {
+        lf_destroy(c);
+        return LF_ENOMEM;
+    }
+    c->off_w[0] = 0; c->off_h[0] = 0; c->off_a[0] = 0;
+    for (int l = 0; l <= L; ++l) {
+        c->width[l] = widths[l];
+        c->off_a[l + 1] = c->off_a[l] + (size_t)widths[l];
+        if (l >= 1) {
+            c->off_w[l] = c->off_w[l - 1] + (size_t)widths[l] * (size_t)widths[l - 1];
+            c->off_h[l] = c->off_h[l - 1] + (size_t)widths[l];
+        }
+    }
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
     c->smem_optin = (int)prop.sharedMemPerBlockOptin;
@@ -214,8 +262,13 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
 
     bool ok = true;
     size_t ws = 0;
-    const int chunks = lfk_delta_row_chunks(N);
-    size_t partial_bytes = (size_t)chunks * N * sizeof(float);
+    // scratch of the B = 1 delta matvec: (row chunks of w^{l+1}) x n_l partial sums, the largest layer
+    size_t partial_floats = 4;
+    for (int l = 1; l < L; ++l) {
+        const size_t need = (size_t)lfk_delta_row_chunks(widths[l + 1]) * (size_t)widths[l];
+        if (need > partial_floats) partial_floats = need;
+    }
+    size_t partial_bytes = partial_floats * sizeof(float);
     size_t counter_bytes = (size_t)(N / 128 + 1) * sizeof(unsigned);
     c->sync_words_count = lf_sync_words_needed(c);
     ok = ok && cudaMalloc(&c->partial, partial_bytes) == cudaSuccess; ws += partial_bytes;
@@ -223,7 +276,7 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k)
     ok = ok && cudaMalloc(&c->sync_words, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
     ws += c->sync_words_count * sizeof(unsigned);
     ok = ok && cudaMalloc(&c->status_dev, sizeof(unsigned)) == cudaSuccess; ws += sizeof(unsigned);
-    const size_t dg_bytes = lf_delta_tc_scratch_bytes(c);
+    const size_t dg_bytes = uniform ? lf_delta_tc_scratch_bytes(c) : 0;
     if (dg_bytes) { ok = ok && cudaMalloc(&c->dg_partial, dg_bytes) == cudaSuccess; ws += dg_bytes; }
     ok = ok && cudaMallocHost(&c->status_host, sizeof(unsigned)) == cudaSuccess;
     if (ok) {
@@ -320,24 +373,25 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
     const void* ps[] = {w, b, x, z, a};
     int rc = check_ptrs(ps, 5);
     if (rc != LF_OK) return rc;
-    const int L = ctx->L, N = ctx->N, B = ctx->B;
+    const int L = ctx->L, B = ctx->B;
     cudaStream_t s = ctx->stream;
     int launches = 0;
-    if (a != x) LF_CUDA_TRY(ctx, lfk_copy_input(x, a, slab(ctx), s));  // Eq. x
+    if (a != x) LF_CUDA_TRY(ctx, lfk_copy_input(x, a, (size_t)B * ctx->width[0], s));  // Eq. x
     for (int l = 1; l <= L; ++l) {
-        const float* w_l = w + (size_t)(l - 1) * mat(ctx);
-        const float* b_l = b + (size_t)(l - 1) * N;
-        const float* a_prev = a + (size_t)(l - 1) * slab(ctx);
-        float* z_l = z + (size_t)(l - 1) * slab(ctx);
-        float* a_l = a + (size_t)l * slab(ctx);
+        const float* w_l = w + w_at(ctx, l);
+        const float* b_l = b + v_at(ctx, l);
+        const float* a_prev = a + a_at(ctx, l - 1);
+        float* z_l = z + h_at(ctx, l);
+        float* a_l = a + a_at(ctx, l);
+        const int n_out = ctx->width[l], n_in = ctx->width[l - 1];
         if (B == 1) {
-            LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, N, ctx->opt_act, s));
+            LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, ctx->opt_act, s));
             ++launches;
         } else if (resolve_delta_math(ctx) == LF_DELTA_MATH_3XTF32) {
             int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, s, &launches);
             if (rc2 != LF_OK) return rc2;
         } else {
-            LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, N, B, ctx->opt_act, s));
+            LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, B, ctx->opt_act, s));
             ++launches;
         }
     }
@@ -374,16 +428,17 @@ int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_
     const void* ps[] = {delta_l, a_prev, gw_l};
     int rc = check_ptrs(ps, 3);
     if (rc != LF_OK) return rc;
+    if (!ctx->uniform) return LF_EINVAL;   // the call names no layer, so it cannot know that layer's shape
     const int gw_math = resolve_gw_math(ctx);
     ctx->stats.gw_math = gw_math;
     const lf_sgd plain = {nullptr, 0.f};
     int launches = 0;
     if (ctx->B == 1)
-        LF_CUDA_TRY(ctx, lfk_gw_rank1(delta_l, a_prev, gw_l, ctx->N, plain, ctx->stream));
+        LF_CUDA_TRY(ctx, lfk_gw_rank1(delta_l, a_prev, gw_l, ctx->N, ctx->N, plain, ctx->stream));
     else if (gw_math == LF_GW_MATH_TF32)
         return lf_gw_gemm_tf32(ctx, delta_l, a_prev, gw_l, plain, ctx->stream, &launches);
     else
-        LF_CUDA_TRY(ctx, lfk_gw_gemm_fp32(delta_l, a_prev, gw_l, ctx->N, ctx->B, plain, ctx->stream));
+        LF_CUDA_TRY(ctx, lfk_gw_gemm_fp32(delta_l, a_prev, gw_l, ctx->N, ctx->N, ctx->B, plain, ctx->stream));
     return LF_OK;
 }
 
@@ -393,7 +448,7 @@ int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a,
     if (!ctx) return LF_ENULL;
     if (!w || !w_new) return LF_ENULL;
     if (!(eta == eta) || eta - eta != 0.f) return LF_EINVAL;          // NaN or infinite
-    const size_t bytes = (size_t)ctx->L * mat(ctx) * sizeof(float);
+    const size_t bytes = ctx->off_w[ctx->L] * sizeof(float);
     const char* lo = reinterpret_cast<const char*>(w);
     const char* out = reinterpret_cast<const char*>(w_new);
     if (out < lo + bytes && lo < out + bytes) return LF_EINVAL;        // w_new overlaps w
@@ -410,10 +465,12 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     const void* ps[] = {w, z, a, y, delta, gw, gb};
     for (int i = 0; i < 7; ++i)
         if (!ps[i]) return LF_ENULL;
-    const size_t L = (size_t)ctx->L, S = slab(ctx), M = mat(ctx), N = (size_t)ctx->N;
+    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
+    const int Li = ctx->L;
+    const size_t Bs = (size_t)ctx->B;
     // staging layout, every block a multiple of 4 floats: w | z | a | y | delta | gw | gb
-    const size_t n_w = L * M, n_z = L * S, n_a = (L + 1) * S, n_y = S, n_d = L * S, n_gw = L * M,
-                 n_gb = L * N;
+    const size_t n_w = ctx->off_w[Li], n_z = Bs * ctx->off_h[Li], n_a = Bs * ctx->off_a[Li + 1],
+                 n_y = Bs * (size_t)ctx->width[Li], n_d = n_z, n_gw = n_w, n_gb = ctx->off_h[Li];
     const size_t total = n_w + n_z + n_a + n_y + n_d + n_gw + n_gb;
     if (!ctx->stage) {
         cudaError_t e = cudaMalloc(&ctx->stage, total * sizeof(float));
@@ -448,7 +505,6 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     // and the worker that finishes gw^l sends it back at once, so the two PCIe directions
     // are busy at the same time.
     cudaStream_t s = ctx->stream, hs = ctx->h2d_stream;
-    const int Li = ctx->L;
     const int gw_math = resolve_gw_math(ctx);
     ctx->stats.variant = LF_VARIANT_STREAMS;
     ctx->stats.gw_math = gw_math;
@@ -464,7 +520,8 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, hs));
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, hs));
     for (int l = Li; l >= 1; --l) {
-        LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w + (size_t)(l - 1) * M, w + (size_t)(l - 1) * M, M * sizeof(float),
+        const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
+        LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w + w_at(ctx, l), w + w_at(ctx, l), M * sizeof(float),
                                          cudaMemcpyHostToDevice, hs));
         LF_CUDA_TRY(ctx, cudaEventRecord(ctx->w_ready_ev[l - 1], hs));
     }
@@ -474,14 +531,14 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
         if (l < Li) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0));   // w^{l+1}
         int rc = enqueue_chain_step(ctx, l, d_w, d_a, d_y, d_d, d_gb, s, &launches);
         if (rc != LF_OK) return rc;
-    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
         LF_CUDA_TRY(ctx, cudaEventRecord(ctx->ready_ev[l - 1], s));
         const int j = (Li - l) % ctx->keff;
         cudaStream_t wsj = ctx->wstreams[j];
         LF_CUDA_TRY(ctx, cudaStreamWaitEvent(wsj, ctx->ready_ev[l - 1], 0));
         rc = enqueue_gradients(ctx, l, d_a, d_d, d_gw, d_gb, gw_math, wsj, &launches);
         if (rc != LF_OK) return rc;
-        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw + (size_t)(l - 1) * M, d_gw + (size_t)(l - 1) * M, M * sizeof(float),
+        const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
+        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw + w_at(ctx, l), d_gw + w_at(ctx, l), M * sizeof(float),
                                          cudaMemcpyDeviceToHost, wsj));
     }
     for (int j = 0; j < ctx->keff; ++j) {
@@ -555,6 +612,10 @@ int lf_destroy(lf_ctx* ctx)
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     if (ctx->stage) cudaFree(ctx->stage);
     if (ctx->h2d_stream) { cudaStreamSynchronize(ctx->h2d_stream); cudaStreamDestroy(ctx->h2d_stream); }
+    delete[] ctx->width;
+    delete[] ctx->off_w;
+    delete[] ctx->off_h;
+    delete[] ctx->off_a;
     if (ctx->w_ready_ev) {
         for (int l = 0; l < ctx->L; ++l)
             if (ctx->w_ready_ev[l]) cudaEventDestroy(ctx->w_ready_ev[l]);

@@ -56,7 +56,14 @@ __device__ __forceinline__ float4 lf_sgd_apply4(float eta, float4 w, float4 g)
 #endif
 
 struct lf_ctx {
-    int L, N, B, k, keff;
+    int L, N, B, k, keff;    // N: the common width, or the widest layer of a context with per-layer widths
+    // per-layer widths n_0..n_L and where each layer's block starts inside the caller's arrays
+    // (in floats; the per-sample arrays multiply by B).  Uniform contexts fill them with N.
+    bool uniform;            // all widths equal: every kernel family applies
+    int* width;              // [L+1]  n_l
+    size_t* off_w;           // [L+1]  off_w[l-1]: start of w^l (n_l x n_{l-1}); off_w[L]: total
+    size_t* off_h;           // [L+1]  off_h[l-1]: n_1 + ... + n_{l-1} (b, gb; z, delta times B)
+    size_t* off_a;           // [L+2]  off_a[l]:   n_0 + ... + n_{l-1} (a times B)
     int device;
     int sm_count;
     int smem_optin;  // max dynamic shared memory per block
@@ -130,24 +137,25 @@ struct lf_ctx {
 // ---- launchers (each enqueues on `s` and returns the cudaError_t of the launch) -------------
 
 // B = 1 kernels
+// A layer's matrix is n_out x n_in, row-major: n_out neurons above, n_in below.
 cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* a_prev,
-                               float* z_l, float* a_l, int N, int act, cudaStream_t s);
+                               float* z_l, float* a_l, int n_out, int n_in, int act, cudaStream_t s);
 cudaError_t lfk_copy_input(const float* x, float* a0, size_t n, cudaStream_t s);
 cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, float* gbL, int N,
                              int B, int cost, int act, cudaStream_t s);
-int lfk_delta_row_chunks(int N);  // number of row chunks the delta matvec splits N rows into
+int lfk_delta_row_chunks(int n_up);  // number of row chunks the delta matvec splits n_up rows into
 cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,
-                             int N, int act, cudaStream_t s);
-cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
+                             int n_up, int n_l, int act, cudaStream_t s);
+cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                          lf_sgd sgd, cudaStream_t s);
 
 // B > 1 kernels (fp32 on the CUDA cores)
 cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
-                             float* z_l, float* a_l, int N, int B, int act, cudaStream_t s);
+                             float* z_l, float* a_l, int n_out, int n_in, int B, int act, cudaStream_t s);
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
-                           float* delta_l, int N, int B, int act, cudaStream_t s);
-cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
+                           float* delta_l, int n_up, int n_l, int B, int act, cudaStream_t s);
+cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                              int B, lf_sgd sgd, cudaStream_t s);
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s);
 

@@ -1,6 +1,7 @@
 // Single-sample (B = 1) kernels, one launch per layer: the forward matvec (Eq. z, Eq. a),
 // the output error (Eq. bp1), the transposed matvec of the delta recurrence (Eq. bp2) and the
-// rank-1 weight-gradient writer (Eq. bp4).  All are HBM-bound streams over one N x N matrix:
+// rank-1 weight-gradient writer (Eq. bp4).  All are HBM-bound streams over one layer's matrix
+// (n_out x n_in, row-major; square when all layers have one width):
 // 128-bit accesses, rows walked in the order they sit in memory.
 #include <mutex>
 
@@ -20,14 +21,14 @@ constexpr int FWD_WARPS = 8;
 __global__ void __launch_bounds__(FWD_WARPS * 32)
 k_forward_matvec(const float* __restrict__ w, const float* __restrict__ b,
                  const float* __restrict__ a_prev, float* __restrict__ z,
-                 float* __restrict__ a, int N, int act)
+                 float* __restrict__ a, int n_out, int n_in, int act)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = blockIdx.x * FWD_WARPS + warp;
-    if (j >= N) return;
-    const float4* wr = reinterpret_cast<const float4*>(w + (size_t)j * N);
+    if (j >= n_out) return;
+    const float4* wr = reinterpret_cast<const float4*>(w + (size_t)j * n_in);
     const float4* av = reinterpret_cast<const float4*>(a_prev);
-    const int n4 = N >> 2;
+    const int n4 = n_in >> 2;
     float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
     int c = lane;
     for (; c + 96 < n4; c += 128) {  // four independent 128-bit loads in flight per lane
@@ -78,23 +79,24 @@ __global__ void k_output_error(const float* __restrict__ aL, const float* __rest
 constexpr int DMV_WARPS = 8;
 constexpr int DMV_STRIP4 = 32;  // float4 columns per strip (128 floats)
 
-__host__ __device__ inline int dmv_rows_per_chunk(int N) { return N <= 2048 ? 32 : 64; }
+__host__ __device__ inline int dmv_rows_per_chunk(int n_up) { return n_up <= 2048 ? 32 : 64; }
 
 __global__ void __launch_bounds__(DMV_WARPS * 32)
 k_delta_matvec(const float* __restrict__ w_up, const float* __restrict__ delta_up,
                const float* __restrict__ a_l, float* __restrict__ delta_l,
                float* __restrict__ gb_l, float* __restrict__ partial,
-               unsigned* __restrict__ counters, int N, int rows_per_chunk, int chunks, int act)
+               unsigned* __restrict__ counters, int n_up, int n_l, int rows_per_chunk, int chunks, int act)
 {
+    // w_up is n_up x n_l: rows = neurons j of layer l+1, columns = neurons k of layer l
     __shared__ float4 red[DMV_WARPS][DMV_STRIP4];
     __shared__ bool is_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int strip = blockIdx.x, chunk = blockIdx.y;
-    const int n4 = N >> 2;
+    const int n4 = n_l >> 2;
     const int c4 = strip * DMV_STRIP4 + lane;
     const bool col_ok = c4 < n4;
     const int r0 = chunk * rows_per_chunk;
-    const int r1 = min(N, r0 + rows_per_chunk);
+    const int r1 = min(n_up, r0 + rows_per_chunk);
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (col_ok) {
@@ -164,10 +166,10 @@ constexpr int GW1_THREADS = 256;
 
 __global__ void __launch_bounds__(GW1_THREADS)
 k_gw_rank1(const float* __restrict__ delta_l, const float* __restrict__ a_prev,
-           float* __restrict__ gw_l, int N, const lf_sgd sgd)
+           float* __restrict__ gw_l, int n_out, int n_in, const lf_sgd sgd)
 {
-    const int n4 = N >> 2;
-    const size_t total4 = (size_t)N * n4;
+    const int n4 = n_in >> 2;
+    const size_t total4 = (size_t)n_out * n4;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     float4* out = reinterpret_cast<float4*>(gw_l);
     const float4* av = reinterpret_cast<const float4*>(a_prev);
@@ -186,10 +188,10 @@ k_gw_rank1(const float* __restrict__ delta_l, const float* __restrict__ a_prev,
 }  // namespace
 
 cudaError_t lfk_forward_matvec(const float* w_l, const float* b_l, const float* a_prev,
-                               float* z_l, float* a_l, int N, int act, cudaStream_t s)
+                               float* z_l, float* a_l, int n_out, int n_in, int act, cudaStream_t s)
 {
-    int grid = (N + FWD_WARPS - 1) / FWD_WARPS;
-    k_forward_matvec<<<grid, FWD_WARPS * 32, 0, s>>>(w_l, b_l, a_prev, z_l, a_l, N, act);
+    int grid = (n_out + FWD_WARPS - 1) / FWD_WARPS;
+    k_forward_matvec<<<grid, FWD_WARPS * 32, 0, s>>>(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, act);
     return cudaGetLastError();
 }
 
@@ -207,34 +209,34 @@ cudaError_t lfk_output_error(const float* aL, const float* y, float* deltaL, flo
     return cudaGetLastError();
 }
 
-int lfk_delta_row_chunks(int N)
+int lfk_delta_row_chunks(int n_up)
 {
-    int r = dmv_rows_per_chunk(N);
-    return (N + r - 1) / r;
+    int r = dmv_rows_per_chunk(n_up);
+    return (n_up + r - 1) / r;
 }
 
 cudaError_t lfk_delta_matvec(const float* w_up, const float* delta_up, const float* a_l,
                              float* delta_l, float* gb_l, float* partial, unsigned* counters,
-                             int N, int act, cudaStream_t s)
+                             int n_up, int n_l, int act, cudaStream_t s)
 {
-    int n4 = N >> 2;
+    int n4 = n_l >> 2;
     int strips = (n4 + DMV_STRIP4 - 1) / DMV_STRIP4;
-    int rows = dmv_rows_per_chunk(N);
-    int chunks = (N + rows - 1) / rows;
+    int rows = dmv_rows_per_chunk(n_up);
+    int chunks = (n_up + rows - 1) / rows;
     dim3 grid(strips, chunks);
     k_delta_matvec<<<grid, DMV_WARPS * 32, 0, s>>>(w_up, delta_up, a_l, delta_l, gb_l, partial,
-                                                  counters, N, rows, chunks, act);
+                                                  counters, n_up, n_l, rows, chunks, act);
     return cudaGetLastError();
 }
 
-cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int N,
+cudaError_t lfk_gw_rank1(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                          lf_sgd sgd, cudaStream_t s)
 {
-    size_t total4 = (size_t)N * (N >> 2);
+    size_t total4 = (size_t)n_out * (n_in >> 2);
     size_t want = (total4 + GW1_THREADS - 1) / GW1_THREADS;
     int grid = (int)(want < (size_t)148 * 16 ? want : (size_t)148 * 16);
     if (grid < 1) grid = 1;
-    k_gw_rank1<<<grid, GW1_THREADS, 0, s>>>(delta_l, a_prev, gw_l, N, sgd);
+    k_gw_rank1<<<grid, GW1_THREADS, 0, s>>>(delta_l, a_prev, gw_l, n_out, n_in, sgd);
     return cudaGetLastError();
 }
 
@@ -305,6 +307,6 @@ extern "C" int lf_delta_step_static(const float* w_up, const float* delta_up, co
         return LF_ECUDA;
     dim3 grid(strips, chunks);
     k_delta_matvec<<<grid, DMV_WARPS * 32, 0, s>>>(w_up, delta_up, a_l, delta_l, nullptr, partial,
-                                                  counters, N, rows, chunks, LF_ACT_SIGMOID);
+                                                  counters, N, N, rows, chunks, LF_ACT_SIGMOID);
     return cudaGetLastError() == cudaSuccess ? LF_OK : LF_ECUDA;
 }

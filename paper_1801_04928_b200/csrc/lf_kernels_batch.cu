@@ -147,29 +147,29 @@ inline dim3 gemm_grid(int M, int Nn) { return dim3((Nn + BN - 1) / BN, (M + BM -
 }  // namespace
 
 cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_prev,
-                             float* z_l, float* a_l, int N, int B, int act, cudaStream_t s)
+                             float* z_l, float* a_l, int n_out, int n_in, int B, int act, cudaStream_t s)
 {
-    // M = B (samples), Nn = N (neuron j), K = N (neuron k of the layer below)
-    k_gemm_simt<true, true, EPI_FORWARD><<<gemm_grid(B, N), 256, 0, s>>>(
-        a_prev, w_l, z_l, a_l, b_l, B, N, N, N, N, N, 0.f, act);
+    // M = B (samples), Nn = n_out (neuron j), K = n_in (neuron k of the layer below)
+    k_gemm_simt<true, true, EPI_FORWARD><<<gemm_grid(B, n_out), 256, 0, s>>>(
+        a_prev, w_l, z_l, a_l, b_l, B, n_out, n_in, n_in, n_in, n_out, 0.f, act);
     return cudaGetLastError();
 }
 
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
-                           float* delta_l, int N, int B, int act, cudaStream_t s)
+                           float* delta_l, int n_up, int n_l, int B, int act, cudaStream_t s)
 {
-    // M = B, Nn = N (neuron k of layer l), K = N (neuron j of layer l+1); w_up[j][k] is n-contiguous
-    k_gemm_simt<true, false, EPI_DELTA><<<gemm_grid(B, N), 256, 0, s>>>(
-        delta_up, w_up, delta_l, nullptr, a_l, B, N, N, N, N, N, 0.f, act);
+    // M = B, Nn = n_l (neuron k of layer l), K = n_up (neuron j of layer l+1); w_up[j][k] is n-contiguous
+    k_gemm_simt<true, false, EPI_DELTA><<<gemm_grid(B, n_l), 256, 0, s>>>(
+        delta_up, w_up, delta_l, nullptr, a_l, B, n_l, n_up, n_up, n_l, n_l, 0.f, act);
     return cudaGetLastError();
 }
 
-cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int N,
+cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                              int B, lf_sgd sgd, cudaStream_t s)
 {
-    // M = N (j), Nn = N (k), K = B; both operands are contiguous along their M / N index
-    k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(N, N), 256, 0, s>>>(
-        delta_l, a_prev, gw_l, nullptr, sgd.w_sub, N, N, B, N, N, N, sgd.eta, LF_ACT_SIGMOID);
+    // M = n_out (j), Nn = n_in (k), K = B; both operands are contiguous along their M / N index
+    k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(n_out, n_in), 256, 0, s>>>(
+        delta_l, a_prev, gw_l, nullptr, sgd.w_sub, n_out, n_in, B, n_out, n_in, n_in, sgd.eta, LF_ACT_SIGMOID);
     return cudaGetLastError();
 }
 

@@ -1,0 +1,148 @@
+"""GPU parity for networks whose layers differ in width (lf_create_widths): Eq. x, z, a and
+Eq. bp1-bp4 with w^l of shape n_l x n_{l-1}, flat per-layer-block layouts, against the oracle's
+functions for the same layout on the same seeded inputs, layer by layer, to the fp32 gate."""
+import numpy as np
+import pytest
+import torch
+
+import lf_inputs
+import paper_1801_04928_b200 as lf
+from lf_testlib import FP32_TOL, assert_layer_close
+from oracle import lf_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+# widths span several tiles of every kernel with ragged tails: the forward matvec's 128-column
+# loop, the delta matvec's 128-column strips and 32/64-row chunks, the 64 x 64 x 16 GEMM tiles
+SHAPES = [
+    [8, 4],                          # one layer, wider below than above
+    [4, 12, 8],
+    [260, 132, 516, 64, 200],        # up and down, nothing a multiple of 128
+    [1028, 2052, 36, 772],           # a row count beyond 2048 (64-row chunks) and a 36-wide bottleneck
+    [784, 512, 512, 256, 12],        # the shape of a small classifier
+]
+
+
+def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0):
+    n = [int(v) for v in widths]
+    L = len(n) - 1
+    cpu = lf_inputs.make_inputs_widths(n, B, y, lf_inputs.SEED_BASE + 700 + seed, "cpu")
+    t = {key: v.cuda() for key, v in cpu.items()}
+    sz = orc.sizes_widths(n, B)
+    dev = t["w"].device
+    z = torch.empty(sz["z"], dtype=torch.float32, device=dev)
+    a = torch.empty(sz["a"], dtype=torch.float32, device=dev)
+    delta = torch.full((sz["z"],), float("nan"), dtype=torch.float32, device=dev)
+    gw = torch.full((sz["w"],), float("nan"), dtype=torch.float32, device=dev)
+    gb = torch.full((sz["b"],), float("nan"), dtype=torch.float32, device=dev)
+    st = torch.cuda.Stream(device=dev)
+    st.wait_stream(torch.cuda.current_stream(dev))
+    with lf.Leapfrog(0, 0, B, k, stream=st.cuda_stream, widths=n) as ctx:
+        ctx.set_option(lf.LF_OPT_COST, cost)
+        ctx.set_option(lf.LF_OPT_ACTIVATION, act)
+        ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED)   # accepted; per-layer launches run
+        ctx.forward(t["w"], t["b"], t["x"], z, a)
+        if host:
+            ctx.sync()
+            hz, ha = z.cpu().pin_memory(), a.cpu().pin_memory()
+            hw, hy = cpu["w"].pin_memory(), cpu["y"].pin_memory()
+            hd = torch.full((sz["z"],), float("nan")).pin_memory()
+            hgw = torch.full((sz["w"],), float("nan")).pin_memory()
+            hgb = torch.full((sz["b"],), float("nan")).pin_memory()
+            ctx.backward_host(hw, hz, ha, hy, hd, hgw, hgb)
+            ctx.sync()
+            delta, gw, gb = hd, hgw, hgb
+        elif sgd_eta is not None:
+            ctx.backward_sgd(t["w"], z, a, t["y"], sgd_eta, delta, gw, gb)
+        else:
+            ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        ctx.sync()
+        stats = ctx.stats()
+    torch.cuda.current_stream(dev).wait_stream(st)
+    torch.cuda.synchronize(dev)
+    out = {key: v.cpu().numpy() for key, v in dict(z=z, a=a, delta=delta, gw=gw, gb=gb).items()}
+    return n, L, cpu, out, stats
+
+
+def _compare(n, B, cpu, out, cross_entropy=False, sgd_eta=None):
+    w = cpu["w"].numpy()
+    z, a = orc.forward_widths(n, w, cpu["b"].numpy(), cpu["x"].numpy())
+    delta, gw, gb = orc.backward_widths(n, w, z, a, cpu["y"].numpy(), cross_entropy=cross_entropy)
+    ref = dict(z=z, a=a, delta=delta, gb=gb, gw=gw)
+    if sgd_eta is not None:
+        ref["gw"] = w.astype(np.float64) - sgd_eta * gw
+    kinds = dict(z="z", a="a", delta="z", gb="b", gw="w")
+    for name, kind in kinds.items():
+        Bk = 1 if kind in ("b", "w") else B
+        got = orc.split(out[name], n, kind, Bk)
+        want = orc.split(ref[name], n, kind, Bk)
+        for l, (g, r) in enumerate(zip(got, want)):
+            assert_layer_close(name, l, g, r, tol=FP32_TOL, n_terms=max(n) + B)
+
+
+@pytest.mark.parametrize("B,k", [(1, 1), (1, 3), (5, 2), (130, 2)])
+@pytest.mark.parametrize("widths", SHAPES, ids=lambda s: "-".join(map(str, s)))
+def test_widths_parity(widths, B, k):
+    n, L, cpu, out, stats = _run(widths, B, k, y="onehot" if B > 1 else "uniform", seed=len(widths) + B)
+    assert stats["device_status"] == 0
+    assert stats["variant"] == lf.LF_VARIANT_STREAMS and stats["N"] == max(n)
+    assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] in (0, lf.LF_DELTA_MATH_FP32)
+    _compare(n, B, cpu, out)
+
+
+@pytest.mark.parametrize("B", [1, 6])
+def test_widths_cross_entropy_and_tanh(B):
+    widths = [260, 132, 516, 64]
+    n, L, cpu, out, stats = _run(widths, B, 2, cost=lf.LF_COST_CROSS_ENTROPY, seed=31)
+    assert stats["cost"] == lf.LF_COST_CROSS_ENTROPY
+    _compare(n, B, cpu, out, cross_entropy=True)
+    n, L, cpu, out, stats = _run(widths, B, 2, act=lf.LF_ACT_TANH, seed=32)
+    with orc.activation("tanh"):
+        _compare(n, B, cpu, out)
+
+
+@pytest.mark.parametrize("B", [1, 9])
+def test_widths_fused_update(B):
+    n, L, cpu, out, stats = _run([132, 516, 260, 8], B, 2, sgd_eta=0.37, seed=41)
+    _compare(n, B, cpu, out, sgd_eta=0.37)
+
+
+@pytest.mark.parametrize("B", [1, 7])
+def test_widths_host_entry_point(B):
+    n, L, cpu, out, stats = _run([200, 64, 328, 12], B, 3, host=True, seed=51)
+    _compare(n, B, cpu, out)
+
+
+def test_equal_widths_give_the_uniform_context():
+    # all widths equal: lf_create_widths is lf_create -- same kernels (the single-launch pass for one
+    # sample), same bits
+    L, N = 6, 516
+    cpu = lf_inputs.make_inputs(L, N, 1, "uniform", lf_inputs.SEED_BASE + 761, "cpu")
+    t = {key: v.cuda() for key, v in cpu.items()}
+    res = []
+    for widths in (None, [N] * (L + 1)):
+        z = torch.empty((L, 1, N), device="cuda"); a = torch.empty((L + 1, 1, N), device="cuda")
+        d = torch.empty((L, 1, N), device="cuda"); gw = torch.empty((L, N, N), device="cuda")
+        gb = torch.empty((L, N), device="cuda")
+        with lf.Leapfrog(L, N, 1, 2, widths=widths) as ctx:
+            ctx.forward(t["w"], t["b"], t["x"], z, a)
+            ctx.backward(t["w"], z, a, t["y"], d, gw, gb)
+            ctx.sync()
+            res.append((ctx.stats()["variant"], z, a, d, gw, gb))
+    assert res[0][0] == res[1][0] != lf.LF_VARIANT_STREAMS
+    for u, v in zip(res[0][1:], res[1][1:]):
+        assert torch.equal(u, v)
+
+
+def test_widths_argument_checks():
+    assert lf.lf_create_widths([8, 6, 8], 1, 1)[0] == lf.LF_EINVAL      # 6 is not a multiple of 4
+    assert lf.lf_create_widths([8, 0, 8], 1, 1)[0] == lf.LF_EINVAL
+    assert lf.lf_create_widths([8], 1, 1)[0] == lf.LF_EINVAL            # no weight layer
+    rc, h = lf.lf_create_widths([8, 4, 12], 1, 1)
+    assert rc == lf.LF_OK
+    try:
+        buf = torch.zeros(64, device="cuda")
+        assert lf.lf_grad_w(h, buf, buf, buf) == lf.LF_EINVAL           # names no layer
+        assert lf.lf_owner(h, 2) == 0 and lf.lf_owner(h, 1) == 0
+    finally:
+        lf.lf_destroy(h)
