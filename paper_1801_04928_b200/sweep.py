@@ -8,6 +8,12 @@ exists at that point: for B = 1 the stream schedule, the persistent leapfrog CTA
 the fused pass; for B > 1 the stream schedule with the fp32 and the TF32 weight gradient.
 One JSON object per line is written, and a table of the fastest variant per (N, B) is printed.
 Inputs are the seeded synthetic tensors of ``lf_inputs`` drawn on the GPU.
+
+    python -m paper_1801_04928_b200.sweep --widths 4096,8192,2048,4096,1024 [--B 1 256]
+
+times instead one network whose layers differ in width (``lf_create_widths``: one launch per
+layer, fp32), for every k of the grid, with the bytes the method must move per pass
+(4 n_l n_{l-1} written for every layer, read for every layer but the first) over the time.
 """
 from __future__ import annotations
 
@@ -40,6 +46,46 @@ def time_point(lf, torch, t, L, N, B, k, variant, gw_math, steps, warmup):
     return e0.elapsed_time(e1) / steps, st
 
 
+def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
+    n = [int(v) for v in widths]
+    L = len(n) - 1
+    mats = [n[l] * n[l - 1] for l in range(1, L + 1)]
+    with open(out, "w") as f:
+        for B in Bs:
+            t = lf_inputs.make_inputs_widths(n, B, "uniform" if B == 1 else "onehot",
+                                             lf_inputs.SEED_BASE + lf_inputs.SWEEP_CONFIG_INDEX, "cuda")
+            hidden = sum(n[1:])
+            t["z"] = torch.empty(B * hidden, device="cuda"); t["a"] = torch.empty(B * sum(n), device="cuda")
+            t["delta"] = torch.empty(B * hidden, device="cuda")
+            t["gw"] = torch.empty(sum(mats), device="cuda"); t["gb"] = torch.empty(hidden, device="cuda")
+            alg = 4.0 * (2 * sum(mats) - mats[0]) + 12.0 * B * hidden
+            flops = 2.0 * B * (2 * sum(mats) - mats[0])
+            steps, warmup = (3, 1) if flops > 2e11 else (30, 5)
+            for k in ks:
+                stream = torch.cuda.Stream()
+                stream.wait_stream(torch.cuda.current_stream())
+                with lf.Leapfrog(0, 0, B, k, stream=stream.cuda_stream, widths=n) as ctx:
+                    with torch.cuda.stream(stream):
+                        ctx.forward(t["w"], t["b"], t["x"], t["z"], t["a"])
+                        for _ in range(warmup):
+                            ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+                        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                        e0.record(stream)
+                        for _ in range(steps):
+                            ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+                        e1.record(stream)
+                        ctx.sync()
+                    st = ctx.stats()
+                ms = e0.elapsed_time(e1) / steps
+                row = dict(widths=n, B=B, k=k, variant="streams", ms=ms, layers_per_s=L / (ms * 1e-3),
+                           alg_GBs=alg / (ms * 1e-3) / 1e9, fp32_TFLOPs=flops / (ms * 1e-3) / 1e12 if B > 1 else None,
+                           launches=st["launches_backward"])
+                f.write(json.dumps(row) + "\n"); f.flush()
+                print(json.dumps(row), flush=True)
+            del t
+            torch.cuda.empty_cache()
+
+
 def main():
     import torch
     import lf_inputs
@@ -51,8 +97,12 @@ def main():
     ap.add_argument("--quick", action="store_true", help="k in {1, 4} only")
     ap.add_argument("--N", type=int, nargs="*", default=list(lf_inputs.SWEEP["N"]))
     ap.add_argument("--B", type=int, nargs="*", default=list(lf_inputs.SWEEP["B"]))
+    ap.add_argument("--widths", default=None, help="n_0,n_1,...,n_L: time one network of these layer widths")
     args = ap.parse_args()
     ks = (1, 4) if args.quick else lf_inputs.SWEEP["k"]
+    if args.widths:
+        sweep_widths(lf, lf_inputs, torch, args.widths.split(","), args.B, ks, args.out)
+        return
     L = args.L
     names = {1: "streams", 2: "persistent", 3: "fused"}
     rows = []
