@@ -34,7 +34,7 @@ int resolve_variant(const lf_ctx* c)
 
 int resolve_gw_math(const lf_ctx* c)
 {
-    if (c->B == 1 || !c->uniform) return LF_GW_MATH_FP32;  // B = 1 is rank-1: one multiply per element, nothing to contract
+    if (c->B == 1) return LF_GW_MATH_FP32;  // rank-1: one multiply per element, nothing to contract
     if (c->opt_gw_math == LF_GW_MATH_FP32) return LF_GW_MATH_FP32;
     return lf_tf32_supported(c) ? LF_GW_MATH_TF32 : LF_GW_MATH_FP32;
 }
@@ -54,7 +54,7 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
         *launches += 1;
     } else {
         if (gw_math == LF_GW_MATH_TF32) {
-            int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, sgd, s, launches);
+            int rc = lf_gw_gemm_tf32(c, d_l, a_prev, gw_l, n_out, n_in, sgd, s, launches);
             if (rc != LF_OK) return rc;
         } else {
             LF_CUDA_TRY(c, lfk_gw_gemm_fp32(d_l, a_prev, gw_l, n_out, n_in, c->B, sgd, s));
@@ -436,7 +436,7 @@ int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_
     if (ctx->B == 1)
         LF_CUDA_TRY(ctx, lfk_gw_rank1(delta_l, a_prev, gw_l, ctx->N, ctx->N, plain, ctx->stream));
     else if (gw_math == LF_GW_MATH_TF32)
-        return lf_gw_gemm_tf32(ctx, delta_l, a_prev, gw_l, plain, ctx->stream, &launches);
+        return lf_gw_gemm_tf32(ctx, delta_l, a_prev, gw_l, ctx->N, ctx->N, plain, ctx->stream, &launches);
     else
         LF_CUDA_TRY(ctx, lfk_gw_gemm_fp32(delta_l, a_prev, gw_l, ctx->N, ctx->N, ctx->B, plain, ctx->stream));
     return LF_OK;

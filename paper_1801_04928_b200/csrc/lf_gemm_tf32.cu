@@ -33,7 +33,7 @@ constexpr int TG_EPI_BYTES = 4 * 32 * TG_EPI_LD * 4;     // one 32 x 32 block pe
 constexpr size_t TG_SMEM_BYTES = (size_t)TG_STAGES * TG_STAGE_BYTES + TG_EPI_BYTES + 1024 /*alignment slack*/ + 256;
 
 struct TgParams {
-    int N, B;
+    int M, N, B;              // gw is M x N (M = neurons of the layer, N = neurons below = row length)
     int tiles_m, tiles_n;
     lf_sgd sgd;               // w_sub != nullptr: store w_sub - eta * (the contraction) instead
     float* gw;
@@ -165,10 +165,10 @@ __device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
 // Fused weight update: ask L2 for the part of the w tile this warp will subtract from (32 rows x
 // `cols` columns starting at row_first, col_first), one 128-byte line per request, while the
 // tile is still being multiplied.
-__device__ __forceinline__ void tg_prefetch_w(const float* w, int N, int row_first, int col_first, int cols, int lane)
+__device__ __forceinline__ void tg_prefetch_w(const float* w, int M, int N, int row_first, int col_first, int cols, int lane)
 {
     const int row = row_first + lane;
-    if (row >= N) return;
+    if (row >= M) return;
     const float* p = w + (size_t)row * N + col_first;
     for (int c = 0; c < cols && col_first + c < N; c += 32)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(p + c));
@@ -278,7 +278,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
         for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_i) {
             const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
             const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
-            if (P.sgd.w_sub) tg_prefetch_w(P.sgd.w_sub, P.N, tm * TG_BM + quad * 32, tn * TG_BN, TG_BN, lane);
+            if (P.sgd.w_sub) tg_prefetch_w(P.sgd.w_sub, P.M, P.N, tm * TG_BM + quad * 32, tn * TG_BN, TG_BN, lane);
             if (!tg_wait(tg_smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
             tg_fence_after();
             // A thread reads one accumulator row (32 columns at a time).  The block is turned
@@ -294,7 +294,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                 if (P.sgd.w_sub && col_w < P.N) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if (row0 + i * 4 + sub_r < P.N)
+                        if (row0 + i * 4 + sub_r < P.M)
                             wv[i] = __ldcs(reinterpret_cast<const float4*>(P.sgd.w_sub + (size_t)(row0 + i * 4 + sub_r) * P.N + col_w));
                 }
                 unsigned r[32];
@@ -310,7 +310,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                 for (int i = 0; i < 8; ++i) {
                     const int rr = i * 4 + sub_r;
                     float4 val = *reinterpret_cast<const float4*>(blk + rr * TG_EPI_LD + sub_c);
-                    if (row0 + rr < P.N && col < P.N) {
+                    if (row0 + rr < P.M && col < P.N) {
                         const size_t off = (size_t)(row0 + rr) * P.N + col;
                         if (P.sgd.w_sub) val = lf_sgd_apply4(P.sgd.eta, wv[i], val);
                         __stcs(reinterpret_cast<float4*>(P.gw + off), val);
@@ -592,7 +592,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             const float* w_row = P.sgd.w_sub ? P.sgd.w_sub + out_off : nullptr;
             const size_t row_step = (size_t)4 * P.N;
             if (w_row)
-                tg_prefetch_w(P.sgd.w_sub, P.N, row0 - sub_r, tn * TP_BN + half * (TP_BN / 2), TP_BN / 2, lane);
+                tg_prefetch_w(P.sgd.w_sub, P.M, P.N, row0 - sub_r, tn * TP_BN + half * (TP_BN / 2), TP_BN / 2, lane);
             if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
             tg_fence_after();
 #pragma unroll 1
@@ -602,7 +602,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 if (w_row && col0 + cchunk * 32 < P.N) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        if (row0 + i * 4 < P.N)
+                        if (row0 + i * 4 < P.M)
                             wv[i] = __ldcs(reinterpret_cast<const float4*>(w_row + i * row_step + cchunk * 32));
                 }
                 unsigned r[32];
@@ -617,7 +617,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         float4 val = *reinterpret_cast<const float4*>(blk + (i * 4 + sub_r) * TG_EPI_LD + sub_c);
-                        if (row0 + i * 4 < P.N) {
+                        if (row0 + i * 4 < P.M) {
                             if (w_row) val = lf_sgd_apply4(P.sgd.eta, wv[i], val);
                             __stcs(reinterpret_cast<float4*>(out_row + i * row_step + cchunk * 32), val);
                         }
@@ -727,16 +727,17 @@ bool lf_tf32_supported(const lf_ctx* c)
     return true;
 }
 
-int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, lf_sgd sgd, cudaStream_t s,
-                    int* launches)
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
+                    lf_sgd sgd, cudaStream_t s, int* launches)
 {
+    // delta_l is [B][n_out], a_prev is [B][n_in], gw_l is n_out x n_in
     alignas(64) CUtensorMap map_d, map_a;
-    if (!tg_encode_operand(&map_d, delta_l, c->N, c->B) || !tg_encode_operand(&map_a, a_prev, c->N, c->B)) {
+    if (!tg_encode_operand(&map_d, delta_l, n_out, c->B) || !tg_encode_operand(&map_a, a_prev, n_in, c->B)) {
         c->last_cuda_error = (int)cudaErrorInvalidValue;
         return LF_ECUDA;
     }
     TgParams P;
-    P.N = c->N; P.B = c->B;
+    P.M = n_out; P.N = n_in; P.B = c->B;
     P.gw = gw_l;
     P.sgd = sgd;
     P.status = c->status_dev;
@@ -744,8 +745,8 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
     const int max_pairs = c->tc_pair_kernels && c->B <= TP_MAX_KS * TG_BK ? tp_max_pairs(c) : 0;
     if (max_pairs > 0) {
         // two-SM kernel: the delta operand of a 256-row block stays in shared memory
-        P.tiles_m = (c->N + 2 * TP_BM - 1) / (2 * TP_BM);
-        P.tiles_n = (c->N + TP_BN - 1) / TP_BN;
+        P.tiles_m = (n_out + 2 * TP_BM - 1) / (2 * TP_BM);
+        P.tiles_n = (n_in + TP_BN - 1) / TP_BN;
         const int tiles = P.tiles_m * P.tiles_n;
         const int pairs = tiles < max_pairs ? tiles : max_pairs;
         cudaLaunchConfig_t cfg = {};
@@ -760,8 +761,8 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
         *launches += 1;
         return LF_OK;
     }
-    P.tiles_m = (c->N + TG_BM - 1) / TG_BM;
-    P.tiles_n = (c->N + TG_BN - 1) / TG_BN;
+    P.tiles_m = (n_out + TG_BM - 1) / TG_BM;
+    P.tiles_n = (n_in + TG_BN - 1) / TG_BN;
     const int tiles = P.tiles_m * P.tiles_n;
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     k_gw_gemm_tf32<<<grid, TG_THREADS, TG_SMEM_BYTES, s>>>(map_d, map_a, P);

@@ -169,8 +169,8 @@ void lf_persistent_release(lf_ctx* c);
 
 // ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------
 bool lf_tf32_supported(const lf_ctx* c);
-int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, lf_sgd sgd,
-                    cudaStream_t s, int* launches);
+int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
+                    lf_sgd sgd, cudaStream_t s, int* launches);
 void lf_tf32_release(lf_ctx* c);
 
 // ---- 3xTF32 tensor-core delta recurrence (B > 1) ----------------------------------------------

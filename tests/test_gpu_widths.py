@@ -7,7 +7,7 @@ import torch
 
 import lf_inputs
 import paper_1801_04928_b200 as lf
-from lf_testlib import FP32_TOL, assert_layer_close
+from lf_testlib import FP32_TOL, TF32_TOL, assert_layer_close, rel_frobenius
 from oracle import lf_oracle as orc
 
 pytestmark = pytest.mark.gpu
@@ -23,7 +23,8 @@ SHAPES = [
 ]
 
 
-def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0):
+def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0,
+         gw_math=lf.LF_GW_MATH_FP32, tiling=0):
     n = [int(v) for v in widths]
     L = len(n) - 1
     cpu = lf_inputs.make_inputs_widths(n, B, y, lf_inputs.SEED_BASE + 700 + seed, "cpu")
@@ -41,6 +42,8 @@ def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, see
         ctx.set_option(lf.LF_OPT_COST, cost)
         ctx.set_option(lf.LF_OPT_ACTIVATION, act)
         ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED)   # accepted; per-layer launches run
+        ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
+        ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
         ctx.forward(t["w"], t["b"], t["x"], z, a)
         if host:
             ctx.sync()
@@ -64,20 +67,38 @@ def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, see
     return n, L, cpu, out, stats
 
 
-def _compare(n, B, cpu, out, cross_entropy=False, sgd_eta=None):
+def _compare(n, B, cpu, out, cross_entropy=False, sgd_eta=None, tf32=False):
     w = cpu["w"].numpy()
     z, a = orc.forward_widths(n, w, cpu["b"].numpy(), cpu["x"].numpy())
     delta, gw, gb = orc.backward_widths(n, w, z, a, cpu["y"].numpy(), cross_entropy=cross_entropy)
-    ref = dict(z=z, a=a, delta=delta, gb=gb, gw=gw)
-    if sgd_eta is not None:
-        ref["gw"] = w.astype(np.float64) - sgd_eta * gw
-    kinds = dict(z="z", a="a", delta="z", gb="b", gw="w")
+    ref = dict(z=z, a=a, delta=delta, gb=gb)
+    kinds = dict(z="z", a="a", delta="z", gb="b")
     for name, kind in kinds.items():
-        Bk = 1 if kind in ("b", "w") else B
+        Bk = 1 if kind == "b" else B
         got = orc.split(out[name], n, kind, Bk)
         want = orc.split(ref[name], n, kind, Bk)
         for l, (g, r) in enumerate(zip(got, want)):
             assert_layer_close(name, l, g, r, tol=FP32_TOL, n_terms=max(n) + B)
+    # the weight gradients (or, under the fused update, w - eta * gw) layer by layer
+    got = orc.split(out["gw"], n, "w")
+    for l, (g, r, wl) in enumerate(zip(got, orc.split(gw, n, "w"), orc.split(w, n, "w"))):
+        assert np.all(np.isfinite(g))
+        if sgd_eta is None:
+            if tf32:
+                e = rel_frobenius(g, r)
+                assert e <= TF32_TOL, f"gw[{l}]: relative Frobenius error {e:.3e}"
+            else:
+                assert_layer_close("gw", l, g, r, tol=FP32_TOL, n_terms=max(n) + B)
+        else:
+            want = wl.astype(np.float64) - sgd_eta * r
+            round_off = 2.0 ** -23 * float(np.max(np.abs(want)))
+            if tf32:
+                err = float(np.linalg.norm(g - want))
+                bound = abs(sgd_eta) * TF32_TOL * float(np.linalg.norm(r)) + round_off * r.shape[1]
+            else:
+                err = float(np.max(np.abs(g - want)))
+                bound = abs(sgd_eta) * FP32_TOL * float(np.max(np.abs(r))) + round_off
+            assert err <= bound, (l, err, bound)
 
 
 @pytest.mark.parametrize("B,k", [(1, 1), (1, 3), (5, 2), (130, 2)])
@@ -88,6 +109,25 @@ def test_widths_parity(widths, B, k):
     assert stats["variant"] == lf.LF_VARIANT_STREAMS and stats["N"] == max(n)
     assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] in (0, lf.LF_DELTA_MATH_FP32)
     _compare(n, B, cpu, out)
+
+
+@pytest.mark.parametrize("tiling", [lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM])
+@pytest.mark.parametrize("B", [5, 130, 256, 300])
+@pytest.mark.parametrize("widths", SHAPES[2:], ids=lambda s: "-".join(map(str, s)))
+def test_widths_weight_gradient_on_the_tensor_cores(widths, B, tiling):
+    # Eq. bp4 of a rectangular layer as an n_l x n_{l-1} x B contraction with TF32 inputs; the two-SM
+    # kernel takes batches up to 256, beyond that the one-SM kernel runs whatever was asked for
+    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=60 + B, gw_math=lf.LF_GW_MATH_AUTO, tiling=tiling)
+    assert stats["device_status"] == 0 and stats["gw_math"] == lf.LF_GW_MATH_TF32
+    assert stats["gw_tiling"] == (tiling if B <= 256 else lf.LF_TC_TILING_ONE_SM)
+    _compare(n, B, cpu, out, tf32=True)
+
+
+@pytest.mark.parametrize("B", [9, 130])
+def test_widths_fused_update_on_the_tensor_cores(B):
+    n, L, cpu, out, stats = _run([132, 516, 260, 8], B, 2, sgd_eta=0.37, seed=43, gw_math=lf.LF_GW_MATH_TF32)
+    assert stats["gw_math"] == lf.LF_GW_MATH_TF32
+    _compare(n, B, cpu, out, sgd_eta=0.37, tf32=True)
 
 
 @pytest.mark.parametrize("B", [1, 6])
