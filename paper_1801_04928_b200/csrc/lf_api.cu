@@ -23,8 +23,8 @@ inline size_t v_at(const lf_ctx* c, int l) { return c->off_h[l - 1]; }          
 inline size_t h_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_h[l - 1]; }       // z, delta
 inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; }           // a: l = 0..L
 
-// Contexts with per-layer widths run one launch per layer with the fp32 kernels; the persistent
-// and the tensor-core kernels are written for one common width.
+// Contexts with per-layer widths run one launch per layer; the persistent kernels are written for
+// one common width (every cluster owns the same column strip of every layer).
 int resolve_variant(const lf_ctx* c)
 {
     if (!c->uniform) return LF_VARIANT_STREAMS;
@@ -68,7 +68,7 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
 
 int resolve_delta_math(const lf_ctx* c)
 {
-    if (c->B == 1 || !c->uniform || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
+    if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
     return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
 }
 
@@ -90,7 +90,7 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
             LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, n_up, n_l,
                                             c->opt_act, s));
         else if (c->stats.delta_math == LF_DELTA_MATH_3XTF32) {
-            int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, s, launches);
+            int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, n_up, n_l, s, launches);
             if (rc != LF_OK) return rc;
             return LF_OK;
         } else
@@ -276,7 +276,7 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
     ok = ok && cudaMalloc(&c->sync_words, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
     ws += c->sync_words_count * sizeof(unsigned);
     ok = ok && cudaMalloc(&c->status_dev, sizeof(unsigned)) == cudaSuccess; ws += sizeof(unsigned);
-    const size_t dg_bytes = uniform ? lf_delta_tc_scratch_bytes(c) : 0;
+    const size_t dg_bytes = lf_delta_tc_scratch_bytes(c);
     if (dg_bytes) { ok = ok && cudaMalloc(&c->dg_partial, dg_bytes) == cudaSuccess; ws += dg_bytes; }
     ok = ok && cudaMallocHost(&c->status_host, sizeof(unsigned)) == cudaSuccess;
     if (ok) {
@@ -388,7 +388,7 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
             LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, ctx->opt_act, s));
             ++launches;
         } else if (resolve_delta_math(ctx) == LF_DELTA_MATH_3XTF32) {
-            int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, s, &launches);
+            int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, n_out, n_in, s, &launches);
             if (rc2 != LF_OK) return rc2;
         } else {
             LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, B, ctx->opt_act, s));

@@ -41,7 +41,8 @@ constexpr int DG_EPI_BYTES = 4 * 32 * DG_EPI_LD * 4;
 constexpr size_t DG_SMEM_BYTES = (size_t)DG_STAGES * DG_STAGE_BYTES + DG_EPI_BYTES + 1024 + 256;
 
 struct DgParams {
-    int N, B;
+    int N, B;                 // the output is [B][N]; the contraction length reaches the kernels only
+                              // through the K-block counts below (loads beyond it are zero-filled)
     int tiles_m, tiles_n, splits;
     int k_per_split;          // j range of one split (multiple of DG_BK)
     int kb_per_tile;          // two-SM kernel: K blocks (of DG_BK) of one tile
@@ -843,15 +844,17 @@ struct DgPlan {
     int g_total;
 };
 
-DgPlan dg_plan(const lf_ctx* c)
+// One contraction out[B][Nc] = lhs[B][K] x W: Nc output columns, contraction length K.  Eq. bp2 of
+// layer l has Nc = n_l, K = n_{l+1}; Eq. z of layer l has Nc = n_l, K = n_{l-1}.
+DgPlan dg_plan(const lf_ctx* c, int Nc, int K)
 {
     DgPlan p = {};
     p.tiles_m = (c->B + DG_BM - 1) / DG_BM;
-    p.tiles_n = (c->N + DG_BN - 1) / DG_BN;
+    p.tiles_n = (Nc + DG_BN - 1) / DG_BN;
     int s = c->sm_count / (p.tiles_m * p.tiles_n);
     if (s < 1) s = 1;
     if (s > 8) s = 8;
-    const int kb = (c->N + DG_BK - 1) / DG_BK;            // K blocks in all
+    const int kb = (K + DG_BK - 1) / DG_BK;               // K blocks in all
     if (s > kb) s = kb;
     const int kb_per = (kb + s - 1) / s;
     p.splits = (kb + kb_per - 1) / kb_per;                 // no empty split
@@ -888,16 +891,16 @@ int dp_max_pairs(const lf_ctx* c)
 }
 
 // The two-SM kernels pay off once a pair's 256 samples are more than half filled.
-bool dp_use_pairs(const lf_ctx* c);
+bool dp_use_pairs(const lf_ctx* c, int Nc, int K);
 
 // Two-SM kernel: tiles x K-blocks cut into one contiguous run per pair; `splits` becomes the
 // largest number of run segments (= partial-sum slots) any tile has.
-DgPlan dp_plan(const lf_ctx* c, int max_pairs)
+DgPlan dp_plan(const lf_ctx* c, int Nc, int K, int max_pairs)
 {
     DgPlan p = {};
     p.tiles_m = (c->B + 2 * DG_BM - 1) / (2 * DG_BM);
-    p.tiles_n = (c->N + DP_BN - 1) / DP_BN;
-    p.kb_per_tile = (c->N + DG_BK - 1) / DG_BK;
+    p.tiles_n = (Nc + DP_BN - 1) / DP_BN;
+    p.kb_per_tile = (K + DG_BK - 1) / DG_BK;
     p.k_per_split = p.kb_per_tile * DG_BK;
     const int tiles = p.tiles_m * p.tiles_n;
     const long long g_total = (long long)tiles * p.kb_per_tile;
@@ -915,11 +918,28 @@ DgPlan dp_plan(const lf_ctx* c, int max_pairs)
     return p;
 }
 
-bool dp_use_pairs(const lf_ctx* c)
+// could the two-SM kernel be chosen for this shape (whatever LF_OPT_TC_TILING says)?
+bool dp_shape_fits_pairs(const lf_ctx* c, int Nc, int K)
 {
     // (narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there)
-    return c->tc_pair_kernels && c->B > DG_BM && c->N >= 512 && dp_max_pairs(c) > 0 &&
-           dp_plan(c, dp_max_pairs(c)).pairs > 0;
+    return c->B > DG_BM && Nc >= 512 && K >= 512 && dp_max_pairs(c) > 0;
+}
+
+bool dp_use_pairs(const lf_ctx* c, int Nc, int K)
+{
+    return c->tc_pair_kernels && dp_shape_fits_pairs(c, Nc, K) && dp_plan(c, Nc, K, dp_max_pairs(c)).pairs > 0;
+}
+
+// floats of partial-sum scratch one contraction of this shape may need: [splits][B][Nc] of
+// whichever tiling has more splits
+size_t dg_partial_floats(const lf_ctx* c, int Nc, int K)
+{
+    int splits = dg_plan(c, Nc, K).splits;
+    if (dp_shape_fits_pairs(c, Nc, K)) {
+        const int s2 = dp_plan(c, Nc, K, dp_max_pairs(c)).splits;
+        if (s2 > splits) splits = s2;
+    }
+    return (size_t)splits * c->B * Nc;
 }
 
 }  // namespace
@@ -927,13 +947,17 @@ bool dp_use_pairs(const lf_ctx* c)
 size_t lf_delta_tc_scratch_bytes(const lf_ctx* c)
 {
     if (c->B < 2) return 0;
-    // K-split partial sums [splits][B][N] of whichever tiling has more splits
-    int splits = dg_plan(c).splits;
-    if (c->B > DG_BM && c->N >= 512 && dp_max_pairs(c) > 0) {
-        const int s2 = dp_plan(c, dp_max_pairs(c)).splits;
-        if (s2 > splits) splits = s2;
+    // the largest need over every contraction of a pass: Eq. z of layers 1..L, Eq. bp2 of layers 1..L-1
+    size_t floats = 0;
+    for (int l = 1; l <= c->L; ++l) {
+        size_t f = dg_partial_floats(c, c->width[l], c->width[l - 1]);
+        if (f > floats) floats = f;
+        if (l < c->L) {
+            f = dg_partial_floats(c, c->width[l], c->width[l + 1]);
+            if (f > floats) floats = f;
+        }
     }
-    return (size_t)splits * c->B * c->N * sizeof(float);
+    return floats * sizeof(float);
 }
 
 bool lf_delta_tc_supported(const lf_ctx* c)
@@ -956,21 +980,24 @@ bool lf_delta_tc_supported(const lf_ctx* c)
     return true;
 }
 
-static DgSlots dg_slots(const lf_ctx* c, const DgPlan& pl)
+static DgSlots dg_slots(int Nc, const DgPlan& pl)
 {
     DgSlots S = {};
     S.splits = pl.splits; S.n_pairs = pl.pairs; S.tiles_n = pl.tiles_n; S.kb_per_tile = pl.kb_per_tile;
-    S.row4 = c->N / 4; S.g_total = pl.g_total;
+    S.row4 = Nc / 4; S.g_total = pl.g_total;
     return S;
 }
 
-// Encode the two operand maps and launch one contraction into c->dg_partial.
-static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kmajor, cudaStream_t s, DgPlan* plan_out)
+// Encode the two operand maps and launch one contraction out[B][Nc] = lhs[B][K] x W into
+// c->dg_partial.  W is [Nc][K] (w_kmajor: row n holds the K values it is contracted over, Eq. z) or
+// [K][Nc] (Eq. bp2: the transposed product read from the same row-major matrix).
+static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kmajor, int Nc, int K, cudaStream_t s,
+                     DgPlan* plan_out)
 {
     alignas(64) CUtensorMap map_d, map_w;
     {
-        cuuint64_t dims[2] = {(cuuint64_t)c->N, (cuuint64_t)c->B};
-        cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
+        cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)c->B};
+        cuuint64_t strides[1] = {(cuuint64_t)K * 4};
         cuuint32_t box[2] = {32, (cuuint32_t)DG_BM};
         cuuint32_t estr[2] = {1, 1};
         if (dg_get_encode()(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(lhs), dims, strides,
@@ -981,8 +1008,9 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
         }
     }
     {
-        cuuint64_t dims[2] = {(cuuint64_t)c->N, (cuuint64_t)c->N};
-        cuuint64_t strides[1] = {(cuuint64_t)c->N * 4};
+        const int inner = w_kmajor ? K : Nc, outer = w_kmajor ? Nc : K;
+        cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+        cuuint64_t strides[1] = {(cuuint64_t)inner * 4};
         cuuint32_t box_mn[2] = {32, (cuuint32_t)DG_BK};      // 32 columns n x 32 rows j
         cuuint32_t box_k[2] = {32, (cuuint32_t)DG_BN};       // 32 values of j x 128 rows n
         cuuint32_t estr[2] = {1, 1};
@@ -994,11 +1022,12 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
             return LF_ECUDA;
         }
     }
-    const bool pairs = dp_use_pairs(c);
+    const bool pairs = dp_use_pairs(c, Nc, K);
     const int max_pairs = pairs ? dp_max_pairs(c) : 0;
-    const DgPlan pl = pairs ? dp_plan(c, max_pairs) : dg_plan(c);
+    const DgPlan pl = pairs ? dp_plan(c, Nc, K, max_pairs) : dg_plan(c, Nc, K);
+    if ((size_t)pl.splits * c->B * Nc > dg_partial_floats(c, Nc, K)) return LF_ERESOURCE;   // cannot happen: same plans
     DgParams P;
-    P.N = c->N; P.B = c->B;
+    P.N = Nc; P.B = c->B;
     P.tiles_m = pl.tiles_m; P.tiles_n = pl.tiles_n; P.splits = pl.splits; P.k_per_split = pl.k_per_split;
     P.kb_per_tile = pl.kb_per_tile; P.g_total = pl.g_total;
     P.partial = c->dg_partial;
@@ -1033,27 +1062,29 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
 }
 
 int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
-                     cudaStream_t s, int* launches)
+                     int n_up, int n_l, cudaStream_t s, int* launches)
 {
+    // w_up = w^{l+1} is n_up x n_l; out[b][k] = sum_j delta_up[b][j] w_up[j][k]
     DgPlan pl;
-    int rc = dg_launch(c, delta_up, w_up, false, s, &pl);
+    int rc = dg_launch(c, delta_up, w_up, false, n_l, n_up, s, &pl);
     if (rc != LF_OK) return rc;
-    const size_t n4 = (size_t)c->B * c->N / 4;
-    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(c, pl), c->opt_act);
+    const size_t n4 = (size_t)c->B * n_l / 4;
+    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(n_l, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
 }
 
 int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const float* a_prev, float* z_l, float* a_l,
-                       cudaStream_t s, int* launches)
+                       int n_out, int n_in, cudaStream_t s, int* launches)
 {
+    // w_l is n_out x n_in; out[b][j] = sum_k a_prev[b][k] w_l[j][k]
     DgPlan pl;
-    int rc = dg_launch(c, a_prev, w_l, true, s, &pl);
+    int rc = dg_launch(c, a_prev, w_l, true, n_out, n_in, s, &pl);
     if (rc != LF_OK) return rc;
-    const size_t n4 = (size_t)c->B * c->N / 4;
-    k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, c->N / 4,
-                                                                  dg_slots(c, pl), c->opt_act);
+    const size_t n4 = (size_t)c->B * n_out / 4;
+    k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, n_out / 4,
+                                                                  dg_slots(n_out, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;

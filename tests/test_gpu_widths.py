@@ -24,7 +24,7 @@ SHAPES = [
 
 
 def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0,
-         gw_math=lf.LF_GW_MATH_FP32, tiling=0):
+         gw_math=lf.LF_GW_MATH_FP32, tiling=0, delta_math=lf.LF_DELTA_MATH_FP32):
     n = [int(v) for v in widths]
     L = len(n) - 1
     cpu = lf_inputs.make_inputs_widths(n, B, y, lf_inputs.SEED_BASE + 700 + seed, "cpu")
@@ -43,6 +43,7 @@ def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, see
         ctx.set_option(lf.LF_OPT_ACTIVATION, act)
         ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED)   # accepted; per-layer launches run
         ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
+        ctx.set_option(lf.LF_OPT_DELTA_MATH, delta_math)
         ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
         ctx.forward(t["w"], t["b"], t["x"], z, a)
         if host:
@@ -107,7 +108,24 @@ def test_widths_parity(widths, B, k):
     n, L, cpu, out, stats = _run(widths, B, k, y="onehot" if B > 1 else "uniform", seed=len(widths) + B)
     assert stats["device_status"] == 0
     assert stats["variant"] == lf.LF_VARIANT_STREAMS and stats["N"] == max(n)
-    assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] in (0, lf.LF_DELTA_MATH_FP32)
+    assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == lf.LF_DELTA_MATH_FP32
+    _compare(n, B, cpu, out)
+
+
+@pytest.mark.parametrize("tiling", [lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM])
+@pytest.mark.parametrize("B", [5, 130, 300])
+@pytest.mark.parametrize("widths", SHAPES[1:], ids=lambda s: "-".join(map(str, s)))
+def test_widths_chain_and_forward_on_the_tensor_cores(widths, B, tiling):
+    # Eq. z and Eq. bp2 of rectangular layers as 3xTF32 contractions (B x n_l x n_{l-1} and
+    # B x n_l x n_{l+1}): fp32-level accuracy, so the fp32 gate applies; the weight gradient stays fp32
+    # here so that every tensor is held to it.  The two-SM kernel serves layers of at least 512 x 512
+    # with more than 128 samples, the one-SM kernel the rest.
+    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=80 + B, delta_math=lf.LF_DELTA_MATH_AUTO,
+                                 tiling=tiling)
+    assert stats["device_status"] == 0 and stats["delta_math"] == lf.LF_DELTA_MATH_3XTF32
+    assert stats["delta_tiling"] in (lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM)
+    if tiling == lf.LF_TC_TILING_ONE_SM or B <= 128:
+        assert stats["delta_tiling"] == lf.LF_TC_TILING_ONE_SM
     _compare(n, B, cpu, out)
 
 
