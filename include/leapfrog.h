@@ -162,10 +162,10 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k);
  *     a        block l = [B][n_l], l = 0..L, a block 0 = x
  *     x [B][n_0],  y [B][n_L]
  * With all widths equal this is lf_create(L, widths[0], B, k) exactly, layouts included.
- * Otherwise the context runs one launch per layer with the k workers as streams
- * (LF_VARIANT_STREAMS) and fp32 arithmetic throughout -- the single-launch and the
- * tensor-core kernels are written for one common width; options asking for them are accepted
- * and lf_get_stats() reports what ran, with N = the widest layer.  lf_forward, lf_backward,
+ * Otherwise the context runs one launch per layer and step with the k workers as streams
+ * (LF_VARIANT_STREAMS) -- the single-launch kernels are written for one common width; an option
+ * asking for them is accepted and lf_get_stats() reports what ran, with N = the widest layer.
+ * The arithmetic options apply as for lf_create (B > 1: tensor-core contractions by default).  lf_forward, lf_backward,
  * lf_backward_sgd and lf_backward_host take such a context; lf_grad_w, which names no layer,
  * returns LF_EINVAL for it.
  * Errors: LF_ENULL (out, widths), LF_EINVAL (sizes), LF_ECUDA, LF_ENOMEM.

@@ -12,8 +12,9 @@ Inputs are the seeded synthetic tensors of ``lf_inputs`` drawn on the GPU.
     python -m paper_1801_04928_b200.sweep --widths 4096,8192,2048,4096,1024 [--B 1 256]
 
 times instead one network whose layers differ in width (``lf_create_widths``: one launch per
-layer, fp32), for every k of the grid, with the bytes the method must move per pass
-(4 n_l n_{l-1} written for every layer, read for every layer but the first) over the time.
+layer and step), for every k of the grid, with the bytes the method must move per pass
+(4 n_l n_{l-1} written for every layer, read for every layer but the first) and, for B > 1, the
+multiply-adds of its contractions (2 B n_l n_{l-1} for every Eq. bp4 and every Eq. bp2) over the time.
 """
 from __future__ import annotations
 
@@ -78,7 +79,7 @@ def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
                     st = ctx.stats()
                 ms = e0.elapsed_time(e1) / steps
                 row = dict(widths=n, B=B, k=k, variant="streams", ms=ms, layers_per_s=L / (ms * 1e-3),
-                           alg_GBs=alg / (ms * 1e-3) / 1e9, fp32_TFLOPs=flops / (ms * 1e-3) / 1e12 if B > 1 else None,
+                           alg_GBs=alg / (ms * 1e-3) / 1e9, alg_TFLOPs=flops / (ms * 1e-3) / 1e12 if B > 1 else None,
                            launches=st["launches_backward"])
                 f.write(json.dumps(row) + "\n"); f.flush()
                 print(json.dumps(row), flush=True)
