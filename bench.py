@@ -349,7 +349,8 @@ def run_ours(args):
                 ("w", "z", "a", "y", "delta", "gw", "gb")}
         for n in ("w", "z", "a", "y"):
             host[n].copy_(t[n])
-        h2d = sum(host[n].numel() * 4 for n in ("w", "z", "a", "y"))
+        # the weights of layer 1 are not read by the backward pass and are not uploaded
+        h2d = sum(host[n].numel() * 4 for n in ("w", "z", "a", "y")) - host["w"][0].numel() * 4
         d2h = sum(host[n].numel() * 4 for n in ("delta", "gw", "gb"))
         ctx = t["ctx"]
         with torch.cuda.stream(stream):

@@ -234,8 +234,8 @@ int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a,
                     float eta, float* delta, float* w_new, float* gb);
 
 /*
- * The same backward pass on HOST buffers (pageable or pinned; same layouts): w, z, a, y are
- * copied to device staging owned by the context (allocated on first use, counted in
+ * The same backward pass on HOST buffers (pageable or pinned; same layouts): w (layers 2..L, the
+ * ones the pass reads), z, a, y are copied to device staging owned by the context (allocated on first use, counted in
  * workspace_bytes), delta, gw, gb are copied back.  The copies are pipelined with the per-layer
  * schedule (LF_VARIANT_STREAMS): weights arrive top layer first on a copy stream, layer l is
  * processed as soon as w^{l+1} is there, and gw^l is sent back as soon as its worker has

@@ -519,7 +519,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, hs));
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, hs));
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, hs));
-    for (int l = Li; l >= 1; --l) {
+    for (int l = Li; l >= 2; --l) {   // w^1 is never read: Eq. bp2 needs w^{l+1} for l = L-1 .. 1
         const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
         LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w + w_at(ctx, l), w + w_at(ctx, l), M * sizeof(float),
                                          cudaMemcpyHostToDevice, hs));

@@ -204,3 +204,25 @@ def test_widths_argument_checks():
         assert lf.lf_owner(h, 2) == 0 and lf.lf_owner(h, 1) == 0
     finally:
         lf.lf_destroy(h)
+
+
+def test_widths_full_size_single_sample():
+    # the network the widths timing runs on (63 M weights): delta, gb, z, a of every layer element by
+    # element; the weight gradients -- rank one for a single sample -- on every 97th row of every layer
+    # against the oracle's delta_j * a_k (one float64 product per entry)
+    widths = [4096, 8192, 2048, 4096, 1024]
+    n, L, cpu, out, stats = _run(widths, 1, 4, seed=91)
+    assert stats["device_status"] == 0
+    w = cpu["w"].numpy()
+    z, a = orc.forward_widths(n, w, cpu["b"].numpy(), cpu["x"].numpy())
+    delta, _, gb = orc.backward_widths(n, w, z, a, cpu["y"].numpy(), want_gw=False)
+    ref = dict(z=z, a=a, delta=delta, gb=gb)
+    for name, kind in dict(z="z", a="a", delta="z", gb="b").items():
+        for l, (g, r) in enumerate(zip(orc.split(out[name], n, kind, 1), orc.split(ref[name], n, kind, 1))):
+            assert_layer_close(name, l, g, r, tol=FP32_TOL, n_terms=max(n))
+    d_l = orc.split(delta, n, "z", 1); a_l = orc.split(a, n, "a", 1)
+    for l, g in enumerate(orc.split(out["gw"], n, "w"), start=1):
+        rows = np.arange(0, n[l], 97)
+        want = d_l[l - 1][0][rows, None] * a_l[l - 1][0][None, :]
+        assert_layer_close("gw", l - 1, g[rows], want, tol=FP32_TOL, n_terms=max(n))
+        assert np.all(np.isfinite(g))
