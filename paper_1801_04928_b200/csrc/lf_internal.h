@@ -118,8 +118,10 @@ struct lf_ctx {
     float* stage;            // one allocation holding w, z, a, y, delta, gw, gb
     size_t stage_bytes;
     cudaStream_t h2d_stream; // host -> device copies of the host entry point
+    cudaStream_t d2h_stream; // device -> host copies of its results, all on this one stream
     cudaEvent_t* w_ready_ev; // L events: w^l has arrived in staging
-    cudaEvent_t small_ev, h2d_done_ev;
+    cudaEvent_t* gw_done_ev; // L events: gw^l (and gb^l) are written
+    cudaEvent_t small_ev, h2d_done_ev, d2h_done_ev;
 
     int last_cuda_error;
     lf_stats stats;
