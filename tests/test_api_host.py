@@ -44,6 +44,18 @@ def test_create_rejects_bad_sizes_before_touching_the_device():
         assert rc == lf.LF_EINVAL and not h.value
 
 
+def test_create_widths_rejects_bad_sizes_before_touching_the_device():
+    for widths, B, k in [([8, 6, 8], 1, 1), ([8, 0, 8], 1, 1), ([8], 1, 1), ([8, 8], 0, 1), ([8, 8], 1, 0),
+                         ([8, -4, 8], 1, 1)]:
+        rc, h = lf.lf_create_widths(widths, B, k)
+        assert rc == lf.LF_EINVAL and not h.value
+    # a NULL widths array or a NULL result pointer is LF_ENULL
+    lib = ctypes.CDLL(lf.LIB_PATH)
+    h = ctypes.c_void_p(None)
+    assert lib.lf_create_widths(ctypes.byref(h), 2, None, 1, 1) == lf.LF_ENULL and not h.value
+    assert lib.lf_create_widths(None, 2, (ctypes.c_int * 3)(8, 8, 8), 1, 1) == lf.LF_ENULL
+
+
 def test_null_context_is_an_error_not_a_crash():
     assert lf.lf_sync(None) == lf.LF_ENULL
     assert lf.lf_destroy(None) == lf.LF_ENULL
@@ -60,4 +72,6 @@ def test_no_device_means_an_error_not_a_fallback():
     if torch.cuda.is_available():
         return
     rc, h = lf.lf_create(4, 64, 1, 2)
+    assert rc == lf.LF_ECUDA and not h.value
+    rc, h = lf.lf_create_widths([64, 32, 16], 1, 2)
     assert rc == lf.LF_ECUDA and not h.value
