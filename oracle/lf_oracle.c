@@ -496,3 +496,30 @@ void lfo_backward_widths(int L, const int *n, int B, int cross_entropy, const lf
     free(oh);
     free(oa);
 }
+
+/* ---- the schedule on k GPUs instead of k threads -------------------------------------------
+ * Section 1 offers the leapfrog schedule for "k threads or k gpus".  On S GPUs nothing is shared:
+ * every GPU walks the whole delta chain (as every thread of Algorithm 1 does) and applies
+ * Eq. bp3 / bp4 only at its own layers, those with (L - l) mod S = r for GPU r -- the residue
+ * classes Algorithm 1 gives its threads (see the header on the three ways the paper names them).
+ * This is GPU r's pass: delta is written completely; gb and gw only at the layers of shard r, the
+ * other layers' slabs are left as they were; wrote[l-1] (may be NULL) is set to 1 at those layers
+ * and to 0 elsewhere.  Returns 0, or -1 for invalid sizes. */
+int lfo_backward_shard(int L, int N, int B, int S, int r, const lfo_w_t *w, const double *z,
+                       const double *a, const double *y, double *delta, double *gw, double *gb,
+                       int *wrote)
+{
+    if (L < 1 || N < 1 || B < 1 || S < 1 || r < 0 || r >= S) return -1;
+    size_t slab = (size_t)B * (size_t)N;
+    lfo_output_error(N, B, a + (size_t)L * slab, y, z + (size_t)(L - 1) * slab,
+                     delta + (size_t)(L - 1) * slab);                          /* bp1 */
+    for (int l = L; l >= 1; --l) {
+        if (l < L)
+            lfo_delta_step(N, B, w + (size_t)l * N * N, delta + (size_t)l * slab,
+                           z + (size_t)(l - 1) * slab, delta + (size_t)(l - 1) * slab);   /* bp2 */
+        int mine = (L - l) % S == r;
+        if (mine) lfo_emit_layer(l, N, B, delta + (size_t)(l - 1) * slab, a, gw, gb);    /* bp3, bp4 */
+        if (wrote) wrote[l - 1] = mine;
+    }
+    return 0;
+}

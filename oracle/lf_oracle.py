@@ -92,6 +92,8 @@ def _lib(tag: str) -> ctypes.CDLL:
             lib.lfo_forward_widths.argtypes = [i, _c_ip, i, wp, _c_dp, _c_dp, _c_dp, _c_dp]
             lib.lfo_backward_widths.restype = None
             lib.lfo_backward_widths.argtypes = [i, _c_ip, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp]
+            lib.lfo_backward_shard.restype = i
+            lib.lfo_backward_shard.argtypes = [i, i, i, i, i, wp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp, _c_dp, _c_ip]
             lib.lfo_sgd_step.restype = None
             lib.lfo_sgd_step.argtypes = [i, i, wp, _c_dp, ctypes.c_double, _c_dp]
             assert lib.lfo_weight_bytes() == (8 if tag == "f64" else 4)
@@ -335,3 +337,23 @@ def backward_widths(widths, w, z, a, y, want_gw: bool = True, cross_entropy: boo
     lib.lfo_backward_widths(n.size - 1, npnt, B, 1 if cross_entropy else 0, wp, _p(z), _p(a), _p(y),
                             _p(delta), _p(gw) if want_gw else None, _p(gb))
     return delta, gw, gb
+
+
+def backward_shard(w, z, a, y, S: int, r: int, want_gw: bool = True):
+    """GPU r's pass of the schedule on S GPUs: the whole delta chain, Eq. bp3/bp4 only at the layers
+    with (L - l) mod S = r.  Returns (delta, gw or None, gb, wrote[L]); layers of other shards hold NaN
+    in gw and gb."""
+    lib, w, wp = _w(w)
+    L, N, _ = w.shape
+    z, a = _d(z), _d(a)
+    B = z.shape[1]
+    y = _d(y).reshape(B, N)
+    delta = np.full((L, B, N), np.nan, dtype=np.float64)
+    gb = np.full((L, N), np.nan, dtype=np.float64)
+    gw = np.full((L, N, N), np.nan, dtype=np.float64) if want_gw else None
+    wrote = np.zeros((L,), dtype=np.int32)
+    rc = lib.lfo_backward_shard(L, N, B, int(S), int(r), wp, _p(z), _p(a), _p(y), _p(delta),
+                                _p(gw) if want_gw else None, _p(gb), wrote.ctypes.data_as(_c_ip))
+    if rc != 0:
+        raise ValueError("lfo_backward_shard: invalid sizes")
+    return delta, gw, gb, wrote

@@ -593,3 +593,53 @@ def test_widths_network_is_the_zero_padded_uniform_network():
         assert np.array_equal(gbl, GB[l - 1][:widths[l]])
     for l, al in enumerate(orc.split(a, widths, "a", B)):
         assert np.array_equal(al, A[l][:, :widths[l]])
+
+
+# ---- the schedule on S GPUs ---------------------------------------------------------------------
+def test_shards_cover_every_layer_once_and_add_up_to_the_sequential_pass():
+    # Catches: a layer no GPU owns or two GPUs own, a GPU that starts its chain from the wrong delta,
+    # gradients emitted before the chain reached the layer.
+    L, N, B = 7, 5, 2
+    w, b, x, y = _net(L, N, B, seed=404)
+    z, a = orc.forward(w, b, x)
+    delta, gw, gb = orc.backward_sequential(w, z, a, y)
+    for S in range(1, L + 3):
+        count = np.zeros(L, dtype=int)
+        for r in range(S):
+            d, g, v, wrote = orc.backward_shard(w, z, a, y, S, r)
+            assert np.array_equal(d, delta)                      # every GPU has the whole chain
+            for l in range(1, L + 1):
+                mine = (L - l) % S == r
+                assert bool(wrote[l - 1]) == mine
+                if mine:
+                    assert np.array_equal(g[l - 1], gw[l - 1]) and np.array_equal(v[l - 1], gb[l - 1])
+                else:
+                    assert np.all(np.isnan(g[l - 1])) and np.all(np.isnan(v[l - 1]))
+            count += wrote
+        assert np.all(count == 1)
+
+
+def test_shard_classes_are_the_thread_classes_of_algorithm_1():
+    # With k GPUs for k threads: all layers one thread of Algorithm 1 saves lie in one shard, and
+    # different threads' layers lie in different shards (the parent's top layers aside, which the
+    # pseudocode handles before it constructs the threads).
+    L, N, B = 11, 3, 1
+    w, b, x, y = _net(L, N, B, seed=405)
+    z, a = orc.forward(w, b, x)
+    for k in range(1, L + 1):
+        _, _, _, writer, writes, _ = orc.backward_leapfrog(w, z, a, y, k, threads=False)
+        cls = {}
+        for l in range(1, L + 1):
+            j = int(writer[l - 1])
+            if j >= 0:
+                cls.setdefault(j, set()).add((L - l) % k)
+        assert all(len(v) == 1 for v in cls.values())
+        residues = [next(iter(v)) for v in cls.values()]
+        assert len(set(residues)) == len(residues)
+
+
+def test_shard_rejects_bad_rank():
+    w, b, x, y = _net(2, 3, 1, seed=1)
+    z, a = orc.forward(w, b, x)
+    with pytest.raises(ValueError):
+        orc.backward_shard(w, z, a, y, 2, 2)
