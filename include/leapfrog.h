@@ -113,6 +113,9 @@ enum lf_option {
                                  lf_forward and lf_backward alike, so set it before both.
                                  LF_COST_CROSS_ENTROPY needs the sigmoid: lf_backward returns
                                  LF_EINVAL for any other pairing                              */
+    LF_OPT_SHARD_COUNT = 10,  /* S >= 1 (default 1): the paper's "k gpus" form (Section 1), see
+                                 below; setting it puts the rank back to 0                    */
+    LF_OPT_SHARD_RANK = 11,   /* r, 0 <= r < S: which of the S shards this context is         */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -136,6 +139,8 @@ typedef struct lf_stats {
     int delta_tiling;         /* the same for the last tensor-core Eq. bp2 / Eq. z launch     */
     int cost;                 /* cost function the last lf_backward used (enum lf_cost)       */
     int activation;           /* activation the last lf_forward / lf_backward used            */
+    int shard_rank;           /* LF_OPT_SHARD_RANK and LF_OPT_SHARD_COUNT of the last lf_backward */
+    int shard_count;
 } lf_stats;
 
 /*
@@ -178,6 +183,20 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k);
  */
 int lf_set_stream(lf_ctx* ctx, void* cuda_stream);
 
+/*
+ * Layer-sharded form (LF_OPT_SHARD_COUNT = S > 1, LF_OPT_SHARD_RANK = r).  The paper offers its
+ * schedule for "k threads or k gpus": with S GPUs every GPU holds w, z, a, runs the whole delta
+ * chain for itself, and does Eq. bp4 (and, for B > 1, Eq. bp3) only for the layers it owns,
+ *     layer l belongs to shard (L - l) mod S,
+ * so that nothing is exchanged during the pass and the gradients end up distributed by owner.
+ * A context with S > 1 writes delta completely (and gb for B = 1, where it is delta), and gw^l
+ * (gb^l for B > 1; w_new^l in lf_backward_sgd) only for its own layers; the other layers' blocks
+ * of those arrays are not touched.  Inside the shard the k leapfrog workers share the shard's
+ * layers in turn: worker ((L - l) / S) mod k.  The S contexts are independent: one per GPU, or
+ * several on one GPU writing into one gw array, give together exactly what one unsharded
+ * context writes.  LF_VARIANT_FUSED, whose tile pass stores every layer, runs as
+ * LF_VARIANT_PERSISTENT (or LF_VARIANT_STREAMS) in a sharded context.
+ */
 /* Set an option (enum lf_option).  LF_EINVAL for unknown keys or out-of-range values. */
 int lf_set_option(lf_ctx* ctx, int key, long long value);
 
@@ -252,7 +271,8 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
  */
 int lf_sync(lf_ctx* ctx);
 
-/* Worker that performs Eq. bp3/bp4 of layer l (1-based): (L - l) mod min(k, L); -1 if out of range. */
+/* Worker that performs Eq. bp3/bp4 of layer l (1-based): (L - l) mod min(k, L); -1 if out of range.
+ * In a sharded context: ((L - l) / S) mod min(k, L) for the shard's own layers, -1 for the others. */
 int lf_owner(const lf_ctx* ctx, int l);
 
 /* Copy the context's counters into *out. */

@@ -28,8 +28,10 @@ inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; 
 int resolve_variant(const lf_ctx* c)
 {
     if (!c->uniform) return LF_VARIANT_STREAMS;
-    if (c->opt_variant != LF_VARIANT_AUTO) return c->opt_variant;
-    return lf_auto_variant(c);
+    int v = c->opt_variant != LF_VARIANT_AUTO ? c->opt_variant : lf_auto_variant(c);
+    // the fused pass stores every layer's tile; a shard stores only its own layers
+    if (v == LF_VARIANT_FUSED && c->shard_count > 1) v = LF_VARIANT_PERSISTENT;
+    return v;
 }
 
 int resolve_gw_math(const lf_ctx* c)
@@ -112,8 +114,9 @@ int enqueue_backward_streams(lf_ctx* c, const float* w, const float* a, const fl
     for (int l = c->L; l >= 1; --l) {
         int rc = enqueue_chain_step(c, l, w, a, y, delta, gb, s, launches);
         if (rc != LF_OK) return rc;
+        if (!lf_layer_owned(c, l)) continue;      // another shard's layer
         LF_CUDA_TRY(c, cudaEventRecord(c->ready_ev[l - 1], s));
-        int j = (c->L - l) % c->keff;
+        int j = lf_layer_worker(c, l);
         LF_CUDA_TRY(c, cudaStreamWaitEvent(c->wstreams[j], c->ready_ev[l - 1], 0));
         rc = enqueue_gradients(c, l, a, delta, gw, gb, gw_math, c->wstreams[j], launches);
         if (rc != LF_OK) return rc;
@@ -144,7 +147,7 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
         return rc;
     }
     lf_graph_key key{w, z, a, y, delta, gw, gb, LF_VARIANT_STREAMS, gw_math * 16 + c->stats.delta_math,
-                     c->sgd_on, c->sgd_eta, c->opt_cost, c->opt_act};
+                     c->shard_rank * 65536 + c->shard_count, c->sgd_on, c->sgd_eta, c->opt_cost, c->opt_act};
     if (!(c->graph_valid && c->graph_key == key)) {
         drop_graph(c);
         LF_CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -259,6 +262,7 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
     c->wait_budget_us = 2000000;
     c->use_graph = 1;
     c->tc_pair_kernels = 1;
+    c->shard_rank = 0; c->shard_count = 1;
 
     bool ok = true;
     size_t ws = 0;
@@ -353,6 +357,15 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value < LF_ACT_SIGMOID || value > LF_ACT_RELU) return LF_EINVAL;
             ctx->opt_act = (int)value;
             return LF_OK;
+        case LF_OPT_SHARD_COUNT:
+            if (value < 1 || value > 65535) return LF_EINVAL;
+            ctx->shard_count = (int)value;
+            ctx->shard_rank = 0;
+            return LF_OK;
+        case LF_OPT_SHARD_RANK:
+            if (value < 0 || value >= ctx->shard_count) return LF_EINVAL;
+            ctx->shard_rank = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -417,6 +430,7 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     ctx->stats.delta_math = resolve_delta_math(ctx);
     ctx->stats.cost = ctx->opt_cost;
     ctx->stats.activation = ctx->opt_act;
+    ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
@@ -517,6 +531,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     ctx->stats.delta_math = resolve_delta_math(ctx);
     ctx->stats.cost = ctx->opt_cost;
     ctx->stats.activation = ctx->opt_act;
+    ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
     int launches = 0;
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
     LF_CUDA_TRY(ctx, cudaStreamWaitEvent(hs, ctx->fork_ev, 0));
@@ -538,8 +553,9 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
         if (l < Li) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0));   // w^{l+1}
         int rc = enqueue_chain_step(ctx, l, d_w, d_a, d_y, d_d, d_gb, s, &launches);
         if (rc != LF_OK) return rc;
+        if (!lf_layer_owned(ctx, l)) continue;    // another shard's layer: nothing to compute or send back
         LF_CUDA_TRY(ctx, cudaEventRecord(ctx->ready_ev[l - 1], s));
-        const int j = (Li - l) % ctx->keff;
+        const int j = lf_layer_worker(ctx, l);
         cudaStream_t wsj = ctx->wstreams[j];
         LF_CUDA_TRY(ctx, cudaStreamWaitEvent(wsj, ctx->ready_ev[l - 1], 0));
         rc = enqueue_gradients(ctx, l, d_a, d_d, d_gw, d_gb, gw_math, wsj, &launches);
@@ -550,9 +566,19 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
         LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw + w_at(ctx, l), d_gw + w_at(ctx, l), M * sizeof(float),
                                          cudaMemcpyDeviceToHost, ds));
     }
-    // by now the download stream has waited for every layer's gw and gb and (through them) delta
+    // the download stream has waited for the gw and gb of every layer done here; the end of the
+    // chain (delta^1, the last thing written on s) it waits for explicitly
+    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, s));
+    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ds, ctx->small_ev, 0));
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(delta, d_d, n_d * sizeof(float), cudaMemcpyDeviceToHost, ds));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, ds));
+    if (ctx->B == 1 || ctx->shard_count == 1) {
+        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, ds));
+    } else {
+        for (int l = 1; l <= Li; ++l)     // B > 1: gb^l exists only for this shard's layers
+            if (lf_layer_owned(ctx, l))
+                LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb + v_at(ctx, l), d_gb + v_at(ctx, l),
+                                                 (size_t)ctx->width[l] * sizeof(float), cudaMemcpyDeviceToHost, ds));
+    }
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->d2h_done_ev, ds));
     for (int j = 0; j < ctx->keff; ++j) {
         LF_CUDA_TRY(ctx, cudaEventRecord(ctx->done_ev[j], ctx->wstreams[j]));
@@ -583,7 +609,7 @@ int lf_sync(lf_ctx* ctx)
 int lf_owner(const lf_ctx* ctx, int l)
 {
     if (!ctx || l < 1 || l > ctx->L) return -1;
-    return (ctx->L - l) % ctx->keff;
+    return lf_layer_owned(ctx, l) ? lf_layer_worker(ctx, l) : -1;
 }
 
 int lf_get_stats(lf_ctx* ctx, lf_stats* out)

@@ -17,6 +17,7 @@ struct lf_graph_key {
     const void *w, *z, *a, *y;
     void *delta, *gw, *gb;
     int variant, gw_math;
+    int shard;      // shard rank * 65536 + shard count
     int sgd;        // 1: the graph writes w - eta * gw instead of gw
     float eta;
     int cost;       // enum lf_cost baked into the Eq. bp1 kernel
@@ -24,7 +25,7 @@ struct lf_graph_key {
     bool operator==(const lf_graph_key& o) const {
         return w == o.w && z == o.z && a == o.a && y == o.y && delta == o.delta &&
                gw == o.gw && gb == o.gb && variant == o.variant && gw_math == o.gw_math &&
-               sgd == o.sgd && (!sgd || eta == o.eta) && cost == o.cost && act == o.act;
+               sgd == o.sgd && (!sgd || eta == o.eta) && cost == o.cost && act == o.act && shard == o.shard;
     }
 };
 
@@ -81,6 +82,7 @@ struct lf_ctx {
     int sgd_on;              // the current backward call is lf_backward_sgd
     float sgd_eta;
     const float* sgd_w;      // its weights (what the update is subtracted from)
+    int shard_rank, shard_count;  // layer l is this context's iff (L - l) % shard_count == shard_rank
     int withhold;            // test hook: one chain CTA withholds its published delta values
 
     // workspace (device)
@@ -126,6 +128,10 @@ struct lf_ctx {
     int last_cuda_error;
     lf_stats stats;
 };
+
+// Layer-sharded form: does this context do Eq. bp3/bp4 of layer l, and on which of its workers?
+inline bool lf_layer_owned(const lf_ctx* c, int l) { return (c->L - l) % c->shard_count == c->shard_rank; }
+inline int lf_layer_worker(const lf_ctx* c, int l) { return ((c->L - l) / c->shard_count) % c->keff; }
 
 #define LF_CUDA_TRY(ctx, expr)                                  \
     do {                                                        \

@@ -48,6 +48,7 @@ struct PkParams {
     int C;         // CTAs per cluster
     int Qc;        // chain clusters
     int Qw;        // worker clusters (0 in the fused variant)
+    int shard_rank, shard_count;   // the workers store layer l only if (L - l) % shard_count == shard_rank
     int fused;     // 1: chain CTAs store gw tiles
     int Wc;        // columns per column block (32, 64, 128 or 256)
     int nCB;       // column blocks per strip
@@ -378,7 +379,8 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         float* a_sm = stages;                         // N floats (N <= 16384: two stages)
         float* dr = stages + 16384;                   // up to N floats
         for (int l = L; l >= 1; --l) {
-            if ((((L - l) % P.keff) % G) != g) continue;   // not a layer of my group
+            if ((L - l) % P.shard_count != P.shard_rank) continue;        // another shard's layer
+            if (((((L - l) / P.shard_count) % P.keff) % G) != g) continue;   // not a layer of my group
             if (row0 < row1) worker_store_rows<UPDATE>(P, l, row0, row1, dr, a_sm, sh);
         }
         cluster_sync_all();   // the cluster's CTAs leave together
@@ -794,7 +796,14 @@ PkPlan plan_for_cluster(const lf_ctx* c, int variant, int C)
     int Qc_budget = p.Qmax;
     if (variant == LF_VARIANT_PERSISTENT) {
         if (p.Qmax < 2) return p;
+        // Half of the clusters for the chain, half for the workers; a shard stores only every S-th
+        // layer, so its workers get by with 1 / (S + 1) of the clusters.
         Qc_budget = p.Qmax / 2;
+        if (c->shard_count > 1) {
+            int workers = p.Qmax / (c->shard_count + 1);
+            if (workers < 1) workers = 1;
+            Qc_budget = p.Qmax - workers;
+        }
     }
     if (Qc_budget < 1) return p;
     const int N = c->N;
@@ -900,6 +909,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
     P.cost = c->opt_cost; P.act = c->opt_act;
+    P.shard_rank = c->shard_rank; P.shard_count = c->shard_count > 1 ? c->shard_count : 1;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
     P.w_sub = c->sgd_on ? c->sgd_w : nullptr; P.eta = c->sgd_eta;
