@@ -51,6 +51,13 @@ def parse_args():
                         "instead of lf_backward; not the headline metric")
     p.add_argument("--layers", type=int, default=0,
                    help="override the config's L (a smaller case of the same kernels, for profiler captures)")
+    p.add_argument("--shards", type=int, default=1, metavar="S",
+                   help="time ONE shard (rank 0) of the layer-sharded form on S GPUs: the whole delta chain, "
+                        "weight gradients of every S-th layer only; nothing is exchanged, so this is the time "
+                        "each of the S GPUs would take")
+    p.add_argument("--shard-by-rank", action="store_true",
+                   help="with --gpus N > 1: instead of N replicas, run ONE pass layer-sharded over the N ranks "
+                        "(rank r = shard r of N, no exchange); value = L / slowest rank's time, strong scaling")
     p.add_argument("--e2e-steps", type=int, default=5)
     p.add_argument("--cpu-seconds", type=float, default=10.0)
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -263,8 +270,13 @@ def run_ours(args):
     cfg, cpu = lf_inputs.make_config(args.config, **({"L": args.layers} if args.layers else {}))
     if args.k:
         cfg["k"] = args.k
+    elif args.shards > 1 or (args.shard_by_rank and world > 1):
+        # the workload's k leapfrog workers are spread over the S GPUs: k / S of them work here
+        cfg["k"] = max(1, cfg["k"] // (world if args.shard_by_rank and world > 1 else args.shards))
     L, N, B, k = cfg["L"], cfg["N"], cfg["B"], cfg["k"]
     variant = VARIANT_NAMES[args.variant]
+    by_rank = args.shard_by_rank and world > 1
+    shard_count, shard_rank = (world, rank) if by_rank else (args.shards, 0)
 
     # Rotating buffer sets: consecutive steps touch different w / gw, so a step never finds
     # its inputs in the 126 MB L2 left there by the step before.
@@ -285,6 +297,8 @@ def run_ours(args):
         ctx = lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream)
         ctx.set_option(lf.LF_OPT_VARIANT, variant)
         ctx.set_option(lf.LF_OPT_TC_TILING, TC_TILING_NAMES[args.tc_tiling])
+        ctx.set_option(lf.LF_OPT_SHARD_COUNT, shard_count)
+        ctx.set_option(lf.LF_OPT_SHARD_RANK, shard_rank)
         t["ctx"] = ctx
         sets.append(t)
     torch.cuda.synchronize(dev)
@@ -338,7 +352,8 @@ def run_ours(args):
         t["ctx"].sync()
     stats = sets[0]["ctx"].stats()
 
-    value, total_ms_max, _ = aggregate_rate(total_ms, L * args.steps, dist, dev)
+    # replicas: every rank does L layers per step; sharded by rank: the N ranks share one pass
+    value, total_ms_max, _ = aggregate_rate(total_ms, L * args.steps / (world if by_rank else 1), dist, dev)
     ms_per_step = total_ms_max / args.steps
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
@@ -352,6 +367,8 @@ def run_ours(args):
         # the weights of layer 1 are not read by the backward pass and are not uploaded
         h2d = sum(host[n].numel() * 4 for n in ("w", "z", "a", "y")) - host["w"][0].numel() * 4
         d2h = sum(host[n].numel() * 4 for n in ("delta", "gw", "gb"))
+        if shard_count > 1:   # only the shard's own layers of gw come back
+            d2h -= host["gw"][0].numel() * 4 * (L - len(range(L, 0, -shard_count)))
         ctx = t["ctx"]
         with torch.cuda.stream(stream):
             for _ in range(2):
@@ -368,7 +385,7 @@ def run_ours(args):
         e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
         if dist is not None:
             dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * L * args.e2e_steps / (float(e2e_ms.item()) * 1e-3), "unit": UNIT,
+        e2e = {"value": (1 if by_rank else world) * L * args.e2e_steps / (float(e2e_ms.item()) * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": float(e2e_ms.item()) / args.e2e_steps}
 
@@ -381,6 +398,9 @@ def run_ours(args):
     alg = algorithmic_bytes(L, N, B)
     if args.sgd is not None:
         alg += 4 * N * N          # the update also reads w^1, which the plain pass never touches
+    if shard_count > 1:           # shard r stores only the layers L - r, L - r - S, ... (rank 0's figures)
+        owned = len(range(L, 0, -shard_count))
+        alg -= 4 * N * N * (L - owned)
     launches_per_step = stats["launches_backward"]
     if launches_per_step == 1:
         kernel_name = "persistent backward kernel (one launch per step)"
@@ -388,7 +408,10 @@ def run_ours(args):
         kernel_name = f"whole step ({launches_per_step} launches replayed from one CUDA graph)"
     achieved = alg / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC.get((args.config, stats["variant"])),
+                "frac": achieved / peak,
+                # counters exist for the plain pass of the named workload only
+                "traffic": NCU_TRAFFIC.get((args.config, stats["variant"]))
+                if shard_count == 1 and args.sgd is None and not args.layers and not args.k else None,
                 "peak_kind": f"of {peak_kind}",
                 "kernel": kernel_name, "algorithmic_bytes_per_launch": alg,
                 "avg_launch_ms": ms_per_step,
@@ -428,11 +451,14 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "strong" if by_rank else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(args.config, cfg), "L": L, "N": N, "B": B, "k": k,
                    "variant": stats["variant"], "gw_math": stats["gw_math"],
                    **({"fused_sgd_eta": args.sgd} if args.sgd is not None else {}),
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   **({"shard": f"0 of {args.shards} (layer-sharded form, one shard's pass)"}
+                      if args.shards > 1 and not by_rank else {}),
+                   "parallelism": ("one pass, layers sharded over the ranks, no exchange" if by_rank else
+                                   "replicas only") if world > 1 else "single GPU",
                    "l2_policy": f"{n_sets} rotating buffer sets of {set_bytes >> 20} MiB (w + gw); "
                                 "inputs larger than the 126 MB L2"},
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
