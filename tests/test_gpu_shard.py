@@ -157,3 +157,31 @@ def test_shard_option_checks():
             ctx.set_option(lf.LF_OPT_SHARD_RANK, 3)
         ctx.set_option(lf.LF_OPT_SHARD_COUNT, 2)       # the rank goes back to 0
         assert ctx.owner(4) == 0 and ctx.owner(3) == -1
+
+
+def test_one_context_switching_shards_recaptures_its_graph():
+    # the stream schedule is replayed from a captured graph on a non-default stream; the shard is part
+    # of what the graph was captured for, so changing it must not replay the old shard's launches
+    L, N, k, S = 6, 260, 2, 2
+    cpu, t = _inputs(L, N, 1, seed=88)
+    full, _, _ = _shard_pass(L, N, 1, k, 1, 0, t, lf.LF_VARIANT_STREAMS)
+    dev = t["w"].device
+    z = torch.empty((L, 1, N), device=dev); a = torch.empty((L + 1, 1, N), device=dev)
+    delta = torch.full((L, 1, N), float("nan"), device=dev)
+    gw = torch.full((L, N, N), float("nan"), device=dev)
+    gb = torch.full((L, N), float("nan"), device=dev)
+    st = torch.cuda.Stream(device=dev)
+    st.wait_stream(torch.cuda.current_stream(dev))
+    with lf.Leapfrog(L, N, 1, k, stream=st.cuda_stream) as ctx:
+        ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_STREAMS)
+        ctx.forward(t["w"], t["b"], t["x"], z, a)
+        ctx.set_option(lf.LF_OPT_SHARD_COUNT, S)
+        for _ in range(2):                               # second call replays the graph
+            ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        ctx.sync()
+        assert torch.isnan(gw[L - 2]).all() and torch.equal(gw[L - 1], full["gw"][L - 1])
+        ctx.set_option(lf.LF_OPT_SHARD_RANK, 1)
+        ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        ctx.sync()
+    torch.cuda.synchronize()
+    assert torch.equal(gw, full["gw"]) and torch.equal(delta, full["delta"])
