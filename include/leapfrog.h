@@ -170,6 +170,11 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k);
  * Otherwise the context runs one launch per layer and step with the k workers as streams
  * (LF_VARIANT_STREAMS) -- the single-launch kernels are written for one common width; an option
  * asking for them is accepted and lf_get_stats() reports what ran, with N = the widest layer.
+ * One case keeps the single launch: B = 1, L >= 3 and all hidden layers n_1 .. n_{L-1} of one
+ * width (the network of Section 2, whose input and output widths are left open): layers
+ * 2 .. L-1 then run as one persistent launch (LF_VARIANT_PERSISTENT or LF_VARIANT_FUSED, as
+ * asked for or as LF_VARIANT_AUTO picks for that width) between per-layer launches for the top
+ * and the bottom layer.
  * The arithmetic options apply as for lf_create (B > 1: tensor-core contractions by default).  lf_forward, lf_backward,
  * lf_backward_sgd and lf_backward_host take such a context; lf_grad_w, which names no layer,
  * returns LF_EINVAL for it.

@@ -23,11 +23,12 @@ inline size_t v_at(const lf_ctx* c, int l) { return c->off_h[l - 1]; }          
 inline size_t h_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_h[l - 1]; }       // z, delta
 inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; }           // a: l = 0..L
 
-// Contexts with per-layer widths run one launch per layer; the persistent kernels are written for
-// one common width (every cluster owns the same column strip of every layer).
+// The persistent kernels are written for one common width (every cluster owns the same column strip
+// of every layer): they serve uniform contexts and, for one sample, the run of hidden layers of a
+// context whose input and output widths alone differ; other contexts run one launch per layer.
 int resolve_variant(const lf_ctx* c)
 {
-    if (!c->uniform) return LF_VARIANT_STREAMS;
+    if (!c->uniform && (c->B != 1 || c->pk_N <= 0)) return LF_VARIANT_STREAMS;
     int v = c->opt_variant != LF_VARIANT_AUTO ? c->opt_variant : lf_auto_variant(c);
     // the fused pass stores every layer's tile; a shard stores only its own layers
     if (v == LF_VARIANT_FUSED && c->shard_count > 1) v = LF_VARIANT_PERSISTENT;
@@ -178,6 +179,59 @@ int backward_streams(lf_ctx* c, const float* w, const float* z, const float* a, 
     return LF_OK;
 }
 
+// One sample, hidden layers n_1 = ... = n_{L-1} of one width, input and/or output of another (the
+// network of the paper's Section 2): the top layer L and the bottom layer 1, whose matrices are not
+// square, run as launches of their own around ONE persistent launch over layers 2..L-1.
+//   stream:  Eq. bp1 (delta^L) -> Eq. bp2 with w^L (delta^{L-1}) -> persistent launch, which takes
+//            delta^{L-1} as given and goes down to delta^2 -> Eq. bp2 with w^2 (delta^1)
+//   workers: gw^L after delta^L and gw^1 after delta^1, on their leapfrog workers' streams
+int backward_hidden_run(lf_ctx* c, int variant, const float* w, const float* a, const float* y, float* delta,
+                        float* gw, float* gb, int gw_math)
+{
+    const int L = c->L;
+    cudaStream_t s = c->stream;
+    int launches = 0;
+    LF_CUDA_TRY(c, cudaEventRecord(c->fork_ev, s));
+    for (int j = 0; j < c->keff; ++j) LF_CUDA_TRY(c, cudaStreamWaitEvent(c->wstreams[j], c->fork_ev, 0));
+    bool used[2] = {false, false};
+    int worker[2] = {0, 0};
+    const int ends[2] = {L, 1};
+    for (int e = 0; e < 2; ++e) {
+        const int l = ends[e];
+        int rc;
+        if (e == 0) {
+            rc = enqueue_chain_step(c, L, w, a, y, delta, gb, s, &launches);            // delta^L
+        } else {
+            rc = enqueue_chain_step(c, 1, w, a, y, delta, gb, s, &launches);            // delta^1 from delta^2
+        }
+        if (rc != LF_OK) return rc;
+        if (lf_layer_owned(c, l)) {
+            LF_CUDA_TRY(c, cudaEventRecord(c->ready_ev[l - 1], s));
+            worker[e] = lf_layer_worker(c, l);
+            used[e] = true;
+            LF_CUDA_TRY(c, cudaStreamWaitEvent(c->wstreams[worker[e]], c->ready_ev[l - 1], 0));
+            rc = enqueue_gradients(c, l, a, delta, gw, gb, gw_math, c->wstreams[worker[e]], &launches);
+            if (rc != LF_OK) return rc;
+        }
+        if (e == 0) {
+            rc = enqueue_chain_step(c, L - 1, w, a, y, delta, gb, s, &launches);        // delta^{L-1}
+            if (rc != LF_OK) return rc;
+            rc = lf_backward_persistent(c, variant, w + w_at(c, 2), a + a_at(c, 1), y, delta + h_at(c, 2),
+                                        gw + w_at(c, 2), gb + v_at(c, 2),
+                                        c->sgd_on ? c->sgd_w + w_at(c, 2) : nullptr, 1, 1);
+            if (rc != LF_OK) return rc;
+            launches += 1;
+        }
+    }
+    for (int e = 0; e < 2; ++e) {
+        if (!used[e]) continue;
+        LF_CUDA_TRY(c, cudaEventRecord(c->done_ev[worker[e]], c->wstreams[worker[e]]));
+        LF_CUDA_TRY(c, cudaStreamWaitEvent(s, c->done_ev[worker[e]], 0));
+    }
+    c->stats.launches_backward = launches;
+    return LF_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -252,6 +306,13 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
             c->off_w[l] = c->off_w[l - 1] + (size_t)widths[l] * (size_t)widths[l - 1];
             c->off_h[l] = c->off_h[l - 1] + (size_t)widths[l];
         }
+    }
+    if (uniform) {
+        c->pk_N = N; c->pk_L = L;
+    } else if (L >= 3) {
+        bool hidden_equal = true;
+        for (int l = 2; l <= L - 1; ++l) hidden_equal = hidden_equal && widths[l] == widths[1];
+        if (hidden_equal) { c->pk_N = widths[1]; c->pk_L = L - 2; }
     }
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
@@ -433,7 +494,9 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
-    return lf_backward_persistent(ctx, variant, w, z, a, y, delta, gw, gb);
+    if (ctx->uniform)
+        return lf_backward_persistent(ctx, variant, w, a, y, delta, gw, gb, ctx->sgd_w, 0, 0);
+    return backward_hidden_run(ctx, variant, w, a, y, delta, gw, gb, gw_math);
 }
 
 int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_l)

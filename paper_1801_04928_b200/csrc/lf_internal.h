@@ -61,6 +61,10 @@ struct lf_ctx {
     // per-layer widths n_0..n_L and where each layer's block starts inside the caller's arrays
     // (in floats; the per-sample arrays multiply by B).  Uniform contexts fill them with N.
     bool uniform;            // all widths equal: every kernel family applies
+    // what a single-launch (persistent) pass covers: all L layers of a uniform context; the L - 2
+    // layers 2..L-1 when only the hidden layers n_1..n_{L-1} share a width (the top and the bottom
+    // layer then run as launches of their own); pk_N = 0 when there is no such run
+    int pk_N, pk_L;
     int* width;              // [L+1]  n_l
     size_t* off_w;           // [L+1]  off_w[l-1]: start of w^l (n_l x n_{l-1}); off_w[L]: total
     size_t* off_h;           // [L+1]  off_h[l-1]: n_1 + ... + n_{l-1} (b, gb; z, delta times B)
@@ -171,8 +175,8 @@ cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, c
 size_t lf_sync_words_needed(const lf_ctx* c);           // unsigned words of flag/barrier workspace
 bool lf_persistent_supported(const lf_ctx* c, int variant);
 int lf_auto_variant(const lf_ctx* c);                   // table lookup for LF_VARIANT_AUTO
-int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* z, const float* a,
-                           const float* y, float* delta, float* gw, float* gb);
+int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* a, const float* y, float* delta,
+                           float* gw, float* gb, const float* w_sub, int top_given, int depth_shift);
 void lf_persistent_release(lf_ctx* c);
 
 // ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------

@@ -49,6 +49,10 @@ struct PkParams {
     int Qc;        // chain clusters
     int Qw;        // worker clusters (0 in the fused variant)
     int shard_rank, shard_count;   // the workers store layer l only if (L - l) % shard_count == shard_rank
+    int top_given;     // 1: delta of the top layer is already in `delta` (the launch covers a run of layers
+                       //    below the network's own top layer); 0: Eq. bp1 is computed here
+    int depth_shift;   // layers between the run's top layer and the network's: added to (L - l) wherever
+                       //    a layer is given to a shard or a worker group
     int fused;     // 1: chain CTAs store gw tiles
     int Wc;        // columns per column block (32, 64, 128 or 256)
     int nCB;       // column blocks per strip
@@ -379,8 +383,9 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
         float* a_sm = stages;                         // N floats (N <= 16384: two stages)
         float* dr = stages + 16384;                   // up to N floats
         for (int l = L; l >= 1; --l) {
-            if ((L - l) % P.shard_count != P.shard_rank) continue;        // another shard's layer
-            if (((((L - l) / P.shard_count) % P.keff) % G) != g) continue;   // not a layer of my group
+            const int depth = L - l + P.depth_shift;
+            if (depth % P.shard_count != P.shard_rank) continue;        // another shard's layer
+            if ((((depth / P.shard_count) % P.keff) % G) != g) continue;   // not a layer of my group
             if (row0 < row1) worker_store_rows<UPDATE>(P, l, row0, row1, dr, a_sm, sh);
         }
         cluster_sync_all();   // the cluster's CTAs leave together
@@ -534,14 +539,18 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 const int row = row_base + r;
                 float d = 0.f;
                 if (r < Hr && row < N) {
-                    const float av = aL[row];
-                    d = av - P.y[row];
-                    if (P.cost == LF_COST_QUADRATIC) d *= lf_act_prime(av, P.act);   // cross-entropy: sigma' cancels
-                    if (q == 0) {
-                        P.delta[(size_t)(L - 1) * N + row] = d;
-                        P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
-                        if (P.Qw > 0) st_slot(P.xch + (size_t)(L - 1) * N + row, d, P.epoch);
+                    if (P.top_given) {
+                        d = P.delta[(size_t)(L - 1) * N + row];   // written (with gb) by an earlier launch
+                    } else {
+                        const float av = aL[row];
+                        d = av - P.y[row];
+                        if (P.cost == LF_COST_QUADRATIC) d *= lf_act_prime(av, P.act);   // cross-entropy: sigma' cancels
+                        if (q == 0) {
+                            P.delta[(size_t)(L - 1) * N + row] = d;
+                            P.gb[(size_t)(L - 1) * N + row] = d;                  // Eq. bp3
+                        }
                     }
+                    if (q == 0 && P.Qw > 0) st_slot(P.xch + (size_t)(L - 1) * N + row, d, P.epoch);
                 }
                 dr[r] = d;
             }
@@ -806,7 +815,7 @@ PkPlan plan_for_cluster(const lf_ctx* c, int variant, int C)
         }
     }
     if (Qc_budget < 1) return p;
-    const int N = c->N;
+    const int N = c->pk_N;
     int need = (N + Qc_budget - 1) / Qc_budget;      // strip width needed
     int Wc = 32;
     while (Wc < need && Wc < 256) Wc <<= 1;
@@ -833,7 +842,7 @@ PkPlan plan_for_cluster(const lf_ctx* c, int variant, int C)
 PkPlan make_plan(const lf_ctx* c, int variant)
 {
     PkPlan best = {};
-    if (c->B != 1) return best;
+    if (c->B != 1 || c->pk_N <= 0 || c->pk_L < 1) return best;
     if ((size_t)c->smem_optin < PK_SMEM_BYTES) return best;
     if (!get_encode_fn()) return best;
     int best_ctas = 0;
@@ -870,24 +879,26 @@ bool lf_persistent_supported(const lf_ctx* c, int variant)
 // ahead.
 int lf_auto_variant(const lf_ctx* c)
 {
-    if (c->B != 1) return LF_VARIANT_STREAMS;
-    const int N = c->N;
+    if (c->B != 1 || c->pk_N <= 0) return LF_VARIANT_STREAMS;
+    const int N = c->pk_N;
     const bool groups_faster = c->keff <= 4 ? N <= 2048 : (N <= 576 || (N >= 832 && N <= 1280));
     if (groups_faster && make_plan(c, LF_VARIANT_PERSISTENT).ok) return LF_VARIANT_PERSISTENT;
     return make_plan(c, LF_VARIANT_FUSED).ok ? LF_VARIANT_FUSED : LF_VARIANT_STREAMS;
 }
 
-int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* z, const float* a,
-                           const float* y, float* delta, float* gw, float* gb)
+// The launch covers the pk_L layers of width pk_N that w, a, delta, gw, gb (and w_sub) point at --
+// the whole network, or the run of equal-width layers in its middle (top_given, depth_shift = 1).
+int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* a, const float* y, float* delta,
+                           float* gw, float* gb, const float* w_sub, int top_given, int depth_shift)
 {
-    (void)z;
+    const int L_run = c->pk_L, N_run = c->pk_N;
     PkPlan pl = make_plan(c, variant);
     if (!pl.ok) return LF_ERESOURCE;
     // tensor map over w as [L][N][N], box = Wc columns x R rows x 1 layer
     if (!c->w_map_valid || c->w_map_ptr != w || c->w_map_wc != pl.Wc) {
         CUtensorMap* m = reinterpret_cast<CUtensorMap*>(c->w_map_storage);
-        cuuint64_t dims[3] = {(cuuint64_t)c->N, (cuuint64_t)c->N, (cuuint64_t)c->L};
-        cuuint64_t strides[2] = {(cuuint64_t)c->N * 4, (cuuint64_t)c->N * c->N * 4};
+        cuuint64_t dims[3] = {(cuuint64_t)N_run, (cuuint64_t)N_run, (cuuint64_t)L_run};
+        cuuint64_t strides[2] = {(cuuint64_t)N_run * 4, (cuuint64_t)N_run * N_run * 4};
         cuuint32_t box[3] = {(cuuint32_t)pl.Wc, (cuuint32_t)pl.R, 1};
         cuuint32_t estr[3] = {1, 1, 1};
         CUresult r = get_encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(w), dims,
@@ -904,7 +915,8 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     if (c->epoch == 0) c->epoch = 1;
 
     PkParams P = {};
-    P.L = c->L; P.N = c->N; P.C = pl.C; P.Qc = pl.Qc; P.Qw = pl.Qw;
+    P.L = L_run; P.N = N_run; P.C = pl.C; P.Qc = pl.Qc; P.Qw = pl.Qw;
+    P.top_given = top_given; P.depth_shift = depth_shift;
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
     P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
@@ -912,7 +924,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.shard_rank = c->shard_rank; P.shard_count = c->shard_count > 1 ? c->shard_count : 1;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
-    P.w_sub = c->sgd_on ? c->sgd_w : nullptr; P.eta = c->sgd_eta;
+    P.w_sub = c->sgd_on ? w_sub : nullptr; P.eta = c->sgd_eta;
     P.xch = reinterpret_cast<unsigned long long*>(c->sync_words);
     P.status = c->status_dev;
 #ifdef LF_PK_TRACE

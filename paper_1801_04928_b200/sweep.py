@@ -62,10 +62,13 @@ def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
             alg = 4.0 * (2 * sum(mats) - mats[0]) + 12.0 * B * hidden
             flops = 2.0 * B * (2 * sum(mats) - mats[0])
             steps, warmup = (3, 1) if flops > 2e11 else (30, 5)
-            for k in ks:
+            # one sample: the stream schedule, and whatever LF_VARIANT_AUTO picks (the single-launch pass
+            # when the hidden layers share a width)
+            for k, variant in [(k, v) for k in ks for v in ((1, 0) if B == 1 else (1,))]:
                 stream = torch.cuda.Stream()
                 stream.wait_stream(torch.cuda.current_stream())
                 with lf.Leapfrog(0, 0, B, k, stream=stream.cuda_stream, widths=n) as ctx:
+                    ctx.set_option(lf.LF_OPT_VARIANT, variant)
                     with torch.cuda.stream(stream):
                         ctx.forward(t["w"], t["b"], t["x"], t["z"], t["a"])
                         for _ in range(warmup):
@@ -78,7 +81,7 @@ def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
                         ctx.sync()
                     st = ctx.stats()
                 ms = e0.elapsed_time(e1) / steps
-                row = dict(widths=n, B=B, k=k, variant="streams", ms=ms, layers_per_s=L / (ms * 1e-3),
+                row = dict(widths=n, B=B, k=k, variant={1: "streams", 2: "persistent", 3: "fused"}[st["variant"]], ms=ms, layers_per_s=L / (ms * 1e-3),
                            alg_GBs=alg / (ms * 1e-3) / 1e9, alg_TFLOPs=flops / (ms * 1e-3) / 1e12 if B > 1 else None,
                            launches=st["launches_backward"])
                 f.write(json.dumps(row) + "\n"); f.flush()

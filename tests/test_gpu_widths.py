@@ -226,3 +226,82 @@ def test_widths_full_size_single_sample():
         want = d_l[l - 1][0][rows, None] * a_l[l - 1][0][None, :]
         assert_layer_close("gw", l - 1, g[rows], want, tol=FP32_TOL, n_terms=max(n))
         assert np.all(np.isfinite(g))
+
+
+# ---- hidden layers of one width, input / output of another: the single-launch pass over the hidden run
+HIDDEN_RUN_SHAPES = [
+    [260, 516, 516, 516, 516, 132],     # both ends differ
+    [516, 516, 516, 516, 12],           # only the output differs
+    [36, 1028, 1028, 1028],             # only the input differs
+    [200, 132, 132, 64],                # L = 3: a run of one layer
+    [8, 64, 64, 64, 64, 64, 64, 4],
+]
+
+
+def _run_variant(widths, k, variant, seed, sgd_eta=None, shard=None):
+    n = [int(v) for v in widths]
+    cpu = lf_inputs.make_inputs_widths(n, 1, "uniform", lf_inputs.SEED_BASE + 800 + seed, "cpu")
+    t = {key: v.cuda() for key, v in cpu.items()}
+    sz = orc.sizes_widths(n, 1)
+    z = torch.empty(sz["z"], device="cuda"); a = torch.empty(sz["a"], device="cuda")
+    delta = torch.full((sz["z"],), float("nan"), device="cuda")
+    gw = torch.full((sz["w"],), float("nan"), device="cuda")
+    gb = torch.full((sz["b"],), float("nan"), device="cuda")
+    with lf.Leapfrog(0, 0, 1, k, widths=n) as ctx:
+        ctx.set_option(lf.LF_OPT_VARIANT, variant)
+        if shard is not None:
+            ctx.set_option(lf.LF_OPT_SHARD_COUNT, shard[1])
+            ctx.set_option(lf.LF_OPT_SHARD_RANK, shard[0])
+        ctx.forward(t["w"], t["b"], t["x"], z, a)
+        for _ in range(2):     # twice: the second call meets the flags and slots the first one left
+            if sgd_eta is not None:
+                ctx.backward_sgd(t["w"], z, a, t["y"], sgd_eta, delta, gw, gb)
+            else:
+                ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        ctx.sync()
+        stats = ctx.stats()
+    torch.cuda.synchronize()
+    out = {key: v.cpu().numpy() for key, v in dict(z=z, a=a, delta=delta, gw=gw, gb=gb).items()}
+    return n, cpu, out, stats
+
+
+@pytest.mark.parametrize("variant", [lf.LF_VARIANT_AUTO, lf.LF_VARIANT_PERSISTENT, lf.LF_VARIANT_FUSED])
+@pytest.mark.parametrize("k", [1, 3])
+@pytest.mark.parametrize("widths", HIDDEN_RUN_SHAPES, ids=lambda s: "-".join(map(str, s)))
+def test_hidden_run_goes_through_the_single_launch_pass(widths, k, variant):
+    n, cpu, out, stats = _run_variant(widths, k, variant, seed=len(widths) + k)
+    assert stats["device_status"] == 0
+    assert stats["variant"] in (lf.LF_VARIANT_PERSISTENT, lf.LF_VARIANT_FUSED)
+    if variant != lf.LF_VARIANT_AUTO:
+        assert stats["variant"] == variant
+    assert stats["launches_backward"] == 6            # bp1, 2 x bp2, 2 x rank-1 writer, 1 persistent launch
+    _compare(n, 1, cpu, out)
+
+
+@pytest.mark.parametrize("variant", [lf.LF_VARIANT_PERSISTENT, lf.LF_VARIANT_FUSED])
+def test_hidden_run_fused_update(variant):
+    n, cpu, out, stats = _run_variant([260, 516, 516, 516, 132], 2, variant, seed=5, sgd_eta=0.3)
+    assert stats["variant"] == variant
+    _compare(n, 1, cpu, out, sgd_eta=0.3)
+
+
+def test_hidden_run_shards():
+    widths, S = [260, 516, 516, 516, 516, 516, 132], 2
+    n = widths
+    L = len(n) - 1
+    union = None
+    for r in range(S):
+        n, cpu, out, stats = _run_variant(widths, 2, lf.LF_VARIANT_AUTO, seed=9, shard=(r, S))
+        assert stats["variant"] == lf.LF_VARIANT_PERSISTENT and stats["device_status"] == 0
+        w = cpu["w"].numpy()
+        z, a = orc.forward_widths(n, w, cpu["b"].numpy(), cpu["x"].numpy())
+        delta, gw, gb = orc.backward_widths(n, w, z, a, cpu["y"].numpy())
+        for l, (g, ref) in enumerate(zip(orc.split(out["gw"], n, "w"), orc.split(gw, n, "w")), start=1):
+            if (L - l) % S == r:
+                assert_layer_close("gw", l - 1, g, ref, n_terms=max(n))
+            else:
+                assert np.all(np.isnan(g)), f"shard {r} wrote layer {l}"
+        for l, (g, ref) in enumerate(zip(orc.split(out["delta"], n, "z", 1), orc.split(delta, n, "z", 1)), start=1):
+            assert_layer_close("delta", l - 1, g, ref, n_terms=max(n))
+        union = out["gw"] if union is None else np.where(np.isnan(union), out["gw"], union)
+    assert np.all(np.isfinite(union))
