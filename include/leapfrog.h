@@ -18,6 +18,7 @@
  *     gw    [L][N][N]   same indexing as w
  *     gb    [L][N]
  * N must be a multiple of 4 (128-bit accesses); other sizes are rejected with LF_EINVAL.
+ * (lf_create_widths gives every layer its own width; its layouts are stated there.)
  *
  * Execution.  Calls enqueue work on the context's stream and return; lf_sync() waits for it
  * and reports device-side status.  The library never allocates or frees tensors; a context
