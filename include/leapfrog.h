@@ -200,8 +200,8 @@ int lf_set_stream(lf_ctx* ctx, void* cuda_stream);
  * of those arrays are not touched.  Inside the shard the k leapfrog workers share the shard's
  * layers in turn: worker ((L - l) / S) mod k.  The S contexts are independent: one per GPU, or
  * several on one GPU writing into one gw array, give together exactly what one unsharded
- * context writes.  LF_VARIANT_FUSED, whose tile pass stores every layer, runs as
- * LF_VARIANT_PERSISTENT (or LF_VARIANT_STREAMS) in a sharded context.
+ * context writes.  Every variant takes a sharded context (the fused pass skips the stores of
+ * other shards' tiles).
  */
 /* Set an option (enum lf_option).  LF_EINVAL for unknown keys or out-of-range values. */
 int lf_set_option(lf_ctx* ctx, int key, long long value);

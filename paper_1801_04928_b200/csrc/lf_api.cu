@@ -29,10 +29,7 @@ inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; 
 int resolve_variant(const lf_ctx* c)
 {
     if (!c->uniform && (c->B != 1 || c->pk_N <= 0)) return LF_VARIANT_STREAMS;
-    int v = c->opt_variant != LF_VARIANT_AUTO ? c->opt_variant : lf_auto_variant(c);
-    // the fused pass stores every layer's tile; a shard stores only its own layers
-    if (v == LF_VARIANT_FUSED && c->shard_count > 1) v = LF_VARIANT_PERSISTENT;
-    return v;
+    return c->opt_variant != LF_VARIANT_AUTO ? c->opt_variant : lf_auto_variant(c);
 }
 
 int resolve_gw_math(const lf_ctx* c)

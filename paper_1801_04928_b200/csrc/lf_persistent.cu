@@ -462,6 +462,9 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 wait_bar<false>(smem_u32(&sh->d_ready[p]), use & 1u, P, sh);
                 const float* dr = d_rows + p * PK_DROWS;
                 float* gw_s = P.gw + (size_t)(s - 1) * N * N;
+                // layer-sharded form: the tile of another shard's layer is not stored; every wait and
+                // arrival below still takes place, so the chain and the producer see no difference
+                const bool mine = (L - s + P.depth_shift) % P.shard_count == P.shard_rank;
                 if (UPDATE && s >= 2) {
                     // Fused weight update, layers the chain reads: the sub-tiles of w^s pass through
                     // this CTA's shared memory for the chain anyway, so the store warps take w from
@@ -478,7 +481,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                             const int st = it_store % PK_STAGES;
                             wait_bar<false>(smem_u32(&sh->full[st]), (unsigned)((it_store / PK_STAGES) & 1), P, sh);
                             const float4* tile = reinterpret_cast<const float4*>(stages + (size_t)st * PK_STAGE_FLOATS);
-                            if (col < N) {
+                            if (mine && col < N) {
 #pragma unroll 8
                                 for (int i = 0; i < 16; ++i) {
                                     const int rr = rb * R + trow + i * RG;
@@ -500,7 +503,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
                 }
 #pragma unroll
                 for (int cb = 0; cb < PK_MAX_NCB; ++cb) {
-                    if (cb >= nCB) break;
+                    if (cb >= nCB || !mine) break;
                     const int col = col_base + cb * Wc + tcol * 4;
                     if (col >= N) continue;
                     const float4 av = a4[cb];

@@ -69,8 +69,7 @@ def test_single_sample_shards(L, N, k, S, variant):
     for r in range(S):
         bufs, stats, owners = _shard_pass(L, N, 1, k, S, r, t, variant)
         assert stats["device_status"] == 0 and stats["shard_count"] == S and stats["shard_rank"] == r
-        assert stats["variant"] != lf.LF_VARIANT_FUSED
-        if variant in (lf.LF_VARIANT_STREAMS, lf.LF_VARIANT_PERSISTENT):
+        if variant != lf.LF_VARIANT_AUTO:
             assert stats["variant"] == variant
         d_ref, gw_ref, gb_ref, wrote = orc.backward_shard(w, z, a, y, S, r)
         gw = bufs["gw"].cpu().numpy(); gb = bufs["gb"].cpu().numpy(); d = bufs["delta"].cpu().numpy()
@@ -144,6 +143,28 @@ def test_shards_of_the_fused_update_and_of_the_host_entry_point(B):
                 assert np.all(np.isnan(w_new[l - 1])) and np.all(np.isnan(gw_h[l - 1]))
                 if B > 1:
                     assert np.all(np.isnan(gb_h[l - 1]))
+
+
+@pytest.mark.parametrize("variant", [lf.LF_VARIANT_PERSISTENT, lf.LF_VARIANT_FUSED])
+def test_shards_of_the_fused_update_in_the_single_launch_variants(variant):
+    # the fused pass takes w from the chain's shared-memory stages; for another shard's layer it must
+    # still hand every stage back without storing anything
+    L, N, k, S, eta = 7, 516, 2, 3, 0.25
+    cpu, t = _inputs(L, N, 1, seed=63)
+    w, z, a, y = _oracle(cpu)
+    for r in range(S):
+        d_ref, gw_ref, gb_ref, wrote = orc.backward_shard(w, z, a, y, S, r)
+        upd, stats, _ = _shard_pass(L, N, 1, k, S, r, t, variant, sgd_eta=eta)
+        assert stats["variant"] == variant and stats["device_status"] == 0
+        w_new = upd["gw"].cpu().numpy()
+        for l in range(1, L + 1):
+            assert_layer_close("delta", l - 1, upd["delta"].cpu().numpy()[l - 1], d_ref[l - 1], n_terms=N + 1)
+            if wrote[l - 1]:
+                want = w[l - 1].astype(np.float64) - eta * gw_ref[l - 1]
+                bound = eta * FP32_TOL * np.max(np.abs(gw_ref[l - 1])) + 2.0 ** -23 * np.max(np.abs(want))
+                assert np.max(np.abs(w_new[l - 1] - want)) <= bound
+            else:
+                assert np.all(np.isnan(w_new[l - 1]))
 
 
 def test_shard_option_checks():
