@@ -219,7 +219,7 @@ def aggregate_rate(total_ms, units_per_rank, dist=None, device=None):
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu capture
 # summarised under profiles/) of the dominant kernel, keyed by (config, variant); null elsewhere.
-NCU_TRAFFIC = {(2, 2): 206.2e6}
+NCU_TRAFFIC = {(2, 2): 206.4e6}
 
 
 def time_gw_gemm(lf, L, N, B, t, stream, steps, tc_tiling=0):
