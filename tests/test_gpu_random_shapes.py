@@ -72,3 +72,28 @@ def test_random_shards(case, L, N, k, S, variant, eta):
                 want = w[l - 1].astype(np.float64) - eta * gw_ref[l - 1]
                 bound = eta * 1e-5 * np.max(np.abs(gw_ref[l - 1])) + 2.0 ** -23 * np.max(np.abs(want))
                 assert np.max(np.abs(gw[l - 1] - want)) <= bound
+
+
+def _uniform_cases(seed, count):
+    rng = random.Random(seed)
+    cases = []
+    for i in range(count):
+        B = rng.choice([1, 1, 1, 2, 5, 31, 128, 130, 256, 300])
+        cases.append((i, rng.randint(1, 10), 4 * rng.randint(1, 400), B, rng.randint(1, 12),
+                      rng.choice([0, 1, 2, 3]) if B == 1 else 0, rng.choice([0, 1, 2]), rng.choice([0, 1, 2]),
+                      rng.choice([0, 1, 2]), rng.random() < 0.3))
+    return cases
+
+
+@pytest.mark.parametrize("case,L,N,B,k,variant,gw_math,delta_math,tiling,cross_entropy", _uniform_cases(20260116, 24))
+def test_random_uniform_networks(case, L, N, B, k, variant, gw_math, delta_math, tiling, cross_entropy):
+    import lf_inputs
+    from lf_testlib import compare_all, gpu_pass, oracle_pass
+    cpu = lf_inputs.make_inputs(L, N, B, "uniform" if B == 1 else "onehot", lf_inputs.SEED_BASE + 5000 + case, "cpu")
+    t = {name: v.cuda() for name, v in cpu.items()}
+    cfg = dict(L=L, N=N, B=B, k=k)
+    out, stats = gpu_pass(cfg, t, variant=variant, gw_math=gw_math, delta_math=delta_math, tc_tiling=tiling,
+                          cost=lf.LF_COST_CROSS_ENTROPY if cross_entropy else lf.LF_COST_QUADRATIC, repeat=2)
+    assert stats["device_status"] == 0
+    ref = oracle_pass(t, want_gw=False, cross_entropy=cross_entropy)
+    compare_all(cfg, out, ref, gw_tf32=(stats["gw_math"] == lf.LF_GW_MATH_TF32))
