@@ -16,6 +16,9 @@
  *   Section 2, Eq. bp3 : dC/db^l_j = delta^l_j
  *   Section 2, Eq. bp4 : dC/dw^l_jk = a^{l-1}_k delta^l_j
  *   Section 3, Algorithm 1 : the leapfrog schedule with k threads (lfo_backward_leapfrog)
+ *   Section 1 ("k threads or k gpus") : one GPU's pass of the schedule on S GPUs (lfo_backward_shard)
+ *   Section 2 (equations "generally valid") : the same pass for layers of different widths
+ *                            (lfo_forward_widths, lfo_backward_widths)
  *   (not in the paper)     : the gradient-descent step that consumes Eq. bp4, w - eta dC/dw
  *                            (lfo_sgd_step); the paper ends with the gradients of one pass
  *
@@ -24,7 +27,7 @@
  *     bias is added, z = w a + b.
  *   - Indexing: this code counts L WEIGHT layers l = 1..L with a^0 = x.  The paper numbers
  *     the input as layer 1, so paper layer p is l = p - 1 here and the paper's L is L + 1.
- *   - All layers, input and output included, are N wide.
+ *   - All layers, input and output included, are N wide (except in the *_widths functions).
  *   - C is the quadratic cost C = 1/2 sum_b ||a^L_b - y_b||^2 (a SUM over the B samples,
  *     no 1/B), hence grad_a C = a^L - y.  (The *_cross_entropy functions are the same pass
  *     under a second cost, see there.)
