@@ -86,6 +86,17 @@ enum lf_tc_tiling {
                                 N >= 512; other sizes use ONE_SM                                */
 };
 
+/* Tiling of the fused single-launch pass (LF_VARIANT_FUSED, B = 1). */
+enum lf_fused_tiling {
+    LF_FUSED_TILING_AUTO = 0,     /* whole columns at the widths where the delta hand-off is the bound */
+    LF_FUSED_TILING_CLUSTERS = 1, /* thread-block clusters own column strips, their CTAs row blocks of
+                                     them; partial sums cross the cluster's shared memory             */
+    LF_FUSED_TILING_COLUMNS = 2   /* every CTA owns whole columns (all rows): delta crosses CTAs once
+                                     per layer, and each CTA stores the rows of gw it finished itself
+                                     (in lf_backward_sgd it reads those rows of w from memory once
+                                     more, where CLUSTERS takes them from the tile the chain holds)   */
+};
+
 /* The cost function C of Eq. bp1, delta^L = grad_a C (.) sigma'(z^L); Section 2 leaves it open
  * ("the cost function").  Both are sums over the B samples (no 1/B). */
 enum lf_cost {
@@ -117,6 +128,7 @@ enum lf_option {
     LF_OPT_SHARD_COUNT = 10,  /* S >= 1 (default 1): the paper's "k gpus" form (Section 1), see
                                  below; setting it puts the rank back to 0                    */
     LF_OPT_SHARD_RANK = 11,   /* r, 0 <= r < S: which of the S shards this context is         */
+    LF_OPT_FUSED_TILING = 12, /* enum lf_fused_tiling                                         */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -142,6 +154,8 @@ typedef struct lf_stats {
     int activation;           /* activation the last lf_forward / lf_backward used            */
     int shard_rank;           /* LF_OPT_SHARD_RANK and LF_OPT_SHARD_COUNT of the last lf_backward */
     int shard_count;
+    int fused_tiling;         /* tiling of the last fused single-launch pass (enum lf_fused_tiling,
+                                 CLUSTERS or COLUMNS; 0 if the last pass was not a fused one)     */
 } lf_stats;
 
 /*
@@ -149,6 +163,10 @@ typedef struct lf_stats {
  * workers (Section 3: "k threads"; here CTA groups or streams).  k > L is legal and acts as
  * k = L.  Binds to the current CUDA device and allocates the workspace there.
  * *out receives the context; on failure *out is NULL.
+ * Two options take their initial value from the environment, if set, so that a run can be steered
+ * without touching the caller: LF_VARIANT = auto | streams | persistent | fused (LF_OPT_VARIANT) and
+ * LF_FUSED_TILING = auto | clusters | columns (LF_OPT_FUSED_TILING), by name or by number; a later
+ * lf_set_option overrides them, an unknown value is ignored.
  * Errors: LF_ENULL (out), LF_EINVAL (sizes), LF_ECUDA (no device / CUDA failure), LF_ENOMEM.
  */
 int lf_create(lf_ctx** out, int L, int N, int B, int k);

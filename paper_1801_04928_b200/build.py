@@ -18,7 +18,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libleapfrog.so")
 
-SOURCES = ["lf_api.cu", "lf_kernels_b1.cu", "lf_kernels_batch.cu", "lf_persistent.cu",
+SOURCES = ["lf_api.cu", "lf_kernels_b1.cu", "lf_kernels_batch.cu", "lf_persistent.cu", "lf_columns.cu",
            "lf_gemm_tf32.cu", "lf_delta_gemm_tc.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -1,5 +1,6 @@
 // C ABI of libleapfrog: context, validation, scheduling of the per-layer kernels.
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "lf_internal.h"
@@ -7,6 +8,19 @@
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Initial value of an option from the environment: one of `names` (its index) or a number in range;
+// anything else, or no variable, gives `fallback`.
+int option_from_env(const char* var, const char* const* names, int count, int fallback)
+{
+    const char* e = getenv(var);
+    if (!e || !*e) return fallback;
+    for (int i = 0; i < count; ++i)
+        if (strcmp(e, names[i]) == 0) return i;
+    char* end = nullptr;
+    const long v = strtol(e, &end, 10);
+    return (end && *end == 0 && v >= 0 && v < count) ? (int)v : fallback;
+}
 
 int check_ptrs(const void* const* ps, int n)
 {
@@ -315,7 +329,10 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
     c->sm_count = prop.multiProcessorCount;
     c->smem_optin = (int)prop.sharedMemPerBlockOptin;
     c->stream = nullptr;
-    c->opt_variant = LF_VARIANT_AUTO;
+    static const char* const variant_names[] = {"auto", "streams", "persistent", "fused"};
+    static const char* const tiling_names[] = {"auto", "clusters", "columns"};
+    c->opt_variant = option_from_env("LF_VARIANT", variant_names, 4, LF_VARIANT_AUTO);
+    c->opt_fused_tiling = option_from_env("LF_FUSED_TILING", tiling_names, 3, LF_FUSED_TILING_AUTO);
     c->opt_gw_math = LF_GW_MATH_AUTO;
     c->wait_budget_us = 2000000;
     c->use_graph = 1;
@@ -424,6 +441,10 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value < 0 || value >= ctx->shard_count) return LF_EINVAL;
             ctx->shard_rank = (int)value;
             return LF_OK;
+        case LF_OPT_FUSED_TILING:
+            if (value < LF_FUSED_TILING_AUTO || value > LF_FUSED_TILING_COLUMNS) return LF_EINVAL;
+            ctx->opt_fused_tiling = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -489,6 +510,7 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     ctx->stats.cost = ctx->opt_cost;
     ctx->stats.activation = ctx->opt_act;
     ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
+    ctx->stats.fused_tiling = 0;
     if (variant == LF_VARIANT_STREAMS)
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     if (ctx->uniform)

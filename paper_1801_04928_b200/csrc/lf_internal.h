@@ -116,7 +116,13 @@ struct lf_ctx {
     const void* w_map_ptr;
     int w_map_wc;
     unsigned epoch;
-#ifdef LF_PK_TRACE
+    // the whole-columns fused kernel keeps a descriptor of its own (another box shape)
+    alignas(64) unsigned char ck_map_storage[128];
+    bool ck_map_valid;
+    const void* ck_map_ptr;
+    int ck_map_wc;
+    int opt_fused_tiling;    // enum lf_fused_tiling
+#if defined(LF_PK_TRACE) || defined(LF_CK_TRACE)
     unsigned long long* trace_dev;  // debug builds: per-step SM-clock stamps of two CTAs
 #endif
 
@@ -178,6 +184,13 @@ int lf_auto_variant(const lf_ctx* c);                   // table lookup for LF_V
 int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* a, const float* y, float* delta,
                            float* gw, float* gb, const float* w_sub, int top_given, int depth_shift);
 void lf_persistent_release(lf_ctx* c);
+int lf_fused_tiling(const lf_ctx* c);                   // which fused kernel a context gets (enum lf_fused_tiling)
+constexpr int LF_COLUMNS_AUTO_MAX_N = 640;    // widths up to which LF_VARIANT_AUTO takes the fused pass with whole columns
+constexpr int LF_COLUMNS_FUSED_MAX_N = 768;   // widths up to which a fused pass takes whole columns (LF_FUSED_TILING_AUTO)
+// the fused pass with whole columns per CTA (one hop through L2 per layer, no clusters)
+bool lf_columns_supported(const lf_ctx* c);
+int lf_backward_columns(lf_ctx* c, const float* w, const float* a, const float* y, float* delta, float* gw,
+                        float* gb, const float* w_sub, int top_given, int depth_shift);
 
 // ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------
 bool lf_tf32_supported(const lf_ctx* c);

@@ -870,23 +870,39 @@ size_t lf_sync_words_needed(const lf_ctx* c)
 bool lf_persistent_supported(const lf_ctx* c, int variant)
 {
     if (variant != LF_VARIANT_PERSISTENT && variant != LF_VARIANT_FUSED) return false;
+    if (variant == LF_VARIANT_FUSED && lf_columns_supported(c)) return true;
     return make_plan(c, variant).ok;
+}
+
+// Which of the two fused kernels serves a context: whole columns per CTA (one hop per layer), or
+// cluster tiles.  The same rule holds for the plain pass and for the fused weight update, so that
+// the two give the same gradients bit for bit.
+int lf_fused_tiling(const lf_ctx* c)
+{
+    const bool columns_ok = lf_columns_supported(c);
+    const bool clusters_ok = make_plan(c, LF_VARIANT_FUSED).ok;
+    if (c->opt_fused_tiling == LF_FUSED_TILING_COLUMNS && columns_ok) return LF_FUSED_TILING_COLUMNS;
+    if (c->opt_fused_tiling == LF_FUSED_TILING_CLUSTERS && clusters_ok) return LF_FUSED_TILING_CLUSTERS;
+    if (columns_ok && (!clusters_ok || c->pk_N <= LF_COLUMNS_FUSED_MAX_N)) return LF_FUSED_TILING_COLUMNS;
+    return LF_FUSED_TILING_CLUSTERS;
 }
 
 // LF_VARIANT_AUTO for one sample: fused pass or leapfrog CTA groups, from measurement (B200, L = 32,
 // buffers rotated so that nothing is found in L2, N = 256..4096, k = 1..8).  Up to N = 2048 the pass
-// is bound by the delta hand-off, and the groups variant -- whose chain has half of the clusters,
-// hence wider strips and fewer CTAs to wait for -- is 1-12 % ahead with up to four workers; with
-// more workers (fewer CTAs per layer) only at the widths listed.  From N = 2560 the pass is
-// bandwidth-bound and the fused pass, which leaves no SM without a share of the weights, is 4-8 %
-// ahead.
+// is bound by the delta hand-off.  Up to N = 640 the fused pass with whole columns per CTA -- one
+// hop per layer, few CTAs -- is 3-12 % ahead of everything else.  From there to N = 2048 the groups
+// variant -- whose chain has half of the clusters, hence wider strips and fewer CTAs to wait for,
+// and stores nothing itself -- is 1-12 % ahead with up to four workers; with more workers (fewer
+// CTAs per layer) only at the widths listed.  From N = 2560 the pass is bandwidth-bound and the fused
+// pass, which leaves no SM without a share of the weights, is 4-8 % ahead.
 int lf_auto_variant(const lf_ctx* c)
 {
     if (c->B != 1 || c->pk_N <= 0) return LF_VARIANT_STREAMS;
     const int N = c->pk_N;
+    if (N <= LF_COLUMNS_AUTO_MAX_N && lf_columns_supported(c)) return LF_VARIANT_FUSED;
     const bool groups_faster = c->keff <= 4 ? N <= 2048 : (N <= 576 || (N >= 832 && N <= 1280));
     if (groups_faster && make_plan(c, LF_VARIANT_PERSISTENT).ok) return LF_VARIANT_PERSISTENT;
-    return make_plan(c, LF_VARIANT_FUSED).ok ? LF_VARIANT_FUSED : LF_VARIANT_STREAMS;
+    return lf_persistent_supported(c, LF_VARIANT_FUSED) ? LF_VARIANT_FUSED : LF_VARIANT_STREAMS;
 }
 
 // The launch covers the pk_L layers of width pk_N that w, a, delta, gw, gb (and w_sub) point at --
@@ -895,8 +911,14 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
                            float* gw, float* gb, const float* w_sub, int top_given, int depth_shift)
 {
     const int L_run = c->pk_L, N_run = c->pk_N;
+    c->stats.fused_tiling = 0;
+    if (variant == LF_VARIANT_FUSED && lf_fused_tiling(c) == LF_FUSED_TILING_COLUMNS) {
+        c->stats.fused_tiling = LF_FUSED_TILING_COLUMNS;
+        return lf_backward_columns(c, w, a, y, delta, gw, gb, w_sub, top_given, depth_shift);
+    }
     PkPlan pl = make_plan(c, variant);
     if (!pl.ok) return LF_ERESOURCE;
+    if (variant == LF_VARIANT_FUSED) c->stats.fused_tiling = LF_FUSED_TILING_CLUSTERS;
     // tensor map over w as [L][N][N], box = Wc columns x R rows x 1 layer
     if (!c->w_map_valid || c->w_map_ptr != w || c->w_map_wc != pl.Wc) {
         CUtensorMap* m = reinterpret_cast<CUtensorMap*>(c->w_map_storage);
@@ -956,14 +978,14 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
 
 void lf_persistent_release(lf_ctx* c)
 {
-#ifdef LF_PK_TRACE
+#if defined(LF_PK_TRACE) || defined(LF_CK_TRACE)
     if (c->trace_dev) cudaFree(c->trace_dev);
 #else
     (void)c;
 #endif
 }
 
-#ifdef LF_PK_TRACE
+#if defined(LF_PK_TRACE) || defined(LF_CK_TRACE)
 // Debug builds: copy the SM-clock stamps of the last persistent launch to `out` (2 * L * 16 words).
 extern "C" int lf_debug_read_trace(lf_ctx* c, unsigned long long* out)
 {

@@ -1,0 +1,89 @@
+// Inline-PTX wrappers shared by the kernels of libleapfrog: shared-memory addresses, the
+// nanosecond timer that bounds every device-side wait, mbarriers, bulk tensor (TMA) loads and
+// the 8-byte {value, epoch} exchange slots of the single-launch kernels.  Device code only.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+namespace lfptx {
+
+__device__ __forceinline__ unsigned smem_u32(const void* p)
+{
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// ---- mbarriers of the CTA's own shared memory ---------------------------------------------------
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+// Arms a barrier for data written by TMA or st.async (never by the arriving thread itself), so
+// the arrive carries no release fence.
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cta.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar)
+{
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// ---- bulk tensor loads into the CTA's own shared memory (no multicast) ---------------------------
+__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap* map, unsigned bar,
+                                            int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+// ---- exchange slots: a value and the epoch of the call that wrote it, in one 64-bit word ---------
+// One 64-bit store publishes both and one 64-bit load reads both, so neither a fence nor a
+// separate flag is needed; the epoch changes with every call, so the slots are never cleared.
+__device__ __forceinline__ unsigned long long ld_slot(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_slot(unsigned long long* p, float value, unsigned epoch)
+{
+    unsigned long long v = ((unsigned long long)epoch << 32) | (unsigned long long)__float_as_uint(value);
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_stream4(float* p, float4 v)
+{
+    __stcs(reinterpret_cast<float4*>(p), v);
+}
+__device__ __forceinline__ void bar_sync(int id, int threads)   // named barrier of part of a CTA
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+}  // namespace lfptx

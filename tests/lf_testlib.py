@@ -14,7 +14,8 @@ DENORMAL = 2.0 ** -149
 
 
 def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=None,
-             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0, act=0):
+             use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0, act=0,
+             fused_tiling=0):
     """lf_forward + lf_backward on device tensors t (w,b,x,y).  Returns dict of device tensors
     and the stats of the context."""
     L, N, B = cfg["L"], cfg["N"], cfg["B"]
@@ -34,6 +35,7 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
         ctx.set_option(lf.LF_OPT_TC_TILING, tc_tiling)
         ctx.set_option(lf.LF_OPT_COST, cost)
         ctx.set_option(lf.LF_OPT_ACTIVATION, act)
+        ctx.set_option(lf.LF_OPT_FUSED_TILING, fused_tiling)
         ctx.set_option(lf.LF_OPT_USE_GRAPH, 1 if use_graph else 0)
         ctx.forward(t["w"], t["b"], t["x"], z, a)
         for _ in range(repeat):

@@ -246,13 +246,13 @@ def test_grad_w_alone_is_the_layer_slab_of_backward(L, N, B, gw_math):
         assert ctx.stats()["gw_math"] == stats["gw_math"]
 
 
-@pytest.mark.parametrize("N,k,want", [(512, 2, lf.LF_VARIANT_PERSISTENT), (768, 2, lf.LF_VARIANT_PERSISTENT),
+@pytest.mark.parametrize("N,k,want", [(512, 2, lf.LF_VARIANT_FUSED), (640, 8, lf.LF_VARIANT_FUSED), (768, 2, lf.LF_VARIANT_PERSISTENT),
                                       (768, 8, lf.LF_VARIANT_FUSED), (1024, 8, lf.LF_VARIANT_PERSISTENT),
                                       (2048, 4, lf.LF_VARIANT_PERSISTENT), (2052, 2, lf.LF_VARIANT_FUSED)])
 def test_auto_variant_follows_the_measured_table(N, k, want):
-    # LF_VARIANT_AUTO for one sample: leapfrog CTA groups at the widths (and worker counts) where
-    # they were measured faster than the fused pass, the fused pass elsewhere; the result passes
-    # parity either way.
+    # LF_VARIANT_AUTO for one sample: the fused pass with whole columns per CTA up to N = 640,
+    # leapfrog CTA groups at the widths (and worker counts) where they were measured faster than the
+    # fused pass, the fused pass elsewhere; the result passes parity either way.
     cfg = dict(L=9, N=N, B=1, k=k)
     t = _inputs(9, N, 1, seed=N)
     out, stats = gpu_pass(cfg, t)
