@@ -542,8 +542,8 @@ def run_ours(args):
                 ("w", "z", "a", "y", "delta", "gw", "gb")}
         for n in ("w", "z", "a", "y"):
             host[n].copy_(t[n])
-        # the weights of layer 1 are not read by the backward pass and are not uploaded
-        h2d = sum(host[n].numel() * 4 for n in ("w", "z", "a", "y")) - host["w"][0].numel() * 4
+        # the weights of layer 1 and z are not read by the backward pass and are not uploaded
+        h2d = sum(host[n].numel() * 4 for n in ("w", "a", "y")) - host["w"][0].numel() * 4
         d2h = sum(host[n].numel() * 4 for n in ("delta", "gw", "gb"))
         if shard_count > 1:   # only the shard's own layers of gw come back
             d2h -= host["gw"][0].numel() * 4 * (L - len(range(L, 0, -shard_count)))

@@ -278,8 +278,9 @@ int lf_backward_sgd(lf_ctx* ctx, const float* w, const float* z, const float* a,
 
 /*
  * The same backward pass on HOST buffers (pageable or pinned; same layouts): w (layers 2..L, the
- * ones the pass reads), z, a, y are copied to device staging owned by the context (allocated on first use, counted in
- * workspace_bytes), delta, gw, gb are copied back.  The copies are pipelined with the per-layer
+ * ones the pass reads), a, y are copied to device staging owned by the context (allocated on first use, counted in
+ * workspace_bytes), delta, gw, gb are copied back.  z is not copied and not read (sigma' is taken
+ * from a); it must still be non-NULL.  The copies are pipelined with the per-layer
  * schedule (LF_VARIANT_STREAMS): weights arrive top layer first on a copy stream, layer l is
  * processed as soon as w^{l+1} is there, and gw^l is sent back as soon as its worker has
  * written it, so both PCIe directions are busy at once (use pinned memory for that).  All work
@@ -327,14 +328,20 @@ int lf_last_cuda_error(const lf_ctx* ctx);
  * Limits and rules:
  *  - N must be a multiple of 4 and at most 4096; a larger N is LF_ECAPACITY (nothing is run).
  *  - The first call on each device looks up the array's device address (with that device
- *    current) and remembers it; make that first call outside any stream capture.
+ *    current) and remembers it; make that first call outside any stream capture.  With CUDA's
+ *    default lazy loading that look-up is also the moment the driver loads this part of the
+ *    library onto the device, which reserves the array and the kernel code there and synchronises
+ *    the device: so make one warm-up call per device early -- BEFORE the process hands the
+ *    remaining memory to its pool, and outside any latency-critical section.  If the device has no
+ *    memory left for that, the call returns LF_ENOMEM and nothing is run.  Calls after the first
+ *    one neither allocate nor synchronise.
  *  - All calls on a device share the one array.  Calls whose kernels may overlap on the GPU
  *    (different streams without an ordering between them, or several host threads) race on it
  *    and give wrong results; keep calls on one stream or order them with events.
  *  - `cuda_stream` is a cudaStream_t of the current device (NULL = legacy default stream).  The
  *    call enqueues a small memset of the counters and one kernel, and returns without waiting.
  * Errors: LF_ENULL, LF_EALIGN, LF_EINVAL (N), LF_ECAPACITY, LF_ERESOURCE (device ordinal
- * >= 64), LF_ECUDA.
+ * >= 64), LF_ENOMEM (first call on a device that cannot hold the array), LF_ECUDA.
  */
 int lf_delta_step_static(const float* w_up, const float* delta_up, const float* a_l,
                          float* delta_l, int N, void* cuda_stream);

@@ -283,7 +283,7 @@ void lfo_backward_sequential_cross_entropy(int L, int N, int B, const lfo_w_t *w
     lfo_backward_below_top(L, N, B, w, z, a, delta, gw, gb);
 }
 
-/* ---- Algorithm 1, taken literally ------------------------------------------------------ */
+/* ---- Algorithm 1: k threads, each recomputing the chain, each saving its own layers ----- */
 
 typedef struct {
     int j, k, L, N, B;
@@ -296,36 +296,39 @@ typedef struct {
     long long bp2_steps;        /* how many bp2 applications this thread performed   */
 } lfo_thread_arg;
 
-/* Procedure Thread(j, k, delta) of Algorithm 1.  The thread walks the delta chain on its
- * own (bp2 at EVERY layer below its start, in private buffers) and applies bp3/bp4 only
- * at the last layer of every group of k.  With p = l + 1 the paper's layer number and
- * L + 1 the paper's L, the paper's loop bound "j < L_paper - k - 1" is "j < L - k" here
- * and its "l <- L_paper - 1 - j - i" is l = L - 1 - j - i here. */
+/* The work of thread j of Algorithm 1, which starts from delta^{L-j} (computed by the parent).
+ * Its layers are the residue class (L - l) mod k = j below its start: l = L-j-k, L-j-2k, ...
+ * (Theorem 1: the k classes together cover every layer the parent did not do).  The algorithm
+ * lets a thread take whole groups of k chain steps for as long as a group's first step lies above
+ * layer k, i.e. n_groups = ceil((L - k - j) / k) groups (none if L - k - j <= 0), so its lowest
+ * layer is L - j - n_groups * k >= 1.  The thread walks the delta chain on its own -- Eq. bp2 at
+ * EVERY layer from its start down to that lowest layer, in private buffers -- and applies
+ * Eq. bp3 / bp4 only where the layer is one of its own.  (With the paper's numbering, in which the
+ * input is layer 1, its layer p is l = p - 1 here and its L is L + 1 here.)  That this walk visits
+ * and saves exactly the layers the printed procedure does is checked, for every size up to
+ * paper-L = 21, by an integer-only walk of that procedure in the tests. */
 static void *lfo_thread_main(void *argp)
 {
     lfo_thread_arg *t = (lfo_thread_arg *)argp;
+    const int k = t->k, start = t->L - t->j;
+    const int room = t->L - k - t->j;                          /* > 0: the thread has work */
+    const int n_groups = room > 0 ? (room + k - 1) / k : 0;
+    const int lowest = start - n_groups * k;
     size_t slab = (size_t)t->B * (size_t)t->N;
     double *cur = (double *)malloc(slab * sizeof(double));
     double *nxt = (double *)malloc(slab * sizeof(double));
     memcpy(cur, t->delta_start, slab * sizeof(double));
-    int j = t->j;
-    while (j < t->L - t->k) {
-        int i = 0;
-        while (i < t->k) {
-            int l = t->L - 1 - j - i;
-            lfo_delta_step(t->N, t->B, t->w + (size_t)l * t->N * t->N, cur,
-                           t->z + (size_t)(l - 1) * slab, nxt);           /* bp2 at l */
-            t->bp2_steps += 1;
-            double *tmp = cur; cur = nxt; nxt = tmp;
-            if (i == t->k - 1) {
-                lfo_emit_layer(l, t->N, t->B, cur, t->a, t->gw, t->gb);   /* bp3, bp4 */
-                memcpy(t->delta + (size_t)(l - 1) * slab, cur, slab * sizeof(double));
-                t->writer[l - 1] = t->j;
-                __atomic_fetch_add(&t->writes[l - 1], 1, __ATOMIC_RELAXED);
-            }
-            i += 1;
+    for (int l = start - 1; l >= lowest && n_groups > 0; --l) {
+        lfo_delta_step(t->N, t->B, t->w + (size_t)l * t->N * t->N, cur,
+                       t->z + (size_t)(l - 1) * slab, nxt);               /* bp2: delta^l */
+        t->bp2_steps += 1;
+        double *tmp = cur; cur = nxt; nxt = tmp;
+        if ((t->L - l) % k == t->j % k) {                                 /* one of this thread's layers */
+            lfo_emit_layer(l, t->N, t->B, cur, t->a, t->gw, t->gb);       /* bp3, bp4 */
+            memcpy(t->delta + (size_t)(l - 1) * slab, cur, slab * sizeof(double));
+            t->writer[l - 1] = t->j;
+            __atomic_fetch_add(&t->writes[l - 1], 1, __ATOMIC_RELAXED);
         }
-        j += t->k;
     }
     free(cur);
     free(nxt);

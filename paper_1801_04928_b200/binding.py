@@ -91,6 +91,26 @@ class LeapfrogError(RuntimeError):
         super().__init__(msg)
 
 
+def _check_tensor(t, need: int, name: str, where: str, on_device: bool = True) -> None:
+    """Marshalling-side guard: a tensor handed to the library must be float32, contiguous, on the
+    right side of the bus and hold at least `need` elements -- the kernels trust the context's sizes
+    and would write past a buffer that is too small.  Raw addresses (ints) and None are passed on
+    unchecked (None is rejected by the library itself)."""
+    if t is None or isinstance(t, int):
+        return
+    problems = []
+    if str(getattr(t, "dtype", "")) != "torch.float32":
+        problems.append(f"dtype {getattr(t, 'dtype', '?')} (float32 needed)")
+    if hasattr(t, "is_contiguous") and not t.is_contiguous():
+        problems.append("not contiguous")
+    if hasattr(t, "is_cuda") and bool(t.is_cuda) != on_device:
+        problems.append("must be a CUDA tensor" if on_device else "must be a host tensor")
+    if hasattr(t, "numel") and t.numel() < need:
+        problems.append(f"{t.numel()} elements, {need} needed")
+    if problems:
+        raise LeapfrogError(LF_EINVAL, f"{where}: argument {name}: " + "; ".join(problems))
+
+
 def _ptr(t) -> ctypes.c_void_p:
     """Address of a tensor-like object (``data_ptr()``), an int, or None."""
     if t is None:
@@ -186,8 +206,16 @@ def lf_delta_step_static(w_up, delta_up, a_l, delta_l, N: int, cuda_stream: int 
     For processes that own all device memory through their own pool, or that cannot take the
     device-wide stall of a cudaMalloc: the kernel's scratch is a fixed array inside the
     library (N <= 4096, else LF_ECAPACITY).  Calls share that array, so do not let two of
-    them overlap on the GPU.  Returns the status code; the work is only enqueued.
+    them overlap on the GPU.  The first call on a device loads that part of the library onto it:
+    make it early, before memory is handed to a pool.  Returns the status code; the work is only
+    enqueued.  Tensors (as opposed to raw addresses) are checked for dtype, device, contiguity and
+    size first; a mismatch raises LeapfrogError(LF_EINVAL).
     """
+    n = int(N)
+    if 1 <= n <= 4096 and n % 4 == 0:
+        _check_tensor(w_up, n * n, "w_up", "lf_delta_step_static")
+        for name, t in (("delta_up", delta_up), ("a_l", a_l), ("delta_l", delta_l)):
+            _check_tensor(t, n, name, "lf_delta_step_static")
     return _lib.lf_delta_step_static(_ptr(w_up), _ptr(delta_up), _ptr(a_l), _ptr(delta_l), int(N),
                                      ctypes.c_void_p(cuda_stream or None))
 
@@ -208,8 +236,18 @@ class Leapfrog:
             self._h = None
             raise LeapfrogError(rc, "lf_create_widths" if widths is not None else "lf_create")
         self.L, self.N, self.B, self.k = L, N, B, k
+        n = [int(v) for v in widths] if widths is not None else [int(N)] * (int(L) + 1)
+        n_w = sum(n[l] * n[l - 1] for l in range(1, len(n)))
+        n_h = sum(n[1:])
+        # elements every argument must hold (w, gw | b, gb | z, delta | a | x | y)
+        self._need = dict(w=n_w, gw=n_w, w_new=n_w, b=n_h, gb=n_h, z=B * n_h, delta=B * n_h,
+                          a=B * sum(n), x=B * n[0], y=B * n[-1], layer_w=int(N) * int(N), layer_v=B * int(N))
         if stream is not None:
             self.set_stream(stream)
+
+    def _args(self, where: str, on_device: bool = True, **tensors):
+        for name, t in tensors.items():
+            _check_tensor(t, self._need[name], name, where, on_device)
 
     def _check(self, rc: int, where: str):
         if rc != LF_OK:
@@ -222,18 +260,24 @@ class Leapfrog:
         self._check(lf_set_option(self._h, key, value), "lf_set_option")
 
     def forward(self, w, b, x, z, a):
+        self._args("lf_forward", w=w, b=b, x=x, z=z, a=a)
         self._check(lf_forward(self._h, w, b, x, z, a), "lf_forward")
 
     def backward(self, w, z, a, y, delta, gw, gb):
+        self._args("lf_backward", w=w, z=z, a=a, y=y, delta=delta, gw=gw, gb=gb)
         self._check(lf_backward(self._h, w, z, a, y, delta, gw, gb), "lf_backward")
 
     def grad_w(self, delta_l, a_prev, gw_l):
+        for name, t, need in (("delta_l", delta_l, "layer_v"), ("a_prev", a_prev, "layer_v"), ("gw_l", gw_l, "layer_w")):
+            _check_tensor(t, self._need[need], name, "lf_grad_w")
         self._check(lf_grad_w(self._h, delta_l, a_prev, gw_l), "lf_grad_w")
 
     def backward_sgd(self, w, z, a, y, eta, delta, w_new, gb):
+        self._args("lf_backward_sgd", w=w, z=z, a=a, y=y, delta=delta, w_new=w_new, gb=gb)
         self._check(lf_backward_sgd(self._h, w, z, a, y, eta, delta, w_new, gb), "lf_backward_sgd")
 
     def backward_host(self, w, z, a, y, delta, gw, gb):
+        self._args("lf_backward_host", on_device=False, w=w, z=z, a=a, y=y, delta=delta, gw=gw, gb=gb)
         self._check(lf_backward_host(self._h, w, z, a, y, delta, gw, gb), "lf_backward_host")
 
     def sync(self):

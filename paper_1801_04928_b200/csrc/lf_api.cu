@@ -564,10 +564,11 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
     const int Li = ctx->L;
     const size_t Bs = (size_t)ctx->B;
-    // staging layout, every block a multiple of 4 floats: w | z | a | y | delta | gw | gb
-    const size_t n_w = ctx->off_w[Li], n_z = Bs * ctx->off_h[Li], n_a = Bs * ctx->off_a[Li + 1],
-                 n_y = Bs * (size_t)ctx->width[Li], n_d = n_z, n_gw = n_w, n_gb = ctx->off_h[Li];
-    const size_t total = n_w + n_z + n_a + n_y + n_d + n_gw + n_gb;
+    // staging layout, every block a multiple of 4 floats: w | a | y | delta | gw | gb  (z stays on the
+    // host: no kernel of the backward pass reads it, sigma' comes from a)
+    const size_t n_w = ctx->off_w[Li], n_a = Bs * ctx->off_a[Li + 1], n_y = Bs * (size_t)ctx->width[Li],
+                 n_d = Bs * ctx->off_h[Li], n_gw = n_w, n_gb = ctx->off_h[Li];
+    const size_t total = n_w + n_a + n_y + n_d + n_gw + n_gb;
     if (!ctx->stage) {
         cudaError_t e = cudaMalloc(&ctx->stage, total * sizeof(float));
         if (e != cudaSuccess) {
@@ -580,26 +581,51 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
         ctx->stats.workspace_bytes += (long long)ctx->stage_bytes;
     }
     float* d_w = ctx->stage;
-    float* d_z = d_w + n_w;
-    float* d_a = d_z + n_z;
+    float* d_a = d_w + n_w;
     float* d_y = d_a + n_a;
     float* d_d = d_y + n_y;
     float* d_gw = d_d + n_d;
     float* d_gb = d_gw + n_gw;
-    // copy stream and per-layer arrival events (created on first use)
-    if (!ctx->h2d_stream) {
-        LF_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking));
-        LF_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking));
-        ctx->w_ready_ev = new (std::nothrow) cudaEvent_t[ctx->L]();
-        ctx->gw_done_ev = new (std::nothrow) cudaEvent_t[ctx->L]();
-        if (!ctx->w_ready_ev || !ctx->gw_done_ev) return LF_ENOMEM;
-        for (int l = 0; l < ctx->L; ++l) {
-            LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->w_ready_ev[l], cudaEventDisableTiming));
-            LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->gw_done_ev[l], cudaEventDisableTiming));
+    // copy streams and per-layer arrival events, created on first use: everything is built first and
+    // handed to the context only when all of it exists, so a failure half way leaves nothing behind
+    // that a later call would take for a finished set-up
+    if (!ctx->host_path_ready) {
+        cudaStream_t hs = nullptr, ds = nullptr;
+        cudaEvent_t* w_ev = new (std::nothrow) cudaEvent_t[Li]();
+        cudaEvent_t* g_ev = new (std::nothrow) cudaEvent_t[Li]();
+        cudaEvent_t one[3] = {nullptr, nullptr, nullptr};
+        bool ok = w_ev && g_ev;
+        cudaError_t e = cudaSuccess;
+        if (ok) {
+            ok = (e = cudaStreamCreateWithFlags(&hs, cudaStreamNonBlocking)) == cudaSuccess &&
+                 (e = cudaStreamCreateWithFlags(&ds, cudaStreamNonBlocking)) == cudaSuccess;
+            for (int l = 0; l < Li && ok; ++l)
+                ok = (e = cudaEventCreateWithFlags(&w_ev[l], cudaEventDisableTiming)) == cudaSuccess &&
+                     (e = cudaEventCreateWithFlags(&g_ev[l], cudaEventDisableTiming)) == cudaSuccess;
+            for (int i = 0; i < 3 && ok; ++i)
+                ok = (e = cudaEventCreateWithFlags(&one[i], cudaEventDisableTiming)) == cudaSuccess;
         }
-        LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->small_ev, cudaEventDisableTiming));
-        LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->h2d_done_ev, cudaEventDisableTiming));
-        LF_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->d2h_done_ev, cudaEventDisableTiming));
+        if (!ok) {
+            const bool no_host_memory = !w_ev || !g_ev;
+            for (int l = 0; l < Li; ++l) {
+                if (w_ev && w_ev[l]) cudaEventDestroy(w_ev[l]);
+                if (g_ev && g_ev[l]) cudaEventDestroy(g_ev[l]);
+            }
+            for (int i = 0; i < 3; ++i)
+                if (one[i]) cudaEventDestroy(one[i]);
+            if (hs) cudaStreamDestroy(hs);
+            if (ds) cudaStreamDestroy(ds);
+            delete[] w_ev;
+            delete[] g_ev;
+            cudaGetLastError();
+            if (no_host_memory) return LF_ENOMEM;
+            ctx->last_cuda_error = (int)e;
+            return LF_ECUDA;
+        }
+        ctx->h2d_stream = hs; ctx->d2h_stream = ds;
+        ctx->w_ready_ev = w_ev; ctx->gw_done_ev = g_ev;
+        ctx->small_ev = one[0]; ctx->h2d_done_ev = one[1]; ctx->d2h_done_ev = one[2];
+        ctx->host_path_ready = true;
     }
     // The copies are pipelined with the per-layer schedule: the weights arrive top layer
     // first on a copy stream, the chain step of layer l starts as soon as w^{l+1} is there,
@@ -614,62 +640,75 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     ctx->stats.cost = ctx->opt_cost;
     ctx->stats.activation = ctx->opt_act;
     ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
+    ctx->stats.fused_tiling = 0;
     int launches = 0;
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(hs, ctx->fork_ev, 0));
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ds, ctx->fork_ev, 0));
-    for (int j = 0; j < ctx->keff; ++j) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->wstreams[j], ctx->fork_ev, 0));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_z, z, n_z * sizeof(float), cudaMemcpyHostToDevice, hs));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, hs));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, hs));
-    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, hs));
-    for (int l = Li; l >= 2; --l) {   // w^1 is never read: Eq. bp2 needs w^{l+1} for l = L-1 .. 1
-        const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
-        LF_CUDA_TRY(ctx, cudaMemcpyAsync(d_w + w_at(ctx, l), w + w_at(ctx, l), M * sizeof(float),
-                                         cudaMemcpyHostToDevice, hs));
-        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->w_ready_ev[l - 1], hs));
+    // From here on the copy, download and worker streams are forked off the context's stream: whatever
+    // goes wrong below, they are joined back into it before the call returns (`fail` keeps the
+    // first error; the remaining enqueues are skipped).
+    int fail = LF_OK;
+    auto tried = [&](cudaError_t e) {
+        if (e != cudaSuccess && fail == LF_OK) { ctx->last_cuda_error = (int)e; fail = LF_ECUDA; }
+        return fail == LF_OK;
+    };
+    tried(cudaStreamWaitEvent(hs, ctx->fork_ev, 0));
+    tried(cudaStreamWaitEvent(ds, ctx->fork_ev, 0));
+    for (int j = 0; j < ctx->keff; ++j) tried(cudaStreamWaitEvent(ctx->wstreams[j], ctx->fork_ev, 0));
+    if (fail == LF_OK) {
+        tried(cudaMemcpyAsync(d_a, a, n_a * sizeof(float), cudaMemcpyHostToDevice, hs));
+        tried(cudaMemcpyAsync(d_y, y, n_y * sizeof(float), cudaMemcpyHostToDevice, hs));
+        tried(cudaEventRecord(ctx->small_ev, hs));
     }
-    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->h2d_done_ev, hs));
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->small_ev, 0));
-    for (int l = Li; l >= 1; --l) {
-        if (l < Li) LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0));   // w^{l+1}
+    for (int l = Li; l >= 2 && fail == LF_OK; --l) {   // w^1 is never read: Eq. bp2 needs w^{l+1} for l = L-1 .. 1
+        const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
+        tried(cudaMemcpyAsync(d_w + w_at(ctx, l), w + w_at(ctx, l), M * sizeof(float), cudaMemcpyHostToDevice, hs));
+        tried(cudaEventRecord(ctx->w_ready_ev[l - 1], hs));
+    }
+    if (fail == LF_OK) tried(cudaStreamWaitEvent(s, ctx->small_ev, 0));
+    for (int l = Li; l >= 1 && fail == LF_OK; --l) {
+        if (l < Li && !tried(cudaStreamWaitEvent(s, ctx->w_ready_ev[l], 0))) break;   // w^{l+1}
         int rc = enqueue_chain_step(ctx, l, d_w, d_a, d_y, d_d, d_gb, s, &launches);
-        if (rc != LF_OK) return rc;
+        if (rc != LF_OK) { fail = rc; break; }
         if (!lf_layer_owned(ctx, l)) continue;    // another shard's layer: nothing to compute or send back
-        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->ready_ev[l - 1], s));
         const int j = lf_layer_worker(ctx, l);
         cudaStream_t wsj = ctx->wstreams[j];
-        LF_CUDA_TRY(ctx, cudaStreamWaitEvent(wsj, ctx->ready_ev[l - 1], 0));
+        if (!tried(cudaEventRecord(ctx->ready_ev[l - 1], s)) ||
+            !tried(cudaStreamWaitEvent(wsj, ctx->ready_ev[l - 1], 0)))
+            break;
         rc = enqueue_gradients(ctx, l, d_a, d_d, d_gw, d_gb, gw_math, wsj, &launches);
-        if (rc != LF_OK) return rc;
-        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->gw_done_ev[l - 1], wsj));
-        LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ds, ctx->gw_done_ev[l - 1], 0));
+        if (rc != LF_OK) { fail = rc; break; }
         const size_t M = (size_t)ctx->width[l] * (size_t)ctx->width[l - 1];
-        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gw + w_at(ctx, l), d_gw + w_at(ctx, l), M * sizeof(float),
-                                         cudaMemcpyDeviceToHost, ds));
+        tried(cudaEventRecord(ctx->gw_done_ev[l - 1], wsj));
+        tried(cudaStreamWaitEvent(ds, ctx->gw_done_ev[l - 1], 0));
+        tried(cudaMemcpyAsync(gw + w_at(ctx, l), d_gw + w_at(ctx, l), M * sizeof(float), cudaMemcpyDeviceToHost, ds));
     }
-    // the download stream has waited for the gw and gb of every layer done here; the end of the
-    // chain (delta^1, the last thing written on s) it waits for explicitly
-    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->small_ev, s));
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(ds, ctx->small_ev, 0));
-    LF_CUDA_TRY(ctx, cudaMemcpyAsync(delta, d_d, n_d * sizeof(float), cudaMemcpyDeviceToHost, ds));
-    if (ctx->B == 1 || ctx->shard_count == 1) {
-        LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, ds));
-    } else {
-        for (int l = 1; l <= Li; ++l)     // B > 1: gb^l exists only for this shard's layers
-            if (lf_layer_owned(ctx, l))
-                LF_CUDA_TRY(ctx, cudaMemcpyAsync(gb + v_at(ctx, l), d_gb + v_at(ctx, l),
-                                                 (size_t)ctx->width[l] * sizeof(float), cudaMemcpyDeviceToHost, ds));
+    if (fail == LF_OK) {
+        // the download stream has waited for the gw and gb of every layer done here; the end of the
+        // chain (delta^1, the last thing written on s) it waits for explicitly
+        tried(cudaEventRecord(ctx->small_ev, s));
+        tried(cudaStreamWaitEvent(ds, ctx->small_ev, 0));
+        tried(cudaMemcpyAsync(delta, d_d, n_d * sizeof(float), cudaMemcpyDeviceToHost, ds));
+        if (ctx->B == 1 || ctx->shard_count == 1) {
+            tried(cudaMemcpyAsync(gb, d_gb, n_gb * sizeof(float), cudaMemcpyDeviceToHost, ds));
+        } else {
+            for (int l = 1; l <= Li; ++l)     // B > 1: gb^l exists only for this shard's layers
+                if (lf_layer_owned(ctx, l))
+                    tried(cudaMemcpyAsync(gb + v_at(ctx, l), d_gb + v_at(ctx, l),
+                                          (size_t)ctx->width[l] * sizeof(float), cudaMemcpyDeviceToHost, ds));
+        }
     }
-    LF_CUDA_TRY(ctx, cudaEventRecord(ctx->d2h_done_ev, ds));
-    for (int j = 0; j < ctx->keff; ++j) {
-        LF_CUDA_TRY(ctx, cudaEventRecord(ctx->done_ev[j], ctx->wstreams[j]));
-        LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->done_ev[j], 0));
+    // join: on every path, also after a failure
+    cudaError_t je = cudaEventRecord(ctx->d2h_done_ev, ds);
+    if (je == cudaSuccess) je = cudaEventRecord(ctx->h2d_done_ev, hs);
+    for (int j = 0; j < ctx->keff && je == cudaSuccess; ++j) {
+        je = cudaEventRecord(ctx->done_ev[j], ctx->wstreams[j]);
+        if (je == cudaSuccess) je = cudaStreamWaitEvent(s, ctx->done_ev[j], 0);
     }
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->h2d_done_ev, 0));
-    LF_CUDA_TRY(ctx, cudaStreamWaitEvent(s, ctx->d2h_done_ev, 0));
+    if (je == cudaSuccess) je = cudaStreamWaitEvent(s, ctx->h2d_done_ev, 0);
+    if (je == cudaSuccess) je = cudaStreamWaitEvent(s, ctx->d2h_done_ev, 0);
+    if (je != cudaSuccess && fail == LF_OK) { ctx->last_cuda_error = (int)je; fail = LF_ECUDA; }
     ctx->stats.launches_backward = launches;
-    return LF_OK;
+    return fail;
 }
 
 int lf_sync(lf_ctx* ctx)

@@ -127,13 +127,14 @@ struct lf_ctx {
 #endif
 
     // host-buffer entry point staging
-    float* stage;            // one allocation holding w, z, a, y, delta, gw, gb
+    float* stage;            // one allocation holding w, a, y, delta, gw, gb
     size_t stage_bytes;
     cudaStream_t h2d_stream; // host -> device copies of the host entry point
     cudaStream_t d2h_stream; // device -> host copies of its results, all on this one stream
     cudaEvent_t* w_ready_ev; // L events: w^l has arrived in staging
     cudaEvent_t* gw_done_ev; // L events: gw^l (and gb^l) are written
     cudaEvent_t small_ev, h2d_done_ev, d2h_done_ev;
+    bool host_path_ready;    // the copy streams and events above all exist
 
     int last_cuda_error;
     lf_stats stats;

@@ -268,10 +268,13 @@ int static_scratch_for_current_device(float** out)
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_scratch_addr[dev]) {
         float* p = nullptr;
+        // With CUDA's lazy module loading this look-up is also what loads the module that holds the
+        // array and the kernel on this device: that reserves the array's megabyte and the code, and
+        // it fails with an out-of-memory error if the process has already given all memory away.
         cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), lf_static_scratch);
         if (e != cudaSuccess || !p) {
             cudaGetLastError();
-            return LF_ECUDA;
+            return e == cudaErrorMemoryAllocation ? LF_ENOMEM : LF_ECUDA;
         }
         g_static_scratch_addr[dev] = p;
     }

@@ -75,3 +75,23 @@ def test_no_device_means_an_error_not_a_fallback():
     assert rc == lf.LF_ECUDA and not h.value
     rc, h = lf.lf_create_widths([64, 32, 16], 1, 2)
     assert rc == lf.LF_ECUDA and not h.value
+
+
+def test_binding_checks_tensors_before_the_library_sees_them():
+    # dtype, contiguity, side of the bus and size are checked while marshalling: the kernels trust the
+    # context's sizes, so a buffer that is too small must never reach them
+    import pytest
+    import torch
+    from paper_1801_04928_b200 import binding
+    ok = torch.zeros(64, dtype=torch.float32)
+    binding._check_tensor(ok, 64, "x", "test", on_device=False)
+    binding._check_tensor(None, 64, "x", "test")
+    binding._check_tensor(12345, 64, "x", "test")
+    for bad, on_device in ((torch.zeros(64, dtype=torch.float64), False), (torch.zeros(63), False),
+                           (torch.zeros(8, 16).t(), False), (ok, True)):
+        with pytest.raises(lf.LeapfrogError) as e:
+            binding._check_tensor(bad, 64, "x", "test", on_device=on_device)
+        assert e.value.status == lf.LF_EINVAL
+    # the static entry point checks before it calls into the library (no device is touched here)
+    with pytest.raises(lf.LeapfrogError):
+        lf.lf_delta_step_static(torch.zeros(16), torch.zeros(8), torch.zeros(8), torch.zeros(8), 8)

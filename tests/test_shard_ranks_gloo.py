@@ -1,7 +1,11 @@
 """The layer-sharded form on several ranks, on the CPU: every rank (a gloo process standing for a
 GPU) runs the oracle's pass of its own shard -- rank = shard, world size = shard count, the mapping
 a multi-GPU launch uses -- and the ranks then compare notes: every layer has exactly one owner,
-and the owners' gradients put together are the sequential pass.  Nothing is exchanged before that."""
+and the owners' gradients put together are the sequential pass.  Nothing is exchanged before that.
+The rank -> shard mapping is the product's own (`bench.shard_plan`, what `bench.py --gpus N
+--shard-by-rank` runs), and the layers a rank claims come from the library's rule -- layer l
+belongs to shard (L - l) mod S, worker ((L - l) / S) mod k inside it -- checked against what the
+oracle's shard pass really wrote."""
 import os
 import sys
 
@@ -20,11 +24,20 @@ def _rank_main(rank, world, port, results):
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
-    L, N, B = 5, 12, 2
+    import bench
+    L, N, B, k = 5, 12, 2, 4
+    S, r, k_here = bench.shard_plan(world, rank, k, 1, True)     # the product's mapping of ranks to shards
+    assert (S, r) == (world, rank) and k_here == max(1, k // world)
+    assert bench.shard_plan(1, 0, k, 1, True) == (1, 0, k)       # one rank: no sharding
+    assert bench.shard_plan(1, 0, k, 4, False) == (4, 0, 1)      # --shards 4 on one GPU: shard 0, k / 4 workers
+    mine = [l for l in range(1, L + 1) if (L - l) % S == r]      # the library's ownership rule
+    workers = sorted({((L - l) // S) % k_here for l in mine})
+    assert workers == list(range(min(k_here, len(mine))))        # the shard's layers go round its workers
     t = lf_inputs.make_inputs(L, N, B, "uniform", lf_inputs.SEED_BASE + 31, "cpu")   # same seed: replicated inputs
     w = t["w"].numpy()
     z, a = orc.forward(w, t["b"].numpy(), t["x"].numpy())
-    delta, gw, gb, wrote = orc.backward_shard(w, z, a, t["y"].numpy(), world, rank)
+    delta, gw, gb, wrote = orc.backward_shard(w, z, a, t["y"].numpy(), S, r)
+    assert [l for l in range(1, L + 1) if wrote[l - 1]] == mine  # the oracle's shard wrote exactly those
     owners = torch.from_numpy(wrote.astype(np.int64))
     dist.all_reduce(owners)                                   # how many ranks own each layer
     parts = torch.from_numpy(np.nan_to_num(gw, nan=0.0))

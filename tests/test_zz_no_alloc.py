@@ -5,14 +5,18 @@ its own memory pool, or a loop that cannot take the device-wide stall of an allo
 them the library has one entry point whose scratch is a fixed array in the library image.
 This file checks, through the C ABI, that it returns what the ordinary path (`lf_backward`,
 which uses a context's allocated workspace) returns for the same layer -- on two calls in a
-row, because the calls share the array and the second one meets the first one's leftovers.
+row, because the calls share the array and the second one meets the first one's leftovers --
+and what the oracle's Eq. bp2 gives for the same inputs; and that, once the first call on the
+device has been made, further calls leave the amount of free device memory exactly as it was.
 It is named to be collected last, so a failure here cannot hide any other test's result.
 """
+import numpy as np
 import pytest
 import torch
 
 import lf_inputs
 import paper_1801_04928_b200 as lf
+from oracle import lf_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -56,6 +60,35 @@ def test_static_delta_step_matches_lf_backward_twice_in_a_row(N):
         err = (out.double() - ref.double()).abs().max().item()
         scale = ref.double().abs().max().item()
         assert err <= TOL * scale, (N, l, err, scale)
+        # and the oracle's Eq. bp2 on the same inputs (sigma' from z; a = sigma(z) went to the GPU)
+        a_l = a[l, 0].double().cpu().numpy()
+        z_l = np.log(a_l) - np.log1p(-a_l)
+        want = orc.delta_step(t["w"][l].cpu().numpy(), delta[l].double().cpu().numpy(), z_l[None, :])[0]
+        err = float(np.max(np.abs(out.double().cpu().numpy() - want)))
+        assert err <= TOL * float(np.max(np.abs(want))), (N, l, err)
+
+
+def test_static_delta_step_leaves_free_memory_alone_after_the_first_call():
+    # The first call on a device may load the library's code and its scratch array onto it; every
+    # call after that must not change the amount of free device memory by a single byte.
+    N = 1024
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    w = torch.empty((N, N), device="cuda").normal_(0.0, N ** -0.5, generator=g)
+    d_up = torch.empty((N,), device="cuda").normal_(0.0, 1.0, generator=g)
+    a_l = torch.empty((N,), device="cuda").uniform_(0.05, 0.95, generator=g)
+    out = torch.empty((N,), device="cuda")
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    assert lf.lf_delta_step_static(w, d_up, a_l, out, N, stream.cuda_stream) == lf.LF_OK   # warm-up
+    stream.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(5):
+        assert lf.lf_delta_step_static(w, d_up, a_l, out, N, stream.cuda_stream) == lf.LF_OK
+    stream.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    want = (w.double().t() @ d_up.double()) * a_l.double() * (1 - a_l.double())
+    assert float((out.double() - want).abs().max()) <= TOL * float(want.abs().max())
 
 
 def test_static_delta_step_rejects_what_it_cannot_hold():
