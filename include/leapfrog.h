@@ -113,6 +113,20 @@ enum lf_activation {
     LF_ACT_RELU = 2     /* sigma(t) = max(t, 0),          sigma' = [a > 0]  (0 where t <= 0)       */
 };
 
+/*
+ * LF_OPT_SHARD_COUNT = S > 1 and LF_OPT_SHARD_RANK = r (in the enum below) select the
+ * layer-sharded form.  The paper offers its schedule for "k threads or k gpus": with S GPUs every GPU holds w, z, a, runs the whole delta
+ * chain for itself, and does Eq. bp4 (and, for B > 1, Eq. bp3) only for the layers it owns,
+ *     layer l belongs to shard (L - l) mod S,
+ * so that nothing is exchanged during the pass and the gradients end up distributed by owner.
+ * A context with S > 1 writes delta completely (and gb for B = 1, where it is delta), and gw^l
+ * (gb^l for B > 1; w_new^l in lf_backward_sgd) only for its own layers; the other layers' blocks
+ * of those arrays are not touched.  Inside the shard the k leapfrog workers share the shard's
+ * layers in turn: worker ((L - l) / S) mod k.  The S contexts are independent: one per GPU, or
+ * several on one GPU writing into one gw array, give together exactly what one unsharded
+ * context writes.  Every variant takes a sharded context (the fused pass skips the stores of
+ * other shards' tiles).
+ */
 enum lf_option {
     LF_OPT_VARIANT = 1,       /* enum lf_variant                                              */
     LF_OPT_GW_MATH = 2,       /* enum lf_gw_math                                              */
@@ -126,9 +140,12 @@ enum lf_option {
                                  LF_COST_CROSS_ENTROPY needs the sigmoid: lf_backward returns
                                  LF_EINVAL for any other pairing                              */
     LF_OPT_SHARD_COUNT = 10,  /* S >= 1 (default 1): the paper's "k gpus" form (Section 1), see
-                                 below; setting it puts the rank back to 0                    */
+                                 above; setting it puts the rank back to 0                    */
     LF_OPT_SHARD_RANK = 11,   /* r, 0 <= r < S: which of the S shards this context is         */
     LF_OPT_FUSED_TILING = 12, /* enum lf_fused_tiling                                         */
+    LF_OPT_TIME_CALLS = 13,   /* 0/1 (default 0): bracket every backward call with two events on
+                                 the context's stream; lf_sync then puts the elapsed device time
+                                 of the last one into lf_stats.last_backward_ms                 */
     LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
                                  publish its share of delta, so the bounded waits of the others
                                  expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
@@ -156,6 +173,10 @@ typedef struct lf_stats {
     int shard_count;
     int fused_tiling;         /* tiling of the last fused single-launch pass (enum lf_fused_tiling,
                                  CLUSTERS or COLUMNS; 0 if the last pass was not a fused one)     */
+    float last_backward_ms;   /* device time of the last lf_backward / lf_backward_sgd /
+                                 lf_backward_host between two events on the context's stream, as
+                                 of the last lf_sync (0 before the first; filled only while
+                                 LF_OPT_TIME_CALLS is on)                                         */
 } lf_stats;
 
 /*
@@ -207,20 +228,6 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k);
  */
 int lf_set_stream(lf_ctx* ctx, void* cuda_stream);
 
-/*
- * Layer-sharded form (LF_OPT_SHARD_COUNT = S > 1, LF_OPT_SHARD_RANK = r).  The paper offers its
- * schedule for "k threads or k gpus": with S GPUs every GPU holds w, z, a, runs the whole delta
- * chain for itself, and does Eq. bp4 (and, for B > 1, Eq. bp3) only for the layers it owns,
- *     layer l belongs to shard (L - l) mod S,
- * so that nothing is exchanged during the pass and the gradients end up distributed by owner.
- * A context with S > 1 writes delta completely (and gb for B = 1, where it is delta), and gw^l
- * (gb^l for B > 1; w_new^l in lf_backward_sgd) only for its own layers; the other layers' blocks
- * of those arrays are not touched.  Inside the shard the k leapfrog workers share the shard's
- * layers in turn: worker ((L - l) / S) mod k.  The S contexts are independent: one per GPU, or
- * several on one GPU writing into one gw array, give together exactly what one unsharded
- * context writes.  Every variant takes a sharded context (the fused pass skips the stores of
- * other shards' tiles).
- */
 /* Set an option (enum lf_option).  LF_EINVAL for unknown keys or out-of-range values. */
 int lf_set_option(lf_ctx* ctx, int key, long long value);
 

@@ -25,6 +25,7 @@ LF_OPT_COST = 8
 LF_OPT_ACTIVATION = 9
 LF_OPT_SHARD_COUNT, LF_OPT_SHARD_RANK = 10, 11
 LF_OPT_FUSED_TILING = 12
+LF_OPT_TIME_CALLS = 13
 LF_FUSED_TILING_AUTO, LF_FUSED_TILING_CLUSTERS, LF_FUSED_TILING_COLUMNS = 0, 1, 2
 LF_ACT_SIGMOID, LF_ACT_TANH, LF_ACT_RELU = 0, 1, 2
 LF_COST_QUADRATIC, LF_COST_CROSS_ENTROPY = 0, 1
@@ -45,7 +46,7 @@ class lf_stats(ctypes.Structure):
                 ("device_status", ctypes.c_uint), ("workspace_bytes", ctypes.c_longlong),
                 ("delta_math", ctypes.c_int), ("gw_tiling", ctypes.c_int), ("delta_tiling", ctypes.c_int), ("cost", ctypes.c_int), ("activation", ctypes.c_int),
                 ("shard_rank", ctypes.c_int), ("shard_count", ctypes.c_int),
-                ("fused_tiling", ctypes.c_int)]
+                ("fused_tiling", ctypes.c_int), ("last_backward_ms", ctypes.c_float)]
 
 
 def _load() -> ctypes.CDLL:

@@ -445,6 +445,19 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             if (value < LF_FUSED_TILING_AUTO || value > LF_FUSED_TILING_COLUMNS) return LF_EINVAL;
             ctx->opt_fused_tiling = (int)value;
             return LF_OK;
+        case LF_OPT_TIME_CALLS:
+            if (value != 0 && value != 1) return LF_EINVAL;
+            if (value && !ctx->t_begin_ev) {
+                cudaEvent_t b = nullptr, e = nullptr;
+                if (cudaEventCreate(&b) != cudaSuccess || cudaEventCreate(&e) != cudaSuccess) {
+                    if (b) cudaEventDestroy(b);
+                    ctx->last_cuda_error = (int)cudaGetLastError();
+                    return LF_ECUDA;
+                }
+                ctx->t_begin_ev = b; ctx->t_end_ev = e;
+            }
+            ctx->time_calls = (int)value;
+            return LF_OK;
         case LF_OPT_WITHHOLD:
             if (value != 0 && value != 1) return LF_EINVAL;
             ctx->withhold = (int)value;
@@ -492,14 +505,30 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
     return LF_OK;
 }
 
-int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
-                float* delta, float* gw, float* gb)
+// LF_OPT_TIME_CALLS: events around a backward call on the context's stream (not during a capture
+// the caller may have open on it: an event recorded there could not be read back).
+struct call_timer {
+    lf_ctx* c;
+    bool on;
+    explicit call_timer(lf_ctx* ctx) : c(ctx), on(false)
+    {
+        if (!c->time_calls || !c->t_begin_ev) return;
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(c->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+            cudaGetLastError();
+            return;
+        }
+        on = cudaEventRecord(c->t_begin_ev, c->stream) == cudaSuccess;
+    }
+    void done(int rc)
+    {
+        if (on && rc == LF_OK && cudaEventRecord(c->t_end_ev, c->stream) == cudaSuccess) c->timed_call_pending = true;
+    }
+};
+
+static int backward_impl(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                         float* delta, float* gw, float* gb)
 {
-    if (!ctx) return LF_ENULL;
-    const void* ps[] = {w, z, a, y, delta, gw, gb};
-    int rc = check_ptrs(ps, 7);
-    if (rc != LF_OK) return rc;
-    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
     int variant = resolve_variant(ctx);
     const int gw_math = resolve_gw_math(ctx);
     if (variant != LF_VARIANT_STREAMS && !lf_persistent_supported(ctx, variant))
@@ -516,6 +545,20 @@ int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, con
     if (ctx->uniform)
         return lf_backward_persistent(ctx, variant, w, a, y, delta, gw, gb, ctx->sgd_w, 0, 0);
     return backward_hidden_run(ctx, variant, w, a, y, delta, gw, gb, gw_math);
+}
+
+int lf_backward(lf_ctx* ctx, const float* w, const float* z, const float* a, const float* y,
+                float* delta, float* gw, float* gb)
+{
+    if (!ctx) return LF_ENULL;
+    const void* ps[] = {w, z, a, y, delta, gw, gb};
+    int rc = check_ptrs(ps, 7);
+    if (rc != LF_OK) return rc;
+    if (ctx->opt_cost == LF_COST_CROSS_ENTROPY && ctx->opt_act != LF_ACT_SIGMOID) return LF_EINVAL;
+    call_timer timer(ctx);
+    rc = backward_impl(ctx, w, z, a, y, delta, gw, gb);
+    timer.done(rc);
+    return rc;
 }
 
 int lf_grad_w(lf_ctx* ctx, const float* delta_l, const float* a_prev, float* gw_l)
@@ -642,6 +685,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     ctx->stats.shard_rank = ctx->shard_rank; ctx->stats.shard_count = ctx->shard_count;
     ctx->stats.fused_tiling = 0;
     int launches = 0;
+    call_timer timer(ctx);
     LF_CUDA_TRY(ctx, cudaEventRecord(ctx->fork_ev, s));
     // From here on the copy, download and worker streams are forked off the context's stream: whatever
     // goes wrong below, they are joined back into it before the call returns (`fail` keeps the
@@ -708,6 +752,7 @@ int lf_backward_host(lf_ctx* ctx, const float* w, const float* z, const float* a
     if (je == cudaSuccess) je = cudaStreamWaitEvent(s, ctx->d2h_done_ev, 0);
     if (je != cudaSuccess && fail == LF_OK) { ctx->last_cuda_error = (int)je; fail = LF_ECUDA; }
     ctx->stats.launches_backward = launches;
+    timer.done(fail);
     return fail;
 }
 
@@ -717,6 +762,12 @@ int lf_sync(lf_ctx* ctx)
     LF_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(unsigned),
                                      cudaMemcpyDeviceToHost, ctx->stream));
     LF_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->timed_call_pending) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ctx->t_begin_ev, ctx->t_end_ev) == cudaSuccess) ctx->stats.last_backward_ms = ms;
+        else cudaGetLastError();
+        ctx->timed_call_pending = false;
+    }
     unsigned st = *ctx->status_host;
     ctx->stats.device_status = st;
     if (st != 0) {
@@ -787,6 +838,8 @@ int lf_destroy(lf_ctx* ctx)
             if (ctx->w_ready_ev[l]) cudaEventDestroy(ctx->w_ready_ev[l]);
         delete[] ctx->w_ready_ev;
     }
+    if (ctx->t_begin_ev) cudaEventDestroy(ctx->t_begin_ev);
+    if (ctx->t_end_ev) cudaEventDestroy(ctx->t_end_ev);
     if (ctx->small_ev) cudaEventDestroy(ctx->small_ev);
     if (ctx->h2d_done_ev) cudaEventDestroy(ctx->h2d_done_ev);
     lf_persistent_release(ctx);

@@ -267,6 +267,12 @@ k_backward_columns(const __grid_constant__ CUtensorMap w_map, const CkParams P)
             const float4* a_prev = reinterpret_cast<const float4*>(P.a + (size_t)(l - 1) * N);
             float4 a4 = st_tid < n4 ? __ldg(a_prev + st_tid) : make_float4(0.f, 0.f, 0.f, 0.f);
             ck_wait(smem_u32(&sh->d_ready[p]), use & 1u, P, sh);
+            // delta^l and gb^l (Eq. bp3) at this CTA's neurons, for the caller (every shard writes these)
+            if (st_tid < my_cols && !(l == L && P.top_given)) {
+                const float d = d_own[p * CK_MAX_WC + st_tid];
+                P.delta[(size_t)(l - 1) * N + col_base + st_tid] = d;
+                P.gb[(size_t)(l - 1) * N + col_base + st_tid] = d;
+            }
             // layer-sharded form: another shard's layer is not stored (the waits and arrivals stay)
             const bool mine = P.shard_count == 1 || (L - l + P.depth_shift) % P.shard_count == P.shard_rank;
             if (mine) {
@@ -320,10 +326,6 @@ k_backward_columns(const __grid_constant__ CUtensorMap w_map, const CkParams P)
             float d = 0.f;
             if (col_ok) {
                 d = ck_top_delta(P, my_col);
-                if (!P.top_given) {
-                    P.delta[(size_t)(L - 1) * N + my_col] = d;
-                    P.gb[(size_t)(L - 1) * N + my_col] = d;
-                }
             }
             d_own[(L & 1) * CK_MAX_WC + tid] = d;
             mbar_arrive(smem_u32(&sh->d_ready[L & 1]));
@@ -412,11 +414,8 @@ k_backward_columns(const __grid_constant__ CUtensorMap w_map, const CkParams P)
             }
             CK_STAMP(4);
             if (finisher) {
-                if (col_ok) {
-                    P.delta[(size_t)(s - 2) * N + my_col] = d;
-                    P.gb[(size_t)(s - 2) * N + my_col] = d;                                // Eq. bp3
-                }
-                // hand delta^{s-1} of my column to the store warps (row my_col of gw^{s-1})
+                // hand delta^{s-1} of my column to the store warps: it scales row my_col of gw^{s-1},
+                // and they also write it to delta and gb (Eq. bp3), which nothing on the chain reads
                 const int pn = (s - 1) & 1;
                 const unsigned used = (unsigned)((L - (s - 1)) >> 1);   // earlier uses of buffer pn
                 if (used > 0) ck_wait(smem_u32(&sh->d_free[pn]), (used - 1) & 1u, P, sh);

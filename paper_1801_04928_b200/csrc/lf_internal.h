@@ -136,6 +136,11 @@ struct lf_ctx {
     cudaEvent_t small_ev, h2d_done_ev, d2h_done_ev;
     bool host_path_ready;    // the copy streams and events above all exist
 
+    // LF_OPT_TIME_CALLS: two timing events around the last backward call
+    int time_calls;
+    cudaEvent_t t_begin_ev, t_end_ev;
+    bool timed_call_pending;
+
     int last_cuda_error;
     lf_stats stats;
 };

@@ -1,0 +1,138 @@
+"""Where the time of one layer step goes inside the single-launch backward kernels (B = 1).
+
+    python -m paper_1801_04928_b200.step_trace [--N 1024] [--L 32] [--k 4]
+                                               [--kernel groups|clusters|columns|all]
+
+Builds a DEBUG copy of the library (``-DLF_PK_TRACE -DLF_CK_TRACE``: thread 0 of two CTAs writes
+SM-clock stamps at fixed points of every layer step; the release library carries none of this)
+under ``_build/trace/``, runs a few passes of the chosen kernel on seeded inputs and prints, per
+traced CTA, the median number of SM cycles between consecutive stamps over the layers of a pass,
+the whole step, and the event-timed pass.  The weights of the one buffer set stay in L2 between
+passes, so the figures describe the hand-off, not the memory system.
+
+Stamps of the cluster kernel (``groups``: leapfrog CTA groups; ``clusters``: fused pass):
+0 step starts, 1 first weight sub-tile is there, 3 all column blocks multiplied and the partial
+sums sent, 4 the cluster's partial sums for my columns have arrived, 5 delta published,
+6 delta of my rows has arrived from the other clusters.
+Stamps of the whole-columns kernel (``columns``): 0 step starts, 1 delta of this warp's rows has
+arrived, 2 multiplied, 3 the CTA's barrier is passed, 4 delta published.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import os
+import subprocess
+import sys
+from concurrent.futures import ThreadPoolExecutor
+
+PKG = os.path.dirname(os.path.abspath(__file__))
+ROOT = os.path.dirname(PKG)
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1801_04928_b200 import build as lfbuild   # noqa: E402  (sources and flags of the release build)
+
+TRACE_DIR = os.path.join(lfbuild.OBJ, "trace")
+TRACE_LIB = os.path.join(TRACE_DIR, "libleapfrog_trace.so")
+
+KERNELS = {  # name -> (LF_OPT_VARIANT, LF_OPT_FUSED_TILING, stamps in order, names of the intervals)
+    "groups": (2, 0, [0, 1, 3, 4, 5, 6], ["wait for the first weight sub-tile", "multiply, reduce, send partial sums",
+                                          "wait for the cluster's partial sums", "add them, sigma', publish",
+                                          "wait for delta of my rows"]),
+    "clusters": (3, 1, [0, 1, 3, 4, 5, 6], ["wait for the first weight sub-tile", "multiply, reduce, send partial sums",
+                                            "wait for the cluster's partial sums", "add them, sigma', publish",
+                                            "wait for delta of my rows"]),
+    "columns": (3, 2, [0, 1, 2, 3, 4], ["wait for delta of the warp's rows (one hop through L2)", "multiply",
+                                        "reduce in the warp, CTA barrier", "add the warps' sums, sigma', publish"]),
+}
+
+
+def build_trace_library() -> str:
+    os.makedirs(TRACE_DIR, exist_ok=True)
+    nvcc = lfbuild._nvcc()
+    flags = [f for f in lfbuild.NVCC_FLAGS if f not in ("-Xptxas", "-v")] + ["-DLF_PK_TRACE", "-DLF_CK_TRACE"]
+
+    def one(src):
+        obj = os.path.join(TRACE_DIR, src.replace(".cu", ".o"))
+        r = subprocess.run([nvcc, *flags, "-c", os.path.join(lfbuild.CSRC, src), "-o", obj], capture_output=True, text=True)
+        if r.returncode != 0:
+            raise RuntimeError(f"nvcc failed on {src}:\n{r.stderr}")
+        return obj
+
+    with ThreadPoolExecutor(max_workers=len(lfbuild.SOURCES)) as ex:
+        objs = list(ex.map(one, lfbuild.SOURCES))
+    r = subprocess.run([nvcc, "-shared", "-o", TRACE_LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a"],
+                       capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError(f"link failed:\n{r.stderr}")
+    return TRACE_LIB
+
+
+def trace(lib, torch, lf_inputs, np, name, L, N, k):
+    variant, tiling, stamps, names = KERNELS[name]
+    vp = ctypes.c_void_p
+    P = lambda x: vp(x.data_ptr())
+    t = lf_inputs.make_inputs(L, N, 1, "uniform", lf_inputs.SEED_BASE + 2, "cuda")
+    z = torch.empty((L, 1, N), device="cuda"); a = torch.empty((L + 1, 1, N), device="cuda")
+    d = torch.empty((L, 1, N), device="cuda"); gw = torch.empty((L, N, N), device="cuda"); gb = torch.empty((L, N), device="cuda")
+    h = vp()
+    assert lib.lf_create(ctypes.byref(h), L, N, 1, k) == 0
+    lib.lf_set_option(h, 1, variant); lib.lf_set_option(h, 12, tiling)
+    lib.lf_forward(h, P(t["w"]), P(t["b"]), P(t["x"]), P(z), P(a))
+    back = lambda: lib.lf_backward(h, P(t["w"]), P(z), P(a), P(t["y"]), P(d), P(gw), P(gb))
+    for _ in range(3):
+        assert back() == 0
+    assert lib.lf_sync(h) == 0
+    buf = (ctypes.c_ulonglong * (2 * L * 16))()
+    assert lib.lf_debug_read_trace(h, buf) == 0
+    stride = 8 if name == "columns" else 16
+    tr = np.array(buf, dtype=np.int64)[:2 * L * stride].reshape(2, L, stride)
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(); e0.record()
+    for _ in range(20):
+        back()
+    e1.record(); torch.cuda.synchronize()
+    assert lib.lf_sync(h) == 0
+    lib.lf_destroy(h)
+    print(f"\n## {name}: L = {L}, N = {N}, k = {k}; pass (weights L2-warm, debug build): {e0.elapsed_time(e1) / 20 * 1e3:.1f} us")
+    print("| interval | " + " | ".join(f"CTA {'0' if c == 0 else 'other'} (median cycles)" for c in range(2)) + " |")
+    print("|---|---|---|")
+    med = []
+    for c in range(2):
+        seg = []
+        for i in range(2, L - 3):          # steady-state layers: not the first two, not the last two
+            r, nx = tr[c][i], tr[c][i + 1]
+            if r[stamps[0]] == 0 or nx[stamps[0]] == 0:
+                continue
+            seg.append([r[stamps[j + 1]] - r[stamps[j]] for j in range(len(stamps) - 1)] +
+                       [nx[stamps[0]] - r[stamps[-1]], nx[stamps[0]] - r[stamps[0]]])
+        med.append(np.median(np.array(seg), axis=0) if seg else None)
+    rows = names + ["rest of the step (housekeeping off the chain)", "whole layer step"]
+    for j, nm in enumerate(rows):
+        print(f"| {nm} | " + " | ".join("n/a" if m is None else f"{int(m[j])}" for m in med) + " |")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--N", type=int, default=1024)
+    ap.add_argument("--L", type=int, default=32)
+    ap.add_argument("--k", type=int, default=4)
+    ap.add_argument("--kernel", default="all", choices=["all"] + sorted(KERNELS))
+    args = ap.parse_args()
+    import numpy as np
+    import torch
+    import lf_inputs
+    if not torch.cuda.is_available():
+        raise SystemExit("step_trace: no CUDA device")
+    lib = ctypes.CDLL(build_trace_library())
+    lib.lf_set_option.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong]
+    clock = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader"],
+                           capture_output=True, text=True).stdout.strip()
+    print(f"SM clock now / max: {clock} (cycles -> ns: divide by the GHz under load)")
+    for name in (sorted(KERNELS) if args.kernel == "all" else [args.kernel]):
+        trace(lib, torch, lf_inputs, np, name, args.L, args.N, args.k)
+
+
+if __name__ == "__main__":
+    main()

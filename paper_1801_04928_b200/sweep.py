@@ -7,7 +7,15 @@ k in {1, 2, 4, 8, 16}) the backward pass is timed with CUDA events for each vari
 exists at that point: for B = 1 the stream schedule, the persistent leapfrog CTA groups and
 the fused pass; for B > 1 the stream schedule with the fp32 and the TF32 weight gradient.
 One JSON object per line is written, and a table of the fastest variant per (N, B) is printed.
-Inputs are the seeded synthetic tensors of ``lf_inputs`` drawn on the GPU.
+Inputs are the seeded synthetic tensors of ``lf_inputs`` drawn on the GPU.  With ``--rotate`` the
+single-sample points run on several buffer sets in turn (as ``bench.py`` does), so that a pass never
+finds its weights in L2; without it widths up to about 1024 are partly L2-resident.
+
+    python -m paper_1801_04928_b200.sweep --emit-table sweep.jsonl
+
+prints, from the single-sample rows of an earlier run, the fastest variant per width and worker
+class (k <= 4, k > 4) and the width ranges in which each one wins: the table
+``LF_VARIANT_AUTO`` encodes.
 
     python -m paper_1801_04928_b200.sweep --widths 4096,8192,2048,4096,1024 [--B 1 256]
 
@@ -28,23 +36,74 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
-def time_point(lf, torch, t, L, N, B, k, variant, gw_math, steps, warmup):
+def time_point(lf, torch, sets, L, N, B, k, variant, gw_math, steps, warmup, fused_tiling=0):
+    """`sets`: one or more buffer sets (dicts of tensors) used in turn."""
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
-    with lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream) as ctx:
+    ctxs = []
+    for _ in sets:     # one context per set: the single-launch kernels keep a descriptor of w
+        ctx = lf.Leapfrog(L, N, B, k, stream=stream.cuda_stream)
         ctx.set_option(lf.LF_OPT_VARIANT, variant)
         ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
-        with torch.cuda.stream(stream):
-            for _ in range(warmup):
-                ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
-            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(steps):
-                ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
-            e1.record(stream)
+        ctx.set_option(lf.LF_OPT_FUSED_TILING, fused_tiling)
+        ctxs.append(ctx)
+
+    def step(i):
+        t, ctx = sets[i % len(sets)], ctxs[i % len(sets)]
+        ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, len(sets))):
+            step(i)
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        e1.record(stream)
+        for ctx in ctxs:
             ctx.sync()
-        st = ctx.stats()
+    st = ctxs[0].stats()
+    for ctx in ctxs:
+        ctx.close()
     return e0.elapsed_time(e1) / steps, st
+
+
+def emit_table(path):
+    """The choice LF_VARIANT_AUTO should make for one sample, from the rows of a sweep."""
+    rows = [json.loads(l) for l in open(path) if l.strip()]
+    rows = [r for r in rows if r.get("B") == 1 and "N" in r]
+    if not rows:
+        print("no single-sample rows in", path)
+        return
+    label = lambda r: r["variant"] + ("/" + r["fused_tiling"] if r.get("fused_tiling") else "")
+    print("| N | workers | fastest | ms | runner-up | ms |")
+    print("|---|---|---|---|---|---|")
+    winners = {"k<=4": [], "k>4": []}
+    for N in sorted({r["N"] for r in rows}):
+        for cls, pick in (("k<=4", lambda k: k <= 4), ("k>4", lambda k: k > 4)):
+            # the fused pass has no workers: its one row competes in both classes
+            cand = [r for r in rows if r["N"] == N and (pick(r["k"]) or r["variant"] == "fused")]
+            if not cand:
+                continue
+            best = {}
+            for r in cand:                      # best k of every variant
+                if label(r) not in best or r["ms"] < best[label(r)]["ms"]:
+                    best[label(r)] = r
+            order = sorted(best.values(), key=lambda r: r["ms"])
+            second = order[1] if len(order) > 1 else order[0]
+            print(f"| {N} | {cls} | {label(order[0])} | {order[0]['ms']:.4f} | {label(second)} | {second['ms']:.4f} |")
+            winners[cls].append((N, label(order[0])))
+    for cls, seq in winners.items():
+        runs, start, prev_n, cur = [], None, None, None
+        for N, w in seq:
+            if w != cur:
+                if cur is not None:
+                    runs.append(f"{cur}: N = {start}..{prev_n}")
+                cur, start = w, N
+            prev_n = N
+        if cur is not None:
+            runs.append(f"{cur}: N = {start}..{prev_n}")
+        print(f"{cls}: " + "; ".join(runs))
 
 
 def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
@@ -90,19 +149,31 @@ def sweep_widths(lf, lf_inputs, torch, widths, Bs, ks, out):
             torch.cuda.empty_cache()
 
 
+SWEEP_L = 48
+SWEEP_N = (256, 1024, 4096, 8192)
+SWEEP_B = (1, 16, 128, 1024)
+
+
 def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--L", type=int, default=SWEEP_L)
+    ap.add_argument("--out", default="sweep.jsonl")
+    ap.add_argument("--quick", action="store_true", help="k in {1, 4} only")
+    ap.add_argument("--N", type=int, nargs="*", default=list(SWEEP_N))
+    ap.add_argument("--B", type=int, nargs="*", default=list(SWEEP_B))
+    ap.add_argument("--widths", default=None, help="n_0,n_1,...,n_L: time one network of these layer widths")
+    ap.add_argument("--rotate", action="store_true",
+                    help="single-sample points: run on rotating buffer sets of at least 1 GiB in total")
+    ap.add_argument("--emit-table", default=None, metavar="SWEEP_JSONL",
+                    help="print the fastest variant per width and worker class from an earlier run, and exit")
+    args = ap.parse_args()
+    if args.emit_table:
+        emit_table(args.emit_table)
+        return
     import torch
     import lf_inputs
     import paper_1801_04928_b200 as lf
-
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--L", type=int, default=lf_inputs.SWEEP["L"])
-    ap.add_argument("--out", default="sweep.jsonl")
-    ap.add_argument("--quick", action="store_true", help="k in {1, 4} only")
-    ap.add_argument("--N", type=int, nargs="*", default=list(lf_inputs.SWEEP["N"]))
-    ap.add_argument("--B", type=int, nargs="*", default=list(lf_inputs.SWEEP["B"]))
-    ap.add_argument("--widths", default=None, help="n_0,n_1,...,n_L: time one network of these layer widths")
-    args = ap.parse_args()
+    assert (SWEEP_L, SWEEP_N, SWEEP_B) == (lf_inputs.SWEEP["L"], lf_inputs.SWEEP["N"], lf_inputs.SWEEP["B"])
     ks = (1, 4) if args.quick else lf_inputs.SWEEP["k"]
     if args.widths:
         sweep_widths(lf, lf_inputs, torch, args.widths.split(","), args.B, ks, args.out)
@@ -122,6 +193,11 @@ def main():
                 with lf.Leapfrog(L, N, B, 1) as ctx:
                     ctx.forward(t["w"], t["b"], t["x"], t["z"], t["a"])
                     ctx.sync()
+                sets = [t]
+                if args.rotate and B == 1:
+                    n_sets = max(2, min(8, int((1 << 30) // (8 * L * N * N))))
+                    for _ in range(n_sets - 1):
+                        sets.append({kk: v.clone() for kk, v in t.items()})
                 flops = 2.0 * N * N * B
                 slow = flops * L > 2e12            # seconds per step on the fp32 chain
                 steps, warmup = (2, 1) if slow else ((5, 2) if N >= 4096 or B > 1 else (50, 5))
@@ -129,23 +205,29 @@ def main():
                 if B == 1:
                     for k in ks:
                         points += [(k, 1, lf.LF_GW_MATH_AUTO), (k, 2, lf.LF_GW_MATH_AUTO)]
-                    points.append((1, 3, lf.LF_GW_MATH_AUTO))   # the fused pass has no k
+                    # the fused pass has no k; both of its tilings
+                    points += [(1, 3, lf.LF_GW_MATH_AUTO, lf.LF_FUSED_TILING_CLUSTERS),
+                               (1, 3, lf.LF_GW_MATH_AUTO, lf.LF_FUSED_TILING_COLUMNS)]
                 else:
                     for k in ks:
                         points.append((k, 1, lf.LF_GW_MATH_TF32))
                     points.append((ks[-1] if len(ks) < 3 else 4, 1, lf.LF_GW_MATH_FP32))
-                for (k, variant, gw_math) in points:
-                    ms, st = time_point(lf, torch, t, L, N, B, k, variant, gw_math, steps, warmup)
+                for point in points:
+                    k, variant, gw_math = point[:3]
+                    tiling = point[3] if len(point) > 3 else 0
+                    ms, st = time_point(lf, torch, sets, L, N, B, k, variant, gw_math, steps, warmup, tiling)
                     alg = 4.0 * N * N * (2 * L - 1) + 12.0 * N * B * L
                     row = dict(L=L, N=N, B=B, k=k, variant=names[st["variant"]], requested=names[variant],
                                gw_math={1: "fp32", 2: "tf32"}[st["gw_math"]], ms=ms,
+                               fused_tiling={0: None, 1: "clusters", 2: "columns"}[st["fused_tiling"]],
+                               buffer_sets=len(sets),
                                layers_per_s=L / (ms * 1e-3), alg_GBs=alg / (ms * 1e-3) / 1e9,
                                chain_ctas=st["chain_ctas"], worker_ctas=st["worker_ctas"],
                                gw_tiling=st["gw_tiling"], delta_tiling=st["delta_tiling"])
                     rows.append(row)
                     f.write(json.dumps(row) + "\n"); f.flush()
                     print(json.dumps(row), flush=True)
-                del t
+                del t, sets
                 torch.cuda.empty_cache()
     print("\n| N | B | fastest | k | ms | layers/s | algorithmic GB/s |")
     print("|---|---|---|---|---|---|---|")

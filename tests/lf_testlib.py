@@ -13,6 +13,28 @@ TF32_TOL = 5e-3      # relative Frobenius error, TF32 tensor-core weight gradien
 DENORMAL = 2.0 ** -149
 
 
+GUARD = 256                      # floats of sentinel on either side of every output buffer
+_SENTINEL = -0x12345679          # an int32 bit pattern no result takes by accident (a NaN with a payload)
+
+
+class Guarded:
+    """An output tensor with a guard band on each side: `t` is what the library gets (NaN-filled),
+    `check()` says whether anything wrote outside it."""
+
+    def __init__(self, shape, device, fill=float("nan")):
+        n = int(np.prod(shape))
+        self.raw = torch.empty(n + 2 * GUARD, dtype=torch.float32, device=device)
+        self.raw.view(torch.int32).fill_(_SENTINEL)
+        self.t = self.raw[GUARD:GUARD + n].view(shape)
+        self.t.fill_(fill)
+
+    def check(self, name):
+        g = self.raw.view(torch.int32)
+        lo, hi = g[:GUARD], g[-GUARD:]
+        assert bool((lo == _SENTINEL).all()), f"{name}: something wrote below the buffer"
+        assert bool((hi == _SENTINEL).all()), f"{name}: something wrote past the end of the buffer"
+
+
 def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=None,
              use_graph=True, stream=None, repeat=1, delta_math=0, tc_tiling=0, cost=0, act=0,
              fused_tiling=0):
@@ -21,11 +43,10 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
     L, N, B = cfg["L"], cfg["N"], cfg["B"]
     k = cfg["k"] if k is None else k
     dev = t["w"].device
-    z = torch.empty((L, B, N), dtype=torch.float32, device=dev)
-    a = torch.empty((L + 1, B, N), dtype=torch.float32, device=dev)
-    delta = torch.full((L, B, N), float("nan"), dtype=torch.float32, device=dev)
-    gw = torch.full((L, N, N), float("nan"), dtype=torch.float32, device=dev)
-    gb = torch.full((L, N), float("nan"), dtype=torch.float32, device=dev)
+    # every output sits between two guard bands that are checked after the pass
+    guards = dict(z=Guarded((L, B, N), dev), a=Guarded((L + 1, B, N), dev), delta=Guarded((L, B, N), dev),
+                  gw=Guarded((L, N, N), dev), gb=Guarded((L, N), dev))
+    z, a, delta, gw, gb = (guards[n].t for n in ("z", "a", "delta", "gw", "gb"))
     st = stream if stream is not None else torch.cuda.Stream(device=dev)
     st.wait_stream(torch.cuda.current_stream(dev))
     with lf.Leapfrog(L, N, B, k, stream=st.cuda_stream) as ctx:
@@ -44,6 +65,8 @@ def gpu_pass(cfg, t, variant=lf.LF_VARIANT_AUTO, gw_math=lf.LF_GW_MATH_AUTO, k=N
         stats = ctx.stats()
     torch.cuda.current_stream(dev).wait_stream(st)
     torch.cuda.synchronize(dev)
+    for name, g in guards.items():
+        g.check(name)
     return dict(z=z, a=a, delta=delta, gw=gw, gb=gb), stats
 
 

@@ -84,3 +84,40 @@ def test_host_buffer_entry_point_matches_device_path():
         assert torch.equal(res[k], out[k].cpu())
     ref = oracle_pass(t)
     compare_all(cfg, dict(z=out["z"], a=out["a"], **{k: v.cuda() for k, v in res.items()}), ref)
+
+
+def test_last_backward_time_is_reported_when_asked_for():
+    # LF_OPT_TIME_CALLS: two events around the call on the context's stream; lf_sync reads them
+    L, N = 8, 1024
+    t = _buffers(L, N)
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with lf.Leapfrog(L, N, 1, 2, stream=st.cuda_stream) as ctx:
+        ctx.forward(t["w"], t["b"], t["x"], t["z"], t["a"])
+        ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+        ctx.sync()
+        assert ctx.stats()["last_backward_ms"] == 0.0            # off by default
+        ctx.set_option(lf.LF_OPT_TIME_CALLS, 1)
+        for variant in (lf.LF_VARIANT_STREAMS, lf.LF_VARIANT_AUTO):
+            ctx.set_option(lf.LF_OPT_VARIANT, variant)
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])
+            e1.record(st)
+            ctx.sync()
+            ms = ctx.stats()["last_backward_ms"]
+            assert 0.0 < ms <= e0.elapsed_time(e1) + 1e-3, (variant, ms, e0.elapsed_time(e1))
+    torch.cuda.synchronize()
+
+
+def test_binding_refuses_buffers_of_the_wrong_size_or_type():
+    L, N = 3, 64
+    t = _buffers(L, N)
+    with lf.Leapfrog(L, N, 1, 2) as ctx:
+        small = torch.empty((L, N, N - 4), device="cuda")
+        for bad in (small, t["gw"].double(), t["gw"].cpu(), t["gw"].transpose(1, 2)):
+            with pytest.raises(lf.LeapfrogError) as e:
+                ctx.backward(t["w"], t["z"], t["a"], t["y"], t["delta"], bad, t["gb"])
+            assert e.value.status == lf.LF_EINVAL
+        with pytest.raises(lf.LeapfrogError):
+            ctx.backward_host(t["w"], t["z"], t["a"], t["y"], t["delta"], t["gw"], t["gb"])   # device tensors
