@@ -274,10 +274,19 @@ def aggregate_rate(total_ms, units_per_rank, dist=None, device=None):
 # launch; the summaries are under profiles/).  A figure is reported only for the workload, variant
 # and tiling it was captured on, and only while the kernel's source file is byte for byte the one
 # that was captured (sha1 below); otherwise `traffic` is null.  configs[2] is too large to capture
-# whole: its figure is the 8-layer capture scaled by the algorithmic bytes (traffic is proportional
-# to the layers processed: every layer's weights are read once and its gradients written once).
+# whole: its figure comes from an 8-layer capture of the same kernel at the same width.  Reads grow
+# in proportion to the layers read (L - 1: every layer's weights once; the capture shows no
+# re-reads); writes are the 4N^2 L bytes of gradients minus what is still dirty in L2 when the
+# kernel ends, which the capture gives as a constant (its own 4N^2 L minus its DRAM writes).
 NCU_TRAFFIC = {
-    # (config, variant, fused tiling): (bytes per launch of the captured case, its L, source file, sha1, summary)
+    # (config, variant, fused tiling): (dram read bytes, dram write bytes per launch of the captured case -- the
+    #                                   mean of two launches --, its L, source file, its sha1, summary)
+    (1, 3, 2): (150528.0, 0.0, 8, "lf_columns.cu", "7e82cab6387d9ce80034afdf0e1346383242a180",
+                "profiles/dram_traffic_single_launch_kernels.md"),
+    (2, 2, 0): (130518400.0, 75710336.0, 32, "lf_persistent.cu", "bedd670278ba61cefa2d84f22a5d7393bcd13f93",
+                "profiles/dram_traffic_single_launch_kernels.md"),
+    (3, 3, 1): (470146432.0, 476348672.0, 8, "lf_persistent.cu", "bedd670278ba61cefa2d84f22a5d7393bcd13f93",
+                "profiles/dram_traffic_single_launch_kernels.md"),
 }
 
 
@@ -294,12 +303,15 @@ def ncu_traffic(index, stats, L, N, B, plain):
     ent = NCU_TRAFFIC.get((index, stats["variant"], stats.get("fused_tiling", 0)))
     if not ent or not plain:
         return None, None
-    cap_bytes, cap_L, src, sha, summary = ent
+    cap_read, cap_write, cap_L, src, sha, summary = ent
     if source_sha1(src) != sha:
         return None, f"stale: {src} has changed since the capture in {summary}"
-    scale = algorithmic_bytes(L, N, B) / algorithmic_bytes(cap_L, N, B)
-    how = "as captured" if cap_L == L else f"captured at L={cap_L}, scaled by algorithmic bytes x{scale:.3f}"
-    return cap_bytes * scale, f"{summary} ({how}; {src} sha1 {sha[:12]})"
+    if cap_L == L:
+        return cap_read + cap_write, f"{summary} (as captured; {src} sha1 {sha[:12]})"
+    dirty_tail = 4.0 * N * N * cap_L - cap_write
+    traffic = cap_read * (L - 1) / max(cap_L - 1, 1) + 4.0 * N * N * L - dirty_tail
+    return traffic, (f"{summary} (captured at L={cap_L}: reads scaled by (L-1)/{cap_L - 1}, writes = 4N^2 L minus the "
+                     f"{dirty_tail / 1e6:.0f} MB still dirty in L2 at the end; {src} sha1 {sha[:12]})")
 
 
 def time_gw_gemm(lf, L, N, B, delta_l, a_prev, gw_slabs, stream, steps, tc_tiling=0):
