@@ -81,9 +81,10 @@ enum lf_delta_math {
 enum lf_tc_tiling {
     LF_TC_TILING_AUTO = 0,   /* CTA pairs where they apply and the device can co-schedule them  */
     LF_TC_TILING_ONE_SM = 1, /* one CTA per tile                                                */
-    LF_TC_TILING_TWO_SM = 2  /* CTA pairs: Eq. bp4 for B <= 256 (the delta operand of a row
-                                block stays in shared memory), Eq. bp2 / Eq. z for B > 128 and
-                                N >= 512; other sizes use ONE_SM                                */
+    LF_TC_TILING_TWO_SM = 2  /* CTA pairs: Eq. bp4 at every B (up to 256 samples the delta operand
+                                of a row block stays in shared memory, beyond that both operands
+                                stream), Eq. bp2 / Eq. z for B > 128 and N >= 512; other sizes use
+                                ONE_SM                                                          */
 };
 
 /* Tiling of the fused single-launch pass (LF_VARIANT_FUSED, B = 1). */

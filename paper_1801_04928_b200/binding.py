@@ -99,17 +99,26 @@ def _check_tensor(t, need: int, name: str, where: str, on_device: bool = True) -
     unchecked (None is rejected by the library itself)."""
     if t is None or isinstance(t, int):
         return
+    global _FLOAT32
+    dt = t.dtype
+    if dt is not _FLOAT32:                   # (the dtype object is remembered: the check costs no string work)
+        if str(dt) == "torch.float32":
+            _FLOAT32 = dt
+    if dt is _FLOAT32 and t.is_cuda == on_device and t.numel() >= need and t.is_contiguous():
+        return
     problems = []
-    if str(getattr(t, "dtype", "")) != "torch.float32":
-        problems.append(f"dtype {getattr(t, 'dtype', '?')} (float32 needed)")
-    if hasattr(t, "is_contiguous") and not t.is_contiguous():
+    if dt is not _FLOAT32:
+        problems.append(f"dtype {dt} (float32 needed)")
+    if not t.is_contiguous():
         problems.append("not contiguous")
-    if hasattr(t, "is_cuda") and bool(t.is_cuda) != on_device:
+    if bool(t.is_cuda) != on_device:
         problems.append("must be a CUDA tensor" if on_device else "must be a host tensor")
-    if hasattr(t, "numel") and t.numel() < need:
+    if t.numel() < need:
         problems.append(f"{t.numel()} elements, {need} needed")
-    if problems:
-        raise LeapfrogError(LF_EINVAL, f"{where}: argument {name}: " + "; ".join(problems))
+    raise LeapfrogError(LF_EINVAL, f"{where}: argument {name}: " + "; ".join(problems))
+
+
+_FLOAT32 = None
 
 
 def _ptr(t) -> ctypes.c_void_p:

@@ -353,6 +353,7 @@ constexpr int TP_BM = 128;                               // rows of gw per CTA (
 constexpr int TP_BN = 256;                               // columns of a pair tile (128 loaded per CTA)
 constexpr int TP_MAX_KS = 8;                             // at most 8 x 32 = 256 samples
 constexpr int TP_STAGES = 3;
+constexpr int TPS_STAGES = 5;                             // streaming form (B > 256): stages of 32 KiB, both operands
 constexpr int TP_ACC = 2;                                // accumulators of TP_BN columns
 constexpr int TP_A_STAGE_BYTES = (TP_BM / 32) * TG_BOX_BYTES;        // 16 KiB: 128 rows x 32 samples
 constexpr int TP_B_STAGE_BYTES = (TP_BN / 2 / 32) * TG_BOX_BYTES;    // 16 KiB: 128 columns x 32 samples
@@ -361,17 +362,20 @@ constexpr int TP_THREADS = 320;                          // producer, issuer, ei
 constexpr int TP_EPI_BYTES = 8 * 32 * TG_EPI_LD * 4;    // one 32 x 32 block per epilogue warp
 constexpr size_t TP_SMEM_BYTES = (size_t)TP_A_BYTES + (size_t)TP_STAGES * TP_B_STAGE_BYTES + TP_EPI_BYTES +
                                  1024 /*alignment slack*/ + 512;
+static_assert((size_t)TPS_STAGES * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES) <= (size_t)TP_A_BYTES + (size_t)TP_STAGES * TP_B_STAGE_BYTES,
+              "the streaming form's ring overlays the resident operand and the activation ring");
 
 struct TpShared {
     unsigned long long a_full[TP_MAX_KS];   // leader: delta operand chunk ks of both CTAs has landed
     unsigned long long a_empty;             // both: the resident delta operand may be replaced
-    unsigned long long b_full[TP_STAGES];   // leader: stage of both CTAs has landed
-    unsigned long long b_empty[TP_STAGES];  // both: stage may be refilled
+    unsigned long long b_full[TPS_STAGES];  // leader: stage of both CTAs has landed
+    unsigned long long b_empty[TPS_STAGES]; // both: stage may be refilled
     unsigned long long acc_full[TP_ACC];    // both: accumulator complete
     unsigned long long acc_empty[TP_ACC];   // leader: accumulator drained by both CTAs
     unsigned tmem_base;
     volatile unsigned abort_flag;
 };
+static_assert(sizeof(TpShared) <= 512, "the barrier block must fit into the space reserved for it");
 
 __device__ __forceinline__ unsigned tp_cluster_rank()
 {
@@ -448,6 +452,12 @@ __device__ __forceinline__ bool tp_wait(unsigned bar, unsigned parity, const TgP
     return true;
 }
 
+// RESIDENT = true: B <= 256, the delta operand of a row block stays in shared memory (above).
+// RESIDENT = false: any B.  Both operands stream: a stage holds 32 samples of the pair's 256 rows of
+// delta and 256 columns of a, half of each loaded by either CTA (32 KiB per CTA and stage, five
+// stages over the same shared memory).  Per multiply-add a CTA then loads two thirds of what the
+// one-SM kernel loads, which is what that kernel waits for at large B.
+template <bool RESIDENT>
 __global__ void __launch_bounds__(TP_THREADS, 1)
 k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_a,
                     const TgParams P)
@@ -464,7 +474,8 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned rank = tp_cluster_rank();          // 0 = leader (issues the multiplications)
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_k = (P.B + TG_BK - 1) / TG_BK;        // <= TP_MAX_KS
+    const int n_k = (P.B + TG_BK - 1) / TG_BK;        // RESIDENT: <= TP_MAX_KS
+    constexpr unsigned N_ST = RESIDENT ? TP_STAGES : TPS_STAGES;
     const int n_tiles = P.tiles_m * P.tiles_n;        // tiles_m counts 256-row blocks here
     const int t_begin = (int)(((long long)n_tiles * pair) / n_pairs);
     const int t_end = (int)(((long long)n_tiles * (pair + 1)) / n_pairs);
@@ -472,7 +483,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     if (threadIdx.x == 0) {
         for (int i = 0; i < TP_MAX_KS; ++i) tg_mbar_init(tg_smem_u32(&sh->a_full[i]), 1);
         tg_mbar_init(tg_smem_u32(&sh->a_empty), 1);
-        for (int i = 0; i < TP_STAGES; ++i) {
+        for (int i = 0; i < TPS_STAGES; ++i) {
             tg_mbar_init(tg_smem_u32(&sh->b_full[i]), 1);
             tg_mbar_init(tg_smem_u32(&sh->b_empty[i]), 1);
         }
@@ -504,7 +515,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             bool ok = true;
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int rb = t / P.tiles_n, tn = t - rb * P.tiles_n;
-                const bool new_rb = rb != cur_rb;
+                const bool new_rb = RESIDENT && rb != cur_rb;
                 if (new_rb) {
                     // the resident delta operand changes: wait until every multiplication that
                     // reads the old one is done
@@ -523,15 +534,29 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                             tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
                                            ks * TG_BK);
                     }
-                    const unsigned st = it % TP_STAGES, use = it / TP_STAGES;
+                    const unsigned st = it % N_ST, use = it / N_ST;
                     if (use > 0 && !tp_wait(tg_smem_u32(&sh->b_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
                     const unsigned lbar = tg_smem_u32(&sh->b_full[st]);
-                    if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
                     const unsigned bar = tp_map_to_rank(lbar, 0);
-                    const unsigned dst = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
+                    if (RESIDENT) {
+                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
+                        const unsigned dst = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
 #pragma unroll
-                    for (int i = 0; i < TP_BN / 2 / 32; ++i)
-                        tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                        for (int i = 0; i < TP_BN / 2 / 32; ++i)
+                            tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                    } else {
+                        // streaming form: this CTA's half of both operands for these 32 samples
+                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                        const unsigned dst_a = tg_smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                        const unsigned dst_b = dst_a + TP_A_STAGE_BYTES;
+#pragma unroll
+                        for (int i = 0; i < TP_BM / 32; ++i)
+                            tp_tma_load_2d(dst_a + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
+                                           ks * TG_BK);
+#pragma unroll
+                        for (int i = 0; i < TP_BN / 2 / 32; ++i)
+                            tp_tma_load_2d(dst_b + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                    }
                 }
             }
         }
@@ -543,7 +568,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             int cur_rb = -1;
             for (int t = t_begin; t < t_end; ++t, ++tile_i) {
                 const int rb = t / P.tiles_n;
-                const bool new_rb = rb != cur_rb;
+                const bool new_rb = RESIDENT && rb != cur_rb;
                 if (new_rb) { cur_rb = rb; ++a_loads; }
                 const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
                 if (ab_use > 0 && !tp_wait(tg_smem_u32(&sh->acc_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
@@ -552,11 +577,13 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 bool ok = true;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     if (new_rb && !tp_wait(tg_smem_u32(&sh->a_full[ks]), (a_loads - 1) & 1u, P, sh)) { ok = false; break; }
-                    const unsigned st = it % TP_STAGES, use = it / TP_STAGES;
+                    const unsigned st = it % N_ST, use = it / N_ST;
                     if (!tp_wait(tg_smem_u32(&sh->b_full[st]), use & 1u, P, sh)) { ok = false; break; }
                     tg_fence_after();
-                    const unsigned a_addr = tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES);
-                    const unsigned b_addr = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
+                    const unsigned a_addr = RESIDENT ? tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES)
+                                                     : tg_smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                    const unsigned b_addr = RESIDENT ? tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES)
+                                                     : a_addr + TP_A_STAGE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < TG_BK / 8; ++kk) {      // eight samples per instruction
                         const unsigned long long da = tg_make_desc(a_addr + kk * 1024, TG_BOX_BYTES);
@@ -567,7 +594,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 }
                 if (!ok) break;
                 // the last tile of a row block frees the resident operand for the next one
-                if (t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(tg_smem_u32(&sh->a_empty));
+                if (RESIDENT && t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(tg_smem_u32(&sh->a_empty));
                 tp_commit_both(tg_smem_u32(&sh->acc_full[ab]));
             }
         }
@@ -693,7 +720,9 @@ static int tp_max_pairs(const lf_ctx* c)
     if (cached_dev == c->device) return cached;
     int n = 0;
     if ((size_t)c->smem_optin >= TP_SMEM_BYTES &&
-        cudaFuncSetAttribute(k_gw_gemm_tf32_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_gw_gemm_tf32_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)TP_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_gw_gemm_tf32_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)TP_SMEM_BYTES) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
@@ -701,7 +730,12 @@ static int tp_max_pairs(const lf_ctx* c)
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        if (cudaOccupancyMaxActiveClusters(&n, k_gw_gemm_tf32_pair, &cfg) != cudaSuccess) n = 0;
+        int n_stream = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_gw_gemm_tf32_pair<true>, &cfg) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n_stream, k_gw_gemm_tf32_pair<false>, &cfg) != cudaSuccess)
+            n = 0;
+        else if (n_stream < n)
+            n = n_stream;
     }
     cudaGetLastError();
     cached_dev = c->device; cached = n;
@@ -742,9 +776,10 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
     P.sgd = sgd;
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
-    const int max_pairs = c->tc_pair_kernels && c->B <= TP_MAX_KS * TG_BK ? tp_max_pairs(c) : 0;
+    const int max_pairs = c->tc_pair_kernels ? tp_max_pairs(c) : 0;
     if (max_pairs > 0) {
-        // two-SM kernel: the delta operand of a 256-row block stays in shared memory
+        // two-SM kernels: up to 256 samples the delta operand of a 256-row block stays in shared
+        // memory; beyond, both operands stream
         P.tiles_m = (n_out + 2 * TP_BM - 1) / (2 * TP_BM);
         P.tiles_n = (n_in + TP_BN - 1) / TP_BN;
         const int tiles = P.tiles_m * P.tiles_n;
@@ -756,7 +791,10 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_gw_gemm_tf32_pair, map_d, map_a, P));
+        if (c->B <= TP_MAX_KS * TG_BK)
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_gw_gemm_tf32_pair<true>, map_d, map_a, P));
+        else
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_gw_gemm_tf32_pair<false>, map_d, map_a, P));
         c->stats.gw_tiling = LF_TC_TILING_TWO_SM;
         *launches += 1;
         return LF_OK;

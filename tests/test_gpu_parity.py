@@ -141,12 +141,15 @@ def test_config3_parity_long_chain():
 
 @pytest.mark.parametrize("tiling", [lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM])
 @pytest.mark.parametrize("L,N,B,k", [(2, 256, 32, 1), (3, 512, 256, 2), (2, 388, 70, 2), (2, 132, 16, 1),
-                                     (2, 1028, 129, 3), (2, 64, 8, 1), (2, 2308, 96, 2)])
+                                     (2, 1028, 129, 3), (2, 64, 8, 1), (2, 2308, 96, 2),
+                                     (2, 772, 300, 2), (2, 1284, 515, 1), (2, 516, 1024, 2)])
 def test_minibatch_tf32_weight_gradient(L, N, B, k, tiling):
     # Eq. bp4 on the tensor cores: relative Frobenius error per layer <= 5e-3 against the
     # float64 oracle; everything else on the path stays fp32 and keeps the 1e-5 gate.  Both
     # tilings: one CTA per tile, and CTA pairs with the delta operand resident (N = 2308 gives
-    # pairs runs of several tiles that cross a row-block boundary, with ragged last tiles).
+    # pairs runs of several tiles that cross a row-block boundary, with ragged last tiles) or, for
+    # more than 256 samples, with both operands streaming (B = 300: a ragged last stage; B = 515:
+    # more stages than the ring holds; B = 1024: the ring goes round six times per tile).
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=3 * N + B)
     out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_TF32, tc_tiling=tiling)
@@ -185,6 +188,31 @@ def test_tf32_pair_kernel_long_runs():
         assert e <= TF32_TOL, (tiling, e)
     # the two tilings multiply the same truncated operands and add the samples in the same order
     assert np.array_equal(outs[lf.LF_TC_TILING_TWO_SM], outs[lf.LF_TC_TILING_ONE_SM])
+
+
+def test_tf32_tilings_agree_bitwise_beyond_256_samples():
+    # more than 256 samples: the CTA pairs stream both operands; they multiply the same truncated
+    # operands and add the samples in the same order as the one-SM kernel.  Eq. bp4 alone
+    # (lf_grad_w) on one delta and one a, so that nothing else depends on the tiling.
+    for N, B in ((1540, 300), (772, 1024)):
+        g = torch.Generator(device="cuda"); g.manual_seed(N + B)
+        d = torch.empty((B, N), device="cuda").normal_(0.0, 1.0, generator=g)
+        a = torch.empty((B, N), device="cuda").uniform_(0.0, 1.0, generator=g)
+        outs = {}
+        for tiling in (lf.LF_TC_TILING_TWO_SM, lf.LF_TC_TILING_ONE_SM):
+            gw = torch.full((N, N), float("nan"), device="cuda")
+            with lf.Leapfrog(1, N, B, 1) as ctx:
+                ctx.set_option(lf.LF_OPT_GW_MATH, lf.LF_GW_MATH_TF32)
+                ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
+                for _ in range(2):
+                    ctx.grad_w(d, a, gw)
+                ctx.sync()
+                assert ctx.stats()["gw_tiling"] == tiling and ctx.stats()["device_status"] == 0
+            outs[tiling] = gw
+        assert torch.equal(outs[lf.LF_TC_TILING_TWO_SM], outs[lf.LF_TC_TILING_ONE_SM]), (N, B)
+        ref = d.double().t() @ a.double()      # (a library product only as a second opinion on the size of the error)
+        err = float((outs[lf.LF_TC_TILING_TWO_SM].double() - ref).norm() / ref.norm())
+        assert err <= 5e-3, err
 
 
 def test_config4_minibatch_full_size_sampled():
