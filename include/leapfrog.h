@@ -147,9 +147,11 @@ enum lf_option {
     LF_OPT_TIME_CALLS = 13,   /* 0/1 (default 0): bracket every backward call with two events on
                                  the context's stream; lf_sync then puts the elapsed device time
                                  of the last one into lf_stats.last_backward_ms                 */
-    LF_OPT_WITHHOLD = 5       /* 0/1, test hook for the persistent variants: one CTA does not
-                                 publish its share of delta, so the bounded waits of the others
-                                 expire and lf_sync() reports LF_ETIMEOUT (no fault, no hang)  */
+    LF_OPT_WITHHOLD = 5       /* test hook, 0 (off), 1 or 2.  1, single-launch variants: one CTA does
+                                 not publish its share of delta.  2, tensor-core weight-gradient
+                                 kernels (B > 1): one producer arms a stage and never loads it.
+                                 Either way the bounded waits of the others expire and lf_sync()
+                                 reports LF_ETIMEOUT (no fault, no hang)                          */
 };
 
 typedef struct lf_stats {

@@ -459,7 +459,7 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             ctx->time_calls = (int)value;
             return LF_OK;
         case LF_OPT_WITHHOLD:
-            if (value != 0 && value != 1) return LF_EINVAL;
+            if (value < 0 || value > 2) return LF_EINVAL;
             ctx->withhold = (int)value;
             return LF_OK;
         case LF_OPT_USE_GRAPH:

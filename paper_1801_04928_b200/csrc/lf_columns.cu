@@ -552,7 +552,7 @@ int lf_backward_columns(lf_ctx* c, const float* w, const float* a, const float* 
     P.nSub = pl.nSub; P.Rw = pl.Rw; P.stages = pl.stages; P.stage_floats = pl.stage_floats;
     P.top_given = top_given; P.depth_shift = depth_shift;
     P.shard_rank = c->shard_rank; P.shard_count = c->shard_count > 1 ? c->shard_count : 1;
-    P.withhold = c->withhold; P.cost = c->opt_cost; P.act = c->opt_act;
+    P.withhold = c->withhold == 1 ? 1 : 0; P.cost = c->opt_cost; P.act = c->opt_act;
     P.epoch = c->epoch;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
     P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;

@@ -39,6 +39,8 @@ struct TgParams {
     float* gw;
     unsigned* status;
     unsigned long long budget_ns;
+    int withhold;             // test hook (LF_OPT_WITHHOLD = 2): one producer leaves out the loads of its first
+                              // stage, so that every wait behind it runs out
 };
 
 struct TgShared {
@@ -222,6 +224,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                     if (use > 0 && !tg_wait(tg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
                     const unsigned bar = tg_smem_u32(&sh->full[st]);
                     tg_mbar_expect_tx(bar, TG_STAGE_BYTES);
+                    if (P.withhold && blockIdx.x == 0 && it == 0) continue;   // test hook: armed, never loaded
                     const unsigned a_dst = tg_smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
                     const unsigned b_dst = a_dst + TG_A_BYTES;
 #pragma unroll
@@ -374,6 +377,10 @@ struct TpShared {
     unsigned long long acc_empty[TP_ACC];   // leader: accumulator drained by both CTAs
     unsigned tmem_base;
     volatile unsigned abort_flag;
+    // what this CTA's producer has issued (read by the leader when a launch is given up)
+    unsigned prog_it;         // stage loads issued
+    unsigned prog_a_loads;    // resident form: loads of the delta operand begun ...
+    unsigned prog_a_ks;       // ... and chunks of the last one issued
 };
 static_assert(sizeof(TpShared) <= 512, "the barrier block must fit into the space reserved for it");
 
@@ -431,6 +438,16 @@ __device__ __forceinline__ bool tp_try_wait_cluster(unsigned bar, unsigned parit
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ void tp_complete_tx(unsigned bar, unsigned bytes)   // bytes that will never arrive
+{
+    asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ unsigned tp_ld_remote(unsigned cluster_addr)
+{
+    unsigned v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+    return v;
 }
 // Bounded wait on a barrier of this CTA; returns false once this CTA has given up.
 __device__ __forceinline__ bool tp_wait(unsigned bar, unsigned parity, const TgParams& P, TpShared* sh)
@@ -508,7 +525,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     if (warp == 0) {
         // ------------------------------ TMA producer (each CTA, its own halves) ----------------
         if (lane == 0) {
-            unsigned it = 0, a_loads = 0;
+            unsigned it = 0, a_loads = 0, a_ks = 0;
             int cur_rb = -1;
             const int my_row0 = (int)rank * TP_BM;
             const int my_col0 = (int)rank * (TP_BN / 2);
@@ -522,9 +539,11 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                     if (a_loads > 0 && !tp_wait(tg_smem_u32(&sh->a_empty), (a_loads - 1) & 1u, P, sh)) break;
                     cur_rb = rb;
                     ++a_loads;
+                    a_ks = 0;
                 }
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     if (new_rb) {
+                        ++a_ks;
                         const unsigned lbar = tg_smem_u32(&sh->a_full[ks]);
                         if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_A_STAGE_BYTES);
                         const unsigned bar = tp_map_to_rank(lbar, 0);
@@ -538,6 +557,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                     if (use > 0 && !tp_wait(tg_smem_u32(&sh->b_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
                     const unsigned lbar = tg_smem_u32(&sh->b_full[st]);
                     const unsigned bar = tp_map_to_rank(lbar, 0);
+                    if (P.withhold && pair == 0 && rank == 1 && it == 0) continue;   // test hook: the peer leaves out its first stage
                     if (RESIDENT) {
                         if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
                         const unsigned dst = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
@@ -559,6 +579,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                     }
                 }
             }
+            sh->prog_it = it; sh->prog_a_loads = a_loads; sh->prog_a_ks = a_ks;
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer (leader CTA only) ---------------------------
@@ -663,10 +684,44 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     // memory, and its commits arrive on the peer's barriers.
     tg_fence_before();
     __syncthreads();
-    if (sh->abort_flag && threadIdx.x == 0 && rank == 0) {
-        // after giving up: let loads that are still landing finish (bounded)
-        const unsigned long long t0 = tg_timer();
-        while (tg_timer() - t0 < 200000ull) { }
+    tp_cluster_sync();     // both producers have stopped; what each has issued is in its prog_* words
+    if (threadIdx.x == 0 && rank == 0) {
+        // A launch that was given up: no CTA of the pair may exit while operand loads are still on
+        // their way into its shared memory.  The loads of BOTH CTAs are credited to the leader's
+        // barriers, so the leader can see all of them land -- once every phase that anyone issued
+        // loads for has been brought to a state it can complete in: a phase only the peer loaded
+        // for gets the arrival (and the byte count) the leader never gave it, a phase only the
+        // leader loaded for is told that the peer's bytes will not come.  Then wait, with a limit.
+        const bool gave_up = sh->abort_flag != 0u || tp_ld_remote(tp_map_to_rank(tg_smem_u32((const void*)&sh->abort_flag), 1)) != 0u;
+        if (gave_up) {
+            const unsigned it_l = sh->prog_it, it_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_it), 1));
+            const unsigned stage_bytes = RESIDENT ? (unsigned)TP_B_STAGE_BYTES : (unsigned)(TP_A_STAGE_BYTES + TP_B_STAGE_BYTES);
+            const unsigned it_hi = it_l > it_p ? it_l : it_p, it_lo = it_l < it_p ? it_l : it_p;
+            for (unsigned j = it_lo; j < it_hi; ++j) {
+                const unsigned bar = tg_smem_u32(&sh->b_full[j % N_ST]);
+                if (j >= it_l) tg_mbar_expect_tx(bar, stage_bytes);      // only the peer loaded
+                else tp_complete_tx(bar, stage_bytes);                  // only the leader loaded
+            }
+            const unsigned long long t0 = tg_timer();
+            for (unsigned j = it_hi > N_ST ? it_hi - N_ST : 0; j < it_hi; ++j) {
+                const unsigned bar = tg_smem_u32(&sh->b_full[j % N_ST]);
+                while (!tg_mbar_try_wait(bar, (j / N_ST) & 1u) && tg_timer() - t0 < 50000000ull) { }
+            }
+            if (RESIDENT) {
+                // the resident operand: chunks of the load that was under way (loads before it were
+                // waited for by the multiplications that freed the operand for this one)
+                const unsigned al_l = sh->prog_a_loads, al_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_a_loads), 1));
+                const unsigned ak_l = sh->prog_a_ks, ak_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_a_ks), 1));
+                const unsigned al = al_l > al_p ? al_l : al_p;
+                const unsigned kl = al_l == al ? ak_l : 0u, kp = al_p == al ? ak_p : 0u;   // chunks of load `al`
+                for (unsigned ks = 0; ks < (kl > kp ? kl : kp) && al > 0; ++ks) {
+                    const unsigned bar = tg_smem_u32(&sh->a_full[ks]);
+                    if (ks >= kl) tg_mbar_expect_tx(bar, (unsigned)TP_A_STAGE_BYTES);
+                    else if (ks >= kp) tp_complete_tx(bar, (unsigned)TP_A_STAGE_BYTES);
+                    while (!tg_mbar_try_wait(bar, (al - 1) & 1u) && tg_timer() - t0 < 50000000ull) { }
+                }
+            }
+        }
     }
     tp_cluster_sync();
     if (warp == 1) {
@@ -776,6 +831,7 @@ int lf_gw_gemm_tf32(lf_ctx* c, const float* delta_l, const float* a_prev, float*
     P.sgd = sgd;
     P.status = c->status_dev;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
+    P.withhold = c->withhold == 2 ? 1 : 0;
     const int max_pairs = c->tc_pair_kernels ? tp_max_pairs(c) : 0;
     if (max_pairs > 0) {
         // two-SM kernels: up to 256 samples the delta operand of a 256-row block stays in shared

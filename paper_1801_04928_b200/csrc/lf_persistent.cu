@@ -944,7 +944,7 @@ int lf_backward_persistent(lf_ctx* c, int variant, const float* w, const float* 
     P.top_given = top_given; P.depth_shift = depth_shift;
     P.fused = variant == LF_VARIANT_FUSED ? 1 : 0;
     P.Wc = pl.Wc; P.nCB = pl.nCB; P.Ws = pl.Ws; P.Hr = pl.Hr; P.R = pl.R; P.nRB = pl.nRB;
-    P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold;
+    P.slice = pl.slice; P.keff = c->keff; P.epoch = c->epoch; P.withhold = c->withhold == 1 ? 1 : 0;
     P.cost = c->opt_cost; P.act = c->opt_act;
     P.shard_rank = c->shard_rank; P.shard_count = c->shard_count > 1 ? c->shard_count : 1;
     P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;

@@ -69,6 +69,37 @@ def test_bounded_waits_expire_and_the_context_recovers(variant):
     compare_all(cfg, {k: t[k] for k in ("z", "a", "delta", "gw", "gb")}, ref)
 
 
+@pytest.mark.parametrize("N,B,tiling", [(256, 32, lf.LF_TC_TILING_ONE_SM), (512, 96, lf.LF_TC_TILING_ONE_SM),
+                                        (512, 64, lf.LF_TC_TILING_TWO_SM), (772, 320, lf.LF_TC_TILING_TWO_SM)])
+def test_tensor_core_kernels_give_up_cleanly(N, B, tiling):
+    # LF_OPT_WITHHOLD = 2: one producer of the weight-gradient kernel arms a stage and never loads it,
+    # so the multiplications behind it never start and every wait runs out (budget 20 ms).  The
+    # kernel must end -- the one-SM kernel, the CTA pairs with the delta operand resident (B <= 256)
+    # and with both operands streaming --, lf_sync must say LF_ETIMEOUT, and the next call must be
+    # right again: Eq. bp4 against the oracle.
+    from oracle import lf_oracle as orc
+    from lf_testlib import rel_frobenius, TF32_TOL
+    g = torch.Generator(device="cuda"); g.manual_seed(N + B)
+    d = torch.empty((B, N), device="cuda").normal_(0.0, 1.0, generator=g)
+    a = torch.empty((B, N), device="cuda").uniform_(0.0, 1.0, generator=g)
+    gw = torch.full((N, N), float("nan"), device="cuda")
+    with lf.Leapfrog(1, N, B, 1) as ctx:
+        ctx.set_option(lf.LF_OPT_GW_MATH, lf.LF_GW_MATH_TF32)
+        ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
+        ctx.set_option(lf.LF_OPT_WAIT_BUDGET_US, 20000)
+        ctx.set_option(lf.LF_OPT_WITHHOLD, 2)
+        ctx.grad_w(d, a, gw)
+        assert lf.lf_sync(ctx._h) == lf.LF_ETIMEOUT
+        assert ctx.stats()["device_status"] != 0 and ctx.stats()["gw_tiling"] == tiling
+        ctx.set_option(lf.LF_OPT_WITHHOLD, 0)
+        gw.fill_(float("nan"))
+        ctx.grad_w(d, a, gw)
+        ctx.sync()
+        assert ctx.stats()["device_status"] == 0
+    ref = orc.grad_w(d.double().cpu().numpy(), a.double().cpu().numpy())
+    assert rel_frobenius(gw.cpu().numpy(), ref) <= TF32_TOL
+
+
 def test_host_buffer_entry_point_matches_device_path():
     L, N = 4, 516
     cfg = dict(L=L, N=N, B=1, k=2)
