@@ -210,14 +210,16 @@ int lf_create(lf_ctx** out, int L, int N, int B, int k);
  *     a        block l = [B][n_l], l = 0..L, a block 0 = x
  *     x [B][n_0],  y [B][n_L]
  * With all widths equal this is lf_create(L, widths[0], B, k) exactly, layouts included.
- * Otherwise the context runs one launch per layer and step with the k workers as streams
- * (LF_VARIANT_STREAMS) -- the single-launch kernels are written for one common width; an option
- * asking for them is accepted and lf_get_stats() reports what ran, with N = the widest layer.
- * One case keeps the single launch: B = 1, L >= 3 and all hidden layers n_1 .. n_{L-1} of one
- * width (the network of Section 2, whose input and output widths are left open): layers
- * 2 .. L-1 then run as one persistent launch (LF_VARIANT_PERSISTENT or LF_VARIANT_FUSED, as
- * asked for or as LF_VARIANT_AUTO picks for that width) between per-layer launches for the top
- * and the bottom layer.
+ * Otherwise, for one sample (B = 1), LF_VARIANT_FUSED -- and LF_VARIANT_AUTO, which picks it --
+ * runs the whole pass as ONE launch whatever the widths are (the whole-columns tiling gives every
+ * layer its own split of columns over the CTAs; up to 64 layers, widths up to 16384);
+ * LF_VARIANT_STREAMS runs one launch per layer and step with the k workers as streams; and
+ * LF_VARIANT_PERSISTENT, or LF_VARIANT_FUSED with LF_FUSED_TILING_CLUSTERS -- kernels written for
+ * one common width -- run over the hidden layers n_1 .. n_{L-1} if those share a width (the
+ * network of Section 2, whose input and output widths are left open; L >= 3), between per-layer
+ * launches for the top and the bottom layer, and fall back to LF_VARIANT_STREAMS if they do not.
+ * A mini-batch (B > 1) runs one launch per layer.  lf_get_stats() reports what ran, with N = the
+ * widest layer.
  * The arithmetic options apply as for lf_create (B > 1: tensor-core contractions by default).  lf_forward, lf_backward,
  * lf_backward_sgd and lf_backward_host take such a context; lf_grad_w, which names no layer,
  * returns LF_EINVAL for it.

@@ -37,11 +37,22 @@ inline size_t v_at(const lf_ctx* c, int l) { return c->off_h[l - 1]; }          
 inline size_t h_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_h[l - 1]; }       // z, delta
 inline size_t a_at(const lf_ctx* c, int l) { return (size_t)c->B * c->off_a[l]; }           // a: l = 0..L
 
+// LF_VARIANT_AUTO for layers of different widths (one sample): the single launch wherever it exists --
+// measured against one launch per layer it is ahead at every shape tried (no launch gaps, the chain
+// never leaves the SMs).
+bool lf_widths_auto_single_launch(const lf_ctx*) { return true; }
+
 // The persistent kernels are written for one common width (every cluster owns the same column strip
 // of every layer): they serve uniform contexts and, for one sample, the run of hidden layers of a
 // context whose input and output widths alone differ; other contexts run one launch per layer.
 int resolve_variant(const lf_ctx* c)
 {
+    // layers of different widths, one sample: the fused pass with whole columns per CTA takes any
+    // shape in one launch (where it was asked for; LF_VARIANT_AUTO: see below)
+    if (!c->uniform && c->B == 1 && c->opt_fused_tiling != LF_FUSED_TILING_CLUSTERS &&
+        (c->opt_variant == LF_VARIANT_FUSED || (c->opt_variant == LF_VARIANT_AUTO && lf_widths_auto_single_launch(c))) &&
+        lf_columns_widths_supported(c))
+        return LF_VARIANT_FUSED;
     if (!c->uniform && (c->B != 1 || c->pk_N <= 0)) return LF_VARIANT_STREAMS;
     return c->opt_variant != LF_VARIANT_AUTO ? c->opt_variant : lf_auto_variant(c);
 }
@@ -531,7 +542,9 @@ static int backward_impl(lf_ctx* ctx, const float* w, const float* z, const floa
 {
     int variant = resolve_variant(ctx);
     const int gw_math = resolve_gw_math(ctx);
-    if (variant != LF_VARIANT_STREAMS && !lf_persistent_supported(ctx, variant))
+    const bool widths_single_launch = !ctx->uniform && variant == LF_VARIANT_FUSED &&
+                                      ctx->opt_fused_tiling != LF_FUSED_TILING_CLUSTERS && lf_columns_widths_supported(ctx);
+    if (variant != LF_VARIANT_STREAMS && !widths_single_launch && !lf_persistent_supported(ctx, variant))
         variant = LF_VARIANT_STREAMS;
     ctx->stats.variant = variant;
     ctx->stats.gw_math = gw_math;
@@ -544,6 +557,8 @@ static int backward_impl(lf_ctx* ctx, const float* w, const float* z, const floa
         return backward_streams(ctx, w, z, a, y, delta, gw, gb, gw_math);
     if (ctx->uniform)
         return lf_backward_persistent(ctx, variant, w, a, y, delta, gw, gb, ctx->sgd_w, 0, 0);
+    if (variant == LF_VARIANT_FUSED && ctx->opt_fused_tiling != LF_FUSED_TILING_CLUSTERS && lf_columns_widths_supported(ctx))
+        return lf_backward_columns_widths(ctx, w, a, y, delta, gw, gb, ctx->sgd_w);
     return backward_hidden_run(ctx, variant, w, a, y, delta, gw, gb, gw_math);
 }
 
@@ -843,6 +858,7 @@ int lf_destroy(lf_ctx* ctx)
     if (ctx->small_ev) cudaEventDestroy(ctx->small_ev);
     if (ctx->h2d_done_ev) cudaEventDestroy(ctx->h2d_done_ev);
     lf_persistent_release(ctx);
+    lf_columns_release(ctx);
     lf_tf32_release(ctx);
     delete ctx;
     return LF_OK;

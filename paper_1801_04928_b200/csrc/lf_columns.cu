@@ -23,6 +23,7 @@
 // Every wait is bounded by a time budget.  On expiry the CTA raises the status word, stops waiting
 // for the rest of the launch and runs to the end with whatever it has, so the kernel always ends.
 #include <cuda.h>
+#include <string.h>
 
 #include "lf_internal.h"
 #include "lf_ptx.cuh"
@@ -117,14 +118,19 @@ __device__ __forceinline__ void ck_wait(unsigned bar, unsigned parity, const CkP
     }
 }
 
-// Eq. bp1 at one neuron of the top layer (or delta^L as an earlier launch left it).
-__device__ __forceinline__ float ck_top_delta(const CkParams& P, int row)
+// Eq. bp1 at one neuron of the top layer (or delta^L as an earlier launch left it); aL, deltaL: the
+// top layer's activations and delta.
+__device__ __forceinline__ float ck_top_delta_at(const CkParams& P, const float* aL, const float* deltaL, int row)
 {
-    if (P.top_given) return P.delta[(size_t)(P.L - 1) * P.N + row];
-    const float av = P.a[(size_t)P.L * P.N + row];
+    if (P.top_given) return deltaL[row];
+    const float av = aL[row];
     float d = av - P.y[row];
     if (P.cost == LF_COST_QUADRATIC) d *= lf_act_prime(av, P.act);   // cross-entropy: sigma' cancels
     return d;
+}
+__device__ __forceinline__ float ck_top_delta(const CkParams& P, int row)
+{
+    return ck_top_delta_at(P, P.a + (size_t)P.L * P.N, P.delta + (size_t)(P.L - 1) * P.N, row);
 }
 
 // Polling delta^s at the rows this warp multiplies (d_sm index = row; rows past N hold 0).  A lane
@@ -137,18 +143,18 @@ struct CkPoll {
     int sub, piece;      // the next item (counted up, never divided: this is the chain)
 };
 
-// rows of the next batch
-__device__ __forceinline__ void ck_poll_setup(CkPoll& q, const CkParams& P, int warp, int lane)
+// rows of the next batch (R rows per sub-tile, Rw of them this warp's, nSub sub-tiles, n_rows rows in all)
+__device__ __forceinline__ void ck_poll_setup(CkPoll& q, int R, int Rw, int nSub, int n_rows, int warp, int lane)
 {
-    const int cpw = (P.Rw + 31) >> 5;             // 32-row pieces of a warp's share of a sub-tile
+    const int cpw = (Rw + 31) >> 5;               // 32-row pieces of a warp's share of a sub-tile
 #pragma unroll
     for (int u = 0; u < CK_POLL_BATCH; ++u) {
         const int off = q.piece * 32 + lane;
-        const int rl = warp * P.Rw + off;
-        q.row[u] = q.sub * P.R + rl;
-        q.valid[u] = q.sub < P.nSub && off < P.Rw && rl < P.R;
+        const int rl = warp * Rw + off;
+        q.row[u] = q.sub * R + rl;
+        q.valid[u] = q.sub < nSub && off < Rw && rl < R;
         if (++q.piece == cpw) { q.piece = 0; ++q.sub; }
-        q.pend[u] = q.valid[u] && q.row[u] < P.N;
+        q.pend[u] = q.valid[u] && q.row[u] < n_rows;
         q.v[u] = 0ull;
     }
 }
@@ -345,14 +351,14 @@ k_backward_columns(const __grid_constant__ CUtensorMap w_map, const CkParams P)
             // delta^s of this warp's rows: Eq. bp1 at the top, polled below it
             if (s == L) {
                 for (int i0 = 0; i0 < n_items; i0 += CK_POLL_BATCH) {
-                    ck_poll_setup(q, P, warp, lane);
+                    ck_poll_setup(q, P.R, P.Rw, P.nSub, P.N, warp, lane);
 #pragma unroll
                     for (int u = 0; u < CK_POLL_BATCH; ++u)
                         if (q.valid[u]) d_sm[q.row[u]] = q.pend[u] ? ck_top_delta(P, q.row[u]) : 0.f;
                 }
             } else {
                 for (int i0 = 0; i0 < n_items; i0 += CK_POLL_BATCH) {
-                    ck_poll_setup(q, P, warp, lane);
+                    ck_poll_setup(q, P.R, P.Rw, P.nSub, P.N, warp, lane);
                     ck_poll_issue(q, slots);
                     ck_poll_collect(q, P, sh, slots, d_sm);
                 }
@@ -423,6 +429,249 @@ k_backward_columns(const __grid_constant__ CUtensorMap w_map, const CkParams P)
                 mbar_arrive(smem_u32(&sh->d_ready[pn]));
             }
             a_mine = a_mine_next;
+        }
+    }
+    __syncthreads();
+}
+
+// ---- the same pass for layers of different widths ------------------------------------------------
+// Step s reads w^s (n_s rows, n_{s-1} columns) and produces delta^{s-1}; CTA q owns the columns
+// [q * Wc_s, (q+1) * Wc_s) of that matrix, with Wc_s following the layer, so every layer keeps all
+// CTAs busy whatever its shape.  Everything a step needs is one entry of a table (copied to shared
+// memory when the kernel starts) and one tensor map per layer.  The uniform kernel above is this
+// one with every entry equal; it stays a kernel of its own because its constants come for free.
+constexpr int CK_TAB_MAX = 64;     // layers the table holds
+struct CkLayer {
+    int rows, cols;        // n_s, n_{s-1}: the shape of w^s
+    int Wc;                // columns of w^s per CTA (= neurons of layer s-1 a CTA finishes)
+    int RH, R, nSub, Rw;   // TMA box (RL x RH rows) and the warps' shares of it
+    unsigned box_bytes;
+    unsigned off_w_lo, off_w_hi;   // start of w^s / gw^s (floats, 64 bits)
+    int off_rows;          // start of delta^s in delta / gb / the exchange slots (B = 1: neurons before layer s)
+    int off_cols;          // start of delta^{s-1} there
+    int off_a_cols;        // start of a^{s-1} in a
+    int Wc_rows;           // neurons of layer s a CTA finishes (its rows of gw^s)
+    int pad0, pad1;
+};
+static_assert(sizeof(CkLayer) == 64, "one table entry is 64 bytes");
+
+template <bool UPDATE>
+__global__ void __launch_bounds__(CK_THREADS, 1)
+k_backward_columns_widths(const CUtensorMap* __restrict__ maps, const CkLayer* __restrict__ table, const CkParams P)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    float* ring = reinterpret_cast<float*>(smem_raw);                                // stages x stage_floats
+    float* d_sm = ring + (size_t)P.stages * P.stage_floats;                          // [max nSub * R]
+    float4* red = reinterpret_cast<float4*>(d_sm + (((size_t)P.nSub * P.R + 3) & ~(size_t)3));   // [2][8 warps][32]
+    float* d_own = reinterpret_cast<float*>(red + 2 * CK_CHAIN_WARPS * 32);          // [2][CK_MAX_WC]
+    CkLayer* tab = reinterpret_cast<CkLayer*>(d_own + 2 * CK_MAX_WC);                // [L + 1], entry s for step s
+    CkShared* sh = reinterpret_cast<CkShared*>(tab + CK_TAB_MAX + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int L = P.L;
+    for (int i = tid; i < (L + 1) * (int)(sizeof(CkLayer) / 16); i += CK_THREADS)
+        reinterpret_cast<float4*>(tab)[i] = reinterpret_cast<const float4*>(table)[i];
+    if (tid == 0) {
+        for (int i = 0; i < P.stages; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->empty[i]), CK_CHAIN_WARPS);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&sh->d_ready[i]), CK_MAX_WC);     // the first 128 chain threads, finishing or not
+            mbar_init(smem_u32(&sh->d_free[i]), CK_STORE_THREADS);
+        }
+        sh->abort_flag = 0u;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    // entry s (2 <= s <= L) describes step s; entry 1 only the top of the table's use by the stores
+    // (rows of gw^1); Wc_rows of entry L is the split of the top layer.
+
+    if (warp == CK_PRODUCER_WARP) {
+        if (lane == 0) {
+            int it = 0, st = 0;
+            unsigned fill = 0;
+            for (int s = L; s >= 2 && !sh->abort_flag; --s) {
+                const CkLayer ly = tab[s];
+                const int col_base = blockIdx.x * ly.Wc;
+                for (int sub = 0; sub < ly.nSub; ++sub, ++it) {
+                    if (fill > 0) {
+                        ck_wait(smem_u32(&sh->empty[st]), (fill - 1) & 1u, P, sh);
+                        if (sh->abort_flag) break;
+                    }
+                    const unsigned bar = smem_u32(&sh->full[st]);
+                    mbar_expect_tx(bar, ly.box_bytes);
+                    // (a CTA whose columns lie beyond the matrix still loads: the box is all fill)
+                    tma_load_3d(smem_u32(ring + (size_t)st * P.stage_floats), maps + (s - 1), bar, col_base, 0, sub * ly.RH);
+                    if (++st == P.stages) { st = 0; ++fill; }
+                }
+            }
+            if (sh->abort_flag) {
+                const unsigned long long t0 = globaltimer_ns();
+                for (int j = it > P.stages ? it - P.stages : 0; j < it; ++j) {
+                    const unsigned bar = smem_u32(&sh->full[j % P.stages]);
+                    const unsigned parity = (unsigned)((j / P.stages) & 1);
+                    while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < 50000000ull) { }
+                }
+            }
+        }
+    } else if (warp >= CK_CHAIN_WARPS) {
+        // ------------------------- store warps: this CTA's rows of every gw^l -----------------------
+        const int st_tid = tid - CK_CHAIN_THREADS;
+        for (int l = L; l >= 1; --l) {
+            const CkLayer ly = tab[l];                       // w^l: rows = n_l, cols = n_{l-1}
+            const int p = l & 1;
+            const unsigned use = (unsigned)((L - l) >> 1);
+            const int n4 = ly.cols >> 2;
+            const int row_base = blockIdx.x * ly.Wc_rows;
+            const int my_rows = min(ly.Wc_rows, ly.rows - row_base);        // <= 0: none of this layer
+            const float4* a_prev = reinterpret_cast<const float4*>(P.a + ly.off_a_cols);
+            float4 a4 = st_tid < n4 ? __ldg(a_prev + st_tid) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ck_wait(smem_u32(&sh->d_ready[p]), use & 1u, P, sh);
+            if (st_tid < my_rows && !(l == L && P.top_given)) {
+                const float d = d_own[p * CK_MAX_WC + st_tid];
+                P.delta[ly.off_rows + row_base + st_tid] = d;
+                P.gb[ly.off_rows + row_base + st_tid] = d;                  // Eq. bp3
+            }
+            const bool mine = P.shard_count == 1 || (L - l + P.depth_shift) % P.shard_count == P.shard_rank;
+            if (mine && my_rows > 0) {
+                const float* dr = d_own + p * CK_MAX_WC;
+                const size_t off_w = ((size_t)ly.off_w_hi << 32) | ly.off_w_lo;
+                float* out = P.gw + off_w + (size_t)row_base * ly.cols;
+                const float* w_in = UPDATE ? P.w_sub + off_w + (size_t)row_base * ly.cols : nullptr;
+                for (int c = st_tid; c < n4; c += CK_STORE_THREADS) {
+                    const float4 av = a4;
+                    if (c + CK_STORE_THREADS < n4) a4 = __ldg(a_prev + c + CK_STORE_THREADS);
+                    if (UPDATE) {
+                        for (int r0 = 0; r0 < my_rows; r0 += 4) {
+                            float4 wv[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (r0 + u < my_rows) wv[u] = __ldcg(reinterpret_cast<const float4*>(w_in + (size_t)(r0 + u) * ly.cols + 4 * c));
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                if (r0 + u < my_rows) {
+                                    const float d = dr[r0 + u];
+                                    st_stream4(out + (size_t)(r0 + u) * ly.cols + 4 * c,
+                                               lf_sgd_apply4(P.eta, wv[u], make_float4(d * av.x, d * av.y, d * av.z, d * av.w)));
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll 4
+                        for (int r = 0; r < my_rows; ++r) {
+                            const float d = dr[r];
+                            st_stream4(out + (size_t)r * ly.cols + 4 * c, make_float4(d * av.x, d * av.y, d * av.z, d * av.w));
+                        }
+                    }
+                }
+            }
+            mbar_arrive(smem_u32(&sh->d_free[p]));
+        }
+    } else {
+        // ------------------------- chain warps ------------------------------------------------------
+        const bool hands_over = tid < CK_MAX_WC;     // these threads fill d_own (with 0 where they finish nothing)
+        // ---- Eq. bp1 at the top layer's neurons of this CTA
+        {
+            const CkLayer top = tab[L];
+            const int r = blockIdx.x * top.Wc_rows + tid;
+            if (hands_over) {
+                float d = 0.f;
+                if (tid < top.Wc_rows && r < top.rows)
+                    d = ck_top_delta_at(P, P.a + top.off_a_cols + top.cols, P.delta + top.off_rows, r);
+                d_own[(L & 1) * CK_MAX_WC + tid] = d;
+                mbar_arrive(smem_u32(&sh->d_ready[L & 1]));
+            }
+        }
+        int st = 0;
+        unsigned full_phase = 0;
+        CkPoll q;
+        for (int s = L; s >= 2; --s) {
+            const CkLayer ly = tab[s];
+            const int Wc = ly.Wc, WC4 = Wc >> 2, rpi = 32 / WC4;
+            const bool active = lane < rpi * WC4;
+            const int rsub = lane / WC4, c4 = lane - rsub * WC4;
+            int pow2 = 1;
+            while (pow2 < rpi) pow2 <<= 1;
+            const int row_lo = warp * ly.Rw, row_hi = min(ly.R, row_lo + ly.Rw);
+            const int my_col = blockIdx.x * Wc + tid;
+            const bool col_ok = tid < Wc && my_col < ly.cols;
+            const float a_mine = col_ok ? P.a[ly.off_a_cols + my_col] : 0.f;
+            const unsigned long long* slots = P.xch + ly.off_rows;
+            const int n_items = ly.nSub * ((ly.Rw + 31) >> 5);
+            q.sub = 0; q.piece = 0;
+            if (s == L) {
+                const CkLayer top = ly;
+                for (int i0 = 0; i0 < n_items; i0 += CK_POLL_BATCH) {
+                    ck_poll_setup(q, ly.R, ly.Rw, ly.nSub, ly.rows, warp, lane);
+#pragma unroll
+                    for (int u = 0; u < CK_POLL_BATCH; ++u)
+                        if (q.valid[u])
+                            d_sm[q.row[u]] = q.pend[u] ? ck_top_delta_at(P, P.a + top.off_a_cols + top.cols, P.delta + top.off_rows, q.row[u]) : 0.f;
+                }
+            } else {
+                for (int i0 = 0; i0 < n_items; i0 += CK_POLL_BATCH) {
+                    ck_poll_setup(q, ly.R, ly.Rw, ly.nSub, ly.rows, warp, lane);
+                    ck_poll_issue(q, slots);
+                    ck_poll_collect(q, P, sh, slots, d_sm);
+                }
+            }
+            __syncwarp();
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int sub = 0; sub < ly.nSub; ++sub) {
+                ck_wait(smem_u32(&sh->full[st]), full_phase, P, sh);
+                const float4* tile = reinterpret_cast<const float4*>(ring + (size_t)st * P.stage_floats);
+                const float* dsub = d_sm + sub * ly.R;
+                if (active) {
+#pragma unroll 4
+                    for (int r = row_lo + rsub; r < row_hi; r += rpi) {
+                        const float4 wv = tile[r * WC4 + c4];
+                        const float d = dsub[r];
+                        acc.x = fmaf(wv.x, d, acc.x);
+                        acc.y = fmaf(wv.y, d, acc.y);
+                        acc.z = fmaf(wv.z, d, acc.z);
+                        acc.w = fmaf(wv.w, d, acc.w);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->empty[st]));
+                if (++st == P.stages) { st = 0; full_phase ^= 1u; }
+            }
+            {
+                int cnt = rpi;
+                for (int stp = pow2 >> 1; stp >= 1; stp >>= 1) {
+                    const float4 o = make_float4(__shfl_down_sync(0xffffffffu, acc.x, stp * WC4),
+                                                 __shfl_down_sync(0xffffffffu, acc.y, stp * WC4),
+                                                 __shfl_down_sync(0xffffffffu, acc.z, stp * WC4),
+                                                 __shfl_down_sync(0xffffffffu, acc.w, stp * WC4));
+                    if (rsub < stp && rsub + stp < cnt) { acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
+                    if (cnt > stp) cnt = stp;
+                }
+            }
+            float4* red_p = red + (s & 1) * CK_CHAIN_WARPS * 32;
+            if (lane < WC4) red_p[warp * 32 + lane] = acc;
+            bar_sync(1, CK_CHAIN_THREADS);
+            float d = 0.f;
+            if (tid < Wc) {
+                const float* rp = reinterpret_cast<const float*>(red_p);
+                float part[CK_CHAIN_WARPS];
+#pragma unroll
+                for (int wq = 0; wq < CK_CHAIN_WARPS; ++wq) part[wq] = rp[wq * 128 + tid];
+                float v = part[0];
+#pragma unroll
+                for (int wq = 1; wq < CK_CHAIN_WARPS; ++wq) v += part[wq];
+                if (col_ok) {
+                    d = v * lf_act_prime(a_mine, P.act);                                   // Eq. bp2
+                    if (!(P.withhold && blockIdx.x == 0)) st_slot(P.xch + ly.off_cols + my_col, d, P.epoch);
+                }
+            }
+            if (hands_over) {
+                const int pn = (s - 1) & 1;
+                const unsigned used = (unsigned)((L - (s - 1)) >> 1);
+                if (used > 0) ck_wait(smem_u32(&sh->d_free[pn]), (used - 1) & 1u, P, sh);
+                d_own[pn * CK_MAX_WC + tid] = d;
+                mbar_arrive(smem_u32(&sh->d_ready[pn]));
+            }
         }
     }
     __syncthreads();
@@ -587,5 +836,188 @@ int lf_backward_columns(lf_ctx* c, const float* w, const float* a, const float* 
     c->stats.launches_backward = 1;
     c->stats.chain_ctas = pl.Q;
     c->stats.worker_ctas = 0;
+    return LF_OK;
+}
+
+
+// ---- layers of different widths: plan, table, tensor maps, launch ----------------------------------
+namespace {
+
+struct CkWidthsPlan {
+    bool ok;
+    int Q, stages, stage_floats, d_floats;
+    size_t smem_bytes;
+};
+
+// Fills `tab` (L + 1 entries, entry 0 unused) and the box shapes; returns the launch plan.
+CkWidthsPlan ck_plan_widths(const lf_ctx* c, CkLayer* tab, int* rl_out)
+{
+    CkWidthsPlan p = {};
+    const int L = c->L;
+    if (c->B != 1 || L < 1 || L > CK_TAB_MAX) return p;
+    if ((size_t)c->smem_optin < CK_SMEM_LIMIT || !ck_get_encode_fn()) return p;
+    const int max_ctas = ck_max_ctas(c);
+    if (max_ctas < 1) return p;
+    auto split = [&](int n) {                       // neurons of a layer per CTA
+        int wc = 4 * ((n + 4 * max_ctas - 1) / (4 * max_ctas));
+        if (wc < CK_MIN_WC && n >= CK_MIN_WC) wc = CK_MIN_WC;
+        return wc;
+    };
+    int q_needed = 1;
+    for (int l = 1; l <= L; ++l) {
+        CkLayer& e = tab[l];
+        e = CkLayer{};
+        e.rows = c->width[l]; e.cols = c->width[l - 1];
+        if (e.rows > CK_MAX_N || e.cols > CK_MAX_N) return p;
+        e.Wc_rows = split(e.rows);
+        e.Wc = split(e.cols);                       // (entry 1: not used, the chain ends at step 2)
+        if (e.Wc_rows > CK_MAX_WC || e.Wc > CK_MAX_WC) return p;
+        const size_t ow = c->off_w[l - 1];
+        e.off_w_lo = (unsigned)(ow & 0xffffffffu); e.off_w_hi = (unsigned)(ow >> 32);
+        if (c->off_h[L] > 0x7fffffffu || c->off_a[L + 1] > 0x7fffffffu) return p;
+        e.off_rows = (int)c->off_h[l - 1];
+        e.off_cols = l >= 2 ? (int)c->off_h[l - 2] : 0;
+        e.off_a_cols = (int)c->off_a[l - 1];
+        const int q_rows = (e.rows + e.Wc_rows - 1) / e.Wc_rows;
+        if (q_rows > q_needed) q_needed = q_rows;
+        if (l >= 2) {
+            int RL = 2;
+            for (int d = CK_STAGE_FLOATS / e.Wc < 256 ? CK_STAGE_FLOATS / e.Wc : 256; d >= 1; --d)
+                if (e.rows % d == 0 && d % 2 == 0) { RL = d; break; }
+            rl_out[l] = RL;
+            e.RH = CK_STAGE_FLOATS / (e.Wc * RL);
+            if (e.RH > e.rows / RL) e.RH = e.rows / RL;
+            if (e.RH > 256) e.RH = 256;
+            if (e.RH < 1) return p;
+            e.R = RL * e.RH;
+            e.nSub = (e.rows / RL + e.RH - 1) / e.RH;
+            e.Rw = 2 * ((e.R + 2 * CK_CHAIN_WARPS - 1) / (2 * CK_CHAIN_WARPS));
+            e.box_bytes = (unsigned)(e.Wc * e.R * sizeof(float));
+            const int sf = (e.R * e.Wc + 31) & ~31;
+            if (sf > p.stage_floats) p.stage_floats = sf;
+            if (e.nSub * e.R > p.d_floats) p.d_floats = e.nSub * e.R;
+            const int q_cols = (e.cols + e.Wc - 1) / e.Wc;
+            if (q_cols > q_needed) q_needed = q_cols;
+        }
+    }
+    // a CTA finishes the same neurons of layer l whether they are columns of w^{l+1} or rows of gw^l
+    for (int l = 1; l < L; ++l)
+        if (tab[l].Wc_rows != tab[l + 1].Wc) return p;
+    if (p.stage_floats == 0) { p.stage_floats = 32; p.d_floats = 4; }      // L == 1: no chain step
+    p.Q = q_needed;
+    if (p.Q > max_ctas) return p;
+    const size_t fixed = (((size_t)p.d_floats + 3) & ~(size_t)3) * 4 + 2 * CK_CHAIN_WARPS * 32 * 16 + 2 * CK_MAX_WC * 4 +
+                         (CK_TAB_MAX + 1) * sizeof(CkLayer) + sizeof(CkShared) + 16;
+    if (fixed + 2 * (size_t)p.stage_floats * 4 > CK_SMEM_LIMIT) return p;
+    size_t st = (CK_SMEM_LIMIT - fixed) / ((size_t)p.stage_floats * 4);
+    if (st > CK_MAX_STAGES) st = CK_MAX_STAGES;
+    p.stages = (int)st;
+    p.smem_bytes = fixed + (size_t)p.stages * p.stage_floats * 4;
+    p.ok = true;
+    return p;
+}
+
+}  // namespace
+
+bool lf_columns_widths_supported(const lf_ctx* c)
+{
+    if (c->uniform) return false;
+    CkLayer tab[CK_TAB_MAX + 1];
+    int rl[CK_TAB_MAX + 1];
+    return ck_plan_widths(c, tab, rl).ok;
+}
+
+void lf_columns_release(lf_ctx* c)
+{
+    if (c->ckw_dev) cudaFree(c->ckw_dev);
+    c->ckw_dev = nullptr;
+}
+
+// One launch over all L layers of a context whose layers differ in width (B = 1).
+int lf_backward_columns_widths(lf_ctx* c, const float* w, const float* a, const float* y, float* delta, float* gw,
+                               float* gb, const float* w_sub)
+{
+    const int L = c->L;
+    CkLayer tab[CK_TAB_MAX + 1];
+    int rl[CK_TAB_MAX + 1] = {};
+    const CkWidthsPlan pl = ck_plan_widths(c, tab, rl);
+    if (!pl.ok) return LF_ERESOURCE;
+    // device copy of the table and of one tensor map per layer, rebuilt when the weights move
+    const size_t maps_bytes = (size_t)L * sizeof(CUtensorMap), tab_bytes = (size_t)(L + 1) * sizeof(CkLayer);
+    if (!c->ckw_dev) {
+        cudaError_t e = cudaMalloc(&c->ckw_dev, maps_bytes + tab_bytes);
+        if (e != cudaSuccess) {
+            c->ckw_dev = nullptr;
+            c->last_cuda_error = (int)e;
+            cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? LF_ENOMEM : LF_ECUDA;
+        }
+        c->stats.workspace_bytes += (long long)(maps_bytes + tab_bytes);
+        c->ckw_ptr = nullptr;
+    }
+    if (c->ckw_ptr != w) {
+        alignas(64) CUtensorMap maps[CK_TAB_MAX];
+        memset(maps, 0, sizeof(maps));
+        for (int s = 2; s <= L; ++s) {        // w^s as [rows / RL][RL][cols]; box = Wc columns x RL rows x RH row blocks
+            const CkLayer& e = tab[s];
+            const size_t ow = ((size_t)e.off_w_hi << 32) | e.off_w_lo;
+            cuuint64_t dims[3] = {(cuuint64_t)e.cols, (cuuint64_t)rl[s], (cuuint64_t)(e.rows / rl[s])};
+            cuuint64_t strides[2] = {(cuuint64_t)e.cols * 4, (cuuint64_t)e.cols * rl[s] * 4};
+            cuuint32_t box[3] = {(cuuint32_t)e.Wc, (cuuint32_t)rl[s], (cuuint32_t)e.RH};
+            cuuint32_t estr[3] = {1, 1, 1};
+            CUresult r = ck_get_encode_fn()(&maps[s - 1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(w + ow), dims,
+                                            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) {
+                c->last_cuda_error = (int)r;
+                return LF_ECUDA;
+            }
+        }
+        // (pageable host memory: the copies are staged by the runtime before the calls return)
+        LF_CUDA_TRY(c, cudaMemcpyAsync(c->ckw_dev, maps, maps_bytes, cudaMemcpyHostToDevice, c->stream));
+        LF_CUDA_TRY(c, cudaMemcpyAsync(static_cast<unsigned char*>(c->ckw_dev) + maps_bytes, tab, tab_bytes,
+                                       cudaMemcpyHostToDevice, c->stream));
+        c->ckw_ptr = w;
+    }
+    c->epoch += 1;
+    if (c->epoch == 0) c->epoch = 1;
+
+    CkParams P = {};
+    P.L = L; P.N = c->N; P.Q = pl.Q;
+    P.R = pl.d_floats; P.nSub = 1;                 // (only the size of the delta buffer is taken from these)
+    P.stages = pl.stages; P.stage_floats = pl.stage_floats;
+    P.top_given = 0; P.depth_shift = 0;
+    P.shard_rank = c->shard_rank; P.shard_count = c->shard_count > 1 ? c->shard_count : 1;
+    P.withhold = c->withhold == 1 ? 1 : 0; P.cost = c->opt_cost; P.act = c->opt_act;
+    P.epoch = c->epoch;
+    P.budget_ns = (unsigned long long)c->wait_budget_us * 1000ull;
+    P.a = a; P.y = y; P.delta = delta; P.gw = gw; P.gb = gb;
+    P.w_sub = c->sgd_on ? w_sub : nullptr; P.eta = c->sgd_eta;
+    P.xch = reinterpret_cast<unsigned long long*>(c->sync_words);
+    P.status = c->status_dev;
+
+    LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_columns_widths<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)CK_SMEM_LIMIT));
+    LF_CUDA_TRY(c, cudaFuncSetAttribute(k_backward_columns_widths<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)CK_SMEM_LIMIT));
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    cfg.gridDim = dim3(pl.Q);
+    cfg.blockDim = dim3(CK_THREADS);
+    cfg.dynamicSmemBytes = pl.smem_bytes;
+    cfg.stream = c->stream;
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    const CUtensorMap* maps_dev = static_cast<const CUtensorMap*>(c->ckw_dev);
+    const CkLayer* tab_dev = reinterpret_cast<const CkLayer*>(static_cast<unsigned char*>(c->ckw_dev) + maps_bytes);
+    if (P.w_sub)
+        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_columns_widths<true>, maps_dev, tab_dev, P));
+    else
+        LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_backward_columns_widths<false>, maps_dev, tab_dev, P));
+    c->stats.launches_backward = 1;
+    c->stats.chain_ctas = pl.Q;
+    c->stats.worker_ctas = 0;
+    c->stats.fused_tiling = LF_FUSED_TILING_COLUMNS;
     return LF_OK;
 }

@@ -122,6 +122,9 @@ struct lf_ctx {
     const void* ck_map_ptr;
     int ck_map_wc;
     int opt_fused_tiling;    // enum lf_fused_tiling
+    // its form for layers of different widths: device copy of one tensor map per layer and the layer table
+    void* ckw_dev;
+    const void* ckw_ptr;     // the weights they describe
 #if defined(LF_PK_TRACE) || defined(LF_CK_TRACE)
     unsigned long long* trace_dev;  // debug builds: per-step SM-clock stamps of two CTAs
 #endif
@@ -197,6 +200,11 @@ constexpr int LF_COLUMNS_FUSED_MAX_N = 768;   // widths up to which a fused pass
 bool lf_columns_supported(const lf_ctx* c);
 int lf_backward_columns(lf_ctx* c, const float* w, const float* a, const float* y, float* delta, float* gw,
                         float* gb, const float* w_sub, int top_given, int depth_shift);
+// ... and over all layers of a context whose layers differ in width (one sample)
+bool lf_columns_widths_supported(const lf_ctx* c);
+int lf_backward_columns_widths(lf_ctx* c, const float* w, const float* a, const float* y, float* delta, float* gw,
+                               float* gb, const float* w_sub);
+void lf_columns_release(lf_ctx* c);
 
 // ---- TF32 tensor-core weight-gradient contraction (B > 1) ------------------------------------
 bool lf_tf32_supported(const lf_ctx* c);

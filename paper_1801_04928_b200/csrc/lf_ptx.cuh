@@ -63,6 +63,15 @@ __device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap* map
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, unsigned bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
 // ---- exchange slots: a value and the epoch of the call that wrote it, in one 64-bit word ---------
 // One 64-bit store publishes both and one 64-bit load reads both, so neither a fence nor a
 // separate flag is needed; the epoch changes with every call, so the slots are never cleared.

@@ -23,7 +23,7 @@ SHAPES = [
 ]
 
 
-def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0,
+def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, seed=0, variant=None,
          gw_math=lf.LF_GW_MATH_FP32, tiling=0, delta_math=lf.LF_DELTA_MATH_FP32):
     n = [int(v) for v in widths]
     L = len(n) - 1
@@ -41,7 +41,9 @@ def _run(widths, B, k, y="uniform", cost=0, act=0, sgd_eta=None, host=False, see
     with lf.Leapfrog(0, 0, B, k, stream=st.cuda_stream, widths=n) as ctx:
         ctx.set_option(lf.LF_OPT_COST, cost)
         ctx.set_option(lf.LF_OPT_ACTIVATION, act)
-        ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED)   # accepted; per-layer launches run
+        # the fused pass is accepted by every context: one sample runs it as one launch over all layers
+        # (whole columns per CTA), a mini-batch runs one launch per layer
+        ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED if variant is None else variant)
         ctx.set_option(lf.LF_OPT_GW_MATH, gw_math)
         ctx.set_option(lf.LF_OPT_DELTA_MATH, delta_math)
         ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
@@ -102,12 +104,19 @@ def _compare(n, B, cpu, out, cross_entropy=False, sgd_eta=None, tf32=False):
             assert err <= bound, (l, err, bound)
 
 
+@pytest.mark.parametrize("variant", [lf.LF_VARIANT_STREAMS, lf.LF_VARIANT_FUSED])
 @pytest.mark.parametrize("B,k", [(1, 1), (1, 3), (5, 2), (130, 2)])
 @pytest.mark.parametrize("widths", SHAPES, ids=lambda s: "-".join(map(str, s)))
-def test_widths_parity(widths, B, k):
-    n, L, cpu, out, stats = _run(widths, B, k, y="onehot" if B > 1 else "uniform", seed=len(widths) + B)
-    assert stats["device_status"] == 0
-    assert stats["variant"] == lf.LF_VARIANT_STREAMS and stats["N"] == max(n)
+def test_widths_parity(widths, B, k, variant):
+    if B > 1 and variant == lf.LF_VARIANT_FUSED:
+        pytest.skip("a mini-batch runs one launch per layer whatever is asked for")
+    n, L, cpu, out, stats = _run(widths, B, k, y="onehot" if B > 1 else "uniform", seed=len(widths) + B, variant=variant)
+    assert stats["device_status"] == 0 and stats["N"] == max(n)
+    if B == 1 and variant == lf.LF_VARIANT_FUSED:       # one launch over all layers, whatever their widths
+        assert stats["variant"] == lf.LF_VARIANT_FUSED and stats["launches_backward"] == 1
+        assert stats["fused_tiling"] == lf.LF_FUSED_TILING_COLUMNS
+    else:
+        assert stats["variant"] == lf.LF_VARIANT_STREAMS
     assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == lf.LF_DELTA_MATH_FP32
     _compare(n, B, cpu, out)
 
@@ -274,7 +283,71 @@ def test_hidden_run_goes_through_the_single_launch_pass(widths, k, variant):
     assert stats["variant"] in (lf.LF_VARIANT_PERSISTENT, lf.LF_VARIANT_FUSED)
     if variant != lf.LF_VARIANT_AUTO:
         assert stats["variant"] == variant
-    assert stats["launches_backward"] == 6            # bp1, 2 x bp2, 2 x rank-1 writer, 1 persistent launch
+    if variant == lf.LF_VARIANT_PERSISTENT:
+        assert stats["launches_backward"] == 6        # bp1, 2 x bp2, 2 x rank-1 writer, 1 persistent launch
+    else:                                             # the fused pass with whole columns takes all layers at once
+        assert stats["launches_backward"] == 1 and stats["fused_tiling"] == lf.LF_FUSED_TILING_COLUMNS
+    _compare(n, 1, cpu, out)
+
+
+@pytest.mark.parametrize("widths", HIDDEN_RUN_SHAPES[:3], ids=lambda s: "-".join(map(str, s)))
+def test_hidden_run_between_per_layer_launches_with_cluster_tiles(widths, monkeypatch):
+    # the cluster-tile fused kernel needs one width: asked for by name it runs over the hidden run,
+    # with per-layer launches for the rectangular top and bottom layer
+    monkeypatch.setenv("LF_FUSED_TILING", "clusters")
+    n, cpu, out, stats = _run_variant(widths, 2, lf.LF_VARIANT_FUSED, seed=len(widths))
+    assert stats["variant"] == lf.LF_VARIANT_FUSED and stats["fused_tiling"] == lf.LF_FUSED_TILING_CLUSTERS
+    assert stats["launches_backward"] == 6 and stats["device_status"] == 0
+    _compare(n, 1, cpu, out)
+
+
+@pytest.mark.parametrize("cost,act", [(lf.LF_COST_CROSS_ENTROPY, lf.LF_ACT_SIGMOID), (lf.LF_COST_QUADRATIC, lf.LF_ACT_TANH)])
+def test_single_launch_over_different_widths_costs_and_activations(cost, act):
+    widths = [260, 132, 516, 64, 200]
+    n, L, cpu, out, stats = _run(widths, 1, 2, y="onehot" if cost else "uniform", cost=cost, act=act, seed=33)
+    assert stats["variant"] == lf.LF_VARIANT_FUSED and stats["launches_backward"] == 1 and stats["device_status"] == 0
+    with orc.activation({lf.LF_ACT_SIGMOID: "sigmoid", lf.LF_ACT_TANH: "tanh"}[act]):
+        _compare(n, 1, cpu, out, cross_entropy=bool(cost))
+
+
+def test_single_launch_over_different_widths_shards_and_bounded_waits():
+    widths = [260, 516, 132, 516, 64, 200]
+    L = len(widths) - 1
+    # two shards: each stores the gradients of its own layers only
+    for S in (2, 3):
+        seen = np.zeros(L, dtype=int)
+        for r in range(S):
+            n, cpu, out, stats = _run_variant(widths, 2, lf.LF_VARIANT_FUSED, seed=12, shard=(r, S))
+            assert stats["launches_backward"] == 1 and stats["device_status"] == 0
+            w = cpu["w"].numpy()
+            z, a = orc.forward_widths(n, w, cpu["b"].numpy(), cpu["x"].numpy())
+            delta, gw, gb = orc.backward_widths(n, w, z, a, cpu["y"].numpy())
+            for l, (g, ref) in enumerate(zip(orc.split(out["gw"], n, "w"), orc.split(gw, n, "w")), start=1):
+                if (L - l) % S == r:
+                    assert_layer_close("gw", l - 1, g, ref, tol=FP32_TOL, n_terms=max(n))
+                    seen[l - 1] += 1
+                else:
+                    assert np.all(np.isnan(g)), (S, r, l)
+        assert np.all(seen == 1)
+    # one CTA publishes nothing: the others give up within the budget and the next call is right again
+    n = widths
+    cpu = lf_inputs.make_inputs_widths(n, 1, "uniform", lf_inputs.SEED_BASE + 5, "cpu")
+    t = {key: v.cuda() for key, v in cpu.items()}
+    sz = orc.sizes_widths(n, 1)
+    z = torch.empty(sz["z"], device="cuda"); a = torch.empty(sz["a"], device="cuda")
+    delta = torch.empty(sz["z"], device="cuda"); gw = torch.empty(sz["w"], device="cuda"); gb = torch.empty(sz["b"], device="cuda")
+    with lf.Leapfrog(0, 0, 1, 2, widths=n) as ctx:
+        ctx.set_option(lf.LF_OPT_VARIANT, lf.LF_VARIANT_FUSED)
+        ctx.set_option(lf.LF_OPT_WAIT_BUDGET_US, 20000)
+        ctx.forward(t["w"], t["b"], t["x"], z, a)
+        ctx.set_option(lf.LF_OPT_WITHHOLD, 1)
+        ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        assert lf.lf_sync(ctx._h) == lf.LF_ETIMEOUT
+        ctx.set_option(lf.LF_OPT_WITHHOLD, 0)
+        ctx.backward(t["w"], z, a, t["y"], delta, gw, gb)
+        ctx.sync()
+        assert ctx.stats()["device_status"] == 0 and ctx.stats()["launches_backward"] == 1
+    out = {key: v.cpu().numpy() for key, v in dict(z=z, a=a, delta=delta, gw=gw, gb=gb).items()}
     _compare(n, 1, cpu, out)
 
 
