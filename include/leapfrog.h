@@ -70,7 +70,9 @@ enum lf_gw_math {
 /* Arithmetic of the B > 1 delta recurrence and forward pass (Eq. bp2 and Eq. z as N x N x B
  * contractions). */
 enum lf_delta_math {
-    LF_DELTA_MATH_AUTO = 0,  /* tensor cores when B > 1 and the device supports it               */
+    LF_DELTA_MATH_AUTO = 0,  /* tensor cores when B > 1 and the device supports it; Eq. bp2 for 2 to
+                                16 samples stays fp32 on the CUDA cores (a batched matrix-vector
+                                product that reads w^{l+1} once, at the memory rate)              */
     LF_DELTA_MATH_FP32 = 1,  /* fp32 FMA on the CUDA cores                                        */
     LF_DELTA_MATH_3XTF32 = 2 /* tensor cores; every operand split into two TF32 numbers, three
                                 products per term, fp32 accumulation: fp32-level accuracy        */

@@ -91,9 +91,20 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
     return LF_OK;
 }
 
+// Arithmetic of the forward pass for B > 1 (Eq. z as a contraction).
+int resolve_forward_math(const lf_ctx* c)
+{
+    if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
+    return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
+}
+
+// Arithmetic of Eq. bp2 for B > 1.  A handful of samples is a batched matrix-vector product: fp32 on
+// the CUDA cores at the memory rate beats tensor-core tiles that are nearly empty (unless the
+// tensor cores are asked for by name).
 int resolve_delta_math(const lf_ctx* c)
 {
     if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
+    if (c->opt_delta_math == LF_DELTA_MATH_AUTO && c->B <= lfk_small_batch_max() && c->sb_partial) return LF_DELTA_MATH_FP32;
     return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
 }
 
@@ -118,7 +129,10 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
             int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, n_up, n_l, s, launches);
             if (rc != LF_OK) return rc;
             return LF_OK;
-        } else
+        } else if (B <= lfk_small_batch_max() && c->sb_partial)
+            LF_CUDA_TRY(c, lfk_delta_small_batch(w_up, d_up, a_l, d_l, c->sb_partial, c->counters, n_up, n_l, B,
+                                                 c->opt_act, s));
+        else
             LF_CUDA_TRY(c, lfk_delta_gemm(w_up, d_up, a_l, d_l, n_up, n_l, B, c->opt_act, s));
     }
     *launches += 1;
@@ -366,6 +380,14 @@ int lf_create_widths(lf_ctx** out, int L, const int* widths, int B, int k)
     ok = ok && cudaMalloc(&c->sync_words, c->sync_words_count * sizeof(unsigned)) == cudaSuccess;
     ws += c->sync_words_count * sizeof(unsigned);
     ok = ok && cudaMalloc(&c->status_dev, sizeof(unsigned)) == cudaSuccess; ws += sizeof(unsigned);
+    if (B > 1 && B <= lfk_small_batch_max()) {
+        size_t sb_floats = 0;
+        for (int l = 1; l < L; ++l) {
+            const size_t f = lfk_delta_small_batch_scratch_floats(widths[l + 1], widths[l], B);
+            if (f > sb_floats) sb_floats = f;
+        }
+        if (sb_floats) { ok = ok && cudaMalloc(&c->sb_partial, sb_floats * sizeof(float)) == cudaSuccess; ws += sb_floats * sizeof(float); }
+    }
     const size_t dg_bytes = lf_delta_tc_scratch_bytes(c);
     if (dg_bytes) { ok = ok && cudaMalloc(&c->dg_partial, dg_bytes) == cudaSuccess; ws += dg_bytes; }
     ok = ok && cudaMallocHost(&c->status_host, sizeof(unsigned)) == cudaSuccess;
@@ -503,7 +525,7 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
         if (B == 1) {
             LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, ctx->opt_act, s));
             ++launches;
-        } else if (resolve_delta_math(ctx) == LF_DELTA_MATH_3XTF32) {
+        } else if (resolve_forward_math(ctx) == LF_DELTA_MATH_3XTF32) {
             int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, n_out, n_in, s, &launches);
             if (rc2 != LF_OK) return rc2;
         } else {
@@ -834,6 +856,7 @@ int lf_destroy(lf_ctx* ctx)
     if (ctx->sync_words) cudaFree(ctx->sync_words);
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     if (ctx->dg_partial) cudaFree(ctx->dg_partial);
+    if (ctx->sb_partial) cudaFree(ctx->sb_partial);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     if (ctx->stage) cudaFree(ctx->stage);
     if (ctx->h2d_stream) { cudaStreamSynchronize(ctx->h2d_stream); cudaStreamDestroy(ctx->h2d_stream); }

@@ -97,6 +97,7 @@ struct lf_ctx {
     unsigned* status_dev;    // device status word
     unsigned* status_host;   // pinned mirror
     float* dg_partial;       // B > 1: K-split partial sums of the tensor-core delta GEMM
+    float* sb_partial;       // 1 < B <= 16: row-chunk partial sums of the small-batch Eq. bp2 kernel
 
     // leapfrog workers as streams
     cudaStream_t* wstreams;  // keff streams
@@ -185,6 +186,11 @@ cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float
 cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                              int B, lf_sgd sgd, cudaStream_t s);
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s);
+// Eq. bp2 for a handful of samples (B <= lfk_small_batch_max()): w read once at the memory rate, fp32
+int lfk_small_batch_max();
+size_t lfk_delta_small_batch_scratch_floats(int n_up, int n_l, int B);
+cudaError_t lfk_delta_small_batch(const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
+                                  float* partial, unsigned* counters, int n_up, int n_l, int B, int act, cudaStream_t s);
 
 // ---- persistent single-launch backward (B = 1) ---------------------------------------------
 size_t lf_sync_words_needed(const lf_ctx* c);           // unsigned words of flag/barrier workspace

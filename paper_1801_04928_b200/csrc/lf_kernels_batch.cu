@@ -155,6 +155,190 @@ cudaError_t lfk_forward_gemm(const float* w_l, const float* b_l, const float* a_
     return cudaGetLastError();
 }
 
+
+namespace {
+
+// ---- Eq. bp2 for a handful of samples (B <= 16) --------------------------------------------------
+// With so few samples the contraction is a batched matrix-vector product: w^{l+1} is read once, at the
+// memory rate, and every loaded weight is used B times from registers (4B fused multiply-adds per
+// 16 bytes).  Tiles of tensor-core size would spend their time staging a nearly empty operand.
+//   grid = column strips (128 columns) x row chunks, sized to one wave of resident CTAs.  A CTA of
+//   eight warps walks the rows of its chunk (warp q: rows q, q+8, ...), each lane four columns and BT
+//   running sums of them.  Every thread prefetches its own 16 bytes of the next SB_DEPTH rows with
+//   cp.async into a ring slot only it reads, so the loads in flight cost no registers and need no
+//   barrier.  The delta values of 256 rows at a time sit in shared memory as float4 over four
+//   samples, so one broadcast 128-bit load feeds four samples.
+//   Partial sums go to scratch [chunks][B][n_l]; the last CTA of a strip to finish adds them in chunk
+//   order (a fixed order: results are reproducible), applies sigma' and writes delta^l.
+constexpr int SB_WARPS = 8, SB_THREADS = SB_WARPS * 32, SB_STRIP4 = 32, SB_BLOCK_ROWS = 256, SB_DEPTH = 8;
+constexpr int SB_MIN_ROWS = 64;     // a chunk has at least this many rows (bounds the number of partial sums)
+
+template <int BT>
+constexpr int sb_smem_bytes()
+{
+    // ring [SB_DEPTH][threads] float4, then delta [BT/4][SB_BLOCK_ROWS] float4; the reduction
+    // ([warps][32 lanes][4 samples] float4 = 16 KiB) reuses the ring
+    return SB_DEPTH * SB_THREADS * 16 + (BT / 4) * SB_BLOCK_ROWS * 16;
+}
+
+__device__ __forceinline__ void sb_cp_async16(unsigned dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void sb_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N_PENDING>
+__device__ __forceinline__ void sb_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N_PENDING) : "memory"); }
+
+template <int BT>
+__global__ void __launch_bounds__(SB_THREADS, BT <= 4 ? 4 : BT <= 8 ? 3 : 2)
+k_delta_small_batch(const float* __restrict__ w_up, const float* __restrict__ delta_up, const float* __restrict__ a_l,
+                    float* __restrict__ delta_l, float* __restrict__ partial, unsigned* __restrict__ counters,
+                    int n_up, int n_l, int B, int rows_per_chunk, int chunks, int act)
+{
+    extern __shared__ __align__(16) unsigned char sb_smem[];
+    float4* ring = reinterpret_cast<float4*>(sb_smem);                                   // [SB_DEPTH][threads]
+    float4* d_sm = reinterpret_cast<float4*>(sb_smem + SB_DEPTH * SB_THREADS * 16);      // [BT/4][SB_BLOCK_ROWS]
+    __shared__ bool is_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int strip = blockIdx.x, chunk = blockIdx.y;
+    const int n4 = n_l >> 2;
+    const int c4 = strip * SB_STRIP4 + lane;
+    const bool col_ok = c4 < n4;
+    const int row0 = chunk * rows_per_chunk;
+    const int rows = min(rows_per_chunk, n_up - row0);
+    const int my_rows = rows > warp ? (rows - warp + SB_WARPS - 1) / SB_WARPS : 0;     // rows warp, warp + 8, ...
+    const float4* wp = reinterpret_cast<const float4*>(w_up) + (size_t)(row0 + warp) * n4 + (col_ok ? c4 : 0);
+    const unsigned ring_u32 = (unsigned)__cvta_generic_to_shared(ring + tid);
+
+    // prologue: my first SB_DEPTH - 1 rows are on their way (one group per row, empty past the end)
+#pragma unroll
+    for (int i = 0; i < SB_DEPTH - 1; ++i) {
+        if (col_ok && i < my_rows) sb_cp_async16(ring_u32 + i * SB_THREADS * 16, wp + (size_t)i * SB_WARPS * n4);
+        sb_cp_commit();
+    }
+
+    float4 acc[BT];
+#pragma unroll
+    for (int b = 0; b < BT; ++b) acc[b] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    int i = 0;     // index of my next row
+    for (int blk0 = 0; blk0 < rows; blk0 += SB_BLOCK_ROWS) {
+        const int blk_rows = min(SB_BLOCK_ROWS, rows - blk0);
+        __syncthreads();      // the previous block's delta values are no longer read
+        for (int idx = tid; idx < (BT / 4) * SB_BLOCK_ROWS; idx += SB_THREADS) {
+            const int j = idx & (SB_BLOCK_ROWS - 1), b4 = idx / SB_BLOCK_ROWS;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j < blk_rows) {
+                const float* src = delta_up + (size_t)(4 * b4) * n_up + row0 + blk0 + j;
+                if (4 * b4 + 0 < B) v.x = __ldcg(src);
+                if (4 * b4 + 1 < B) v.y = __ldcg(src + n_up);
+                if (4 * b4 + 2 < B) v.z = __ldcg(src + 2 * (size_t)n_up);
+                if (4 * b4 + 3 < B) v.w = __ldcg(src + 3 * (size_t)n_up);
+            }
+            d_sm[idx] = v;
+        }
+        __syncthreads();
+        const int i_end = min(my_rows, (blk0 + blk_rows - warp + SB_WARPS - 1) / SB_WARPS);   // my rows below the block's end
+        for (; i < i_end; ++i) {
+            const int nx = i + SB_DEPTH - 1;
+            if (col_ok && nx < my_rows)
+                sb_cp_async16(ring_u32 + (nx % SB_DEPTH) * SB_THREADS * 16, wp + (size_t)nx * SB_WARPS * n4);
+            sb_cp_commit();
+            sb_cp_wait<SB_DEPTH - 1>();      // the group of row i has landed
+            const float4 wv = ring[(i % SB_DEPTH) * SB_THREADS + tid];
+            const int j = warp + i * SB_WARPS - blk0;
+#pragma unroll
+            for (int b4 = 0; b4 < BT / 4; ++b4) {
+                const float4 d = d_sm[b4 * SB_BLOCK_ROWS + j];
+                float4& a0 = acc[4 * b4], &a1 = acc[4 * b4 + 1], &a2 = acc[4 * b4 + 2], &a3 = acc[4 * b4 + 3];
+                a0.x = fmaf(wv.x, d.x, a0.x); a0.y = fmaf(wv.y, d.x, a0.y); a0.z = fmaf(wv.z, d.x, a0.z); a0.w = fmaf(wv.w, d.x, a0.w);
+                a1.x = fmaf(wv.x, d.y, a1.x); a1.y = fmaf(wv.y, d.y, a1.y); a1.z = fmaf(wv.z, d.y, a1.z); a1.w = fmaf(wv.w, d.y, a1.w);
+                a2.x = fmaf(wv.x, d.z, a2.x); a2.y = fmaf(wv.y, d.z, a2.y); a2.z = fmaf(wv.z, d.z, a2.z); a2.w = fmaf(wv.w, d.z, a2.w);
+                a3.x = fmaf(wv.x, d.w, a3.x); a3.y = fmaf(wv.y, d.w, a3.y); a3.z = fmaf(wv.z, d.w, a3.z); a3.w = fmaf(wv.w, d.w, a3.w);
+            }
+        }
+    }
+    sb_cp_wait<0>();
+    __syncthreads();      // the ring is free: the eight warps' sums meet there, four samples per round
+    float4* red = ring;                                          // [8 warps][32 lanes][4 samples]
+#pragma unroll
+    for (int r = 0; r < BT / 4; ++r) {
+#pragma unroll
+        for (int sidx = 0; sidx < 4; ++sidx) red[(warp * 32 + lane) * 4 + sidx] = col_ok ? acc[4 * r + sidx] : make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncthreads();
+        if (tid < 128) {
+            const int l = tid & 31, sidx = tid >> 5, b = 4 * r + sidx, c = strip * SB_STRIP4 + l;
+            float4 sum = red[l * 4 + sidx];
+#pragma unroll
+            for (int q = 1; q < SB_WARPS; ++q) {
+                const float4 t = red[(q * 32 + l) * 4 + sidx];
+                sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+            }
+            if (b < B && c < n4) reinterpret_cast<float4*>(partial)[((size_t)chunk * B + b) * n4 + c] = sum;
+        }
+        __syncthreads();
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = atomicAdd(&counters[strip], 1u) == (unsigned)chunks - 1u;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // last CTA of the strip: every (sample, four columns) of the strip, chunks added in order
+    for (int idx = tid; idx < B * SB_STRIP4; idx += SB_THREADS) {
+        const int b = idx >> 5, c = strip * SB_STRIP4 + (idx & 31);
+        if (c >= n4) continue;
+        const float4* src = reinterpret_cast<const float4*>(partial) + (size_t)b * n4 + c;
+        const size_t step = (size_t)B * n4;
+        float4 sum = __ldcg(src);
+#pragma unroll 8
+        for (int q = 1; q < chunks; ++q) {
+            const float4 t = __ldcg(src + q * step);
+            sum.x += t.x; sum.y += t.y; sum.z += t.z; sum.w += t.w;
+        }
+        const float4 av = reinterpret_cast<const float4*>(a_l)[(size_t)b * n4 + c];
+        reinterpret_cast<float4*>(delta_l)[(size_t)b * n4 + c] =
+            make_float4(sum.x * lf_act_prime(av.x, act), sum.y * lf_act_prime(av.y, act),
+                        sum.z * lf_act_prime(av.z, act), sum.w * lf_act_prime(av.w, act));
+    }
+    if (tid == 0) counters[strip] = 0u;   // ready for the next launch
+}
+
+// CTAs of the kernel (BT running sums per column) that one SM holds; asked of the runtime once.
+template <int BT>
+int sb_ctas_per_sm()
+{
+    static int per_device[64] = {};     // the attribute below belongs to a device's copy of the kernel
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (per_device[dev]) return per_device[dev];
+    cudaFuncSetAttribute(k_delta_small_batch<BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb_smem_bytes<BT>());
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_delta_small_batch<BT>, SB_THREADS, sb_smem_bytes<BT>()) != cudaSuccess || n < 1)
+        n = 1;
+    per_device[dev] = n;
+    return n;
+}
+
+// rows of w^{l+1} per chunk: as many chunks as fill the resident CTA slots once, none shorter than
+// SB_MIN_ROWS rows
+int sb_rows_per_chunk(int n_up, int n_l, int B)
+{
+    const int strips = ((n_l >> 2) + SB_STRIP4 - 1) / SB_STRIP4;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int per_sm = B <= 4 ? sb_ctas_per_sm<4>() : B <= 8 ? sb_ctas_per_sm<8>() : sb_ctas_per_sm<16>();
+    int chunks = sms * per_sm / strips;
+    const int most = (n_up + SB_MIN_ROWS - 1) / SB_MIN_ROWS;
+    if (chunks > most) chunks = most;
+    if (chunks < 1) chunks = 1;
+    int rows = (n_up + chunks - 1) / chunks;
+    rows = (rows + 7) & ~7;
+    return rows;
+}
+
+}  // namespace
+
 cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float* a_l,
                            float* delta_l, int n_up, int n_l, int B, int act, cudaStream_t s)
 {
@@ -176,5 +360,31 @@ cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* g
 cudaError_t lfk_grad_b_colsum(const float* delta_l, float* gb_l, int N, int B, cudaStream_t s)
 {
     k_grad_b_colsum<<<(N + 31) / 32, 256, 0, s>>>(delta_l, gb_l, N, B);
+    return cudaGetLastError();
+}
+
+// ---- Eq. bp2 for B <= 16 samples: scratch sizes and launch ------------------------------------------
+int lfk_small_batch_max() { return 16; }
+
+size_t lfk_delta_small_batch_scratch_floats(int n_up, int n_l, int B)
+{
+    const int rows = sb_rows_per_chunk(n_up, n_l, B);
+    const int chunks = (n_up + rows - 1) / rows;
+    return (size_t)chunks * B * n_l;
+}
+
+cudaError_t lfk_delta_small_batch(const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
+                                  float* partial, unsigned* counters, int n_up, int n_l, int B, int act, cudaStream_t s)
+{
+    const int rows = sb_rows_per_chunk(n_up, n_l, B);
+    const int chunks = (n_up + rows - 1) / rows;
+    const int strips = ((n_l >> 2) + SB_STRIP4 - 1) / SB_STRIP4;
+    dim3 grid(strips, chunks);
+    if (B <= 4)
+        k_delta_small_batch<4><<<grid, SB_THREADS, sb_smem_bytes<4>(), s>>>(w_up, delta_up, a_l, delta_l, partial, counters, n_up, n_l, B, rows, chunks, act);
+    else if (B <= 8)
+        k_delta_small_batch<8><<<grid, SB_THREADS, sb_smem_bytes<8>(), s>>>(w_up, delta_up, a_l, delta_l, partial, counters, n_up, n_l, B, rows, chunks, act);
+    else
+        k_delta_small_batch<16><<<grid, SB_THREADS, sb_smem_bytes<16>(), s>>>(w_up, delta_up, a_l, delta_l, partial, counters, n_up, n_l, B, rows, chunks, act);
     return cudaGetLastError();
 }

@@ -62,6 +62,25 @@ def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
     compare_all(cfg, out, ref)
 
 
+@pytest.mark.parametrize("L,N,B,k", [(3, 516, 2, 2), (3, 1028, 5, 1), (2, 2052, 12, 2), (3, 4096, 16, 2),
+                                     (2, 8, 4, 1), (4, 644, 9, 3)])
+def test_small_batch_delta_chain(L, N, B, k):
+    # Up to 16 samples the library's own choice for Eq. bp2 is fp32 on the CUDA cores (a batched
+    # matrix-vector product that reads w once), not the tensor cores; the forward pass keeps its
+    # tensor-core rule.  B = 2, 5, 12: each of the kernel's three sample-tile sizes with samples
+    # missing from the last group of four; N = 516, 1028, 2052, 644: a last column strip of one or
+    # five float4; N = 4096, B = 16: several 256-row blocks per CTA; N = 8: fewer rows than warps.
+    cfg = dict(L=L, N=N, B=B, k=k)
+    t = _inputs(L, N, B, y="onehot", seed=7 * N + B)
+    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32)
+    assert stats["delta_math"] == lf.LF_DELTA_MATH_FP32 and stats["device_status"] == 0
+    ref = oracle_pass(t, want_gw=True)
+    compare_all(cfg, out, ref)
+    # twice in a row through one context: the strip counters reset themselves
+    out2, _ = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, repeat=3)
+    assert torch.equal(out2["delta"], out["delta"])
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_result_does_not_depend_on_k(variant):
     # Theorem 1 on the GPU: every schedule writes every layer once, and because the delta
