@@ -74,8 +74,14 @@ enum lf_delta_math {
                                 16 samples stays fp32 on the CUDA cores (a batched matrix-vector
                                 product that reads w^{l+1} once, at the memory rate)              */
     LF_DELTA_MATH_FP32 = 1,  /* fp32 FMA on the CUDA cores                                        */
-    LF_DELTA_MATH_3XTF32 = 2 /* tensor cores; every operand split into two TF32 numbers, three
+    LF_DELTA_MATH_3XTF32 = 2, /* tensor cores; every operand split into two TF32 numbers, three
                                 products per term, fp32 accumulation: fp32-level accuracy        */
+    LF_DELTA_MATH_TF32_BF16 = 3 /* tensor cores; the product of the two high parts in TF32, the two
+                                cross terms (each below 2^-11 of the product) in BF16: eight
+                                instead of twelve instructions per K stage, about 2^-20 per
+                                term.  Applies to CTA-pair tiles (one-CTA tiles keep three TF32
+                                products).  Never chosen by AUTO: as measured, splitting the
+                                operands, not the tensor cores, then bounds the kernel.          */
 };
 
 /* Tiling of the tensor-core contractions (B > 1): one CTA per tile, or a pair of CTAs (two

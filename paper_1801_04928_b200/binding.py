@@ -30,7 +30,7 @@ LF_FUSED_TILING_AUTO, LF_FUSED_TILING_CLUSTERS, LF_FUSED_TILING_COLUMNS = 0, 1, 
 LF_ACT_SIGMOID, LF_ACT_TANH, LF_ACT_RELU = 0, 1, 2
 LF_COST_QUADRATIC, LF_COST_CROSS_ENTROPY = 0, 1
 LF_TC_TILING_AUTO, LF_TC_TILING_ONE_SM, LF_TC_TILING_TWO_SM = 0, 1, 2
-LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32 = 0, 1, 2
+LF_DELTA_MATH_AUTO, LF_DELTA_MATH_FP32, LF_DELTA_MATH_3XTF32, LF_DELTA_MATH_TF32_BF16 = 0, 1, 2, 3
 
 EXPORTS = ("lf_create", "lf_create_widths", "lf_set_stream", "lf_set_option", "lf_forward", "lf_backward",
            "lf_backward_sgd", "lf_grad_w", "lf_backward_host", "lf_sync", "lf_owner", "lf_get_stats", "lf_last_cuda_error",

@@ -95,7 +95,8 @@ int enqueue_gradients(lf_ctx* c, int l, const float* a, const float* delta, floa
 int resolve_forward_math(const lf_ctx* c)
 {
     if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
-    return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
+    if (!lf_delta_tc_supported(c)) return LF_DELTA_MATH_FP32;
+    return c->opt_delta_math == LF_DELTA_MATH_TF32_BF16 ? LF_DELTA_MATH_TF32_BF16 : LF_DELTA_MATH_3XTF32;
 }
 
 // Arithmetic of Eq. bp2 for B > 1.  A handful of samples is a batched matrix-vector product: fp32 on
@@ -105,7 +106,8 @@ int resolve_delta_math(const lf_ctx* c)
 {
     if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
     if (c->opt_delta_math == LF_DELTA_MATH_AUTO && c->B <= lfk_small_batch_max() && c->sb_partial) return LF_DELTA_MATH_FP32;
-    return lf_delta_tc_supported(c) ? LF_DELTA_MATH_3XTF32 : LF_DELTA_MATH_FP32;
+    if (!lf_delta_tc_supported(c)) return LF_DELTA_MATH_FP32;
+    return c->opt_delta_math == LF_DELTA_MATH_TF32_BF16 ? LF_DELTA_MATH_TF32_BF16 : LF_DELTA_MATH_3XTF32;
 }
 
 // One delta-chain step on stream s: Eq. bp1 for l = L, Eq. bp2 below.
@@ -125,8 +127,8 @@ int enqueue_chain_step(lf_ctx* c, int l, const float* w, const float* a, const f
         if (B == 1)
             LF_CUDA_TRY(c, lfk_delta_matvec(w_up, d_up, a_l, d_l, gb_l, c->partial, c->counters, n_up, n_l,
                                             c->opt_act, s));
-        else if (c->stats.delta_math == LF_DELTA_MATH_3XTF32) {
-            int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, n_up, n_l, s, launches);
+        else if (c->stats.delta_math >= LF_DELTA_MATH_3XTF32) {
+            int rc = lf_delta_gemm_tc(c, w_up, d_up, a_l, d_l, n_up, n_l, c->stats.delta_math, s, launches);
             if (rc != LF_OK) return rc;
             return LF_OK;
         } else if (B <= lfk_small_batch_max() && c->sb_partial)
@@ -449,7 +451,7 @@ int lf_set_option(lf_ctx* ctx, int key, long long value)
             ctx->wait_budget_us = value;
             return LF_OK;
         case LF_OPT_DELTA_MATH:
-            if (value < LF_DELTA_MATH_AUTO || value > LF_DELTA_MATH_3XTF32) return LF_EINVAL;
+            if (value < LF_DELTA_MATH_AUTO || value > LF_DELTA_MATH_TF32_BF16) return LF_EINVAL;
             ctx->opt_delta_math = (int)value;
             return LF_OK;
         case LF_OPT_TC_TILING:
@@ -525,8 +527,8 @@ int lf_forward(lf_ctx* ctx, const float* w, const float* b, const float* x, floa
         if (B == 1) {
             LF_CUDA_TRY(ctx, lfk_forward_matvec(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, ctx->opt_act, s));
             ++launches;
-        } else if (resolve_forward_math(ctx) == LF_DELTA_MATH_3XTF32) {
-            int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, n_out, n_in, s, &launches);
+        } else if (resolve_forward_math(ctx) >= LF_DELTA_MATH_3XTF32) {
+            int rc2 = lf_forward_gemm_tc(ctx, w_l, b_l, a_prev, z_l, a_l, n_out, n_in, resolve_forward_math(ctx), s, &launches);
             if (rc2 != LF_OK) return rc2;
         } else {
             LF_CUDA_TRY(ctx, lfk_forward_gemm(w_l, b_l, a_prev, z_l, a_l, n_out, n_in, B, ctx->opt_act, s));

@@ -244,12 +244,15 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                     const unsigned bar = dg_smem_u32(&sh->full[st]);
                     dg_mbar_expect_tx(bar, DG_RAW_BYTES);
                     const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
-                    dg_tma_load_2d(a_dst, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM);
-                    if (W_KMAJOR) {
-                        dg_tma_load_2d(a_dst + DG_A_BYTES, &map_w, bar, j0 + ks * DG_BK, tn * DG_BN);
-                    } else {
+                    // boxes of 32 rows: the loads of one box are few at a time, several boxes go side by side
 #pragma unroll
-                        for (int i = 0; i < DG_BN / 32; ++i)
+                    for (int i = 0; i < DG_BM / 32; ++i)
+                        dg_tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM + i * 32);
+#pragma unroll
+                    for (int i = 0; i < DG_BN / 32; ++i) {
+                        if (W_KMAJOR)
+                            dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, tn * DG_BN + i * 32);
+                        else
                             dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
                                            j0 + ks * DG_BK);
                     }
@@ -385,14 +388,15 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 // finished stage into the running sums -- have warps of their own here, so they overlap:
 //   warp 0       TMA producer: this CTA's 128 samples of D and its 128 columns of W per stage;
 //   warp 1       leader CTA (cluster rank 0) only: issues the products for both CTAs;
-//   warps 2-7    split this CTA's stage into hi/lo (in place + beside it);
+//   warps 2-7    split this CTA's stage into hi/lo (high parts in place, the rest into a second ring);
 //   warps 8-15   running sums of this CTA's 128 samples: a thread holds one sample and 128 of
 //                the 256 columns in registers.  They need about 200 registers per thread and the
 //                other warps few, so the warpgroups re-divide the register file at the start
 //                (setmaxnreg: 2 x 128 threads x 48 + 2 x 128 threads x 208 = 512 x 128).
 // Hand-offs across the pair: the splitting warps of both CTAs arrive on the leader's "split done"
-// barrier, the leader's tcgen05.commit reaches the "stage free" and "accumulator full" barriers
-// of both CTAs, the summing warps of both arrive on the leader's "accumulator drained" barrier.
+// barrier, the leader's tcgen05.commit reaches the "raw slot free", "second-ring slot free" and
+// "accumulator full" barriers of both CTAs, the summing warps of both arrive on the leader's
+// "accumulator drained" barrier.
 // Work is dealt by K block, not by tile: the tiles x K-blocks sequence is cut into one contiguous
 // run per pair (runs differ by at most one block), so a pair may finish one tile's tail and
 // start the next tile.  Every run segment inside a tile writes its partial sums to the slot
@@ -401,10 +405,17 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 // Arithmetic per output element is that of the one-SM kernel above.
 constexpr int DP_BN = 256;                               // columns of a pair tile (128 loaded per CTA)
 constexpr int DP_BNH = DP_BN / 2;
-constexpr int DP_STAGES = 3;
 constexpr int DP_B_BYTES = (DP_BNH / 32) * DG_BOX_BYTES; // 16 KiB (either operand form)
 constexpr int DP_RAW_BYTES = DG_A_BYTES + DP_B_BYTES;    // 32 KiB per CTA and stage from TMA
-constexpr int DP_STAGE_BYTES = 2 * DP_RAW_BYTES;         // hi (in place) + lo
+// A stage lives in two rings.  Its raw tile (where the high parts then stand) holds a slot from the
+// moment its load is issued until its products are done; what the split adds (remainders, or the
+// 16-bit tiles) is only needed from the split on.  Four raw slots keep loads in the air behind the
+// stage being worked on, and two slots of the second ring let the split of one stage run under the
+// products of the one before.  With the hand-offs cheap (see dp_arrive_cluster) a stage of twelve
+// TF32 instructions then takes about 2100 cycles, which is the rate the tensor cores issue them at.
+constexpr int DP_RAW_SLOTS = 4, DP_LO_SLOTS = 2;
+constexpr int DP_LO_BASE = DP_RAW_SLOTS * DP_RAW_BYTES;
+constexpr int DP_RING_BYTES = (DP_RAW_SLOTS + DP_LO_SLOTS) * DP_RAW_BYTES;
 constexpr int DP_THREADS = 512;                          // four warpgroups
 constexpr int DP_SPLITTERS = 192;                        // warps 2-7
 constexpr int DP_REGS_LAUNCH = 128, DP_REGS_SMALL = 48, DP_REGS_SUM = 208;
@@ -413,12 +424,14 @@ static_assert(2 * 128 * DP_REGS_SMALL + 2 * 128 * DP_REGS_SUM <= DP_THREADS * DP
 constexpr int DP_TMEM_COLS = 512;                        // two stage accumulators of 256 columns
 constexpr int DP_EPI_LD = 20;                            // 16 columns + padding
 constexpr int DP_EPI_BYTES = 8 * 32 * DP_EPI_LD * 4;
-constexpr size_t DP_SMEM_BYTES = (size_t)DP_STAGES * DP_STAGE_BYTES + DP_EPI_BYTES + 1024 + 256;
+constexpr size_t DP_SMEM_BYTES = (size_t)DP_RING_BYTES + DP_EPI_BYTES + 1024 + 256;
+static_assert(DP_SMEM_BYTES <= 227 * 1024, "the two rings, the output staging and the barriers must fit one CTA");
 
 struct DpShared {
-    unsigned long long full[DP_STAGES];        // this CTA's TMA data of the stage has landed
-    unsigned long long split_done[DP_STAGES];  // leader: hi/lo of both CTAs written (12 warp arrivals)
-    unsigned long long empty[DP_STAGES];       // both: the multiplications that read the stage are done
+    unsigned long long full[DP_RAW_SLOTS];      // this CTA's TMA data of the stage has landed
+    unsigned long long raw_empty[DP_RAW_SLOTS]; // both: the products that read the raw slot are done
+    unsigned long long split_done[DP_LO_SLOTS]; // leader: the stage is split in both CTAs (12 warp arrivals)
+    unsigned long long lo_empty[DP_LO_SLOTS];   // both: the products that read the second-ring slot are done
     unsigned long long acc_full[2];            // both: stage accumulator p holds a finished stage
     unsigned long long acc_empty[2];           // leader: accumulator p drained by both CTAs (16 warp arrivals)
     unsigned tmem_base;
@@ -450,6 +463,41 @@ __device__ __forceinline__ void dp_mma(unsigned d_tmem, unsigned long long a_des
         "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same instruction on 16-bit operands (here BF16 x BF16, sixteen values of the contraction index)
+__device__ __forceinline__ void dp_mma16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                         unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// MN-major 16-bit operand, 128-byte swizzle: 64 values along N per 128-byte row, eight K rows per
+// 1024-byte atom (SBO), the next 64 columns one 32-row block (4 KiB) further (LBO).
+__device__ __forceinline__ unsigned long long dp_desc_mnmajor16(unsigned smem_addr)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (unsigned long long)((4096u >> 4) & 0x3FFFu) << 16;
+    d |= (unsigned long long)((1024u >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+// BF16 operand of K step kk (sixteen values of the contraction index) of the W tile: part 0 = the
+// high parts, part 1 = the remainders
+template <bool W_KMAJOR>
+__device__ __forceinline__ unsigned long long dp_desc_w16(unsigned tile16_addr, int part, int kk)
+{
+    return W_KMAJOR ? dg_desc_kmajor(tile16_addr + part * 64 + kk * 32)
+                    : dp_desc_mnmajor16(tile16_addr + part * (DP_B_BYTES / 2) + kk * 2048);
+}
+// two fp32 values as BF16 (round to nearest, ties away from zero) in one word, the first in the low half
+__device__ __forceinline__ unsigned dp_pack_bf16(float a, float b)
+{
+    return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+}
 // arrive on the barrier at this offset in both CTAs once the tensor-core work issued so far is done
 __device__ __forceinline__ void dp_commit_both(unsigned bar)
 {
@@ -459,7 +507,10 @@ __device__ __forceinline__ void dp_commit_both(unsigned bar)
 }
 __device__ __forceinline__ void dp_arrive_cluster(unsigned cluster_bar)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+    // What the arriving warp wrote for the tensor cores has passed a proxy fence, what it read from
+    // tensor memory a tcgen05 fence.  A release at cluster scope here (.release.cluster) was measured
+    // at about 1300 cycles per hand-off, which then bounded the kernel at 3000 cycles per K stage.
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ bool dp_try_wait(unsigned bar, unsigned parity)
 {
@@ -513,12 +564,13 @@ __device__ __forceinline__ bool dp_next_segment(int& g, int g1, const DgParams& 
     g += sg.kb1 - sg.kb0;
     return true;
 }
-__device__ __forceinline__ unsigned dp_idesc(bool w_kmajor)
+// fmt: operand format of the instruction kind (kind::tf32: 2 = TF32; kind::f16: 1 = BF16)
+__device__ __forceinline__ unsigned dp_idesc(bool w_kmajor, unsigned fmt = 2u)
 {
     unsigned d = 0;
     d |= 1u << 4;                             // fp32 accumulator
-    d |= 2u << 7;                             // A: TF32
-    d |= 2u << 10;                            // B: TF32
+    d |= fmt << 7;                            // A
+    d |= fmt << 10;                           // B
     d |= 0u << 15;                            // A is K-major
     d |= (w_kmajor ? 0u : 1u) << 16;          // B operand: K-major or MN-major
     d |= (unsigned)(DP_BN >> 3) << 17;
@@ -549,7 +601,90 @@ __device__ __forceinline__ void dp_tmem_ld64(unsigned taddr, unsigned (&r)[64])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-template <bool W_KMAJOR>
+// What a splitting thread needs to place its pieces.  A raw stage is 256 rows of 128 bytes (the D
+// tile, then the W tile), eight 16-byte pieces per row.  In round i a warp takes four rows of one
+// group of eight rows -- its lanes 0-7, 8-15, 16-23, 24-31 the rows g, g + 4, g + 1, g + 5 of the
+// group (g = 0 or 2) -- so that the 8-byte BF16 stores of a half-warp, which for rows g and g + 4 fall
+// into opposite halves of the 128-byte lines, meet no bank twice.  A thread keeps its piece (tt & 7)
+// and its row within the group, which all swizzle terms depend on; its row advances by 24 per round.
+struct DpSplitPlace {
+    unsigned idx0;        // 16-byte piece of round 0: row * 8 + (tt & 7)
+    unsigned k_hi, k_lo;  // K-major tiles: byte offset in the BF16 row of the high parts / the remainders
+    unsigned mn0, mn1;    // MN-major W: the same for an even / odd 32-column box (high parts)
+};
+__device__ __forceinline__ DpSplitPlace dp_split_place(int tt)
+{
+    DpSplitPlace pl;
+    const unsigned p = tt & 7u, q = (tt >> 3) & 3u, w = (unsigned)tt >> 5;
+    const unsigned sw = (w & 1u) * 2u + (q >> 1) + (q & 1u) * 4u;      // row within its group of eight = row & 7
+    pl.idx0 = (8u * (w >> 1) + sw) * 8u + p;
+    // K-major, 128-byte swizzle: piece p of a row holds K values 4c .. 4c+3, c = p ^ sw; as BF16 they
+    // are eight bytes of piece c >> 1 (high parts) or 4 + (c >> 1) (remainders) of the BF16 row
+    const unsigned ck = p ^ sw;
+    pl.k_hi = (((ck >> 1) ^ sw) << 4) + (ck & 1u) * 8u;
+    pl.k_lo = (((4u + (ck >> 1)) ^ sw) << 4) + (ck & 1u) * 8u;
+    // MN-major W (32-byte swizzle atoms): piece p of K row k of a 32-column box holds columns
+    // 4c .. 4c+3, c = p ^ ((k & 3) << 1); as BF16: K row k of a 64-column block, piece
+    // ((box & 1) * 4 + (c >> 1)) ^ (k & 7), and k & 7 = sw here
+    const unsigned cm = p ^ ((sw & 3u) << 1);
+    pl.mn0 = (((cm >> 1) ^ sw) << 4) + (cm & 1u) * 8u;
+    pl.mn1 = (((4u + (cm >> 1)) ^ sw) << 4) + (cm & 1u) * 8u;
+    return pl;
+}
+// fp32 to TF32, round to nearest, ties away from zero (what cvt.rna.tf32.f32 gives), on the integer pipe
+__device__ __forceinline__ float dp_tf32_rn(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+}
+// Round I (compile-time) of a thread's pieces: the TF32 high parts replace the raw values; the
+// remainders go to the same place of the second-ring slot `lo`, or (CROSS_BF16) high parts and
+// remainders go there as BF16.
+template <bool W_KMAJOR, bool CROSS_BF16, int I>
+__device__ __forceinline__ void dp_split_piece(float4* raw, float4* lo, const DpSplitPlace& pl, const float4 v)
+{
+    const unsigned idx = pl.idx0 + (unsigned)(I * DP_SPLITTERS), row = idx >> 3;     // rows 0 .. 127: D tile, 128 .. 255: W tile
+    const float4 h = make_float4(dp_tf32_rn(v.x), dp_tf32_rn(v.y), dp_tf32_rn(v.z), dp_tf32_rn(v.w));
+    raw[idx] = h;
+    const float4 r = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
+    if (!CROSS_BF16) {
+        lo[idx] = r;
+        return;
+    }
+    constexpr bool MAYBE_D = 24 * I < DG_BM, MAYBE_W = 23 + 24 * I >= DG_BM;
+    unsigned off_h, off_r;
+    if (W_KMAJOR || !MAYBE_W || (MAYBE_D && row < (unsigned)DG_BM)) {
+        off_h = row * 128u + pl.k_hi;                // (the W tile follows the D tile at the same row pitch)
+        off_r = row * 128u + pl.k_lo;
+    } else {
+        const unsigned box = (row - DG_BM) >> 5, k = row & 31u;
+        off_h = (unsigned)DG_A_BYTES + (box >> 1) * 4096u + k * 128u + ((box & 1u) ? pl.mn1 : pl.mn0);
+        off_r = off_h + (unsigned)(DP_B_BYTES / 2);
+    }
+    unsigned char* t16 = reinterpret_cast<unsigned char*>(lo);
+    *reinterpret_cast<uint2*>(t16 + off_h) = make_uint2(dp_pack_bf16(h.x, h.y), dp_pack_bf16(h.z, h.w));
+    *reinterpret_cast<uint2*>(t16 + off_r) = make_uint2(dp_pack_bf16(r.x, r.y), dp_pack_bf16(r.z, r.w));
+}
+// rounds I0 .. I0 + BATCH - 1: all loads first, then the arithmetic and the stores
+template <bool W_KMAJOR, bool CROSS_BF16, int I0, int BATCH>
+__device__ __forceinline__ void dp_split_batch(float4* raw, float4* lo, const DpSplitPlace& pl)
+{
+    float4 v[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) v[j] = raw[pl.idx0 + (unsigned)((I0 + j) * DP_SPLITTERS)];
+    if constexpr (BATCH > 0) dp_split_piece<W_KMAJOR, CROSS_BF16, I0>(raw, lo, pl, v[0]);
+    if constexpr (BATCH > 1) dp_split_piece<W_KMAJOR, CROSS_BF16, I0 + 1>(raw, lo, pl, v[1]);
+    if constexpr (BATCH > 2) dp_split_piece<W_KMAJOR, CROSS_BF16, I0 + 2>(raw, lo, pl, v[2]);
+    if constexpr (BATCH > 3) dp_split_piece<W_KMAJOR, CROSS_BF16, I0 + 3>(raw, lo, pl, v[3]);
+    if constexpr (BATCH > 4) dp_split_piece<W_KMAJOR, CROSS_BF16, I0 + 4>(raw, lo, pl, v[4]);
+}
+
+// CROSS_BF16 = false: hi*hi + hi*lo + lo*hi in TF32 (twelve instructions per 32-wide K stage).
+// CROSS_BF16 = true : hi*hi in TF32, the two cross terms in BF16 (eight instructions per stage): next to
+//   the TF32 high parts the split warps write, where the fp32 remainders went, the high parts and the
+//   remainders rounded to BF16 (K-major operands: both in one 128-byte row, high parts first; the
+//   MN-major W tile: two tiles of 64-column blocks).  A cross term is below 2^-11 of its product, so
+//   the 2^-9 of a BF16 rounding leaves about 2^-20 of the product.
+template <bool W_KMAJOR, bool CROSS_BF16>
 __global__ void __launch_bounds__(DP_THREADS, 1)
 k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_w,
                      const DgParams P)
@@ -558,8 +693,8 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     // the same offsets in both CTAs: one descriptor addresses the shared memory of both
     unsigned char* stages = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(dg_smem_raw) + 1023u) & ~(uintptr_t)1023u);
-    float* epi = reinterpret_cast<float*>(stages + (size_t)DP_STAGES * DP_STAGE_BYTES);
-    DpShared* sh = reinterpret_cast<DpShared*>(stages + (size_t)DP_STAGES * DP_STAGE_BYTES + DP_EPI_BYTES);
+    float* epi = reinterpret_cast<float*>(stages + (size_t)DP_RING_BYTES);
+    DpShared* sh = reinterpret_cast<DpShared*>(stages + (size_t)DP_RING_BYTES + DP_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned rank = dp_cluster_rank();
@@ -567,10 +702,13 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     const int g_begin = (int)((long long)P.g_total * pair / n_pairs), g_end = (int)((long long)P.g_total * (pair + 1) / n_pairs);
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < DP_STAGES; ++i) {
+        for (int i = 0; i < DP_RAW_SLOTS; ++i) {
             dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->raw_empty[i]), 1);
+        }
+        for (int i = 0; i < DP_LO_SLOTS; ++i) {
             dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 2 * DP_SPLITTERS / 32);
-            dg_mbar_init(dg_smem_u32(&sh->empty[i]), 1);
+            dg_mbar_init(dg_smem_u32(&sh->lo_empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             dg_mbar_init(dg_smem_u32(&sh->acc_full[i]), 1);
@@ -604,17 +742,20 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM;       // my samples
                     const int col0 = tn * DP_BN + (int)rank * DP_BNH;          // my columns of W
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
-                        const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
-                        if (use > 0 && !dp_wait(dg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                        const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS;
+                        if (use > 0 && !dp_wait(dg_smem_u32(&sh->raw_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
                         const unsigned bar = dg_smem_u32(&sh->full[st]);
                         dg_mbar_expect_tx(bar, DP_RAW_BYTES);
-                        const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DP_STAGE_BYTES);
-                        dg_tma_load_2d(a_dst, &map_d, bar, j0 + ks * DG_BK, row0);
-                        if (W_KMAJOR) {
-                            dg_tma_load_2d(a_dst + DG_A_BYTES, &map_w, bar, j0 + ks * DG_BK, col0);
-                        } else {
+                        const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
+                        // boxes of 32 rows: the loads of one box are few at a time, several boxes go side by side
 #pragma unroll
-                            for (int i = 0; i < DP_BNH / 32; ++i)
+                        for (int i = 0; i < DG_BM / 32; ++i)
+                            dg_tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, row0 + i * 32);
+#pragma unroll
+                        for (int i = 0; i < DP_BNH / 32; ++i) {
+                            if (W_KMAJOR)
+                                dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, col0 + i * 32);
+                            else
                                 dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, col0 + i * 32,
                                                j0 + ks * DG_BK);
                         }
@@ -623,41 +764,52 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 // after giving up: do not let the CTA exit under loads that are still landing
                 if (sh->abort_flag) {
                     const unsigned long long t0 = dg_timer();
-                    for (unsigned j = it > DP_STAGES ? it - DP_STAGES : 0; j < it; ++j) {
-                        const unsigned bar = dg_smem_u32(&sh->full[j % DP_STAGES]);
-                        while (!dg_mbar_try_wait(bar, (j / DP_STAGES) & 1u) && dg_timer() - t0 < 50000000ull) { }
+                    for (unsigned j = it > DP_RAW_SLOTS ? it - DP_RAW_SLOTS : 0; j < it; ++j) {
+                        const unsigned bar = dg_smem_u32(&sh->full[j % DP_RAW_SLOTS]);
+                        while (!dg_mbar_try_wait(bar, (j / DP_RAW_SLOTS) & 1u) && dg_timer() - t0 < 50000000ull) { }
                     }
                 }
             }
         } else if (warp == 1) {
             // ------------------------------ MMA issuer (leader CTA only) -----------------------
             if (lane == 0 && rank == 0) {
-                const unsigned idesc = dp_idesc(W_KMAJOR);
+                const unsigned idesc = dp_idesc(W_KMAJOR), idesc16 = dp_idesc(W_KMAJOR, 1u);
                 unsigned it = 0;
                 bool ok = true;
                 DpSegment sg;
                 for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
                     const int n_k = sg.kb1 - sg.kb0;
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
-                        const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
-                        const unsigned p = it & 1u, p_use = it >> 1;
-                        if (!dp_wait(dg_smem_u32(&sh->split_done[st]), use & 1u, P, sh)) { ok = false; break; }
+                        // second-ring slot and stage accumulator alternate together
+                        const unsigned st = it % DP_RAW_SLOTS, p = it & 1u, p_use = it >> 1;
+                        if (!dp_wait(dg_smem_u32(&sh->split_done[p]), p_use & 1u, P, sh)) { ok = false; break; }
                         if (p_use > 0 && !dp_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
                         dg_fence_after();
-                        const unsigned hi = dg_smem_u32(stages + (size_t)st * DP_STAGE_BYTES);
-                        const unsigned lo = hi + DP_RAW_BYTES;
+                        const unsigned hi = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
+                        const unsigned lo = dg_smem_u32(stages + (size_t)DP_LO_BASE + (size_t)p * DP_RAW_BYTES);
                         const unsigned d_tmem = tmem_base + p * (unsigned)DP_BN;
-                        // the eight small products first, then the four large ones
+                        // the small products first, then the four large ones
+                        if (CROSS_BF16) {
 #pragma unroll
-                        for (int kk = 0; kk < DG_BK / 8; ++kk) {
-                            dp_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
-                                   kk > 0 ? 1u : 0u);
-                            dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
+                            for (int kk = 0; kk < DG_BK / 16; ++kk) {
+                                dp_mma16(d_tmem, dg_desc_kmajor(lo + 64 + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 0, kk),
+                                         idesc16, kk > 0 ? 1u : 0u);
+                                dp_mma16(d_tmem, dg_desc_kmajor(lo + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 1, kk),
+                                         idesc16, 1u);
+                            }
+                        } else {
+#pragma unroll
+                            for (int kk = 0; kk < DG_BK / 8; ++kk) {
+                                dp_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
+                                       kk > 0 ? 1u : 0u);
+                                dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
+                            }
                         }
 #pragma unroll
                         for (int kk = 0; kk < DG_BK / 8; ++kk)
                             dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
-                        dp_commit_both(dg_smem_u32(&sh->empty[st]));
+                        dp_commit_both(dg_smem_u32(&sh->raw_empty[st]));
+                        dp_commit_both(dg_smem_u32(&sh->lo_empty[p]));
                         dp_commit_both(dg_smem_u32(&sh->acc_full[p]));
                     }
                 }
@@ -665,6 +817,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
         } else {
             // ------------------------------ operand split (hi/lo): warps 2..7 ------------------
             const int tt = threadIdx.x - 64;
+            const DpSplitPlace place = dp_split_place(tt);
             const unsigned leader_split_done0 = dp_map_to_rank(dg_smem_u32(&sh->split_done[0]), 0);
             unsigned it = 0;
             bool ok = true;
@@ -672,23 +825,23 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
                 const int n_k = sg.kb1 - sg.kb0;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
-                    const unsigned st = it % DP_STAGES, use = it / DP_STAGES;
+                    const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS, ls = it & 1u, ls_use = it >> 1;
                     if (!dp_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
-                    float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES);
-                    float4* lo = reinterpret_cast<float4*>(stages + (size_t)st * DP_STAGE_BYTES + DP_RAW_BYTES);
-#pragma unroll 4
-                    for (int i = 0; i < (DP_RAW_BYTES / 16 + DP_SPLITTERS - 1) / DP_SPLITTERS; ++i) {
-                        const int idx = tt + i * DP_SPLITTERS;
-                        if (idx >= DP_RAW_BYTES / 16) break;
-                        const float4 v = raw[idx];
-                        const float4 h = make_float4(dg_tf32_rn(v.x), dg_tf32_rn(v.y), dg_tf32_rn(v.z), dg_tf32_rn(v.w));
-                        raw[idx] = h;
-                        lo[idx] = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);
-                    }
+                    if (ls_use > 0 && !dp_wait(dg_smem_u32(&sh->lo_empty[ls]), (ls_use - 1) & 1u, P, sh)) { ok = false; break; }
+                    float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_RAW_BYTES);
+                    float4* lo = reinterpret_cast<float4*>(stages + (size_t)DP_LO_BASE + (size_t)ls * DP_RAW_BYTES);
+                    // 2048 16-byte pieces for 192 threads: ten rounds, a few loads in flight at a time, then 128 left
+                    static_assert(DP_RAW_BYTES / 16 == 10 * DP_SPLITTERS + 128, "ten rounds and 128 pieces");
+                    dp_split_batch<W_KMAJOR, CROSS_BF16, 0, 2>(raw, lo, place);
+                    dp_split_batch<W_KMAJOR, CROSS_BF16, 2, 2>(raw, lo, place);
+                    dp_split_batch<W_KMAJOR, CROSS_BF16, 4, 2>(raw, lo, place);
+                    dp_split_batch<W_KMAJOR, CROSS_BF16, 6, 2>(raw, lo, place);
+                    dp_split_batch<W_KMAJOR, CROSS_BF16, 8, 2>(raw, lo, place);
+                    if (tt < 128) dp_split_batch<W_KMAJOR, CROSS_BF16, 10, 1>(raw, lo, place);
                     // the tensor cores (of both CTAs) read this shared memory through the async proxy
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0) dp_arrive_cluster(leader_split_done0 + st * (unsigned)sizeof(unsigned long long));
+                    if (lane == 0) dp_arrive_cluster(leader_split_done0 + ls * (unsigned)sizeof(unsigned long long));
                 }
             }
         }
@@ -870,9 +1023,13 @@ int dp_max_pairs(const lf_ctx* c)
     if (cached_dev == c->device) return cached;
     int n = 0;
     if ((size_t)c->smem_optin >= DP_SMEM_BYTES &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
@@ -880,10 +1037,15 @@ int dp_max_pairs(const lf_ctx* c)
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        int n0 = 0, n1 = 0;
-        if (cudaOccupancyMaxActiveClusters(&n0, k_delta_gemm_tc_pair<false>, &cfg) == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n1, k_delta_gemm_tc_pair<true>, &cfg) == cudaSuccess)
+        int n0 = 0, n1 = 0, n2 = 0, n3 = 0;
+        if (cudaOccupancyMaxActiveClusters(&n0, k_delta_gemm_tc_pair<false, false>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n1, k_delta_gemm_tc_pair<true, false>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n2, k_delta_gemm_tc_pair<false, true>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n3, k_delta_gemm_tc_pair<true, true>, &cfg) == cudaSuccess) {
             n = n0 < n1 ? n0 : n1;
+            if (n2 < n) n = n2;
+            if (n3 < n) n = n3;
+        }
     }
     cudaGetLastError();
     cached_dev = c->device; cached = n;
@@ -991,14 +1153,14 @@ static DgSlots dg_slots(int Nc, const DgPlan& pl)
 // Encode the two operand maps and launch one contraction out[B][Nc] = lhs[B][K] x W into
 // c->dg_partial.  W is [Nc][K] (w_kmajor: row n holds the K values it is contracted over, Eq. z) or
 // [K][Nc] (Eq. bp2: the transposed product read from the same row-major matrix).
-static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kmajor, int Nc, int K, cudaStream_t s,
-                     DgPlan* plan_out)
+static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kmajor, bool cross_bf16, int Nc, int K,
+                     cudaStream_t s, DgPlan* plan_out)
 {
     alignas(64) CUtensorMap map_d, map_w;
     {
         cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)c->B};
         cuuint64_t strides[1] = {(cuuint64_t)K * 4};
-        cuuint32_t box[2] = {32, (cuuint32_t)DG_BM};
+        cuuint32_t box[2] = {32, 32};                        // 32 values of j x 32 samples
         cuuint32_t estr[2] = {1, 1};
         if (dg_get_encode()(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(lhs), dims, strides,
                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1012,7 +1174,7 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
         cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
         cuuint64_t strides[1] = {(cuuint64_t)inner * 4};
         cuuint32_t box_mn[2] = {32, (cuuint32_t)DG_BK};      // 32 columns n x 32 rows j
-        cuuint32_t box_k[2] = {32, (cuuint32_t)DG_BN};       // 32 values of j x 128 rows n
+        cuuint32_t box_k[2] = {32, 32};                      // 32 values of j x 32 rows n
         cuuint32_t estr[2] = {1, 1};
         if (dg_get_encode()(&map_w, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(w_mat), dims, strides,
                             w_kmajor ? box_k : box_mn, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -1042,10 +1204,14 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
         at[0].id = cudaLaunchAttributeClusterDimension;
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        if (w_kmajor)
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true>, map_d, map_w, P));
+        if (w_kmajor && cross_bf16)
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, true>, map_d, map_w, P));
+        else if (w_kmajor)
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, false>, map_d, map_w, P));
+        else if (cross_bf16)
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, true>, map_d, map_w, P));
         else
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false>, map_d, map_w, P));
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, false>, map_d, map_w, P));
         c->stats.delta_tiling = LF_TC_TILING_TWO_SM;
         *plan_out = pl;
         return LF_OK;
@@ -1062,11 +1228,11 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
 }
 
 int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
-                     int n_up, int n_l, cudaStream_t s, int* launches)
+                     int n_up, int n_l, int math, cudaStream_t s, int* launches)
 {
     // w_up = w^{l+1} is n_up x n_l; out[b][k] = sum_j delta_up[b][j] w_up[j][k]
     DgPlan pl;
-    int rc = dg_launch(c, delta_up, w_up, false, n_l, n_up, s, &pl);
+    int rc = dg_launch(c, delta_up, w_up, false, math == LF_DELTA_MATH_TF32_BF16, n_l, n_up, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_l / 4;
     k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(n_l, pl), c->opt_act);
@@ -1076,11 +1242,11 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
 }
 
 int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const float* a_prev, float* z_l, float* a_l,
-                       int n_out, int n_in, cudaStream_t s, int* launches)
+                       int n_out, int n_in, int math, cudaStream_t s, int* launches)
 {
     // w_l is n_out x n_in; out[b][j] = sum_k a_prev[b][k] w_l[j][k]
     DgPlan pl;
-    int rc = dg_launch(c, a_prev, w_l, true, n_out, n_in, s, &pl);
+    int rc = dg_launch(c, a_prev, w_l, true, math == LF_DELTA_MATH_TF32_BF16, n_out, n_in, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_out / 4;
     k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, n_out / 4,

@@ -222,6 +222,6 @@ void lf_tf32_release(lf_ctx* c);
 size_t lf_delta_tc_scratch_bytes(const lf_ctx* c);
 bool lf_delta_tc_supported(const lf_ctx* c);
 int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const float* a_l, float* delta_l,
-                     int n_up, int n_l, cudaStream_t s, int* launches);
+                     int n_up, int n_l, int math, cudaStream_t s, int* launches);
 int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const float* a_prev, float* z_l, float* a_l,
-                       int n_out, int n_in, cudaStream_t s, int* launches);
+                       int n_out, int n_in, int math, cudaStream_t s, int* launches);

@@ -39,7 +39,8 @@ def test_single_sample_parity(L, N, k, variant):
 
 @pytest.mark.parametrize("delta_math,tiling", [(lf.LF_DELTA_MATH_FP32, lf.LF_TC_TILING_AUTO),
                                                (lf.LF_DELTA_MATH_3XTF32, lf.LF_TC_TILING_ONE_SM),
-                                               (lf.LF_DELTA_MATH_3XTF32, lf.LF_TC_TILING_TWO_SM)])
+                                               (lf.LF_DELTA_MATH_3XTF32, lf.LF_TC_TILING_TWO_SM),
+                                               (lf.LF_DELTA_MATH_TF32_BF16, lf.LF_TC_TILING_TWO_SM)])
 @pytest.mark.parametrize("L,N,B,k", [(2, 8, 2, 1), (3, 68, 3, 2), (3, 256, 16, 4),
                                      (4, 132, 70, 3), (2, 320, 129, 2), (5, 1028, 260, 2),
                                      (3, 772, 256, 1), (2, 2052, 515, 2)])
@@ -48,13 +49,14 @@ def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
     # forward pass, which shares its kernels): fp32 on the CUDA cores, and the tensor cores with
     # every operand split into two TF32 numbers, one CTA per tile or a CTA pair per tile (pairs
     # take over above 128 samples and from 512 columns: B = 260 leaves a pair's second half nearly
-    # empty, B = 515 needs three 256-sample blocks, N = 2052 gives runs that end inside a tile).
+    # empty, B = 515 needs three 256-sample blocks, N = 2052 gives runs that end inside a tile);
+    # and the CTA pairs with the two cross terms in BF16 (one-CTA tiles keep three TF32 products).
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=N + B)
     out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math, tc_tiling=tiling)
     assert stats["gw_math"] == lf.LF_GW_MATH_FP32 and stats["delta_math"] == delta_math
     assert stats["device_status"] == 0
-    if delta_math == lf.LF_DELTA_MATH_3XTF32 and L > 1:
+    if delta_math >= lf.LF_DELTA_MATH_3XTF32 and L > 1:
         pairs = tiling == lf.LF_TC_TILING_TWO_SM and B > 128 and N >= 512   # the library's rule for CTA pairs
         want = lf.LF_TC_TILING_TWO_SM if pairs else lf.LF_TC_TILING_ONE_SM
         assert stats["delta_tiling"] == want

@@ -129,7 +129,7 @@ def test_widths_chain_and_forward_on_the_tensor_cores(widths, B, tiling):
     # B x n_l x n_{l+1}): fp32-level accuracy, so the fp32 gate applies; the weight gradient stays fp32
     # here so that every tensor is held to it.  The two-SM kernel serves layers of at least 512 x 512
     # with more than 128 samples, the one-SM kernel the rest.
-    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=80 + B, delta_math=lf.LF_DELTA_MATH_AUTO,
+    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=80 + B, delta_math=lf.LF_DELTA_MATH_3XTF32,
                                  tiling=tiling)
     assert stats["device_status"] == 0 and stats["delta_math"] == lf.LF_DELTA_MATH_3XTF32
     assert stats["delta_tiling"] in (lf.LF_TC_TILING_ONE_SM, lf.LF_TC_TILING_TWO_SM)
