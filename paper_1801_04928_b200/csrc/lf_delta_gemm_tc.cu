@@ -25,6 +25,29 @@
 
 #include "lf_internal.h"
 
+// Debug builds (-DLF_DG_TRACE): the leader CTA of pair 0 of the two-SM kernel stamps its SM clock at
+// nine points of each of its first DG_TRACE_STAGES K stages (see DG_STAMP below); the release
+// library carries none of this.
+#ifdef LF_DG_TRACE
+constexpr int DG_TRACE_STAGES = 128;
+__device__ long long dg_trace[DG_TRACE_STAGES * 16];
+extern "C" int lf_debug_read_pair_trace(long long* out)
+{
+    if (!out) return LF_ENULL;
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(out, dg_trace, sizeof(dg_trace)) == cudaSuccess ? LF_OK : LF_ECUDA;
+}
+// 0 loads issued, 1 loads landed, 2 second-ring slot free, 3 split written, 4 issuer sees the split,
+// 5 issuer has the accumulator, 6 products and commits issued, 7 products done, 8 accumulator drained
+#define DG_STAMP(slot) do { if (pair == 0 && rank == 0 && it < (unsigned)DG_TRACE_STAGES) dg_trace[it * 16 + (slot)] = clock64(); } while (0)
+// once per launch, in the words 9 .. 12 of stage 0: 9 kernel entered, 10 set-up done (barriers, tensor
+// memory, cluster barrier), 11 a summing warp has written its last partial sums, 12 before the exit
+#define DG_STAMP_ONCE(slot) do { if (pair == 0 && rank == 0 && (threadIdx.x == 256 || ((slot) < 11 && threadIdx.x == 0))) dg_trace[slot] = clock64(); } while (0)
+#else
+#define DG_STAMP(slot) do { } while (0)
+#define DG_STAMP_ONCE(slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int DG_BM = 128, DG_BN = 128, DG_BK = 32;
@@ -700,6 +723,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     const unsigned rank = dp_cluster_rank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int g_begin = (int)((long long)P.g_total * pair / n_pairs), g_end = (int)((long long)P.g_total * (pair + 1) / n_pairs);
+    DG_STAMP_ONCE(9);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < DP_RAW_SLOTS; ++i) {
@@ -727,6 +751,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     dp_cluster_sync();   // the peer's barriers exist before anything can arrive on them
     dg_fence_after();
     const unsigned tmem_base = sh->tmem_base;
+    DG_STAMP_ONCE(10);
 
     if (warp < 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(DP_REGS_SMALL));
@@ -744,6 +769,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
                         const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS;
                         if (use > 0 && !dp_wait(dg_smem_u32(&sh->raw_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                        DG_STAMP(0);
                         const unsigned bar = dg_smem_u32(&sh->full[st]);
                         dg_mbar_expect_tx(bar, DP_RAW_BYTES);
                         const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
@@ -783,7 +809,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                         // second-ring slot and stage accumulator alternate together
                         const unsigned st = it % DP_RAW_SLOTS, p = it & 1u, p_use = it >> 1;
                         if (!dp_wait(dg_smem_u32(&sh->split_done[p]), p_use & 1u, P, sh)) { ok = false; break; }
+                        DG_STAMP(4);
                         if (p_use > 0 && !dp_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
+                        DG_STAMP(5);
                         dg_fence_after();
                         const unsigned hi = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
                         const unsigned lo = dg_smem_u32(stages + (size_t)DP_LO_BASE + (size_t)p * DP_RAW_BYTES);
@@ -811,6 +839,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                         dp_commit_both(dg_smem_u32(&sh->raw_empty[st]));
                         dp_commit_both(dg_smem_u32(&sh->lo_empty[p]));
                         dp_commit_both(dg_smem_u32(&sh->acc_full[p]));
+                        DG_STAMP(6);
                     }
                 }
             }
@@ -827,7 +856,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS, ls = it & 1u, ls_use = it >> 1;
                     if (!dp_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    if (tt == 0) DG_STAMP(1);
                     if (ls_use > 0 && !dp_wait(dg_smem_u32(&sh->lo_empty[ls]), (ls_use - 1) & 1u, P, sh)) { ok = false; break; }
+                    if (tt == 0) DG_STAMP(2);
                     float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_RAW_BYTES);
                     float4* lo = reinterpret_cast<float4*>(stages + (size_t)DP_LO_BASE + (size_t)ls * DP_RAW_BYTES);
                     // 2048 16-byte pieces for 192 threads: ten rounds, a few loads in flight at a time, then 128 left
@@ -841,6 +872,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     // the tensor cores (of both CTAs) read this shared memory through the async proxy
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
+                    if (tt == 0) DG_STAMP(3);
                     if (lane == 0) dp_arrive_cluster(leader_split_done0 + ls * (unsigned)sizeof(unsigned long long));
                 }
             }
@@ -864,6 +896,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 // add the finished stage (accumulator it & 1) into the registers
                 const unsigned p = it & 1u;
                 if (!dp_wait(dg_smem_u32(&sh->acc_full[p]), (it >> 1) & 1u, P, sh)) { ok = false; break; }
+                if (threadIdx.x == 256) DG_STAMP(7);
                 dg_fence_after();
 #pragma unroll
                 for (int cchunk = 0; cchunk < DP_BNH / 64; ++cchunk) {
@@ -875,6 +908,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 }
                 dg_fence_before();
                 __syncwarp();
+                if (threadIdx.x == 256) DG_STAMP(8);
                 if (lane == 0) dp_arrive_cluster(leader_acc_empty0 + p * (unsigned)sizeof(unsigned long long));
             }
             if (!ok) break;
@@ -904,12 +938,14 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 __syncwarp();
             }
         }
+        DG_STAMP_ONCE(11);
     }
 
     // neither CTA may leave, or free tensor memory, while the other can still reach it
     dg_fence_before();
     __syncthreads();
     dp_cluster_sync();
+    DG_STAMP_ONCE(12);
     if (warp == 1) {
         dg_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DP_TMEM_COLS)
