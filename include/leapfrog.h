@@ -71,8 +71,9 @@ enum lf_gw_math {
  * contractions). */
 enum lf_delta_math {
     LF_DELTA_MATH_AUTO = 0,  /* tensor cores when B > 1 and the device supports it; Eq. bp2 for 2 to
-                                16 samples stays fp32 on the CUDA cores (a batched matrix-vector
-                                product that reads w^{l+1} once, at the memory rate)              */
+                                8 samples, and for 9 to 16 samples of layers at least 2048 wide,
+                                stays fp32 on the CUDA cores (a batched matrix-vector product
+                                that reads w^{l+1} once, at the memory rate)                      */
     LF_DELTA_MATH_FP32 = 1,  /* fp32 FMA on the CUDA cores                                        */
     LF_DELTA_MATH_3XTF32 = 2, /* tensor cores; every operand split into two TF32 numbers, three
                                 products per term, fp32 accumulation: fp32-level accuracy        */

@@ -101,11 +101,14 @@ int resolve_forward_math(const lf_ctx* c)
 
 // Arithmetic of Eq. bp2 for B > 1.  A handful of samples is a batched matrix-vector product: fp32 on
 // the CUDA cores at the memory rate beats tensor-core tiles that are nearly empty (unless the
-// tensor cores are asked for by name).
+// tensor cores are asked for by name).  Measured, whole pass per layer, widths 256 .. 8192: up to 8
+// samples the fp32 kernel is ahead at every width; with 9 to 16 samples from a width of 2048.
 int resolve_delta_math(const lf_ctx* c)
 {
     if (c->B == 1 || c->opt_delta_math == LF_DELTA_MATH_FP32) return LF_DELTA_MATH_FP32;
-    if (c->opt_delta_math == LF_DELTA_MATH_AUTO && c->B <= lfk_small_batch_max() && c->sb_partial) return LF_DELTA_MATH_FP32;
+    if (c->opt_delta_math == LF_DELTA_MATH_AUTO && c->sb_partial && c->B <= lfk_small_batch_max() &&
+        (c->B <= 8 || c->N >= 2048))
+        return LF_DELTA_MATH_FP32;
     if (!lf_delta_tc_supported(c)) return LF_DELTA_MATH_FP32;
     return c->opt_delta_math == LF_DELTA_MATH_TF32_BF16 ? LF_DELTA_MATH_TF32_BF16 : LF_DELTA_MATH_3XTF32;
 }

@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include "lf_internal.h"
+#include "lf_ptx.cuh"
 
 // Debug builds (-DLF_DG_TRACE): the leader CTA of pair 0 of the two-SM kernel stamps its SM clock at
 // nine points of each of its first DG_TRACE_STAGES K stages (see DG_STAMP below); the release
@@ -84,45 +85,16 @@ struct DgShared {
     volatile unsigned abort_flag;
 };
 
-__device__ __forceinline__ unsigned dg_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long dg_timer()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void dg_mbar_init(unsigned bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void dg_mbar_expect_tx(unsigned bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void dg_mbar_arrive(unsigned bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool dg_mbar_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ bool dg_wait(unsigned bar, unsigned parity, const DgParams& P, DgShared* sh)
 {
-    if (dg_mbar_try_wait(bar, parity)) return true;
+    if (lfptx::mbar_try_wait(bar, parity)) return true;
     if (sh->abort_flag) return false;
-    const unsigned long long t0 = dg_timer();
+    const unsigned long long t0 = lfptx::globaltimer_ns();
     unsigned spins = 0;
-    while (!dg_mbar_try_wait(bar, parity)) {
+    while (!lfptx::mbar_try_wait(bar, parity)) {
         if ((++spins & 15u) == 0u) {
             if (sh->abort_flag) return false;
-            if (dg_timer() - t0 > P.budget_ns) {
+            if (lfptx::globaltimer_ns() - t0 > P.budget_ns) {
                 atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
                 sh->abort_flag = 1u;
                 return false;
@@ -130,12 +102,6 @@ __device__ __forceinline__ bool dg_wait(unsigned bar, unsigned parity, const DgP
         }
     }
     return true;
-}
-__device__ __forceinline__ void dg_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 // K-major operand, 128-byte swizzle: rows of 128 bytes (32 floats along K), eight rows per
 // 1024-byte atom (SBO); one instruction consumes 32 bytes of every row.
@@ -192,26 +158,11 @@ __device__ __forceinline__ void dg_commit(unsigned bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void dg_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void dg_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ float dg_tf32_rn(float x)
 {
     unsigned r;
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
     return __uint_as_float(r);
-}
-__device__ __forceinline__ void dg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
 // W_KMAJOR = false: T = D * W   (Eq. bp2: w^{l+1}[j][n], contraction over its rows j; MN-major operand)
@@ -233,25 +184,25 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < DG_STAGES; ++i) {
-            dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
-            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 128);
-            dg_mbar_init(dg_smem_u32(&sh->empty[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->split_done[i]), 128);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            dg_mbar_init(dg_smem_u32(&sh->acc_full[i]), 1);
-            dg_mbar_init(dg_smem_u32(&sh->acc_empty[i]), 128);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_empty[i]), 128);
         }
         sh->abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        lfptx::mbar_fence_init();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(dg_smem_u32(&sh->tmem_base)), "r"((unsigned)DG_TMEM_COLS) : "memory");
+                     ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)DG_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    dg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    dg_fence_after();
+    lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
 
     if (warp == 0) {
@@ -263,20 +214,20 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                 const int j0 = sp * P.k_per_split;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
-                    if (use > 0 && !dg_wait(dg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
-                    const unsigned bar = dg_smem_u32(&sh->full[st]);
-                    dg_mbar_expect_tx(bar, DG_RAW_BYTES);
-                    const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
+                    if (use > 0 && !dg_wait(lfptx::smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
+                    const unsigned bar = lfptx::smem_u32(&sh->full[st]);
+                    lfptx::mbar_arrive_expect_tx(bar, DG_RAW_BYTES);
+                    const unsigned a_dst = lfptx::smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
                     // boxes of 32 rows: the loads of one box are few at a time, several boxes go side by side
 #pragma unroll
                     for (int i = 0; i < DG_BM / 32; ++i)
-                        dg_tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM + i * 32);
+                        lfptx::tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, tm * DG_BM + i * 32);
 #pragma unroll
                     for (int i = 0; i < DG_BN / 32; ++i) {
                         if (W_KMAJOR)
-                            dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, tn * DG_BN + i * 32);
+                            lfptx::tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, tn * DG_BN + i * 32);
                         else
-                            dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
+                            lfptx::tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, tn * DG_BN + i * 32,
                                            j0 + ks * DG_BK);
                     }
                 }
@@ -284,10 +235,10 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
             }
             // after giving up: do not let the CTA exit under loads that are still landing
             if (sh->abort_flag) {
-                const unsigned long long t0 = dg_timer();
+                const unsigned long long t0 = lfptx::globaltimer_ns();
                 for (unsigned j = it > DG_STAGES ? it - DG_STAGES : 0; j < it; ++j) {
-                    const unsigned bar = dg_smem_u32(&sh->full[j % DG_STAGES]);
-                    while (!dg_mbar_try_wait(bar, (j / DG_STAGES) & 1u) && dg_timer() - t0 < 50000000ull) { }
+                    const unsigned bar = lfptx::smem_u32(&sh->full[j % DG_STAGES]);
+                    while (!lfptx::mbar_try_wait(bar, (j / DG_STAGES) & 1u) && lfptx::globaltimer_ns() - t0 < 50000000ull) { }
                 }
             }
         }
@@ -301,10 +252,10 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
                     const unsigned p = it & 1u, p_use = it >> 1;
-                    if (!dg_wait(dg_smem_u32(&sh->split_done[st]), use & 1u, P, sh)) { ok = false; break; }
-                    if (p_use > 0 && !dg_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
-                    dg_fence_after();
-                    const unsigned hi = dg_smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
+                    if (!dg_wait(lfptx::smem_u32(&sh->split_done[st]), use & 1u, P, sh)) { ok = false; break; }
+                    if (p_use > 0 && !dg_wait(lfptx::smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
+                    lfptx::tc_fence_after();
+                    const unsigned hi = lfptx::smem_u32(stages + (size_t)st * DG_STAGE_BYTES);
                     const unsigned lo = hi + DG_RAW_BYTES;
                     const unsigned d_tmem = tmem_base + p * (unsigned)DG_BN;
                     // the eight small products first, then the four large ones
@@ -317,8 +268,8 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
 #pragma unroll
                     for (int kk = 0; kk < DG_BK / 8; ++kk)
                         dg_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
-                    dg_commit(dg_smem_u32(&sh->empty[st]));
-                    dg_commit(dg_smem_u32(&sh->acc_full[p]));
+                    dg_commit(lfptx::smem_u32(&sh->empty[st]));
+                    dg_commit(lfptx::smem_u32(&sh->acc_full[p]));
                 }
             }
         }
@@ -332,25 +283,25 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
         // add the finished stage `j` (accumulator j & 1) into the registers; first == overwrite
         auto drain = [&](unsigned j, bool first) -> bool {
             const unsigned p = j & 1u;
-            if (!dg_wait(dg_smem_u32(&sh->acc_full[p]), (j >> 1) & 1u, P, sh)) return false;
-            dg_fence_after();
+            if (!dg_wait(lfptx::smem_u32(&sh->acc_full[p]), (j >> 1) & 1u, P, sh)) return false;
+            lfptx::tc_fence_after();
 #pragma unroll
             for (int cchunk = 0; cchunk < DG_BN / 32; ++cchunk) {
                 unsigned r[32];
-                dg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DG_BN + cchunk * 32, r);
+                lfptx::tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DG_BN + cchunk * 32, r);
 #pragma unroll
                 for (int v = 0; v < 32; ++v)
                     acc[cchunk * 32 + v] = first ? __uint_as_float(r[v]) : acc[cchunk * 32 + v] + __uint_as_float(r[v]);
             }
-            dg_fence_before();
-            dg_mbar_arrive(dg_smem_u32(&sh->acc_empty[p]));
+            lfptx::tc_fence_before();
+            lfptx::mbar_arrive(lfptx::smem_u32(&sh->acc_empty[p]));
             return true;
         };
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
             const int tn = u % P.tiles_n, tm = (u / P.tiles_n) % P.tiles_m, sp = u / (P.tiles_n * P.tiles_m);
             for (int ks = 0; ks < n_k; ++ks, ++it) {
                 const unsigned st = it % DG_STAGES, use = it / DG_STAGES;
-                if (!dg_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                if (!dg_wait(lfptx::smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
                 float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DG_STAGE_BYTES);
                 float4* lo = reinterpret_cast<float4*>(stages + (size_t)st * DG_STAGE_BYTES + DG_RAW_BYTES);
 #pragma unroll 4
@@ -363,7 +314,7 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
                 }
                 // the tensor core reads shared memory through the async proxy
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                dg_mbar_arrive(dg_smem_u32(&sh->split_done[st]));
+                lfptx::mbar_arrive(lfptx::smem_u32(&sh->split_done[st]));
                 if (ks > 0 && !drain(it - 1, ks == 1)) { ok = false; break; }
             }
             if (!ok) break;
@@ -393,10 +344,10 @@ k_delta_gemm_tc(const __grid_constant__ CUtensorMap map_d, const __grid_constant
         }
     }
 
-    dg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        dg_fence_after();
+        lfptx::tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DG_TMEM_COLS)
                      : "memory");
     }
@@ -461,22 +412,6 @@ struct DpShared {
     volatile unsigned abort_flag;
 };
 
-__device__ __forceinline__ unsigned dp_cluster_rank()
-{
-    unsigned r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ unsigned dp_map_to_rank(unsigned local_addr, unsigned rank)
-{
-    unsigned r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void dp_cluster_sync()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 __device__ __forceinline__ void dp_mma(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                        unsigned idesc, unsigned accumulate)
 {
@@ -535,26 +470,16 @@ __device__ __forceinline__ void dp_arrive_cluster(unsigned cluster_bar)
     // at about 1300 cycles per hand-off, which then bounded the kernel at 3000 cycles per K stage.
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
-__device__ __forceinline__ bool dp_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ bool dp_wait(unsigned bar, unsigned parity, const DgParams& P, DpShared* sh)
 {
-    if (dp_try_wait(bar, parity)) return true;
+    if (lfptx::mbar_try_wait_cluster(bar, parity)) return true;
     if (sh->abort_flag) return false;
-    const unsigned long long t0 = dg_timer();
+    const unsigned long long t0 = lfptx::globaltimer_ns();
     unsigned spins = 0;
-    while (!dp_try_wait(bar, parity)) {
+    while (!lfptx::mbar_try_wait_cluster(bar, parity)) {
         if ((++spins & 15u) == 0u) {
             if (sh->abort_flag) return false;
-            if (dg_timer() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
+            if (lfptx::globaltimer_ns() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
                 atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
                 sh->abort_flag = 1u;
                 return false;
@@ -720,36 +645,36 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     DpShared* sh = reinterpret_cast<DpShared*>(stages + (size_t)DP_RING_BYTES + DP_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned rank = dp_cluster_rank();
+    const unsigned rank = lfptx::cluster_ctarank();
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int g_begin = (int)((long long)P.g_total * pair / n_pairs), g_end = (int)((long long)P.g_total * (pair + 1) / n_pairs);
     DG_STAMP_ONCE(9);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < DP_RAW_SLOTS; ++i) {
-            dg_mbar_init(dg_smem_u32(&sh->full[i]), 1);
-            dg_mbar_init(dg_smem_u32(&sh->raw_empty[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->raw_empty[i]), 1);
         }
         for (int i = 0; i < DP_LO_SLOTS; ++i) {
-            dg_mbar_init(dg_smem_u32(&sh->split_done[i]), 2 * DP_SPLITTERS / 32);
-            dg_mbar_init(dg_smem_u32(&sh->lo_empty[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->split_done[i]), 2 * DP_SPLITTERS / 32);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->lo_empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            dg_mbar_init(dg_smem_u32(&sh->acc_full[i]), 1);
-            dg_mbar_init(dg_smem_u32(&sh->acc_empty[i]), 16);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_empty[i]), 16);
         }
         sh->abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        lfptx::mbar_fence_init();
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(dg_smem_u32(&sh->tmem_base)), "r"((unsigned)DP_TMEM_COLS) : "memory");
+                     ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)DP_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
-    dg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    dp_cluster_sync();   // the peer's barriers exist before anything can arrive on them
-    dg_fence_after();
+    lfptx::cluster_sync_all();   // the peer's barriers exist before anything can arrive on them
+    lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
     DG_STAMP_ONCE(10);
 
@@ -768,31 +693,31 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     const int col0 = tn * DP_BN + (int)rank * DP_BNH;          // my columns of W
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
                         const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS;
-                        if (use > 0 && !dp_wait(dg_smem_u32(&sh->raw_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                        if (use > 0 && !dp_wait(lfptx::smem_u32(&sh->raw_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
                         DG_STAMP(0);
-                        const unsigned bar = dg_smem_u32(&sh->full[st]);
-                        dg_mbar_expect_tx(bar, DP_RAW_BYTES);
-                        const unsigned a_dst = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
+                        const unsigned bar = lfptx::smem_u32(&sh->full[st]);
+                        lfptx::mbar_arrive_expect_tx(bar, DP_RAW_BYTES);
+                        const unsigned a_dst = lfptx::smem_u32(stages + (size_t)st * DP_RAW_BYTES);
                         // boxes of 32 rows: the loads of one box are few at a time, several boxes go side by side
 #pragma unroll
                         for (int i = 0; i < DG_BM / 32; ++i)
-                            dg_tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, row0 + i * 32);
+                            lfptx::tma_load_2d(a_dst + i * DG_BOX_BYTES, &map_d, bar, j0 + ks * DG_BK, row0 + i * 32);
 #pragma unroll
                         for (int i = 0; i < DP_BNH / 32; ++i) {
                             if (W_KMAJOR)
-                                dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, col0 + i * 32);
+                                lfptx::tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, j0 + ks * DG_BK, col0 + i * 32);
                             else
-                                dg_tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, col0 + i * 32,
+                                lfptx::tma_load_2d(a_dst + DG_A_BYTES + i * DG_BOX_BYTES, &map_w, bar, col0 + i * 32,
                                                j0 + ks * DG_BK);
                         }
                     }
                 }
                 // after giving up: do not let the CTA exit under loads that are still landing
                 if (sh->abort_flag) {
-                    const unsigned long long t0 = dg_timer();
+                    const unsigned long long t0 = lfptx::globaltimer_ns();
                     for (unsigned j = it > DP_RAW_SLOTS ? it - DP_RAW_SLOTS : 0; j < it; ++j) {
-                        const unsigned bar = dg_smem_u32(&sh->full[j % DP_RAW_SLOTS]);
-                        while (!dg_mbar_try_wait(bar, (j / DP_RAW_SLOTS) & 1u) && dg_timer() - t0 < 50000000ull) { }
+                        const unsigned bar = lfptx::smem_u32(&sh->full[j % DP_RAW_SLOTS]);
+                        while (!lfptx::mbar_try_wait(bar, (j / DP_RAW_SLOTS) & 1u) && lfptx::globaltimer_ns() - t0 < 50000000ull) { }
                     }
                 }
             }
@@ -808,13 +733,13 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
                         // second-ring slot and stage accumulator alternate together
                         const unsigned st = it % DP_RAW_SLOTS, p = it & 1u, p_use = it >> 1;
-                        if (!dp_wait(dg_smem_u32(&sh->split_done[p]), p_use & 1u, P, sh)) { ok = false; break; }
+                        if (!dp_wait(lfptx::smem_u32(&sh->split_done[p]), p_use & 1u, P, sh)) { ok = false; break; }
                         DG_STAMP(4);
-                        if (p_use > 0 && !dp_wait(dg_smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
+                        if (p_use > 0 && !dp_wait(lfptx::smem_u32(&sh->acc_empty[p]), (p_use - 1) & 1u, P, sh)) { ok = false; break; }
                         DG_STAMP(5);
-                        dg_fence_after();
-                        const unsigned hi = dg_smem_u32(stages + (size_t)st * DP_RAW_BYTES);
-                        const unsigned lo = dg_smem_u32(stages + (size_t)DP_LO_BASE + (size_t)p * DP_RAW_BYTES);
+                        lfptx::tc_fence_after();
+                        const unsigned hi = lfptx::smem_u32(stages + (size_t)st * DP_RAW_BYTES);
+                        const unsigned lo = lfptx::smem_u32(stages + (size_t)DP_LO_BASE + (size_t)p * DP_RAW_BYTES);
                         const unsigned d_tmem = tmem_base + p * (unsigned)DP_BN;
                         // the small products first, then the four large ones
                         if (CROSS_BF16) {
@@ -836,9 +761,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
 #pragma unroll
                         for (int kk = 0; kk < DG_BK / 8; ++kk)
                             dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
-                        dp_commit_both(dg_smem_u32(&sh->raw_empty[st]));
-                        dp_commit_both(dg_smem_u32(&sh->lo_empty[p]));
-                        dp_commit_both(dg_smem_u32(&sh->acc_full[p]));
+                        dp_commit_both(lfptx::smem_u32(&sh->raw_empty[st]));
+                        dp_commit_both(lfptx::smem_u32(&sh->lo_empty[p]));
+                        dp_commit_both(lfptx::smem_u32(&sh->acc_full[p]));
                         DG_STAMP(6);
                     }
                 }
@@ -847,7 +772,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             // ------------------------------ operand split (hi/lo): warps 2..7 ------------------
             const int tt = threadIdx.x - 64;
             const DpSplitPlace place = dp_split_place(tt);
-            const unsigned leader_split_done0 = dp_map_to_rank(dg_smem_u32(&sh->split_done[0]), 0);
+            const unsigned leader_split_done0 = lfptx::map_to_cta(lfptx::smem_u32(&sh->split_done[0]), 0);
             unsigned it = 0;
             bool ok = true;
             DpSegment sg;
@@ -855,9 +780,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 const int n_k = sg.kb1 - sg.kb0;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS, ls = it & 1u, ls_use = it >> 1;
-                    if (!dp_wait(dg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    if (!dp_wait(lfptx::smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
                     if (tt == 0) DG_STAMP(1);
-                    if (ls_use > 0 && !dp_wait(dg_smem_u32(&sh->lo_empty[ls]), (ls_use - 1) & 1u, P, sh)) { ok = false; break; }
+                    if (ls_use > 0 && !dp_wait(lfptx::smem_u32(&sh->lo_empty[ls]), (ls_use - 1) & 1u, P, sh)) { ok = false; break; }
                     if (tt == 0) DG_STAMP(2);
                     float4* raw = reinterpret_cast<float4*>(stages + (size_t)st * DP_RAW_BYTES);
                     float4* lo = reinterpret_cast<float4*>(stages + (size_t)DP_LO_BASE + (size_t)ls * DP_RAW_BYTES);
@@ -882,7 +807,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(DP_REGS_SUM));
         const int quad = warp & 3;               // the TMEM lane quadrant this warp may read
         const int half = (warp - 8) >> 2;        // which 128 of the 256 accumulator columns
-        const unsigned leader_acc_empty0 = dp_map_to_rank(dg_smem_u32(&sh->acc_empty[0]), 0);
+        const unsigned leader_acc_empty0 = lfptx::map_to_cta(lfptx::smem_u32(&sh->acc_empty[0]), 0);
         unsigned it = 0;
         bool ok = true;
         float acc[DP_BNH];     // this thread's sample, its 128 columns of the tile
@@ -895,9 +820,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             for (int ks = 0; ks < n_k; ++ks, ++it) {
                 // add the finished stage (accumulator it & 1) into the registers
                 const unsigned p = it & 1u;
-                if (!dp_wait(dg_smem_u32(&sh->acc_full[p]), (it >> 1) & 1u, P, sh)) { ok = false; break; }
+                if (!dp_wait(lfptx::smem_u32(&sh->acc_full[p]), (it >> 1) & 1u, P, sh)) { ok = false; break; }
                 if (threadIdx.x == 256) DG_STAMP(7);
-                dg_fence_after();
+                lfptx::tc_fence_after();
 #pragma unroll
                 for (int cchunk = 0; cchunk < DP_BNH / 64; ++cchunk) {
                     unsigned r[64];
@@ -906,7 +831,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                     for (int v = 0; v < 64; ++v)
                         acc[cchunk * 64 + v] += __uint_as_float(r[v]);
                 }
-                dg_fence_before();
+                lfptx::tc_fence_before();
                 __syncwarp();
                 if (threadIdx.x == 256) DG_STAMP(8);
                 if (lane == 0) dp_arrive_cluster(leader_acc_empty0 + p * (unsigned)sizeof(unsigned long long));
@@ -942,12 +867,12 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     }
 
     // neither CTA may leave, or free tensor memory, while the other can still reach it
-    dg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    dp_cluster_sync();
+    lfptx::cluster_sync_all();
     DG_STAMP_ONCE(12);
     if (warp == 1) {
-        dg_fence_after();
+        lfptx::tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DP_TMEM_COLS)
                      : "memory");
     }

@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include "lf_internal.h"
+#include "lf_ptx.cuh"
 
 namespace {
 
@@ -52,46 +53,17 @@ struct TgShared {
     volatile unsigned abort_flag;
 };
 
-__device__ __forceinline__ unsigned tg_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long tg_timer()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void tg_mbar_init(unsigned bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void tg_mbar_expect_tx(unsigned bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void tg_mbar_arrive(unsigned bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool tg_mbar_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 // Bounded wait; returns false once this CTA has given up.
 __device__ __forceinline__ bool tg_wait(unsigned bar, unsigned parity, const TgParams& P, TgShared* sh)
 {
-    if (tg_mbar_try_wait(bar, parity)) return true;
+    if (lfptx::mbar_try_wait(bar, parity)) return true;
     if (sh->abort_flag) return false;
-    const unsigned long long t0 = tg_timer();
+    const unsigned long long t0 = lfptx::globaltimer_ns();
     unsigned spins = 0;
-    while (!tg_mbar_try_wait(bar, parity)) {
+    while (!lfptx::mbar_try_wait(bar, parity)) {
         if ((++spins & 15u) == 0u) {
             if (sh->abort_flag) return false;
-            if (tg_timer() - t0 > P.budget_ns) {
+            if (lfptx::globaltimer_ns() - t0 > P.budget_ns) {
                 atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
                 sh->abort_flag = 1u;
                 return false;
@@ -99,12 +71,6 @@ __device__ __forceinline__ bool tg_wait(unsigned bar, unsigned parity, const TgP
         }
     }
     return true;
-}
-__device__ __forceinline__ void tg_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 // Shared-memory matrix descriptor of an MN-major 32-bit operand (128-byte swizzle, 32-byte
 // atoms): 32 floats (128 B) run along M/N, four consecutive samples form one 512-byte swizzle
@@ -146,23 +112,7 @@ __device__ __forceinline__ void tg_commit(unsigned bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tg_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tg_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 32 lanes x 32 consecutive fp32 columns of tensor memory -> 32 registers per thread
-__device__ __forceinline__ void tg_tmem_ld32(unsigned taddr, unsigned (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
 // Fused weight update: ask L2 for the part of the w tile this warp will subtract from (32 rows x
 // `cols` columns starting at row_first, col_first), one 128-byte line per request, while the
@@ -193,24 +143,24 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < TG_STAGES; ++i) {
-            tg_mbar_init(tg_smem_u32(&sh->full[i]), 1);
-            tg_mbar_init(tg_smem_u32(&sh->empty[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
-            tg_mbar_init(tg_smem_u32(&sh->tmem_full[i]), 1);
-            tg_mbar_init(tg_smem_u32(&sh->tmem_empty[i]), 128);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->tmem_full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->tmem_empty[i]), 128);
         }
         sh->abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        lfptx::mbar_fence_init();
     }
     if (warp == 1) {   // tensor memory for both accumulators
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(tg_smem_u32(&sh->tmem_base)), "r"((unsigned)TG_TMEM_COLS) : "memory");
+                     ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)TG_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    tg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    tg_fence_after();
+    lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
 
     if (warp == 0) {
@@ -221,27 +171,27 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                 const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % TG_STAGES, use = it / TG_STAGES;
-                    if (use > 0 && !tg_wait(tg_smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
-                    const unsigned bar = tg_smem_u32(&sh->full[st]);
-                    tg_mbar_expect_tx(bar, TG_STAGE_BYTES);
+                    if (use > 0 && !tg_wait(lfptx::smem_u32(&sh->empty[st]), (use - 1) & 1u, P, sh)) break;
+                    const unsigned bar = lfptx::smem_u32(&sh->full[st]);
+                    lfptx::mbar_arrive_expect_tx(bar, TG_STAGE_BYTES);
                     if (P.withhold && blockIdx.x == 0 && it == 0) continue;   // test hook: armed, never loaded
-                    const unsigned a_dst = tg_smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
+                    const unsigned a_dst = lfptx::smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
                     const unsigned b_dst = a_dst + TG_A_BYTES;
 #pragma unroll
                     for (int i = 0; i < TG_BM / 32; ++i)
-                        tg_tma_load_2d(a_dst + i * TG_BOX_BYTES, &map_d, bar, tm * TG_BM + i * 32, ks * TG_BK);
+                        lfptx::tma_load_2d(a_dst + i * TG_BOX_BYTES, &map_d, bar, tm * TG_BM + i * 32, ks * TG_BK);
 #pragma unroll
                     for (int i = 0; i < TG_BN / 32; ++i)
-                        tg_tma_load_2d(b_dst + i * TG_BOX_BYTES, &map_a, bar, tn * TG_BN + i * 32, ks * TG_BK);
+                        lfptx::tma_load_2d(b_dst + i * TG_BOX_BYTES, &map_a, bar, tn * TG_BN + i * 32, ks * TG_BK);
                 }
                 if (sh->abort_flag) break;
             }
             // after giving up: do not let the CTA exit under loads that are still landing
             if (sh->abort_flag) {
-                const unsigned long long t0 = tg_timer();
+                const unsigned long long t0 = lfptx::globaltimer_ns();
                 for (unsigned j = it > TG_STAGES ? it - TG_STAGES : 0; j < it; ++j) {
-                    const unsigned bar = tg_smem_u32(&sh->full[j % TG_STAGES]);
-                    while (!tg_mbar_try_wait(bar, (j / TG_STAGES) & 1u) && tg_timer() - t0 < 50000000ull) { }
+                    const unsigned bar = lfptx::smem_u32(&sh->full[j % TG_STAGES]);
+                    while (!lfptx::mbar_try_wait(bar, (j / TG_STAGES) & 1u) && lfptx::globaltimer_ns() - t0 < 50000000ull) { }
                 }
             }
         }
@@ -252,15 +202,15 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
             unsigned it = 0, tile_i = 0;
             for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_i) {
                 const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
-                if (ab_use > 0 && !tg_wait(tg_smem_u32(&sh->tmem_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
-                tg_fence_after();
+                if (ab_use > 0 && !tg_wait(lfptx::smem_u32(&sh->tmem_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
+                lfptx::tc_fence_after();
                 const unsigned d_tmem = tmem_base + ab * (unsigned)TG_BN;
                 bool ok = true;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     const unsigned st = it % TG_STAGES, use = it / TG_STAGES;
-                    if (!tg_wait(tg_smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
-                    tg_fence_after();
-                    const unsigned a_addr = tg_smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
+                    if (!tg_wait(lfptx::smem_u32(&sh->full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    lfptx::tc_fence_after();
+                    const unsigned a_addr = lfptx::smem_u32(stages + (size_t)st * TG_STAGE_BYTES);
                     const unsigned b_addr = a_addr + TG_A_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < TG_BK / 8; ++kk) {      // eight samples per instruction
@@ -268,10 +218,10 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                         const unsigned long long db = tg_make_desc(b_addr + kk * 1024, TG_BOX_BYTES);
                         tg_mma_tf32(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
                     }
-                    tg_commit(tg_smem_u32(&sh->empty[st]));      // the stage may be refilled once these are done
+                    tg_commit(lfptx::smem_u32(&sh->empty[st]));      // the stage may be refilled once these are done
                 }
                 if (!ok) break;
-                tg_commit(tg_smem_u32(&sh->tmem_full[ab]));      // accumulator complete
+                tg_commit(lfptx::smem_u32(&sh->tmem_full[ab]));      // accumulator complete
             }
         }
     } else {
@@ -282,8 +232,8 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
             const int tm = t / P.tiles_n, tn = t - tm * P.tiles_n;
             const unsigned ab = tile_i & 1u, ab_use = tile_i >> 1;
             if (P.sgd.w_sub) tg_prefetch_w(P.sgd.w_sub, P.M, P.N, tm * TG_BM + quad * 32, tn * TG_BN, TG_BN, lane);
-            if (!tg_wait(tg_smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
-            tg_fence_after();
+            if (!tg_wait(lfptx::smem_u32(&sh->tmem_full[ab]), ab_use & 1u, P, sh)) break;
+            lfptx::tc_fence_after();
             // A thread reads one accumulator row (32 columns at a time).  The block is turned
             // through shared memory so that the warp stores whole 128-byte row segments.
             float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
@@ -301,7 +251,7 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                             wv[i] = __ldcs(reinterpret_cast<const float4*>(P.sgd.w_sub + (size_t)(row0 + i * 4 + sub_r) * P.N + col_w));
                 }
                 unsigned r[32];
-                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TG_BN + cchunk * 32, r);
+                lfptx::tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TG_BN + cchunk * 32, r);
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
                     *reinterpret_cast<float4*>(blk + lane * TG_EPI_LD + 4 * v) =
@@ -321,15 +271,15 @@ k_gw_gemm_tf32(const __grid_constant__ CUtensorMap map_d, const __grid_constant_
                 }
                 __syncwarp();
             }
-            tg_fence_before();
-            tg_mbar_arrive(tg_smem_u32(&sh->tmem_empty[ab]));
+            lfptx::tc_fence_before();
+            lfptx::mbar_arrive(lfptx::smem_u32(&sh->tmem_empty[ab]));
         }
     }
 
-    tg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        tg_fence_after();
+        lfptx::tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)TG_TMEM_COLS)
                      : "memory");
     }
@@ -384,30 +334,6 @@ struct TpShared {
 };
 static_assert(sizeof(TpShared) <= 512, "the barrier block must fit into the space reserved for it");
 
-__device__ __forceinline__ unsigned tp_cluster_rank()
-{
-    unsigned r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ unsigned tp_map_to_rank(unsigned local_addr, unsigned rank)
-{
-    unsigned r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void tp_cluster_sync()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA load into this CTA's shared memory whose bytes are credited to an mbarrier that may sit in
-// the other CTA of the pair (`bar` is a shared::cluster address).
-__device__ __forceinline__ void tp_tma_load_2d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
 __device__ __forceinline__ void tp_mma_tf32(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                             unsigned idesc, unsigned accumulate)
 {
@@ -429,16 +355,6 @@ __device__ __forceinline__ void tp_arrive_remote(unsigned cluster_bar)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
-__device__ __forceinline__ bool tp_try_wait_cluster(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ void tp_complete_tx(unsigned bar, unsigned bytes)   // bytes that will never arrive
 {
     asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -452,14 +368,14 @@ __device__ __forceinline__ unsigned tp_ld_remote(unsigned cluster_addr)
 // Bounded wait on a barrier of this CTA; returns false once this CTA has given up.
 __device__ __forceinline__ bool tp_wait(unsigned bar, unsigned parity, const TgParams& P, TpShared* sh)
 {
-    if (tp_try_wait_cluster(bar, parity)) return true;
+    if (lfptx::mbar_try_wait_cluster(bar, parity)) return true;
     if (sh->abort_flag) return false;
-    const unsigned long long t0 = tg_timer();
+    const unsigned long long t0 = lfptx::globaltimer_ns();
     unsigned spins = 0;
-    while (!tp_try_wait_cluster(bar, parity)) {
+    while (!lfptx::mbar_try_wait_cluster(bar, parity)) {
         if ((++spins & 15u) == 0u) {
             if (sh->abort_flag) return false;
-            if (tg_timer() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
+            if (lfptx::globaltimer_ns() - t0 > P.budget_ns || (((spins & 1023u) == 0u) && *((volatile unsigned*)P.status) != 0u)) {
                 atomicOr(P.status, LF_DEV_TIMEOUT_BARRIER);
                 sh->abort_flag = 1u;
                 return false;
@@ -489,7 +405,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     TpShared* sh = reinterpret_cast<TpShared*>(reinterpret_cast<unsigned char*>(epi) + TP_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned rank = tp_cluster_rank();          // 0 = leader (issues the multiplications)
+    const unsigned rank = lfptx::cluster_ctarank();          // 0 = leader (issues the multiplications)
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int n_k = (P.B + TG_BK - 1) / TG_BK;        // RESIDENT: <= TP_MAX_KS
     constexpr unsigned N_ST = RESIDENT ? TP_STAGES : TPS_STAGES;
@@ -498,28 +414,28 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     const int t_end = (int)(((long long)n_tiles * (pair + 1)) / n_pairs);
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < TP_MAX_KS; ++i) tg_mbar_init(tg_smem_u32(&sh->a_full[i]), 1);
-        tg_mbar_init(tg_smem_u32(&sh->a_empty), 1);
+        for (int i = 0; i < TP_MAX_KS; ++i) lfptx::mbar_init(lfptx::smem_u32(&sh->a_full[i]), 1);
+        lfptx::mbar_init(lfptx::smem_u32(&sh->a_empty), 1);
         for (int i = 0; i < TPS_STAGES; ++i) {
-            tg_mbar_init(tg_smem_u32(&sh->b_full[i]), 1);
-            tg_mbar_init(tg_smem_u32(&sh->b_empty[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->b_full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->b_empty[i]), 1);
         }
         for (int i = 0; i < TP_ACC; ++i) {
-            tg_mbar_init(tg_smem_u32(&sh->acc_full[i]), 1);
-            tg_mbar_init(tg_smem_u32(&sh->acc_empty[i]), 16);  // eight epilogue warps of each CTA
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_full[i]), 1);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_empty[i]), 16);  // eight epilogue warps of each CTA
         }
         sh->abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        lfptx::mbar_fence_init();
     }
     if (warp == 1) {   // tensor memory for the accumulators, the same columns in both CTAs
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(tg_smem_u32(&sh->tmem_base)), "r"((unsigned)(TP_ACC * TP_BN)) : "memory");
+                     ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)(TP_ACC * TP_BN)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
-    tg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    tp_cluster_sync();   // the peer's barriers exist before anything can arrive on them
-    tg_fence_after();
+    lfptx::cluster_sync_all();   // the peer's barriers exist before anything can arrive on them
+    lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
 
     if (warp == 0) {
@@ -536,7 +452,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 if (new_rb) {
                     // the resident delta operand changes: wait until every multiplication that
                     // reads the old one is done
-                    if (a_loads > 0 && !tp_wait(tg_smem_u32(&sh->a_empty), (a_loads - 1) & 1u, P, sh)) break;
+                    if (a_loads > 0 && !tp_wait(lfptx::smem_u32(&sh->a_empty), (a_loads - 1) & 1u, P, sh)) break;
                     cur_rb = rb;
                     ++a_loads;
                     a_ks = 0;
@@ -544,38 +460,38 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     if (new_rb) {
                         ++a_ks;
-                        const unsigned lbar = tg_smem_u32(&sh->a_full[ks]);
-                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_A_STAGE_BYTES);
-                        const unsigned bar = tp_map_to_rank(lbar, 0);
-                        const unsigned dst = tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES);
+                        const unsigned lbar = lfptx::smem_u32(&sh->a_full[ks]);
+                        if (rank == 0) lfptx::mbar_arrive_expect_tx(lbar, 2u * TP_A_STAGE_BYTES);
+                        const unsigned bar = lfptx::map_to_cta(lbar, 0);
+                        const unsigned dst = lfptx::smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES);
 #pragma unroll
                         for (int i = 0; i < TP_BM / 32; ++i)
-                            tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
+                            lfptx::tma_load_2d_pair(dst + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
                                            ks * TG_BK);
                     }
                     const unsigned st = it % N_ST, use = it / N_ST;
-                    if (use > 0 && !tp_wait(tg_smem_u32(&sh->b_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
-                    const unsigned lbar = tg_smem_u32(&sh->b_full[st]);
-                    const unsigned bar = tp_map_to_rank(lbar, 0);
+                    if (use > 0 && !tp_wait(lfptx::smem_u32(&sh->b_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
+                    const unsigned lbar = lfptx::smem_u32(&sh->b_full[st]);
+                    const unsigned bar = lfptx::map_to_cta(lbar, 0);
                     if (P.withhold && pair == 0 && rank == 1 && it == 0) continue;   // test hook: the peer leaves out its first stage
                     if (RESIDENT) {
-                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
-                        const unsigned dst = tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
+                        if (rank == 0) lfptx::mbar_arrive_expect_tx(lbar, 2u * TP_B_STAGE_BYTES);
+                        const unsigned dst = lfptx::smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES);
 #pragma unroll
                         for (int i = 0; i < TP_BN / 2 / 32; ++i)
-                            tp_tma_load_2d(dst + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                            lfptx::tma_load_2d_pair(dst + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
                     } else {
                         // streaming form: this CTA's half of both operands for these 32 samples
-                        if (rank == 0) tg_mbar_expect_tx(lbar, 2u * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
-                        const unsigned dst_a = tg_smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                        if (rank == 0) lfptx::mbar_arrive_expect_tx(lbar, 2u * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                        const unsigned dst_a = lfptx::smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
                         const unsigned dst_b = dst_a + TP_A_STAGE_BYTES;
 #pragma unroll
                         for (int i = 0; i < TP_BM / 32; ++i)
-                            tp_tma_load_2d(dst_a + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
+                            lfptx::tma_load_2d_pair(dst_a + i * TG_BOX_BYTES, &map_d, bar, rb * 2 * TP_BM + my_row0 + i * 32,
                                            ks * TG_BK);
 #pragma unroll
                         for (int i = 0; i < TP_BN / 2 / 32; ++i)
-                            tp_tma_load_2d(dst_b + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
+                            lfptx::tma_load_2d_pair(dst_b + i * TG_BOX_BYTES, &map_a, bar, tn * TP_BN + my_col0 + i * 32, ks * TG_BK);
                     }
                 }
             }
@@ -592,18 +508,18 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 const bool new_rb = RESIDENT && rb != cur_rb;
                 if (new_rb) { cur_rb = rb; ++a_loads; }
                 const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
-                if (ab_use > 0 && !tp_wait(tg_smem_u32(&sh->acc_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
-                tg_fence_after();
+                if (ab_use > 0 && !tp_wait(lfptx::smem_u32(&sh->acc_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
+                lfptx::tc_fence_after();
                 const unsigned d_tmem = tmem_base + ab * (unsigned)TP_BN;
                 bool ok = true;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
-                    if (new_rb && !tp_wait(tg_smem_u32(&sh->a_full[ks]), (a_loads - 1) & 1u, P, sh)) { ok = false; break; }
+                    if (new_rb && !tp_wait(lfptx::smem_u32(&sh->a_full[ks]), (a_loads - 1) & 1u, P, sh)) { ok = false; break; }
                     const unsigned st = it % N_ST, use = it / N_ST;
-                    if (!tp_wait(tg_smem_u32(&sh->b_full[st]), use & 1u, P, sh)) { ok = false; break; }
-                    tg_fence_after();
-                    const unsigned a_addr = RESIDENT ? tg_smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES)
-                                                     : tg_smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
-                    const unsigned b_addr = RESIDENT ? tg_smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES)
+                    if (!tp_wait(lfptx::smem_u32(&sh->b_full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    lfptx::tc_fence_after();
+                    const unsigned a_addr = RESIDENT ? lfptx::smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES)
+                                                     : lfptx::smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
+                    const unsigned b_addr = RESIDENT ? lfptx::smem_u32(b_ring + (size_t)st * TP_B_STAGE_BYTES)
                                                      : a_addr + TP_A_STAGE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < TG_BK / 8; ++kk) {      // eight samples per instruction
@@ -611,12 +527,12 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                         const unsigned long long db = tg_make_desc(b_addr + kk * 1024, TG_BOX_BYTES);
                         tp_mma_tf32(d_tmem, da, db, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
                     }
-                    tp_commit_both(tg_smem_u32(&sh->b_empty[st]));
+                    tp_commit_both(lfptx::smem_u32(&sh->b_empty[st]));
                 }
                 if (!ok) break;
                 // the last tile of a row block frees the resident operand for the next one
-                if (RESIDENT && t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(tg_smem_u32(&sh->a_empty));
-                tp_commit_both(tg_smem_u32(&sh->acc_full[ab]));
+                if (RESIDENT && t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(lfptx::smem_u32(&sh->a_empty));
+                tp_commit_both(lfptx::smem_u32(&sh->acc_full[ab]));
             }
         }
     } else {
@@ -626,7 +542,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
         // row segments.
         const int quad = warp & 3;                 // the TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;
-        const unsigned leader_acc_empty0 = tp_map_to_rank(tg_smem_u32(&sh->acc_empty[0]), 0);
+        const unsigned leader_acc_empty0 = lfptx::map_to_cta(lfptx::smem_u32(&sh->acc_empty[0]), 0);
         float* blk = epi + (warp - 2) * 32 * TG_EPI_LD;
         const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
         unsigned tile_i = 0;
@@ -641,8 +557,8 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             const size_t row_step = (size_t)4 * P.N;
             if (w_row)
                 tg_prefetch_w(P.sgd.w_sub, P.M, P.N, row0 - sub_r, tn * TP_BN + half * (TP_BN / 2), TP_BN / 2, lane);
-            if (!tp_wait(tg_smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
-            tg_fence_after();
+            if (!tp_wait(lfptx::smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
+            lfptx::tc_fence_after();
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TP_BN / 2 / 32; ++cchunk) {
                 // fused weight update: the loads of w go out before the accumulator is fetched
@@ -654,7 +570,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                             wv[i] = __ldcs(reinterpret_cast<const float4*>(w_row + i * row_step + cchunk * 32));
                 }
                 unsigned r[32];
-                tg_tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + half * (TP_BN / 2) + cchunk * 32, r);
+                lfptx::tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + ab * (unsigned)TP_BN + half * (TP_BN / 2) + cchunk * 32, r);
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
                     *reinterpret_cast<float4*>(blk + lane * TG_EPI_LD + 4 * v) =
@@ -673,7 +589,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 }
                 __syncwarp();
             }
-            tg_fence_before();
+            lfptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) tp_arrive_remote(leader_acc_empty0 + ab * (unsigned)sizeof(unsigned long long));
         }
@@ -682,9 +598,9 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     // Neither CTA may leave (or free tensor memory) while the other can still reach it: the
     // leader's multiplications read the peer's shared memory and write the peer's tensor
     // memory, and its commits arrive on the peer's barriers.
-    tg_fence_before();
+    lfptx::tc_fence_before();
     __syncthreads();
-    tp_cluster_sync();     // both producers have stopped; what each has issued is in its prog_* words
+    lfptx::cluster_sync_all();     // both producers have stopped; what each has issued is in its prog_* words
     if (threadIdx.x == 0 && rank == 0) {
         // A launch that was given up: no CTA of the pair may exit while operand loads are still on
         // their way into its shared memory.  The loads of BOTH CTAs are credited to the leader's
@@ -692,40 +608,40 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
         // loads for has been brought to a state it can complete in: a phase only the peer loaded
         // for gets the arrival (and the byte count) the leader never gave it, a phase only the
         // leader loaded for is told that the peer's bytes will not come.  Then wait, with a limit.
-        const bool gave_up = sh->abort_flag != 0u || tp_ld_remote(tp_map_to_rank(tg_smem_u32((const void*)&sh->abort_flag), 1)) != 0u;
+        const bool gave_up = sh->abort_flag != 0u || tp_ld_remote(lfptx::map_to_cta(lfptx::smem_u32((const void*)&sh->abort_flag), 1)) != 0u;
         if (gave_up) {
-            const unsigned it_l = sh->prog_it, it_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_it), 1));
+            const unsigned it_l = sh->prog_it, it_p = tp_ld_remote(lfptx::map_to_cta(lfptx::smem_u32(&sh->prog_it), 1));
             const unsigned stage_bytes = RESIDENT ? (unsigned)TP_B_STAGE_BYTES : (unsigned)(TP_A_STAGE_BYTES + TP_B_STAGE_BYTES);
             const unsigned it_hi = it_l > it_p ? it_l : it_p, it_lo = it_l < it_p ? it_l : it_p;
             for (unsigned j = it_lo; j < it_hi; ++j) {
-                const unsigned bar = tg_smem_u32(&sh->b_full[j % N_ST]);
-                if (j >= it_l) tg_mbar_expect_tx(bar, stage_bytes);      // only the peer loaded
+                const unsigned bar = lfptx::smem_u32(&sh->b_full[j % N_ST]);
+                if (j >= it_l) lfptx::mbar_arrive_expect_tx(bar, stage_bytes);      // only the peer loaded
                 else tp_complete_tx(bar, stage_bytes);                  // only the leader loaded
             }
-            const unsigned long long t0 = tg_timer();
+            const unsigned long long t0 = lfptx::globaltimer_ns();
             for (unsigned j = it_hi > N_ST ? it_hi - N_ST : 0; j < it_hi; ++j) {
-                const unsigned bar = tg_smem_u32(&sh->b_full[j % N_ST]);
-                while (!tg_mbar_try_wait(bar, (j / N_ST) & 1u) && tg_timer() - t0 < 50000000ull) { }
+                const unsigned bar = lfptx::smem_u32(&sh->b_full[j % N_ST]);
+                while (!lfptx::mbar_try_wait(bar, (j / N_ST) & 1u) && lfptx::globaltimer_ns() - t0 < 50000000ull) { }
             }
             if (RESIDENT) {
                 // the resident operand: chunks of the load that was under way (loads before it were
                 // waited for by the multiplications that freed the operand for this one)
-                const unsigned al_l = sh->prog_a_loads, al_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_a_loads), 1));
-                const unsigned ak_l = sh->prog_a_ks, ak_p = tp_ld_remote(tp_map_to_rank(tg_smem_u32(&sh->prog_a_ks), 1));
+                const unsigned al_l = sh->prog_a_loads, al_p = tp_ld_remote(lfptx::map_to_cta(lfptx::smem_u32(&sh->prog_a_loads), 1));
+                const unsigned ak_l = sh->prog_a_ks, ak_p = tp_ld_remote(lfptx::map_to_cta(lfptx::smem_u32(&sh->prog_a_ks), 1));
                 const unsigned al = al_l > al_p ? al_l : al_p;
                 const unsigned kl = al_l == al ? ak_l : 0u, kp = al_p == al ? ak_p : 0u;   // chunks of load `al`
                 for (unsigned ks = 0; ks < (kl > kp ? kl : kp) && al > 0; ++ks) {
-                    const unsigned bar = tg_smem_u32(&sh->a_full[ks]);
-                    if (ks >= kl) tg_mbar_expect_tx(bar, (unsigned)TP_A_STAGE_BYTES);
+                    const unsigned bar = lfptx::smem_u32(&sh->a_full[ks]);
+                    if (ks >= kl) lfptx::mbar_arrive_expect_tx(bar, (unsigned)TP_A_STAGE_BYTES);
                     else if (ks >= kp) tp_complete_tx(bar, (unsigned)TP_A_STAGE_BYTES);
-                    while (!tg_mbar_try_wait(bar, (al - 1) & 1u) && tg_timer() - t0 < 50000000ull) { }
+                    while (!lfptx::mbar_try_wait(bar, (al - 1) & 1u) && lfptx::globaltimer_ns() - t0 < 50000000ull) { }
                 }
             }
         }
     }
-    tp_cluster_sync();
+    lfptx::cluster_sync_all();
     if (warp == 1) {
-        tg_fence_after();
+        lfptx::tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((unsigned)(TP_ACC * TP_BN)) : "memory");
     }

@@ -27,6 +27,7 @@
 #include <cuda.h>
 
 #include "lf_internal.h"
+#include "lf_ptx.cuh"
 
 namespace {
 
@@ -81,85 +82,11 @@ struct PkParams {
 #endif
 };
 
-// ---- small PTX wrappers ----------------------------------------------------------------------
-__device__ __forceinline__ unsigned smem_u32(const void* p)
-{
-    return (unsigned)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-// The barriers armed this way guard data written by TMA or st.async, never by the arriving
-// thread itself, so the arrive carries no release fence.
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.relaxed.cta.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar)
-{
-    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, unsigned bar,
-                                            int x, int y, int z)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
-        : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;"
-                 ::: "memory");
-}
+// ---- PTX wrappers: the shared ones of lf_ptx.cuh, and two of this kernel's own -------------------
+using namespace lfptx;
 __device__ __forceinline__ void chain_sync()   // the four chain warps only
 {
     asm volatile("bar.sync 1, 128;" ::: "memory");
-}
-__device__ __forceinline__ unsigned cluster_ctarank()
-{
-    unsigned r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ unsigned map_to_cta(unsigned local_addr, unsigned rank)
-{
-    unsigned r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
 }
 // Store four floats into the shared memory of a CTA of the cluster and credit 16 bytes to an
 // mbarrier there (both addresses from mapa): data and "it has arrived" travel together, no fence.
@@ -169,21 +96,6 @@ __device__ __forceinline__ void st_async_f32x4(unsigned cluster_addr, float4 v, 
         "st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
         ::"r"(cluster_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(cluster_bar)
         : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_slot(const unsigned long long* p)
-{
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_slot(unsigned long long* p, float value, unsigned epoch)
-{
-    unsigned long long v = ((unsigned long long)epoch << 32) | (unsigned long long)__float_as_uint(value);
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ void st_stream4(float* p, float4 v)
-{
-    __stcs(reinterpret_cast<float4*>(p), v);
 }
 
 // Debug builds (-DLF_PK_TRACE) record SM-clock stamps of each chain step of two CTAs.
@@ -366,7 +278,7 @@ k_backward_persistent(const __grid_constant__ CUtensorMap w_map, const PkParams 
             mbar_init(smem_u32(&sh->d_free[i]), PK_THREADS - PK_CHAIN_THREADS);
         }
         sh->abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_fence_init();
     }
     __syncthreads();
     cluster_sync_all();   // every CTA's barriers exist before a peer can arrive on them

@@ -67,20 +67,24 @@ def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
 @pytest.mark.parametrize("L,N,B,k", [(3, 516, 2, 2), (3, 1028, 5, 1), (2, 2052, 12, 2), (3, 4096, 16, 2),
                                      (2, 8, 4, 1), (4, 644, 9, 3)])
 def test_small_batch_delta_chain(L, N, B, k):
-    # Up to 16 samples the library's own choice for Eq. bp2 is fp32 on the CUDA cores (a batched
-    # matrix-vector product that reads w once), not the tensor cores; the forward pass keeps its
-    # tensor-core rule.  B = 2, 5, 12: each of the kernel's three sample-tile sizes with samples
+    # For a handful of samples Eq. bp2 has an fp32 kernel on the CUDA cores (a batched matrix-vector
+    # product that reads w once; what LF_DELTA_MATH_FP32 runs up to 16 samples); the forward pass keeps
+    # its tensor-core rule.  B = 2, 5, 12: each of the kernel's three sample-tile sizes with samples
     # missing from the last group of four; N = 516, 1028, 2052, 644: a last column strip of one or
     # five float4; N = 4096, B = 16: several 256-row blocks per CTA; N = 8: fewer rows than warps.
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=7 * N + B)
-    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32)
+    out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=lf.LF_DELTA_MATH_FP32)
     assert stats["delta_math"] == lf.LF_DELTA_MATH_FP32 and stats["device_status"] == 0
     ref = oracle_pass(t, want_gw=True)
     compare_all(cfg, out, ref)
     # twice in a row through one context: the strip counters reset themselves
-    out2, _ = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, repeat=3)
+    out2, _ = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=lf.LF_DELTA_MATH_FP32, repeat=3)
     assert torch.equal(out2["delta"], out["delta"])
+    # the library's own choice: fp32 up to 8 samples, and up to 16 from a width of 2048
+    _, auto = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32)
+    want = lf.LF_DELTA_MATH_FP32 if (B <= 8 or N >= 2048) else lf.LF_DELTA_MATH_3XTF32
+    assert auto["delta_math"] == want
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
