@@ -1042,10 +1042,15 @@ DgPlan dp_plan(const lf_ctx* c, int Nc, int K, int max_pairs)
 }
 
 // could the two-SM kernel be chosen for this shape (whatever LF_OPT_TC_TILING says)?
+// Measured per layer, forward / backward, pairs against one CTA per tile: with 32 to 128 samples the
+// pairs (second CTA's samples empty) lose at widths up to 4096 (N = 2048: 27-31 against 22 us) and win
+// at 8192 (139-148 against 155-157 us): there the weight tile each CTA need not load outweighs the
+// empty half.  Narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there.
+constexpr long long DP_WIDE_LAYER = 6144ll * 6144ll;
 bool dp_shape_fits_pairs(const lf_ctx* c, int Nc, int K)
 {
-    // (narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there)
-    return c->B > DG_BM && Nc >= 512 && K >= 512 && dp_max_pairs(c) > 0;
+    const bool enough = c->B > DG_BM || (long long)Nc * K >= DP_WIDE_LAYER;
+    return enough && Nc >= 512 && K >= 512 && dp_max_pairs(c) > 0;
 }
 
 bool dp_use_pairs(const lf_ctx* c, int Nc, int K)

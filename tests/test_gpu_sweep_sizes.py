@@ -44,6 +44,9 @@ def _sampled_minibatch_parity(L, N, B, tiling, seed, n_chain=3, grid=512):
     t = _inputs(L, N, B, "onehot", seed)
     out, stats = gpu_pass(cfg, t, tc_tiling=tiling)
     assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
+    # CTA pairs serve more than 128 samples, and layers of at least 6144 x 6144 at any batch
+    if tiling == lf.LF_TC_TILING_TWO_SM and (B > 128 or N >= 6144):
+        assert stats["delta_tiling"] == lf.LF_TC_TILING_TWO_SM
     # the library's own choice: a handful of samples (up to 8, or up to 16 from a width of 2048) keeps Eq. bp2 in fp32 on the CUDA cores
     assert stats["delta_math"] == (lf.LF_DELTA_MATH_FP32 if (B <= 8 or (B <= 16 and N >= 2048)) else lf.LF_DELTA_MATH_3XTF32)
 
