@@ -62,7 +62,8 @@ enum lf_variant {
 
 /* Arithmetic of the B > 1 weight-gradient contraction. */
 enum lf_gw_math {
-    LF_GW_MATH_AUTO = 0, /* TF32 tensor cores when B > 1 and the shape is supported          */
+    LF_GW_MATH_AUTO = 0, /* TF32 tensor cores when B > 16 and the shape is supported; up to 16
+                            samples Eq. bp4 is a store stream and stays fp32 (faster and exact)  */
     LF_GW_MATH_FP32 = 1, /* fp32 FMA on the CUDA cores                                        */
     LF_GW_MATH_TF32 = 2  /* inputs rounded to TF32, fp32 accumulation in tensor memory        */
 };

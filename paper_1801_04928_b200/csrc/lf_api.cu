@@ -61,6 +61,9 @@ int resolve_gw_math(const lf_ctx* c)
 {
     if (c->B == 1) return LF_GW_MATH_FP32;  // rank-1: one multiply per element, nothing to contract
     if (c->opt_gw_math == LF_GW_MATH_FP32) return LF_GW_MATH_FP32;
+    // up to 16 samples Eq. bp4 is a store stream (4B multiply-adds per 16 bytes): the fp32 writer is ahead
+    // of the tensor-core tiles at every width measured (256 .. 8192), and exact
+    if (c->opt_gw_math == LF_GW_MATH_AUTO && c->B <= 16) return LF_GW_MATH_FP32;
     return lf_tf32_supported(c) ? LF_GW_MATH_TF32 : LF_GW_MATH_FP32;
 }
 

@@ -348,9 +348,75 @@ cudaError_t lfk_delta_gemm(const float* w_up, const float* delta_up, const float
     return cudaGetLastError();
 }
 
+namespace {
+
+// ---- Eq. bp4 for a handful of samples (B <= 16) --------------------------------------------------
+// gw[j][k] = sum_b delta[b][j] a[b][k] is then a store stream like the rank-1 writer of B = 1: 4B
+// multiply-adds per 16 bytes stored, nothing to tile.  A thread keeps four columns of a (BT float4)
+// in registers and walks the rows of its block; the block's delta values sit in shared memory as
+// float4 over four samples (broadcast loads).  grid = 1024-column blocks x row chunks.
+constexpr int GS_THREADS = 256, GS_ROWS = 32;
+
+template <int BT>
+__global__ void __launch_bounds__(GS_THREADS)
+k_gw_small_batch(const float* __restrict__ delta_l, const float* __restrict__ a_prev, float* __restrict__ gw_l,
+                 int n_out, int n_in, int B, const lf_sgd sgd)
+{
+    __shared__ __align__(16) float4 d_sm[(BT / 4) * GS_ROWS];     // [sample group][row of the chunk]
+    const int n4 = n_in >> 2;
+    const int c4 = blockIdx.x * GS_THREADS + threadIdx.x;
+    const int row0 = blockIdx.y * GS_ROWS;
+    const int rows = min(GS_ROWS, n_out - row0);
+    for (int idx = threadIdx.x; idx < (BT / 4) * GS_ROWS; idx += GS_THREADS) {
+        const int j = idx % GS_ROWS, b4 = idx / GS_ROWS;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < rows) {
+            const float* src = delta_l + (size_t)(4 * b4) * n_out + row0 + j;
+            if (4 * b4 + 0 < B) v.x = src[0];
+            if (4 * b4 + 1 < B) v.y = src[n_out];
+            if (4 * b4 + 2 < B) v.z = src[2 * (size_t)n_out];
+            if (4 * b4 + 3 < B) v.w = src[3 * (size_t)n_out];
+        }
+        d_sm[idx] = v;
+    }
+    __syncthreads();
+    if (c4 >= n4) return;
+    float4 av[BT];
+#pragma unroll
+    for (int b = 0; b < BT; ++b)
+        av[b] = b < B ? reinterpret_cast<const float4*>(a_prev)[(size_t)b * n4 + c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4* out = reinterpret_cast<float4*>(gw_l) + (size_t)row0 * n4 + c4;
+    const float4* wsub = sgd.w_sub ? reinterpret_cast<const float4*>(sgd.w_sub) + (size_t)row0 * n4 + c4 : nullptr;
+#pragma unroll 2
+    for (int j = 0; j < rows; ++j) {
+        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int b4 = 0; b4 < BT / 4; ++b4) {
+            const float4 d = d_sm[b4 * GS_ROWS + j];
+            const float4 &a0 = av[4 * b4], &a1 = av[4 * b4 + 1], &a2 = av[4 * b4 + 2], &a3 = av[4 * b4 + 3];
+            g.x = fmaf(d.x, a0.x, g.x); g.y = fmaf(d.x, a0.y, g.y); g.z = fmaf(d.x, a0.z, g.z); g.w = fmaf(d.x, a0.w, g.w);
+            g.x = fmaf(d.y, a1.x, g.x); g.y = fmaf(d.y, a1.y, g.y); g.z = fmaf(d.y, a1.z, g.z); g.w = fmaf(d.y, a1.w, g.w);
+            g.x = fmaf(d.z, a2.x, g.x); g.y = fmaf(d.z, a2.y, g.y); g.z = fmaf(d.z, a2.z, g.z); g.w = fmaf(d.z, a2.w, g.w);
+            g.x = fmaf(d.w, a3.x, g.x); g.y = fmaf(d.w, a3.y, g.y); g.z = fmaf(d.w, a3.z, g.z); g.w = fmaf(d.w, a3.w, g.w);
+        }
+        if (wsub)   // fused update: w - eta * g, the weights streamed through once
+            g = lf_sgd_apply4(sgd.eta, __ldcs(wsub + (size_t)j * n4), g);
+        __stcs(out + (size_t)j * n4, g);
+    }
+}
+
+}  // namespace
+
 cudaError_t lfk_gw_gemm_fp32(const float* delta_l, const float* a_prev, float* gw_l, int n_out, int n_in,
                              int B, lf_sgd sgd, cudaStream_t s)
 {
+    if (B <= 16) {      // a handful of samples: a store stream, not a contraction
+        dim3 grid(((n_in >> 2) + GS_THREADS - 1) / GS_THREADS, (n_out + GS_ROWS - 1) / GS_ROWS);
+        if (B <= 4) k_gw_small_batch<4><<<grid, GS_THREADS, 0, s>>>(delta_l, a_prev, gw_l, n_out, n_in, B, sgd);
+        else if (B <= 8) k_gw_small_batch<8><<<grid, GS_THREADS, 0, s>>>(delta_l, a_prev, gw_l, n_out, n_in, B, sgd);
+        else k_gw_small_batch<16><<<grid, GS_THREADS, 0, s>>>(delta_l, a_prev, gw_l, n_out, n_in, B, sgd);
+        return cudaGetLastError();
+    }
     // M = n_out (j), Nn = n_in (k), K = B; both operands are contiguous along their M / N index
     k_gemm_simt<false, false, EPI_PLAIN><<<gemm_grid(n_out, n_in), 256, 0, s>>>(
         delta_l, a_prev, gw_l, nullptr, sgd.w_sub, n_out, n_in, B, n_out, n_in, n_in, sgd.eta, LF_ACT_SIGMOID);

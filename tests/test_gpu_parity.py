@@ -199,20 +199,32 @@ def test_tf32_pair_kernel_long_runs():
     L, N, B = 1, 6148, 64
     cfg = dict(L=L, N=N, B=B, k=1)
     t = _inputs(L, N, B, y="onehot", seed=77)
-    outs = {}
+    passes = {}
     for tiling in (lf.LF_TC_TILING_TWO_SM, lf.LF_TC_TILING_ONE_SM):
         out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_TF32, tc_tiling=tiling, repeat=2)
         assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
         assert stats["gw_tiling"] == tiling
-        outs[tiling] = out["gw"][0].cpu().numpy()
-    ref = orc.grad_w(out["delta"][0].cpu().numpy().astype(np.float64),
-                     out["a"][0].cpu().numpy().astype(np.float64))
-    for tiling, g in outs.items():
+        g = out["gw"][0].cpu().numpy()
+        ref = orc.grad_w(out["delta"][0].cpu().numpy().astype(np.float64),
+                         out["a"][0].cpu().numpy().astype(np.float64))
         assert np.all(np.isfinite(g))
         e = rel_frobenius(g, ref)
         assert e <= TF32_TOL, (tiling, e)
-    # the two tilings multiply the same truncated operands and add the samples in the same order
-    assert np.array_equal(outs[lf.LF_TC_TILING_TWO_SM], outs[lf.LF_TC_TILING_ONE_SM])
+        passes[tiling] = out
+    # on one delta and one a (the forward pass of so wide a layer depends on the tiling in its last
+    # bits) the two tilings multiply the same truncated operands and add the samples in the same order
+    d, a = passes[lf.LF_TC_TILING_TWO_SM]["delta"][0].contiguous(), passes[lf.LF_TC_TILING_TWO_SM]["a"][0].contiguous()
+    outs = {}
+    for tiling in (lf.LF_TC_TILING_TWO_SM, lf.LF_TC_TILING_ONE_SM):
+        gw = torch.full((N, N), float("nan"), device="cuda")
+        with lf.Leapfrog(1, N, B, 1) as ctx:
+            ctx.set_option(lf.LF_OPT_GW_MATH, lf.LF_GW_MATH_TF32)
+            ctx.set_option(lf.LF_OPT_TC_TILING, tiling)
+            ctx.grad_w(d, a, gw)
+            ctx.sync()
+            assert ctx.stats()["gw_tiling"] == tiling and ctx.stats()["device_status"] == 0
+        outs[tiling] = gw
+    assert torch.equal(outs[lf.LF_TC_TILING_TWO_SM], outs[lf.LF_TC_TILING_ONE_SM])
 
 
 def test_tf32_tilings_agree_bitwise_beyond_256_samples():

@@ -43,7 +43,9 @@ def _sampled_minibatch_parity(L, N, B, tiling, seed, n_chain=3, grid=512):
     cfg = dict(L=L, N=N, B=B, k=2)
     t = _inputs(L, N, B, "onehot", seed)
     out, stats = gpu_pass(cfg, t, tc_tiling=tiling)
-    assert stats["gw_math"] == lf.LF_GW_MATH_TF32 and stats["device_status"] == 0
+    # the library's own choice for Eq. bp4: up to 16 samples the fp32 store stream, beyond that TF32 tensor cores
+    assert stats["gw_math"] == (lf.LF_GW_MATH_FP32 if B <= 16 else lf.LF_GW_MATH_TF32) and stats["device_status"] == 0
+    tol = 2e-5 if B <= 16 else TF32_TOL      # the fp32 writer is held to fp32 level
     # CTA pairs serve more than 128 samples, and layers of at least 6144 x 6144 at any batch
     if tiling == lf.LF_TC_TILING_TWO_SM and (B > 128 or N >= 6144):
         assert stats["delta_tiling"] == lf.LF_TC_TILING_TWO_SM
@@ -79,17 +81,17 @@ def _sampled_minibatch_parity(L, N, B, tiling, seed, n_chain=3, grid=512):
         ref = orc.grad_w(np.ascontiguousarray(d_gpu[l][:, rows]), np.ascontiguousarray(a_gpu[l][:, cols]))
         got = g[np.ix_(rows, cols)]
         e = rel_frobenius(got, ref)
-        assert e <= TF32_TOL, ("grid", l, e)
+        assert e <= tol, ("grid", l, e)
         # tile by tile as well: a wrong tile must not hide in the whole-matrix norm
         gt = (got - ref).reshape(blocks, per, blocks, per)
         rt = ref.reshape(blocks, per, blocks, per)
         et = np.sqrt((gt * gt).sum(axis=(1, 3)) / (rt * rt).sum(axis=(1, 3)))
-        assert float(et.max()) <= 4 * TF32_TOL, ("tile", l, np.unravel_index(et.argmax(), et.shape), et.max())
+        assert float(et.max()) <= 4 * tol, ("tile", l, np.unravel_index(et.argmax(), et.shape), et.max())
         rms = np.sqrt(np.mean(g * g))
         for _ in range(32):
             j, k = int(rng.integers(N)), int(rng.integers(N))
             r1 = orc.grad_w_entry(d_gpu[l], a_gpu[l], j, k)
-            assert abs(g[j, k] - r1) <= TF32_TOL * max(abs(r1), rms), (l, j, k, g[j, k], r1)
+            assert abs(g[j, k] - r1) <= tol * max(abs(r1), rms), (l, j, k, g[j, k], r1)
     return stats
 
 

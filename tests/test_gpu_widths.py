@@ -144,7 +144,7 @@ def test_widths_chain_and_forward_on_the_tensor_cores(widths, B, tiling):
 def test_widths_weight_gradient_on_the_tensor_cores(widths, B, tiling):
     # Eq. bp4 of a rectangular layer as an n_l x n_{l-1} x B contraction with TF32 inputs; the two-SM
     # kernel takes batches up to 256, beyond that the one-SM kernel runs whatever was asked for
-    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=60 + B, gw_math=lf.LF_GW_MATH_AUTO, tiling=tiling)
+    n, L, cpu, out, stats = _run(widths, B, 2, y="onehot", seed=60 + B, gw_math=lf.LF_GW_MATH_TF32, tiling=tiling)
     assert stats["device_status"] == 0 and stats["gw_math"] == lf.LF_GW_MATH_TF32
     assert stats["gw_tiling"] == tiling      # CTA pairs at every batch (beyond 256 samples both operands stream)
     _compare(n, B, cpu, out, tf32=True)
