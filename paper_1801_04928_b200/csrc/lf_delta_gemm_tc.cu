@@ -886,27 +886,43 @@ struct DgSlots {
     int n_pairs, tiles_n, kb_per_tile, row4;   // row4 = N / 4
     int g_total;
 };
-__device__ __forceinline__ int dg_slot_count(const DgSlots& S, size_t i)
+// slots that hold a contribution to the output elements of sample b, columns n .. n+3
+__device__ __forceinline__ int dg_slot_count(const DgSlots& S, int b, int n)
 {
     if (S.n_pairs == 0) return S.splits;
-    const int b = (int)(i / (size_t)S.row4), n = (int)(i % (size_t)S.row4) * 4;
     const int g0 = ((b / (2 * DG_BM)) * S.tiles_n + n / DP_BN) * S.kb_per_tile;
     return dp_owner(g0 + S.kb_per_tile - 1, S.g_total, S.n_pairs) - dp_owner(g0, S.g_total, S.n_pairs) + 1;
 }
+// the sum of an element's slots, in slot order; the loads go out four at a time
+__device__ __forceinline__ float4 dg_slot_sum(const float4* __restrict__ p, size_t slot_stride, int splits)
+{
+    float4 s = __ldcg(p);
+    int sp = 1;
+    for (; sp + 4 <= splits; sp += 4) {
+        const float4 t0 = __ldcg(p + (size_t)sp * slot_stride), t1 = __ldcg(p + (size_t)(sp + 1) * slot_stride);
+        const float4 t2 = __ldcg(p + (size_t)(sp + 2) * slot_stride), t3 = __ldcg(p + (size_t)(sp + 3) * slot_stride);
+        s.x += t0.x; s.y += t0.y; s.z += t0.z; s.w += t0.w;
+        s.x += t1.x; s.y += t1.y; s.z += t1.z; s.w += t1.w;
+        s.x += t2.x; s.y += t2.y; s.z += t2.z; s.w += t2.w;
+        s.x += t3.x; s.y += t3.y; s.z += t3.z; s.w += t3.w;
+    }
+    for (; sp < splits; ++sp) {
+        const float4 t = __ldcg(p + (size_t)sp * slot_stride);
+        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+    return s;
+}
 
+// grid of the finish kernels: x = blocks of 256 float4 along a row of the output, y = sample
 // delta^l = (sum over the partial-sum slots, in slot order) * sigma'(z^l), sigma' = a (1 - a)
 __global__ void __launch_bounds__(256)
 k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
                size_t n4, const DgSlots S, int act)
 {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n4) return;
-    const int splits = dg_slot_count(S, i);
-    float4 s = reinterpret_cast<const float4*>(partial)[i];
-    for (int sp = 1; sp < splits; ++sp) {
-        const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
-        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
-    }
+    const int c4 = blockIdx.x * blockDim.x + threadIdx.x, b = blockIdx.y;
+    if (c4 >= S.row4) return;
+    const size_t i = (size_t)b * S.row4 + c4;
+    const float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
     const float4 av = reinterpret_cast<const float4*>(a_l)[i];
     reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * lf_act_prime(av.x, act), s.y * lf_act_prime(av.y, act),
                                                         s.z * lf_act_prime(av.z, act), s.w * lf_act_prime(av.w, act));
@@ -915,17 +931,13 @@ k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l,
 // forward: z^l = (sum over the partial-sum slots) + b^l ; a^l = sigma(z^l)
 __global__ void __launch_bounds__(256)
 k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_l, float* __restrict__ z_l,
-                 float* __restrict__ a_l, size_t n4, int n4_row, const DgSlots S, int act)
+                 float* __restrict__ a_l, size_t n4, const DgSlots S, int act)
 {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n4) return;
-    const int splits = dg_slot_count(S, i);
-    float4 s = reinterpret_cast<const float4*>(partial)[i];
-    for (int sp = 1; sp < splits; ++sp) {
-        const float4 t = reinterpret_cast<const float4*>(partial)[(size_t)sp * n4 + i];
-        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
-    }
-    const float4 bb = reinterpret_cast<const float4*>(b_l)[i % n4_row];
+    const int c4 = blockIdx.x * blockDim.x + threadIdx.x, b = blockIdx.y;
+    if (c4 >= S.row4) return;
+    const size_t i = (size_t)b * S.row4 + c4;
+    float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
+    const float4 bb = reinterpret_cast<const float4*>(b_l)[c4];
     s.x += bb.x; s.y += bb.y; s.z += bb.z; s.w += bb.w;
     reinterpret_cast<float4*>(z_l)[i] = s;
     reinterpret_cast<float4*>(a_l)[i] = make_float4(lf_act(s.x, act), lf_act(s.y, act), lf_act(s.z, act), lf_act(s.w, act));
@@ -1201,7 +1213,8 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     int rc = dg_launch(c, delta_up, w_up, false, math == LF_DELTA_MATH_TF32_BF16, n_l, n_up, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_l / 4;
-    k_delta_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4, dg_slots(n_l, pl), c->opt_act);
+    k_delta_finish<<<dim3((unsigned)((n_l / 4 + 255) / 256), (unsigned)c->B), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4,
+                                                                                       dg_slots(n_l, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
@@ -1215,8 +1228,8 @@ int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const floa
     int rc = dg_launch(c, a_prev, w_l, true, math == LF_DELTA_MATH_TF32_BF16, n_out, n_in, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_out / 4;
-    k_forward_finish<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4, n_out / 4,
-                                                                  dg_slots(n_out, pl), c->opt_act);
+    k_forward_finish<<<dim3((unsigned)((n_out / 4 + 255) / 256), (unsigned)c->B), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4,
+                                                                                           dg_slots(n_out, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
     return LF_OK;
