@@ -217,9 +217,13 @@ k_delta_small_batch(const float* __restrict__ w_up, const float* __restrict__ de
         sb_cp_commit();
     }
 
-    float4 acc[BT];
+    // running sums as pairs of samples, acc[p][c] = (sample 2p, sample 2p + 1) of column c: the two
+    // multiply-adds of a pair are one packed instruction (fma.rn.f32x2; each half an ordinary fp32 fma)
+    float2 acc[BT / 2][4];
 #pragma unroll
-    for (int b = 0; b < BT; ++b) acc[b] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = 0; p < BT / 2; ++p)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[p][c] = make_float2(0.f, 0.f);
 
     int i = 0;     // index of my next row
     for (int blk0 = 0; blk0 < rows; blk0 += SB_BLOCK_ROWS) {
@@ -247,14 +251,16 @@ k_delta_small_batch(const float* __restrict__ w_up, const float* __restrict__ de
             sb_cp_wait<SB_DEPTH - 1>();      // the group of row i has landed
             const float4 wv = ring[(i % SB_DEPTH) * SB_THREADS + tid];
             const int j = warp + i * SB_WARPS - blk0;
+            const float2 w2[4] = {make_float2(wv.x, wv.x), make_float2(wv.y, wv.y), make_float2(wv.z, wv.z), make_float2(wv.w, wv.w)};
 #pragma unroll
             for (int b4 = 0; b4 < BT / 4; ++b4) {
                 const float4 d = d_sm[b4 * SB_BLOCK_ROWS + j];
-                float4& a0 = acc[4 * b4], &a1 = acc[4 * b4 + 1], &a2 = acc[4 * b4 + 2], &a3 = acc[4 * b4 + 3];
-                a0.x = fmaf(wv.x, d.x, a0.x); a0.y = fmaf(wv.y, d.x, a0.y); a0.z = fmaf(wv.z, d.x, a0.z); a0.w = fmaf(wv.w, d.x, a0.w);
-                a1.x = fmaf(wv.x, d.y, a1.x); a1.y = fmaf(wv.y, d.y, a1.y); a1.z = fmaf(wv.z, d.y, a1.z); a1.w = fmaf(wv.w, d.y, a1.w);
-                a2.x = fmaf(wv.x, d.z, a2.x); a2.y = fmaf(wv.y, d.z, a2.y); a2.z = fmaf(wv.z, d.z, a2.z); a2.w = fmaf(wv.w, d.z, a2.w);
-                a3.x = fmaf(wv.x, d.w, a3.x); a3.y = fmaf(wv.y, d.w, a3.y); a3.z = fmaf(wv.z, d.w, a3.z); a3.w = fmaf(wv.w, d.w, a3.w);
+                const float2 d01 = make_float2(d.x, d.y), d23 = make_float2(d.z, d.w);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    acc[2 * b4][c] = __ffma2_rn(w2[c], d01, acc[2 * b4][c]);
+                    acc[2 * b4 + 1][c] = __ffma2_rn(w2[c], d23, acc[2 * b4 + 1][c]);
+                }
             }
         }
     }
@@ -264,7 +270,11 @@ k_delta_small_batch(const float* __restrict__ w_up, const float* __restrict__ de
 #pragma unroll
     for (int r = 0; r < BT / 4; ++r) {
 #pragma unroll
-        for (int sidx = 0; sidx < 4; ++sidx) red[(warp * 32 + lane) * 4 + sidx] = col_ok ? acc[4 * r + sidx] : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sidx = 0; sidx < 4; ++sidx) {
+            const float2* ap = acc[2 * r + (sidx >> 1)];      // the pair that holds sample 4r + sidx
+            const float4 v = (sidx & 1) ? make_float4(ap[0].y, ap[1].y, ap[2].y, ap[3].y) : make_float4(ap[0].x, ap[1].x, ap[2].x, ap[3].x);
+            red[(warp * 32 + lane) * 4 + sidx] = col_ok ? v : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         __syncthreads();
         if (tid < 128) {
             const int l = tid & 31, sidx = tid >> 5, b = 4 * r + sidx, c = strip * SB_STRIP4 + l;
@@ -389,16 +399,21 @@ k_gw_small_batch(const float* __restrict__ delta_l, const float* __restrict__ a_
     const float4* wsub = sgd.w_sub ? reinterpret_cast<const float4*>(sgd.w_sub) + (size_t)row0 * n4 + c4 : nullptr;
 #pragma unroll 2
     for (int j = 0; j < rows; ++j) {
-        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+        // two columns per packed multiply-add (fma.rn.f32x2: each half an ordinary fp32 fma, samples in order)
+        float2 g01 = make_float2(0.f, 0.f), g23 = make_float2(0.f, 0.f);
 #pragma unroll
         for (int b4 = 0; b4 < BT / 4; ++b4) {
             const float4 d = d_sm[b4 * GS_ROWS + j];
-            const float4 &a0 = av[4 * b4], &a1 = av[4 * b4 + 1], &a2 = av[4 * b4 + 2], &a3 = av[4 * b4 + 3];
-            g.x = fmaf(d.x, a0.x, g.x); g.y = fmaf(d.x, a0.y, g.y); g.z = fmaf(d.x, a0.z, g.z); g.w = fmaf(d.x, a0.w, g.w);
-            g.x = fmaf(d.y, a1.x, g.x); g.y = fmaf(d.y, a1.y, g.y); g.z = fmaf(d.y, a1.z, g.z); g.w = fmaf(d.y, a1.w, g.w);
-            g.x = fmaf(d.z, a2.x, g.x); g.y = fmaf(d.z, a2.y, g.y); g.z = fmaf(d.z, a2.z, g.z); g.w = fmaf(d.z, a2.w, g.w);
-            g.x = fmaf(d.w, a3.x, g.x); g.y = fmaf(d.w, a3.y, g.y); g.z = fmaf(d.w, a3.z, g.z); g.w = fmaf(d.w, a3.w, g.w);
+            const float dv[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 dd = make_float2(dv[q], dv[q]);
+                const float4& ab = av[4 * b4 + q];
+                g01 = __ffma2_rn(dd, make_float2(ab.x, ab.y), g01);
+                g23 = __ffma2_rn(dd, make_float2(ab.z, ab.w), g23);
+            }
         }
+        float4 g = make_float4(g01.x, g01.y, g23.x, g23.y);
         if (wsub)   // fused update: w - eta * g, the weights streamed through once
             g = lf_sgd_apply4(sgd.eta, __ldcs(wsub + (size_t)j * n4), g);
         __stcs(out + (size_t)j * n4, g);
