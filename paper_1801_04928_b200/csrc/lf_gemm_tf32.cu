@@ -19,6 +19,26 @@
 #include "lf_internal.h"
 #include "lf_ptx.cuh"
 
+// Debug builds (-DLF_TG_TRACE): the leader CTA of pair 0 of the two-SM kernel stamps its SM clock per
+// tile (words 16 t + slot) and once per launch (words 8 .. 11 of tile 0); the release library carries
+// none of this.
+#ifdef LF_TG_TRACE
+constexpr int TG_TRACE_TILES = 32;
+__device__ long long tg_trace[TG_TRACE_TILES * 16];
+extern "C" int lf_debug_read_gw_pair_trace(long long* out)
+{
+    if (!out) return LF_ENULL;
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(out, tg_trace, sizeof(tg_trace)) == cudaSuccess ? LF_OK : LF_ECUDA;
+}
+// per tile: 0 issuer has the accumulator, 1 first stage's operands seen, 2 all products and commits issued,
+// 3 an epilogue warp sees the finished accumulator, 4 that warp has stored its part of the tile
+// once: 8 kernel entered, 9 set-up done, 10 first operand load issued
+#define TG_STAMP(tile, slot) do { if (pair == 0 && rank == 0 && (tile) < (unsigned)TG_TRACE_TILES) tg_trace[(tile) * 16 + (slot)] = clock64(); } while (0)
+#else
+#define TG_STAMP(tile, slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int TG_BM = 128, TG_BN = 256, TG_BK = 32;      // tile and samples per stage
@@ -412,6 +432,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     const int n_tiles = P.tiles_m * P.tiles_n;        // tiles_m counts 256-row blocks here
     const int t_begin = (int)(((long long)n_tiles * pair) / n_pairs);
     const int t_end = (int)(((long long)n_tiles * (pair + 1)) / n_pairs);
+    if (threadIdx.x == 0) TG_STAMP(0u, 8);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < TP_MAX_KS; ++i) lfptx::mbar_init(lfptx::smem_u32(&sh->a_full[i]), 1);
@@ -437,12 +458,14 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
     lfptx::cluster_sync_all();   // the peer's barriers exist before anything can arrive on them
     lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
+    if (threadIdx.x == 0) TG_STAMP(0u, 9);
 
     if (warp == 0) {
         // ------------------------------ TMA producer (each CTA, its own halves) ----------------
         if (lane == 0) {
             unsigned it = 0, a_loads = 0, a_ks = 0;
             int cur_rb = -1;
+            TG_STAMP(0u, 10);
             const int my_row0 = (int)rank * TP_BM;
             const int my_col0 = (int)rank * (TP_BN / 2);
             bool ok = true;
@@ -510,12 +533,14 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 const unsigned ab = tile_i % TP_ACC, ab_use = tile_i / TP_ACC;
                 if (ab_use > 0 && !tp_wait(lfptx::smem_u32(&sh->acc_empty[ab]), (ab_use - 1) & 1u, P, sh)) break;
                 lfptx::tc_fence_after();
+                TG_STAMP(tile_i, 0);
                 const unsigned d_tmem = tmem_base + ab * (unsigned)TP_BN;
                 bool ok = true;
                 for (int ks = 0; ks < n_k; ++ks, ++it) {
                     if (new_rb && !tp_wait(lfptx::smem_u32(&sh->a_full[ks]), (a_loads - 1) & 1u, P, sh)) { ok = false; break; }
                     const unsigned st = it % N_ST, use = it / N_ST;
                     if (!tp_wait(lfptx::smem_u32(&sh->b_full[st]), use & 1u, P, sh)) { ok = false; break; }
+                    if (ks == 0) TG_STAMP(tile_i, 1);
                     lfptx::tc_fence_after();
                     const unsigned a_addr = RESIDENT ? lfptx::smem_u32(a_res + (size_t)ks * TP_A_STAGE_BYTES)
                                                      : lfptx::smem_u32(a_res + (size_t)st * (TP_A_STAGE_BYTES + TP_B_STAGE_BYTES));
@@ -533,6 +558,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
                 // the last tile of a row block frees the resident operand for the next one
                 if (RESIDENT && t + 1 < t_end && (t + 1) / P.tiles_n != rb) tp_commit_both(lfptx::smem_u32(&sh->a_empty));
                 tp_commit_both(lfptx::smem_u32(&sh->acc_full[ab]));
+                TG_STAMP(tile_i, 2);
             }
         }
     } else {
@@ -558,6 +584,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             if (w_row)
                 tg_prefetch_w(P.sgd.w_sub, P.M, P.N, row0 - sub_r, tn * TP_BN + half * (TP_BN / 2), TP_BN / 2, lane);
             if (!tp_wait(lfptx::smem_u32(&sh->acc_full[ab]), ab_use & 1u, P, sh)) break;
+            if (threadIdx.x == 64) TG_STAMP(tile_i, 3);
             lfptx::tc_fence_after();
 #pragma unroll 1
             for (int cchunk = 0; cchunk < TP_BN / 2 / 32; ++cchunk) {
@@ -591,6 +618,7 @@ k_gw_gemm_tf32_pair(const __grid_constant__ CUtensorMap map_d, const __grid_cons
             }
             lfptx::tc_fence_before();
             __syncwarp();
+            if (threadIdx.x == 64) TG_STAMP(tile_i, 4);
             if (lane == 0) tp_arrive_remote(leader_acc_empty0 + ab * (unsigned)sizeof(unsigned long long));
         }
     }

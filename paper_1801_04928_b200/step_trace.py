@@ -4,8 +4,9 @@ and inside the two-SM tensor-core kernel of the mini-batch chain, one K stage at
     python -m paper_1801_04928_b200.step_trace [--N 1024] [--L 32] [--k 4]
                                                [--kernel groups|clusters|columns|all]
     python -m paper_1801_04928_b200.step_trace --kernel pair [--N 4096] [--B 256] [--delta-math 2|3]
+    python -m paper_1801_04928_b200.step_trace --kernel gwpair [--N 4096] [--B 256]
 
-Builds a DEBUG copy of the library (``-DLF_PK_TRACE -DLF_CK_TRACE -DLF_DG_TRACE``: thread 0 of two
+Builds a DEBUG copy of the library (``-DLF_PK_TRACE -DLF_CK_TRACE -DLF_DG_TRACE -DLF_TG_TRACE``: thread 0 of two
 CTAs, or the leader CTA of the first CTA pair, writes SM-clock stamps at fixed points of every
 layer step or K stage; the release library carries none of this) under ``_build/trace/``, runs a
 few passes of the chosen kernel on seeded inputs and prints the median number of SM cycles
@@ -59,7 +60,7 @@ KERNELS = {  # name -> (LF_OPT_VARIANT, LF_OPT_FUSED_TILING, stamps in order, na
 def build_trace_library() -> str:
     os.makedirs(TRACE_DIR, exist_ok=True)
     nvcc = lfbuild._nvcc()
-    flags = [f for f in lfbuild.NVCC_FLAGS if f not in ("-Xptxas", "-v")] + ["-DLF_PK_TRACE", "-DLF_CK_TRACE", "-DLF_DG_TRACE"]
+    flags = [f for f in lfbuild.NVCC_FLAGS if f not in ("-Xptxas", "-v")] + ["-DLF_PK_TRACE", "-DLF_CK_TRACE", "-DLF_DG_TRACE", "-DLF_TG_TRACE"]
 
     def one(src):
         obj = os.path.join(TRACE_DIR, src.replace(".cu", ".o"))
@@ -170,12 +171,45 @@ def trace_pair(lib, torch, lf_inputs, np, N, B, what, delta_math):
     print(f"| kernel entered -> before the exit | {int(once[3] - once[0])} |")
 
 
+def trace_gw_pair(lib, torch, np, N, B):
+    """Eq. bp4 of one layer through lf_grad_w on the two-SM kernel: stamps per 256 x 256 tile of the
+    first pair's leader CTA: 0 the issuing thread has the accumulator, 1 it sees the first stage's
+    operands, 2 all products and commits of the tile are issued, 3 an epilogue warp sees the finished
+    accumulator, 4 that warp has stored its part of the tile."""
+    vp = ctypes.c_void_p
+    P = lambda x: vp(x.data_ptr())
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    d = torch.empty((B, N), device="cuda").normal_(0.0, 1.0, generator=g)
+    a = torch.empty((B, N), device="cuda").uniform_(0.0, 1.0, generator=g)
+    gw = torch.empty((N, N), device="cuda")
+    h = vp()
+    assert lib.lf_create(ctypes.byref(h), 1, N, B, 1) == 0
+    lib.lf_set_option(h, 2, 2); lib.lf_set_option(h, 7, 2)      # LF_OPT_GW_MATH = TF32, LF_OPT_TC_TILING = two-SM
+    for _ in range(3):
+        assert lib.lf_grad_w(h, P(d), P(a), P(gw)) == 0
+    assert lib.lf_sync(h) == 0
+    buf = (ctypes.c_longlong * (32 * 16))()
+    assert lib.lf_debug_read_gw_pair_trace(buf) == 0
+    lib.lf_destroy(h)
+    tr = np.array(buf, dtype=np.int64).reshape(32, 16)
+    n = 0
+    while n < 32 and tr[n, 2] != 0 and (n == 0 or tr[n, 2] > tr[n - 1, 2]):
+        n += 1
+    t0 = tr[0, 8]
+    print(f"\n## weight-gradient pair kernel (Eq. bp4): N = {N}, B = {B}; {n} tiles in the first pair's run; cycles since the kernel was entered")
+    print(f"set-up done {int(tr[0, 9] - t0)}, first operand load issued {int(tr[0, 10] - t0)}")
+    print("| tile | issuer has the accumulator | first operands seen | products issued | epilogue sees the accumulator | epilogue warp done |")
+    print("|---|---|---|---|---|---|")
+    for t in range(n):
+        print(f"| {t} | " + " | ".join(str(int(tr[t, j] - t0)) for j in range(5)) + " |")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--N", type=int, default=1024)
     ap.add_argument("--L", type=int, default=32)
     ap.add_argument("--k", type=int, default=4)
-    ap.add_argument("--kernel", default="all", choices=["all", "pair"] + sorted(KERNELS))
+    ap.add_argument("--kernel", default="all", choices=["all", "pair", "gwpair"] + sorted(KERNELS))
     ap.add_argument("--B", type=int, default=256, help="pair: samples")
     ap.add_argument("--delta-math", type=int, default=2, help="pair: 2 = three TF32 products, 3 = cross terms in BF16")
     ap.add_argument("--what", default="both", choices=["forward", "backward", "both"], help="pair: which contraction")
@@ -190,6 +224,9 @@ def main():
     clock = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader"],
                            capture_output=True, text=True).stdout.strip()
     print(f"SM clock now / max: {clock} (cycles -> ns: divide by the GHz under load)")
+    if args.kernel == "gwpair":
+        trace_gw_pair(lib, torch, np, args.N, args.B)
+        return
     if args.kernel == "pair":
         for what in (("forward", "backward") if args.what == "both" else (args.what,)):
             trace_pair(lib, torch, lf_inputs, np, args.N, args.B, what, args.delta_math)
