@@ -919,13 +919,16 @@ __global__ void __launch_bounds__(256)
 k_delta_finish(const float* __restrict__ partial, const float* __restrict__ a_l, float* __restrict__ delta_l,
                size_t n4, const DgSlots S, int act)
 {
-    const int c4 = blockIdx.x * blockDim.x + threadIdx.x, b = blockIdx.y;
+    const int c4 = blockIdx.x * blockDim.x + threadIdx.x;
     if (c4 >= S.row4) return;
-    const size_t i = (size_t)b * S.row4 + c4;
-    const float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
-    const float4 av = reinterpret_cast<const float4*>(a_l)[i];
-    reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * lf_act_prime(av.x, act), s.y * lf_act_prime(av.y, act),
-                                                        s.z * lf_act_prime(av.z, act), s.w * lf_act_prime(av.w, act));
+    const int B = (int)(n4 / (size_t)S.row4);
+    for (int b = blockIdx.y; b < B; b += gridDim.y) {       // (the grid holds at most 65535 samples)
+        const size_t i = (size_t)b * S.row4 + c4;
+        const float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
+        const float4 av = reinterpret_cast<const float4*>(a_l)[i];
+        reinterpret_cast<float4*>(delta_l)[i] = make_float4(s.x * lf_act_prime(av.x, act), s.y * lf_act_prime(av.y, act),
+                                                            s.z * lf_act_prime(av.z, act), s.w * lf_act_prime(av.w, act));
+    }
 }
 
 // forward: z^l = (sum over the partial-sum slots) + b^l ; a^l = sigma(z^l)
@@ -933,14 +936,17 @@ __global__ void __launch_bounds__(256)
 k_forward_finish(const float* __restrict__ partial, const float* __restrict__ b_l, float* __restrict__ z_l,
                  float* __restrict__ a_l, size_t n4, const DgSlots S, int act)
 {
-    const int c4 = blockIdx.x * blockDim.x + threadIdx.x, b = blockIdx.y;
+    const int c4 = blockIdx.x * blockDim.x + threadIdx.x;
     if (c4 >= S.row4) return;
-    const size_t i = (size_t)b * S.row4 + c4;
-    float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
+    const int B = (int)(n4 / (size_t)S.row4);
     const float4 bb = reinterpret_cast<const float4*>(b_l)[c4];
-    s.x += bb.x; s.y += bb.y; s.z += bb.z; s.w += bb.w;
-    reinterpret_cast<float4*>(z_l)[i] = s;
-    reinterpret_cast<float4*>(a_l)[i] = make_float4(lf_act(s.x, act), lf_act(s.y, act), lf_act(s.z, act), lf_act(s.w, act));
+    for (int b = blockIdx.y; b < B; b += gridDim.y) {
+        const size_t i = (size_t)b * S.row4 + c4;
+        float4 s = dg_slot_sum(reinterpret_cast<const float4*>(partial) + i, n4, dg_slot_count(S, b, 4 * c4));
+        s.x += bb.x; s.y += bb.y; s.z += bb.z; s.w += bb.w;
+        reinterpret_cast<float4*>(z_l)[i] = s;
+        reinterpret_cast<float4*>(a_l)[i] = make_float4(lf_act(s.x, act), lf_act(s.y, act), lf_act(s.z, act), lf_act(s.w, act));
+    }
 }
 
 typedef CUresult (*dg_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1213,7 +1219,7 @@ int lf_delta_gemm_tc(lf_ctx* c, const float* w_up, const float* delta_up, const 
     int rc = dg_launch(c, delta_up, w_up, false, math == LF_DELTA_MATH_TF32_BF16, n_l, n_up, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_l / 4;
-    k_delta_finish<<<dim3((unsigned)((n_l / 4 + 255) / 256), (unsigned)c->B), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4,
+    k_delta_finish<<<dim3((unsigned)((n_l / 4 + 255) / 256), (unsigned)(c->B < 65535 ? c->B : 65535)), 256, 0, s>>>(c->dg_partial, a_l, delta_l, n4,
                                                                                        dg_slots(n_l, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
@@ -1228,7 +1234,7 @@ int lf_forward_gemm_tc(lf_ctx* c, const float* w_l, const float* b_l, const floa
     int rc = dg_launch(c, a_prev, w_l, true, math == LF_DELTA_MATH_TF32_BF16, n_out, n_in, s, &pl);
     if (rc != LF_OK) return rc;
     const size_t n4 = (size_t)c->B * n_out / 4;
-    k_forward_finish<<<dim3((unsigned)((n_out / 4 + 255) / 256), (unsigned)c->B), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4,
+    k_forward_finish<<<dim3((unsigned)((n_out / 4 + 255) / 256), (unsigned)(c->B < 65535 ? c->B : 65535)), 256, 0, s>>>(c->dg_partial, b_l, z_l, a_l, n4,
                                                                                            dg_slots(n_out, pl), c->opt_act);
     LF_CUDA_TRY(c, cudaGetLastError());
     *launches += 2;
