@@ -395,7 +395,6 @@ constexpr int DP_SPLITTERS = 192;                        // warps 2-7
 constexpr int DP_REGS_LAUNCH = 128, DP_REGS_SMALL = 48, DP_REGS_SUM = 208;
 static_assert(2 * 128 * DP_REGS_SMALL + 2 * 128 * DP_REGS_SUM <= DP_THREADS * DP_REGS_LAUNCH,
               "the warpgroups' register shares must fit into what the CTA is launched with");
-constexpr int DP_TMEM_COLS = 512;                        // two stage accumulators of 256 columns
 constexpr int DP_EPI_LD = 20;                            // 16 columns + padding
 constexpr int DP_EPI_BYTES = 8 * 32 * DP_EPI_LD * 4;
 constexpr size_t DP_SMEM_BYTES = (size_t)DP_RING_BYTES + DP_EPI_BYTES + 1024 + 256;
@@ -513,7 +512,7 @@ __device__ __forceinline__ bool dp_next_segment(int& g, int g1, const DgParams& 
     return true;
 }
 // fmt: operand format of the instruction kind (kind::tf32: 2 = TF32; kind::f16: 1 = BF16)
-__device__ __forceinline__ unsigned dp_idesc(bool w_kmajor, unsigned fmt = 2u)
+__device__ __forceinline__ unsigned dp_idesc(bool w_kmajor, unsigned fmt = 2u, int tile_m = 2 * DG_BM, int tile_n = DP_BN)
 {
     unsigned d = 0;
     d |= 1u << 4;                             // fp32 accumulator
@@ -521,9 +520,35 @@ __device__ __forceinline__ unsigned dp_idesc(bool w_kmajor, unsigned fmt = 2u)
     d |= fmt << 10;                           // B
     d |= 0u << 15;                            // A is K-major
     d |= (w_kmajor ? 0u : 1u) << 16;          // B operand: K-major or MN-major
-    d |= (unsigned)(DP_BN >> 3) << 17;
-    d |= (unsigned)((2 * DG_BM) >> 4) << 24;
+    d |= (unsigned)(tile_n >> 3) << 17;
+    d |= (unsigned)(tile_m >> 4) << 24;
     return d;
+}
+// One product of a stage: a CTA pair's instruction (cta_group::2) or a single CTA's (cta_group::1);
+// WIDE = false: TF32 operands, eight values of the contraction index; WIDE = true: BF16, sixteen.
+template <bool PAIR, bool WIDE>
+__device__ __forceinline__ void dp_product(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                           unsigned idesc, unsigned accumulate)
+{
+    if (PAIR) {
+        if (WIDE) dp_mma16(d_tmem, a_desc, b_desc, idesc, accumulate);
+        else dp_mma(d_tmem, a_desc, b_desc, idesc, accumulate);
+    } else if (WIDE) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+    } else {
+        dg_mma(d_tmem, a_desc, b_desc, idesc, accumulate);
+    }
+}
+// "everything issued so far is done" to a barrier of this CTA and, for a pair, of its peer
+template <bool PAIR>
+__device__ __forceinline__ void dp_commit(unsigned bar)
+{
+    if (PAIR) dp_commit_both(bar);
+    else dg_commit(bar);
 }
 // 32 lanes x 64 consecutive fp32 columns of tensor memory as two loads in flight together
 __device__ __forceinline__ void dp_tmem_ld64(unsigned taddr, unsigned (&r)[64])
@@ -632,7 +657,10 @@ __device__ __forceinline__ void dp_split_batch(float4* raw, float4* lo, const Dp
 //   remainders rounded to BF16 (K-major operands: both in one 128-byte row, high parts first; the
 //   MN-major W tile: two tiles of 64-column blocks).  A cross term is below 2^-11 of its product, so
 //   the 2^-9 of a BF16 rounding leaves about 2^-20 of the product.
-template <bool W_KMAJOR, bool CROSS_BF16>
+// PAIR = false: the same kernel on single CTAs (no cluster): a CTA works alone on 128 samples x 128 columns
+//   with cta_group::1 instructions (M = 128, N = 128) -- the warp-specialised form for 17 to 128 samples, where
+//   a pair's second half would be empty; its summing warps hold 64 columns per thread.
+template <bool W_KMAJOR, bool CROSS_BF16, bool PAIR>
 __global__ void __launch_bounds__(DP_THREADS, 1)
 k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_w,
                      const DgParams P)
@@ -645,8 +673,10 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     DpShared* sh = reinterpret_cast<DpShared*>(stages + (size_t)DP_RING_BYTES + DP_EPI_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned rank = lfptx::cluster_ctarank();
-    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    constexpr int TILE_M = PAIR ? 2 * DG_BM : DG_BM, TILE_N = PAIR ? DP_BN : DP_BNH;   // tile of a pair / of a single CTA
+    constexpr int SUM_COLS = TILE_N / 2;                    // columns a summing thread holds
+    const unsigned rank = PAIR ? lfptx::cluster_ctarank() : 0u;
+    const int pair = PAIR ? blockIdx.x >> 1 : blockIdx.x, n_pairs = PAIR ? gridDim.x >> 1 : gridDim.x;   // worker index and count
     const int g_begin = (int)((long long)P.g_total * pair / n_pairs), g_end = (int)((long long)P.g_total * (pair + 1) / n_pairs);
     DG_STAMP_ONCE(9);
 
@@ -656,24 +686,30 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             lfptx::mbar_init(lfptx::smem_u32(&sh->raw_empty[i]), 1);
         }
         for (int i = 0; i < DP_LO_SLOTS; ++i) {
-            lfptx::mbar_init(lfptx::smem_u32(&sh->split_done[i]), 2 * DP_SPLITTERS / 32);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->split_done[i]), (PAIR ? 2 : 1) * DP_SPLITTERS / 32);
             lfptx::mbar_init(lfptx::smem_u32(&sh->lo_empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             lfptx::mbar_init(lfptx::smem_u32(&sh->acc_full[i]), 1);
-            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_empty[i]), 16);
+            lfptx::mbar_init(lfptx::smem_u32(&sh->acc_empty[i]), PAIR ? 16 : 8);
         }
         sh->abort_flag = 0u;
         lfptx::mbar_fence_init();
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)DP_TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)(2 * TILE_N)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(lfptx::smem_u32(&sh->tmem_base)), "r"((unsigned)(2 * TILE_N)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     lfptx::tc_fence_before();
     __syncthreads();
-    lfptx::cluster_sync_all();   // the peer's barriers exist before anything can arrive on them
+    if (PAIR) lfptx::cluster_sync_all();   // the peer's barriers exist before anything can arrive on them
     lfptx::tc_fence_after();
     const unsigned tmem_base = sh->tmem_base;
     DG_STAMP_ONCE(10);
@@ -689,8 +725,8 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
                     const int tn = sg.tile % P.tiles_n, tm = sg.tile / P.tiles_n;
                     const int j0 = sg.kb0 * DG_BK, n_k = sg.kb1 - sg.kb0;
-                    const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM;       // my samples
-                    const int col0 = tn * DP_BN + (int)rank * DP_BNH;          // my columns of W
+                    const int row0 = tm * TILE_M + (int)rank * DG_BM;          // my samples
+                    const int col0 = tn * TILE_N + (int)rank * DP_BNH;         // my columns of W
                     for (int ks = 0; ks < n_k; ++ks, ++it) {
                         const unsigned st = it % DP_RAW_SLOTS, use = it / DP_RAW_SLOTS;
                         if (use > 0 && !dp_wait(lfptx::smem_u32(&sh->raw_empty[st]), (use - 1) & 1u, P, sh)) { ok = false; break; }
@@ -724,7 +760,7 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
         } else if (warp == 1) {
             // ------------------------------ MMA issuer (leader CTA only) -----------------------
             if (lane == 0 && rank == 0) {
-                const unsigned idesc = dp_idesc(W_KMAJOR), idesc16 = dp_idesc(W_KMAJOR, 1u);
+                const unsigned idesc = dp_idesc(W_KMAJOR, 2u, TILE_M, TILE_N), idesc16 = dp_idesc(W_KMAJOR, 1u, TILE_M, TILE_N);
                 unsigned it = 0;
                 bool ok = true;
                 DpSegment sg;
@@ -740,30 +776,30 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                         lfptx::tc_fence_after();
                         const unsigned hi = lfptx::smem_u32(stages + (size_t)st * DP_RAW_BYTES);
                         const unsigned lo = lfptx::smem_u32(stages + (size_t)DP_LO_BASE + (size_t)p * DP_RAW_BYTES);
-                        const unsigned d_tmem = tmem_base + p * (unsigned)DP_BN;
+                        const unsigned d_tmem = tmem_base + p * (unsigned)TILE_N;
                         // the small products first, then the four large ones
                         if (CROSS_BF16) {
 #pragma unroll
                             for (int kk = 0; kk < DG_BK / 16; ++kk) {
-                                dp_mma16(d_tmem, dg_desc_kmajor(lo + 64 + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 0, kk),
-                                         idesc16, kk > 0 ? 1u : 0u);
-                                dp_mma16(d_tmem, dg_desc_kmajor(lo + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 1, kk),
-                                         idesc16, 1u);
+                                dp_product<PAIR, true>(d_tmem, dg_desc_kmajor(lo + 64 + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 0, kk),
+                                                       idesc16, kk > 0 ? 1u : 0u);
+                                dp_product<PAIR, true>(d_tmem, dg_desc_kmajor(lo + kk * 32), dp_desc_w16<W_KMAJOR>(lo + DG_A_BYTES, 1, kk),
+                                                       idesc16, 1u);
                             }
                         } else {
 #pragma unroll
                             for (int kk = 0; kk < DG_BK / 8; ++kk) {
-                                dp_mma(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
-                                       kk > 0 ? 1u : 0u);
-                                dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
+                                dp_product<PAIR, false>(d_tmem, dg_desc_kmajor(lo + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc,
+                                                        kk > 0 ? 1u : 0u);
+                                dp_product<PAIR, false>(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(lo + DG_A_BYTES, kk), idesc, 1u);
                             }
                         }
 #pragma unroll
                         for (int kk = 0; kk < DG_BK / 8; ++kk)
-                            dp_mma(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
-                        dp_commit_both(lfptx::smem_u32(&sh->raw_empty[st]));
-                        dp_commit_both(lfptx::smem_u32(&sh->lo_empty[p]));
-                        dp_commit_both(lfptx::smem_u32(&sh->acc_full[p]));
+                            dp_product<PAIR, false>(d_tmem, dg_desc_kmajor(hi + kk * 32), dg_desc_w<W_KMAJOR>(hi + DG_A_BYTES, kk), idesc, 1u);
+                        dp_commit<PAIR>(lfptx::smem_u32(&sh->raw_empty[st]));
+                        dp_commit<PAIR>(lfptx::smem_u32(&sh->lo_empty[p]));
+                        dp_commit<PAIR>(lfptx::smem_u32(&sh->acc_full[p]));
                         DG_STAMP(6);
                     }
                 }
@@ -806,17 +842,17 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
         // ------------------------------ running sums and output: warps 8..15 -------------------
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(DP_REGS_SUM));
         const int quad = warp & 3;               // the TMEM lane quadrant this warp may read
-        const int half = (warp - 8) >> 2;        // which 128 of the 256 accumulator columns
+        const int half = (warp - 8) >> 2;        // which half of the accumulator's columns
         const unsigned leader_acc_empty0 = lfptx::map_to_cta(lfptx::smem_u32(&sh->acc_empty[0]), 0);
         unsigned it = 0;
         bool ok = true;
-        float acc[DP_BNH];     // this thread's sample, its 128 columns of the tile
+        float acc[SUM_COLS];   // this thread's sample, its columns of the tile (128 for a pair, 64 for a single CTA)
         DpSegment sg;
         for (int g = g_begin; ok && dp_next_segment(g, g_end, P, pair, n_pairs, sg);) {
             const int tn = sg.tile % P.tiles_n, tm = sg.tile / P.tiles_n, sp = sg.slot;
             const int n_k = sg.kb1 - sg.kb0;
 #pragma unroll
-            for (int v = 0; v < DP_BNH; ++v) acc[v] = 0.f;
+            for (int v = 0; v < SUM_COLS; ++v) acc[v] = 0.f;
             for (int ks = 0; ks < n_k; ++ks, ++it) {
                 // add the finished stage (accumulator it & 1) into the registers
                 const unsigned p = it & 1u;
@@ -824,9 +860,9 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
                 if (threadIdx.x == 256) DG_STAMP(7);
                 lfptx::tc_fence_after();
 #pragma unroll
-                for (int cchunk = 0; cchunk < DP_BNH / 64; ++cchunk) {
+                for (int cchunk = 0; cchunk < SUM_COLS / 64; ++cchunk) {
                     unsigned r[64];
-                    dp_tmem_ld64(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)DP_BN + half * DP_BNH + cchunk * 64, r);
+                    dp_tmem_ld64(tmem_base + ((unsigned)(quad * 32) << 16) + p * (unsigned)TILE_N + half * SUM_COLS + cchunk * 64, r);
 #pragma unroll
                     for (int v = 0; v < 64; ++v)
                         acc[cchunk * 64 + v] += __uint_as_float(r[v]);
@@ -839,13 +875,13 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
             if (!ok) break;
             float* blk = epi + (warp - 8) * 32 * DP_EPI_LD;
             const int sub_r = lane >> 2, sub_c = (lane & 3) * 4;
-            const int row0 = tm * 2 * DG_BM + (int)rank * DG_BM + quad * 32 + sub_r;
-            const int col0 = tn * DP_BN + half * DP_BNH + sub_c;
+            const int row0 = tm * TILE_M + (int)rank * DG_BM + quad * 32 + sub_r;
+            const int col0 = tn * TILE_N + half * SUM_COLS + sub_c;
             // four rows per lane (row0 + 8 i), 16 columns per pass; constant offsets from one pointer per row
             float* out_row = P.partial + (size_t)sp * P.B * P.N + (size_t)row0 * P.N + col0;
             const size_t row_step = (size_t)8 * P.N;
 #pragma unroll
-            for (int cchunk = 0; cchunk < DP_BNH / 16; ++cchunk) {
+            for (int cchunk = 0; cchunk < SUM_COLS / 16; ++cchunk) {
 #pragma unroll
                 for (int v = 0; v < 4; ++v)
                     *reinterpret_cast<float4*>(blk + lane * DP_EPI_LD + 4 * v) =
@@ -869,12 +905,14 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
     // neither CTA may leave, or free tensor memory, while the other can still reach it
     lfptx::tc_fence_before();
     __syncthreads();
-    lfptx::cluster_sync_all();
+    if (PAIR) lfptx::cluster_sync_all();
     DG_STAMP_ONCE(12);
     if (warp == 1) {
         lfptx::tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)DP_TMEM_COLS)
-                     : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)(2 * TILE_N)) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((unsigned)(2 * TILE_N)) : "memory");
     }
 }
 
@@ -883,14 +921,15 @@ k_delta_gemm_tc_pair(const __grid_constant__ CUtensorMap map_d, const __grid_con
 // there are run segments in the element's tile.
 struct DgSlots {
     int splits;
-    int n_pairs, tiles_n, kb_per_tile, row4;   // row4 = N / 4
+    int n_pairs, tiles_n, kb_per_tile, row4;   // row4 = N / 4; n_pairs: workers (pairs or single CTAs) of the run-dealing kernel
     int g_total;
+    int tile_m, tile_n;                        // its tile: 256 x 256 for pairs, 128 x 128 for single CTAs
 };
 // slots that hold a contribution to the output elements of sample b, columns n .. n+3
 __device__ __forceinline__ int dg_slot_count(const DgSlots& S, int b, int n)
 {
     if (S.n_pairs == 0) return S.splits;
-    const int g0 = ((b / (2 * DG_BM)) * S.tiles_n + n / DP_BN) * S.kb_per_tile;
+    const int g0 = ((b / S.tile_m) * S.tiles_n + n / S.tile_n) * S.kb_per_tile;
     return dp_owner(g0 + S.kb_per_tile - 1, S.g_total, S.n_pairs) - dp_owner(g0, S.g_total, S.n_pairs) + 1;
 }
 // the sum of an element's slots, in slot order; the loads go out four at a time
@@ -972,8 +1011,10 @@ dg_encode_fn dg_get_encode()
 
 struct DgPlan {
     int tiles_m, tiles_n, splits, k_per_split;
-    int pairs, kb_per_tile;      // two-SM kernel (pairs > 0): launched pairs and K blocks per tile
+    int pairs, kb_per_tile;      // run-dealing kernel (pairs > 0): launched pairs (or single CTAs) and K blocks per tile
     int g_total;
+    int tile_m, tile_n;          // its tile (0: the plain one-SM kernel's fixed 128 x 128)
+    bool solo;                   // run-dealing kernel on single CTAs
 };
 
 // One contraction out[B][Nc] = lhs[B][K] x W: Nc output columns, contraction length K.  Eq. bp2 of
@@ -1002,13 +1043,13 @@ int dp_max_pairs(const lf_ctx* c)
     if (cached_dev == c->device) return cached;
     int n = 0;
     if ((size_t)c->smem_optin >= DP_SMEM_BYTES &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)DP_SMEM_BYTES) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute at[1];
@@ -1017,14 +1058,37 @@ int dp_max_pairs(const lf_ctx* c)
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
         int n0 = 0, n1 = 0, n2 = 0, n3 = 0;
-        if (cudaOccupancyMaxActiveClusters(&n0, k_delta_gemm_tc_pair<false, false>, &cfg) == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n1, k_delta_gemm_tc_pair<true, false>, &cfg) == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n2, k_delta_gemm_tc_pair<false, true>, &cfg) == cudaSuccess &&
-            cudaOccupancyMaxActiveClusters(&n3, k_delta_gemm_tc_pair<true, true>, &cfg) == cudaSuccess) {
+        if (cudaOccupancyMaxActiveClusters(&n0, k_delta_gemm_tc_pair<false, false, true>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n1, k_delta_gemm_tc_pair<true, false, true>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n2, k_delta_gemm_tc_pair<false, true, true>, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&n3, k_delta_gemm_tc_pair<true, true, true>, &cfg) == cudaSuccess) {
             n = n0 < n1 ? n0 : n1;
             if (n2 < n) n = n2;
             if (n3 < n) n = n3;
         }
+    }
+    cudaGetLastError();
+    cached_dev = c->device; cached = n;
+    return n;
+}
+
+// Largest number of CTAs of the single-CTA form of that kernel that can be resident at once (0: unusable).
+int dp_max_solo(const lf_ctx* c)
+{
+    static int cached_dev = -1, cached = 0;
+    if (cached_dev == c->device) return cached;
+    int n = 0;
+    if ((size_t)c->smem_optin >= DP_SMEM_BYTES &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(k_delta_gemm_tc_pair<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)DP_SMEM_BYTES) == cudaSuccess) {
+        int n0 = 0, n1 = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n0, k_delta_gemm_tc_pair<false, false, false>, DP_THREADS,
+                                                          DP_SMEM_BYTES) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n1, k_delta_gemm_tc_pair<true, false, false>, DP_THREADS,
+                                                          DP_SMEM_BYTES) == cudaSuccess)
+            n = (n0 < n1 ? n0 : n1) > 0 ? c->sm_count : 0;      // one CTA per SM: each holds most of its shared memory
     }
     cudaGetLastError();
     cached_dev = c->device; cached = n;
@@ -1036,11 +1100,13 @@ bool dp_use_pairs(const lf_ctx* c, int Nc, int K);
 
 // Two-SM kernel: tiles x K-blocks cut into one contiguous run per pair; `splits` becomes the
 // largest number of run segments (= partial-sum slots) any tile has.
-DgPlan dp_plan(const lf_ctx* c, int Nc, int K, int max_pairs)
+DgPlan dp_plan(const lf_ctx* c, int Nc, int K, int max_pairs, bool solo = false)
 {
     DgPlan p = {};
-    p.tiles_m = (c->B + 2 * DG_BM - 1) / (2 * DG_BM);
-    p.tiles_n = (Nc + DP_BN - 1) / DP_BN;
+    p.solo = solo;
+    p.tile_m = solo ? DG_BM : 2 * DG_BM; p.tile_n = solo ? DP_BNH : DP_BN;
+    p.tiles_m = (c->B + p.tile_m - 1) / p.tile_m;
+    p.tiles_n = (Nc + p.tile_n - 1) / p.tile_n;
     p.kb_per_tile = (K + DG_BK - 1) / DG_BK;
     p.k_per_split = p.kb_per_tile * DG_BK;
     const int tiles = p.tiles_m * p.tiles_n;
@@ -1060,20 +1126,34 @@ DgPlan dp_plan(const lf_ctx* c, int Nc, int K, int max_pairs)
 }
 
 // could the two-SM kernel be chosen for this shape (whatever LF_OPT_TC_TILING says)?
-// Measured per layer, forward / backward, pairs against one CTA per tile: with 32 to 128 samples the
-// pairs (second CTA's samples empty) lose at widths up to 4096 (N = 2048: 27-31 against 22 us) and win
-// at 8192 (139-148 against 155-157 us): there the weight tile each CTA need not load outweighs the
-// empty half.  Narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there.
-constexpr long long DP_WIDE_LAYER = 6144ll * 6144ll;
+// Pairs need more than 128 samples: with fewer, their second CTA's samples are empty, and the
+// warp-specialised kernel on single CTAs (below) is ahead at every width measured (N = 8192, 17 to 128
+// samples, forward / backward per layer: 122-128 / 161-171 us against the pairs' 138-146 / 175-188).
+// Narrow layers are launch-latency-bound: the lighter one-SM kernel is faster there.
 bool dp_shape_fits_pairs(const lf_ctx* c, int Nc, int K)
 {
-    const bool enough = c->B > DG_BM || (long long)Nc * K >= DP_WIDE_LAYER;
-    return enough && Nc >= 512 && K >= 512 && dp_max_pairs(c) > 0;
+    return c->B > DG_BM && Nc >= 512 && K >= 512 && dp_max_pairs(c) > 0;
 }
 
 bool dp_use_pairs(const lf_ctx* c, int Nc, int K)
 {
     return c->tc_pair_kernels && dp_shape_fits_pairs(c, Nc, K) && dp_plan(c, Nc, K, dp_max_pairs(c)).pairs > 0;
+}
+
+// The warp-specialised kernel on single CTAs, where pairs do not apply: for layers of at least
+// DP_SOLO_MIN_WIDTH.  Measured per layer (forward / backward, 17 to 128 samples) against the plain
+// one-SM kernel: N = 2048 and 3072 level, N = 4096: 41-45 / 53-59 against 48-50 / 59-63 us,
+// N = 5120: 57-60 / 74-81 against 73-75 / 88-93 us.  With fewer than 17 samples only the forward pass comes here.
+#ifndef DP_SOLO_MIN_WIDTH
+#define DP_SOLO_MIN_WIDTH 4096
+#endif
+bool dp_shape_fits_solo(const lf_ctx* c, int Nc, int K)
+{
+    return Nc >= DP_SOLO_MIN_WIDTH && K >= DP_SOLO_MIN_WIDTH && dp_max_solo(c) > 0;
+}
+bool dp_use_solo(const lf_ctx* c, int Nc, int K)
+{
+    return !dp_use_pairs(c, Nc, K) && dp_shape_fits_solo(c, Nc, K) && dp_plan(c, Nc, K, dp_max_solo(c), true).pairs > 0;
 }
 
 // floats of partial-sum scratch one contraction of this shape may need: [splits][B][Nc] of
@@ -1084,6 +1164,10 @@ size_t dg_partial_floats(const lf_ctx* c, int Nc, int K)
     if (dp_shape_fits_pairs(c, Nc, K)) {
         const int s2 = dp_plan(c, Nc, K, dp_max_pairs(c)).splits;
         if (s2 > splits) splits = s2;
+    }
+    if (dp_shape_fits_solo(c, Nc, K)) {
+        const int s3 = dp_plan(c, Nc, K, dp_max_solo(c), true).splits;
+        if (s3 > splits) splits = s3;
     }
     return (size_t)splits * c->B * Nc;
 }
@@ -1123,6 +1207,7 @@ bool lf_delta_tc_supported(const lf_ctx* c)
         attr_dev = c->device;
     }
     dp_max_pairs(c);
+    dp_max_solo(c);
     return true;
 }
 
@@ -1131,6 +1216,7 @@ static DgSlots dg_slots(int Nc, const DgPlan& pl)
     DgSlots S = {};
     S.splits = pl.splits; S.n_pairs = pl.pairs; S.tiles_n = pl.tiles_n; S.kb_per_tile = pl.kb_per_tile;
     S.row4 = Nc / 4; S.g_total = pl.g_total;
+    S.tile_m = pl.tile_m; S.tile_n = pl.tile_n;
     return S;
 }
 
@@ -1169,8 +1255,8 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
         }
     }
     const bool pairs = dp_use_pairs(c, Nc, K);
-    const int max_pairs = pairs ? dp_max_pairs(c) : 0;
-    const DgPlan pl = pairs ? dp_plan(c, Nc, K, max_pairs) : dg_plan(c, Nc, K);
+    const bool solo = !pairs && dp_use_solo(c, Nc, K);
+    const DgPlan pl = pairs ? dp_plan(c, Nc, K, dp_max_pairs(c)) : solo ? dp_plan(c, Nc, K, dp_max_solo(c), true) : dg_plan(c, Nc, K);
     if ((size_t)pl.splits * c->B * Nc > dg_partial_floats(c, Nc, K)) return LF_ERESOURCE;   // cannot happen: same plans
     DgParams P;
     P.N = Nc; P.B = c->B;
@@ -1189,18 +1275,27 @@ static int dg_launch(lf_ctx* c, const float* lhs, const float* w_mat, bool w_kma
         at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
         if (w_kmajor && cross_bf16)
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, true>, map_d, map_w, P));
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, true, true>, map_d, map_w, P));
         else if (w_kmajor)
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, false>, map_d, map_w, P));
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<true, false, true>, map_d, map_w, P));
         else if (cross_bf16)
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, true>, map_d, map_w, P));
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, true, true>, map_d, map_w, P));
         else
-            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, false>, map_d, map_w, P));
+            LF_CUDA_TRY(c, cudaLaunchKernelEx(&cfg, k_delta_gemm_tc_pair<false, false, true>, map_d, map_w, P));
         c->stats.delta_tiling = LF_TC_TILING_TWO_SM;
         *plan_out = pl;
         return LF_OK;
     }
     c->stats.delta_tiling = LF_TC_TILING_ONE_SM;
+    if (solo) {      // the warp-specialised kernel on single CTAs (the BF16 cross-term form is for pairs)
+        if (w_kmajor)
+            k_delta_gemm_tc_pair<true, false, false><<<pl.pairs, DP_THREADS, DP_SMEM_BYTES, s>>>(map_d, map_w, P);
+        else
+            k_delta_gemm_tc_pair<false, false, false><<<pl.pairs, DP_THREADS, DP_SMEM_BYTES, s>>>(map_d, map_w, P);
+        LF_CUDA_TRY(c, cudaGetLastError());
+        *plan_out = pl;
+        return LF_OK;
+    }
     const int grid = units < c->sm_count ? units : c->sm_count;
     if (w_kmajor)
         k_delta_gemm_tc<true><<<grid, DG_THREADS, DG_SMEM_BYTES, s>>>(map_d, map_w, P);

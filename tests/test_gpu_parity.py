@@ -43,7 +43,7 @@ def test_single_sample_parity(L, N, k, variant):
                                                (lf.LF_DELTA_MATH_TF32_BF16, lf.LF_TC_TILING_TWO_SM)])
 @pytest.mark.parametrize("L,N,B,k", [(2, 8, 2, 1), (3, 68, 3, 2), (3, 256, 16, 4),
                                      (4, 132, 70, 3), (2, 320, 129, 2), (5, 1028, 260, 2),
-                                     (3, 772, 256, 1), (2, 2052, 515, 2)])
+                                     (3, 772, 256, 1), (2, 2052, 515, 2), (2, 4100, 70, 2), (2, 4608, 17, 1)])
 def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
     # fp32 gate (1e-5 per tensor per layer) for every form of the delta recurrence (and of the
     # forward pass, which shares its kernels): fp32 on the CUDA cores, and the tensor cores with
@@ -51,6 +51,8 @@ def test_minibatch_fp32_parity(L, N, B, k, delta_math, tiling):
     # take over above 128 samples and from 512 columns: B = 260 leaves a pair's second half nearly
     # empty, B = 515 needs three 256-sample blocks, N = 2052 gives runs that end inside a tile);
     # and the CTA pairs with the two cross terms in BF16 (one-CTA tiles keep three TF32 products).
+    # N = 4100 and 4608 with up to 128 samples: the warp-specialised kernel on single CTAs (from a
+    # width of 4096), with a ragged last column tile and with a nearly empty sample tile.
     cfg = dict(L=L, N=N, B=B, k=k)
     t = _inputs(L, N, B, y="onehot", seed=N + B)
     out, stats = gpu_pass(cfg, t, gw_math=lf.LF_GW_MATH_FP32, delta_math=delta_math, tc_tiling=tiling)

@@ -46,9 +46,12 @@ def _sampled_minibatch_parity(L, N, B, tiling, seed, n_chain=3, grid=512):
     # the library's own choice for Eq. bp4: up to 16 samples the fp32 store stream, beyond that TF32 tensor cores
     assert stats["gw_math"] == (lf.LF_GW_MATH_FP32 if B <= 16 else lf.LF_GW_MATH_TF32) and stats["device_status"] == 0
     tol = 2e-5 if B <= 16 else TF32_TOL      # the fp32 writer is held to fp32 level
-    # CTA pairs serve more than 128 samples, and layers of at least 6144 x 6144 at any batch
-    if tiling == lf.LF_TC_TILING_TWO_SM and (B > 128 or N >= 6144):
+    # CTA pairs serve more than 128 samples; below that one CTA per tile (from a width of 4096 the
+    # warp-specialised kernel on single CTAs)
+    if tiling == lf.LF_TC_TILING_TWO_SM and B > 128:
         assert stats["delta_tiling"] == lf.LF_TC_TILING_TWO_SM
+    if B <= 128:
+        assert stats["delta_tiling"] == lf.LF_TC_TILING_ONE_SM
     # the library's own choice: a handful of samples (up to 8, or up to 16 from a width of 2048) keeps Eq. bp2 in fp32 on the CUDA cores
     assert stats["delta_math"] == (lf.LF_DELTA_MATH_FP32 if (B <= 8 or (B <= 16 and N >= 2048)) else lf.LF_DELTA_MATH_3XTF32)
 
